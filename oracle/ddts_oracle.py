@@ -1,0 +1,212 @@
+"""ctypes front end of the fp64 CPU oracle (``ddts_ref.c``) plus two slow numpy
+restatements of other forms the paper gives for the same quantity.
+
+TEST INFRASTRUCTURE ONLY: tests, the smoke check and the benchmark's CPU-baseline
+leg may import this module; the CUDA library and its Python binding never do.
+
+* ``ref_fwd`` / ``ref_step`` / ``ref_gates`` call the sequential recurrence
+  (Eq. "alpha_def", Eq. "rodimus_recurrent_form").
+* ``parallel_form`` is the O(T^2) masked form of the appendix on the chunkwise
+  representation (Eq. "rodimus_parallel_form"), for one sequence and one head.
+* ``unrolled_sum`` is the double sum obtained by unfolding the general gated
+  transition (Sec. 3.1.1, the equation after "general_state_transition").
+
+The last two exist to pin the first: they are written from different equations and
+share no code with it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ddts_ref.c")
+_LIB = os.path.join(_HERE, "libddts_ref.so")
+_lock = threading.Lock()
+_lib = None
+
+POW_G = 0        # ahat = g ** tau                (paper, Eq. "alpha_def")
+POW_SIGMOID = 1  # ahat = (1 - exp(-g)) ** tau    (alternate reading)
+
+
+def build(force: bool = False) -> str:
+    """Compile ``ddts_ref.c`` into ``libddts_ref.so`` beside it (gcc, OpenMP)."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + f".tmp{os.getpid()}"
+            cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        f32p = ctypes.POINTER(ctypes.c_float)
+        f64p = ctypes.POINTER(ctypes.c_double)
+        i32p = ctypes.POINTER(ctypes.c_int32)
+        lib.ddts_ref_gates.argtypes = [ctypes.c_int, ctypes.c_int64, f32p, f32p, f64p, f64p]
+        lib.ddts_ref_gates.restype = ctypes.c_int
+        lib.ddts_ref_fwd.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
+                                     ctypes.c_int, ctypes.c_int, ctypes.c_double,
+                                     f32p, f32p, f32p, f32p, f32p, f64p, f64p, f64p, i32p,
+                                     ctypes.c_int]
+        lib.ddts_ref_fwd.restype = ctypes.c_int
+        lib.ddts_ref_step.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                      ctypes.c_int, ctypes.c_double,
+                                      f32p, f32p, f32p, f32p, f32p, f64p, f64p]
+        lib.ddts_ref_step.restype = ctypes.c_int
+        lib.ddts_ref_num_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a, a.ctypes.data_as(ctypes.POINTER(ctypes.c_float))
+
+
+def _f64p(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double)) if a is not None else None
+
+
+def num_threads() -> int:
+    return int(_load().ddts_ref_num_threads())
+
+
+def ref_gates(x, y, ingate: int = POW_G):
+    """alpha = exp(-softplus(x) * sigmoid(y)) and ahat, element by element (fp64)."""
+    lib = _load()
+    xa, xp = _f32(x)
+    ya, yp = _f32(y)
+    alpha = np.empty(xa.shape, dtype=np.float64)
+    ahat = np.empty(xa.shape, dtype=np.float64)
+    rc = lib.ddts_ref_gates(ingate, xa.size, xp, yp, _f64p(alpha), _f64p(ahat))
+    if rc:
+        raise ValueError(f"ddts_ref_gates returned {rc}")
+    return alpha, ahat
+
+
+def ref_fwd(q, k, x, y, v, s0=None, cu_seqlens=None, scale: float = 1.0, ingate: int = POW_G,
+            want_o: bool = True, want_sT: bool = True):
+    """Sequential prefill.  q,k,x,y: [B,H,T,dk]; v: [B,H,T,dv]; s0: [B|N,H,dk,dv] or None.
+
+    Returns (o [B,H,T,dv] float64 or None, sT [B|N,H,dk,dv] float64 or None).
+    """
+    lib = _load()
+    qa, qp = _f32(q)
+    ka, kp = _f32(k)
+    xa, xp = _f32(x)
+    ya, yp = _f32(y)
+    va, vp = _f32(v)
+    B, H, T, dk = qa.shape
+    dv = va.shape[-1]
+    assert ka.shape == qa.shape == xa.shape == ya.shape and va.shape[:3] == (B, H, T)
+    cu = None
+    cup = None
+    nseq = B
+    N = 0
+    if cu_seqlens is not None:
+        cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+        N = cu.size - 1
+        nseq = N
+        cup = cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+    s0a = None
+    if s0 is not None:
+        s0a = np.ascontiguousarray(s0, dtype=np.float64)
+        assert s0a.shape == (nseq, H, dk, dv)
+    o = np.empty((B, H, T, dv), dtype=np.float64) if want_o else None
+    sT = np.empty((nseq, H, dk, dv), dtype=np.float64) if want_sT else None
+    rc = lib.ddts_ref_fwd(ingate, B, H, T, dk, dv, float(scale), qp, kp, xp, yp, vp,
+                          _f64p(s0a), _f64p(o), _f64p(sT), cup, N)
+    if rc:
+        raise ValueError(f"ddts_ref_fwd returned {rc}")
+    return o, sT
+
+
+def ref_step(q, k, x, y, v, state, scale: float = 1.0, ingate: int = POW_G):
+    """One decode step; ``state`` ([Nseq,H,dk,dv] float64, C-contiguous) is updated in place."""
+    lib = _load()
+    qa, qp = _f32(q)
+    ka, kp = _f32(k)
+    xa, xp = _f32(x)
+    ya, yp = _f32(y)
+    va, vp = _f32(v)
+    Nseq, H, dk = qa.shape
+    dv = va.shape[-1]
+    assert state.dtype == np.float64 and state.flags["C_CONTIGUOUS"]
+    assert state.shape == (Nseq, H, dk, dv)
+    o = np.empty((Nseq, H, dv), dtype=np.float64)
+    rc = lib.ddts_ref_step(ingate, Nseq, H, dk, dv, float(scale), qp, kp, xp, yp, vp,
+                           _f64p(o), _f64p(state))
+    if rc:
+        raise ValueError(f"ddts_ref_step returned {rc}")
+    return o
+
+
+# ----------------------------------------------------------------------------------------------
+# Other forms of the same quantity, written from other equations (pins for the recurrence above).
+# ----------------------------------------------------------------------------------------------
+
+def _gates_np(x, y, ingate):
+    x = np.asarray(x, dtype=np.float64)
+    y = np.asarray(y, dtype=np.float64)
+    g = np.logaddexp(0.0, x)
+    tau = 1.0 / (1.0 + np.exp(-y))
+    log_alpha = -g * tau
+    if ingate == POW_G:
+        ahat = np.power(g, tau)
+    else:
+        ahat = np.power(-np.expm1(-g), tau)
+    return log_alpha, ahat
+
+
+def parallel_form(q, k, x, y, v, scale: float = 1.0, ingate: int = POW_G):
+    """O = ((Q . A)(K / A . ahat)^T . M) V for ONE sequence and head, zero initial state.
+
+    Eq. "rodimus_parallel_form": A_t is the cumulative product of alpha up to t and M the
+    causal mask with the diagonal kept.  The quotient A_t / A_i is formed per pair as the
+    exponential of a difference of prefix sums of log(alpha), never as a division.
+    q,k,x,y: [T,dk]; v: [T,dv]; returns [T,dv] float64.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    log_alpha, ahat = _gates_np(x, y, ingate)
+    cum = np.cumsum(log_alpha, axis=0)                      # log A_t, [T,dk]
+    T = q.shape[0]
+    # scores[t,i] = sum_d q[t,d] * k[i,d] * ahat[i,d] * exp(cum[t,d] - cum[i,d])
+    diff = cum[:, None, :] - cum[None, :, :]                 # [T,T,dk]
+    mask = np.tril(np.ones((T, T), dtype=bool))
+    w = np.where(mask[:, :, None], np.exp(np.where(mask[:, :, None], diff, 0.0)), 0.0)
+    scores = np.einsum("td,id,tid->ti", q, k * ahat, w)
+    return scale * (scores @ v)
+
+
+def unrolled_sum(q, k, x, y, v, scale: float = 1.0, ingate: int = POW_G):
+    """o_t = sum_{i<=t} [q_t (prod_{j=i+1..t} alpha_j . ahat_i . k_i)^T] v_i, by explicit loops.
+
+    Sec. 3.1.1, with beta = 1 and no value gate.  Pure Python loops: tiny inputs only.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    log_alpha, ahat = _gates_np(x, y, ingate)
+    alpha = np.exp(log_alpha)
+    T, dk = q.shape
+    o = np.zeros((T, v.shape[1]), dtype=np.float64)
+    for t in range(T):
+        for i in range(t + 1):
+            prod = np.ones(dk)
+            for j in range(i + 1, t + 1):
+                prod = prod * alpha[j]
+            o[t] += float(np.dot(q[t], prod * ahat[i] * k[i])) * v[i]
+    return scale * o

@@ -1,0 +1,203 @@
+/*
+ * ddts_ref.c -- fp64 CPU oracle for the DDTS linear-attention recurrence.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
+ * CUDA library is checked against.  It shares no code with the CUDA path and
+ * must never be called from it; only the tests, the smoke check and the
+ * benchmark's CPU-baseline leg load it.
+ *
+ * What it computes (Rodimus paper, Eq. "alpha_def" of Sec. 3.1.2 and
+ * Eq. "rodimus_recurrent_form" of Sec. 3.1.3, with the value-side decay
+ * beta_t = 1 as Sec. 3.1.1 chooses, and without the value gate and the
+ * feed-through term, which the caller applies outside this path):
+ *
+ *   g_t     = softplus(x_t)                    selection gate,   per key channel
+ *   tau_t   = sigmoid(y_t)                     temperature gate, per key channel
+ *   alpha_t = exp(-g_t * tau_t)                decay
+ *   ahat_t  = g_t ^ tau_t                      input weight (paper, mode 0)
+ *           = (1 - exp(-g_t)) ^ tau_t          input weight (alternate, mode 1)
+ *   S_t[d,:] = alpha_t[d] * S_{t-1}[d,:] + (ahat_t[d] * k_t[d]) * v_t[:]
+ *   o_t[:]   = scale * sum_d q_t[d] * S_t[d,:]          (state AFTER the update)
+ *
+ * Strictly sequential in t, no chunking, no reordering: one loop per symbol of
+ * the equations.  Inputs arrive as float (the caller has already rounded them to
+ * the dtype the GPU sees, so input rounding is not counted as error) and are
+ * promoted to double before any arithmetic.  Outputs and states are double.
+ *
+ * Parity pins (tests, CPU only): equality with the O(T^2) masked parallel form
+ * (App. "Chunkwise Parallel Representation", Eq. "rodimus_parallel_form") and with
+ * the unrolled double sum of Sec. 3.1.1, reduction to unnormalised causal linear
+ * attention when alpha = ahat = 1, a geometric-series closed form, T = 1 by hand,
+ * the gate identities of Sec. 3.1.2 and the derivative product of the
+ * selection-mechanism proof, linearity, prefill == repeated steps == split runs.
+ * The choice between the two input-weight modes cannot be pinned by a printed
+ * value (the paper prints no worked example): for that choice alone, "parity
+ * unpinned"; both modes are implemented and each is pinned by every other test.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { DDTS_REF_POW_G = 0, DDTS_REF_POW_SIGMOID = 1 };
+
+/* softplus(x) = log(1 + e^x), written so that neither branch overflows. */
+static double ref_softplus(double x) {
+  return x > 0.0 ? x + log1p(exp(-x)) : log1p(exp(x));
+}
+
+/* sigmoid(y) = 1 / (1 + e^-y). */
+static double ref_sigmoid(double y) {
+  if (y >= 0.0) return 1.0 / (1.0 + exp(-y));
+  double e = exp(y);
+  return e / (1.0 + e);
+}
+
+/* Eq. "alpha_def": one key channel of one token. */
+static void ref_gate(int ingate, double x, double y, double *alpha, double *ahat) {
+  double g = ref_softplus(x);
+  double tau = ref_sigmoid(y);
+  *alpha = exp(-g * tau);
+  if (ingate == DDTS_REF_POW_G) {
+    *ahat = pow(g, tau);
+  } else {
+    *ahat = pow(-expm1(-g), tau); /* 1 - exp(-g) */
+  }
+}
+
+/* Gates of n (token, channel) pairs; exported so that tests can pin them alone. */
+int ddts_ref_gates(int ingate, int64_t n, const float *x, const float *y, double *alpha,
+                   double *ahat) {
+  if (ingate != DDTS_REF_POW_G && ingate != DDTS_REF_POW_SIGMOID) return 3;
+  for (int64_t i = 0; i < n; ++i) ref_gate(ingate, (double)x[i], (double)y[i], &alpha[i], &ahat[i]);
+  return 0;
+}
+
+/* One sequence, one head: rows [0,len) of q,k,x,y (row stride dk) and v,o (row stride dv). */
+static void ref_one_sequence(int ingate, int64_t len, int dk, int dv, double scale, const float *q,
+                             const float *k, const float *x, const float *y, const float *v,
+                             const double *s0, double *o, double *sT, double *S) {
+  if (s0)
+    memcpy(S, s0, sizeof(double) * (size_t)dk * dv);
+  else
+    memset(S, 0, sizeof(double) * (size_t)dk * dv);
+  for (int64_t t = 0; t < len; ++t) {
+    const float *qt = q + t * dk, *kt = k + t * dk, *xt = x + t * dk, *yt = y + t * dk;
+    const float *vt = v + t * dv;
+    double *ot = o ? o + t * dv : NULL;
+    if (ot)
+      for (int j = 0; j < dv; ++j) ot[j] = 0.0;
+    for (int d = 0; d < dk; ++d) {
+      double alpha, ahat;
+      ref_gate(ingate, (double)xt[d], (double)yt[d], &alpha, &ahat);
+      double w = ahat * (double)kt[d];
+      double *Sd = S + (size_t)d * dv;
+      for (int j = 0; j < dv; ++j) Sd[j] = alpha * Sd[j] + w * (double)vt[j];
+      if (ot) {
+        double qd = (double)qt[d];
+        for (int j = 0; j < dv; ++j) ot[j] += qd * Sd[j];
+      }
+    }
+    if (ot)
+      for (int j = 0; j < dv; ++j) ot[j] *= scale;
+  }
+  if (sT) memcpy(sT, S, sizeof(double) * (size_t)dk * dv);
+}
+
+/*
+ * Prefill.  Dense: q,k,x,y are [B,H,T,dk], v,o are [B,H,T,dv], s0/sT are
+ * [B,H,dk,dv] (either may be NULL: zero initial state / final state not wanted).
+ * Varlen (cu_seqlens != NULL): B must be 1, the N sequences are packed along T,
+ * sequence n owns rows cu_seqlens[n] .. cu_seqlens[n+1]-1 of every head, and
+ * s0/sT are [N,H,dk,dv].  o may be NULL (state only).  Returns 0, or a nonzero
+ * code for arguments that make no sense.
+ */
+int ddts_ref_fwd(int ingate, int B, int H, int64_t T, int dk, int dv, double scale, const float *q,
+                 const float *k, const float *x, const float *y, const float *v, const double *s0,
+                 double *o, double *sT, const int32_t *cu_seqlens, int N) {
+  if (ingate != DDTS_REF_POW_G && ingate != DDTS_REF_POW_SIGMOID) return 3;
+  if (B < 0 || H < 0 || T < 0 || dk <= 0 || dv <= 0) return 2;
+  int nseq = B;
+  if (cu_seqlens) {
+    if (B != 1 || N < 0) return 2;
+    if (cu_seqlens[0] != 0 || cu_seqlens[N] != T) return 5;
+    for (int n = 0; n < N; ++n)
+      if (cu_seqlens[n + 1] < cu_seqlens[n]) return 5;
+    nseq = N;
+  }
+  int64_t items = (int64_t)nseq * H;
+  int failed = 0;
+#pragma omp parallel
+  {
+    double *S = (double *)malloc(sizeof(double) * (size_t)dk * dv);
+    if (!S) {
+#pragma omp atomic write
+      failed = 1;
+    }
+#pragma omp for schedule(dynamic, 1)
+    for (int64_t it = 0; it < items; ++it) {
+      if (!S) continue;
+      int64_t n = it / H, h = it % H;
+      int64_t row0, len;
+      if (cu_seqlens) {
+        row0 = h * T + cu_seqlens[n];
+        len = cu_seqlens[n + 1] - cu_seqlens[n];
+      } else {
+        row0 = (n * H + h) * T;
+        len = T;
+      }
+      size_t so = (size_t)it * dk * dv;
+      ref_one_sequence(ingate, len, dk, dv, scale, q + row0 * dk, k + row0 * dk, x + row0 * dk,
+                       y + row0 * dk, v + row0 * dv, s0 ? s0 + so : NULL, o ? o + row0 * dv : NULL,
+                       sT ? sT + so : NULL, S);
+    }
+    free(S);
+  }
+  return failed ? 8 : 0;
+}
+
+/*
+ * One decode step for Nseq independent sequences: q,k,x,y are [Nseq,H,dk], v,o are
+ * [Nseq,H,dv], state is [Nseq,H,dk,dv] and is updated in place; o reads the state
+ * after the update (Eq. "rodimus_recurrent_form": o_t = q_t S_t).
+ */
+int ddts_ref_step(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
+                  const float *k, const float *x, const float *y, const float *v, double *o,
+                  double *state) {
+  if (ingate != DDTS_REF_POW_G && ingate != DDTS_REF_POW_SIGMOID) return 3;
+  if (Nseq < 0 || H < 0 || dk <= 0 || dv <= 0) return 2;
+  int64_t items = (int64_t)Nseq * H;
+#pragma omp parallel for schedule(static)
+  for (int64_t it = 0; it < items; ++it) {
+    const float *qt = q + it * dk, *kt = k + it * dk, *xt = x + it * dk, *yt = y + it * dk;
+    const float *vt = v + it * dv;
+    double *ot = o + it * dv;
+    double *S = state + (size_t)it * dk * dv;
+    for (int j = 0; j < dv; ++j) ot[j] = 0.0;
+    for (int d = 0; d < dk; ++d) {
+      double alpha, ahat;
+      ref_gate(ingate, (double)xt[d], (double)yt[d], &alpha, &ahat);
+      double w = ahat * (double)kt[d];
+      double qd = (double)qt[d];
+      double *Sd = S + (size_t)d * dv;
+      for (int j = 0; j < dv; ++j) {
+        Sd[j] = alpha * Sd[j] + w * (double)vt[j];
+        ot[j] += qd * Sd[j];
+      }
+    }
+    for (int j = 0; j < dv; ++j) ot[j] *= scale;
+  }
+  return 0;
+}
+
+/* Threads the parallel regions above will use (1 without OpenMP). */
+int ddts_ref_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}

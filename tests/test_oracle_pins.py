@@ -1,0 +1,273 @@
+"""Pins for the fp64 CPU oracle: every check compares the sequential recurrence with
+something the paper or plain mathematics fixes, never with the oracle itself.  CPU only.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import ddts_oracle as orc
+
+MODES = [orc.POW_G, orc.POW_SIGMOID]
+
+
+def _draw(seed, T, dk, dv, gate_mean=-1.0):
+    rng = np.random.default_rng(seed)
+    q = rng.standard_normal((T, dk)).astype(np.float32)
+    k = rng.standard_normal((T, dk)).astype(np.float32)
+    v = rng.standard_normal((T, dv)).astype(np.float32)
+    x = (rng.standard_normal((T, dk)) + gate_mean).astype(np.float32)
+    y = rng.standard_normal((T, dk)).astype(np.float32)
+    return q, k, x, y, v
+
+
+def _fwd1(q, k, x, y, v, s0=None, **kw):
+    """One sequence, one head through the C recurrence."""
+    s = None if s0 is None else s0[None, None]
+    o, sT = orc.ref_fwd(q[None, None], k[None, None], x[None, None], y[None, None], v[None, None],
+                        s0=s, **kw)
+    return o[0, 0], sT[0, 0]
+
+
+def _rel(a, b):
+    return np.max(np.abs(a - b)) / max(np.max(np.abs(b)), 1e-300)
+
+
+# -- golden: hand-derived closed forms -------------------------------------------------------
+
+def _golden_rows():
+    path = os.path.join(os.path.dirname(__file__), "golden", "ddts_hand_example.txt")
+    rows = []
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = line.split()
+        rows.append((int(f[0]),) + tuple(float(t) for t in f[1:]))
+    return rows
+
+
+@pytest.mark.parametrize("row", _golden_rows())
+def test_hand_example(row):
+    mode, alpha, ahat, o1, o2 = row
+    z = np.zeros((2, 1), dtype=np.float32)
+    one = np.ones((2, 1), dtype=np.float32)
+    a, ah = orc.ref_gates(z, z, mode)
+    assert abs(a[0, 0] - alpha) < 1e-15 and abs(ah[0, 0] - ahat) < 1e-15
+    o, sT = _fwd1(one, one, z, z, one, ingate=mode)
+    assert abs(o[0, 0] - o1) < 1e-15 and abs(o[1, 0] - o2) < 4e-16 * 4
+    assert abs(sT[0, 0] - o2) < 4e-16 * 4
+
+
+# -- other forms of the same quantity --------------------------------------------------------
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("T,dk,dv", [(1, 4, 3), (17, 8, 5), (48, 16, 7)])
+def test_recurrence_equals_parallel_form(mode, T, dk, dv):
+    q, k, x, y, v = _draw(10 + T, T, dk, dv)
+    o, _ = _fwd1(q, k, x, y, v, ingate=mode, scale=0.7)
+    ref = orc.parallel_form(q, k, x, y, v, scale=0.7, ingate=mode)
+    assert _rel(o, ref) < 1e-12
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_recurrence_equals_unrolled_sum(mode):
+    q, k, x, y, v = _draw(3, 7, 5, 4, gate_mean=0.5)
+    o, _ = _fwd1(q, k, x, y, v, ingate=mode)
+    ref = orc.unrolled_sum(q, k, x, y, v, ingate=mode)
+    assert _rel(o, ref) < 1e-12
+
+
+def test_parallel_form_is_causal():
+    # a future token must not change earlier outputs (mask keeps i <= t only)
+    q, k, x, y, v = _draw(5, 12, 6, 4)
+    o1, _ = _fwd1(q, k, x, y, v)
+    v2 = v.copy()
+    v2[8:] += 100.0
+    k2 = k.copy()
+    k2[8:] *= -3.0
+    o2, _ = _fwd1(q, k2, x, y, v2)
+    assert np.array_equal(o1[:8], o2[:8]) and not np.allclose(o1[8:], o2[8:])
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_reduces_to_causal_linear_attention(mode):
+    # tau -> 0 gives alpha = 1 and ahat = 1: S_t = S_{t-1} + k_t^T v_t, o_t = q_t S_t
+    T, dk, dv = 33, 8, 6
+    q, k, x, y, v = _draw(7, T, dk, dv)
+    y = np.full_like(y, -100.0)
+    o, sT = _fwd1(q, k, x, y, v, ingate=mode)
+    q64, k64, v64 = (a.astype(np.float64) for a in (q, k, v))
+    ref = np.tril(q64 @ k64.T) @ v64
+    assert _rel(o, ref) < 1e-12
+    assert _rel(sT, k64.T @ v64) < 1e-12
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_geometric_closed_form(mode):
+    # constant x,y,k,v: S_t[d,:] = ahat_d k_d v (1 - alpha_d^t) / (1 - alpha_d)
+    T, dk, dv = 40, 5, 3
+    rng = np.random.default_rng(11)
+    x1 = rng.standard_normal(dk).astype(np.float32)
+    y1 = rng.standard_normal(dk).astype(np.float32)
+    k1 = rng.standard_normal(dk).astype(np.float32)
+    v1 = rng.standard_normal(dv).astype(np.float32)
+    q = rng.standard_normal((T, dk)).astype(np.float32)
+    til = lambda a: np.tile(a, (T, 1))
+    o, sT = _fwd1(q, til(k1), til(x1), til(y1), til(v1), ingate=mode)
+    g = np.log1p(np.exp(x1.astype(np.float64)))
+    tau = 1 / (1 + np.exp(-y1.astype(np.float64)))
+    alpha = np.exp(-g * tau)
+    ahat = g ** tau if mode == orc.POW_G else (1 - np.exp(-g)) ** tau
+    for t in (1, 2, T):
+        S = (ahat * k1 * (1 - alpha ** t) / (1 - alpha))[:, None] * v1[None, :].astype(np.float64)
+        assert _rel(o[t - 1], q[t - 1].astype(np.float64) @ S) < 1e-12
+    assert _rel(sT, S) < 1e-12
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_single_token_by_hand(mode):
+    # o_1 = (q . alpha) S_0 + (q . (ahat . k)) v : the diagonal term is included
+    dk, dv = 6, 4
+    q, k, x, y, v = _draw(13, 1, dk, dv)
+    s0 = np.random.default_rng(14).standard_normal((dk, dv))
+    o, sT = _fwd1(q, k, x, y, v, s0=s0, ingate=mode, scale=2.0)
+    alpha, ahat = orc.ref_gates(x, y, mode)
+    S1 = alpha[0][:, None] * s0 + (ahat[0] * k[0])[:, None] * v[0][None, :].astype(np.float64)
+    assert _rel(sT, S1) < 1e-14
+    assert _rel(o[0], 2.0 * (q[0].astype(np.float64) @ S1)) < 1e-14
+    # and the state-only part really is weighted by alpha, not by 1
+    assert not np.allclose(S1, s0 + (ahat[0] * k[0])[:, None] * v[0][None, :])
+
+
+# -- gate functions ---------------------------------------------------------------------------
+
+def test_gate_identities():
+    x = np.linspace(-20, 20, 161).astype(np.float32)
+    big = np.full_like(x, 60.0)           # tau = 1 to fp64 precision
+    alpha, ahat = orc.ref_gates(x, big, orc.POW_G)
+    sig = 1 / (1 + np.exp(-x.astype(np.float64)))
+    # exp(-g) = 1 - sigmoid(x) = 1 / (1 + e^x)   (second form avoids cancellation in the test)
+    one_minus_sig = 1 / (1 + np.exp(x.astype(np.float64)))
+    assert np.max(np.abs(alpha - one_minus_sig) / one_minus_sig) < 1e-12
+    assert np.max(np.abs(alpha - (1 - sig))) < 1e-15
+    # at tau = 1: ahat = g (paper) and ahat = sigmoid(x) (alternate)
+    assert np.max(np.abs(ahat / np.logaddexp(0, x.astype(np.float64)) - 1)) < 1e-12
+    _, ahat1 = orc.ref_gates(x, big, orc.POW_SIGMOID)
+    assert np.max(np.abs(ahat1 / sig - 1)) < 1e-12
+    # ranges: 0 < alpha <= 1 always; the paper's ahat exceeds 1 for large gates, the alternate never
+    y = np.linspace(-6, 6, 161).astype(np.float32)
+    X, Y = np.meshgrid(x, y)
+    a, ah = orc.ref_gates(X, Y, orc.POW_G)
+    assert np.all(a > 0) and np.all(a <= 1)
+    assert ah.max() > 1.0
+    _, ah1 = orc.ref_gates(X, Y, orc.POW_SIGMOID)
+    assert np.all(ah1 <= 1.0) and np.all(ah1 > 0)
+
+
+def test_temperature_flattens_both_gates():
+    # smaller tau => alpha and ahat vary more slowly with the gate pre-activation
+    x = np.array([-2.0, -1.0], dtype=np.float32)
+    spans = []
+    for yv in (3.0, 0.0, -3.0):           # tau decreasing
+        a, ah = orc.ref_gates(x, np.full_like(x, yv), orc.POW_G)
+        spans.append((abs(a[1] - a[0]), abs(np.log(ah[1]) - np.log(ah[0]))))
+    assert spans[0][0] > spans[1][0] > spans[2][0]
+    assert spans[0][1] > spans[1][1] > spans[2][1]
+
+
+def test_selection_derivative_product():
+    # proof of the selection property: d(exp(-g))/d(eta) * d(g)/d(eta) = -sigma^2 (1 - sigma), tau = 1
+    h = 2.0 ** -9
+    for eta in (-2.0, -0.5, 0.0, 0.75, 3.0):
+        xs = np.array([eta - h, eta + h], dtype=np.float32)
+        a, ah = orc.ref_gates(xs, np.full_like(xs, 60.0), orc.POW_G)
+        dA = (a[1] - a[0]) / (2 * h)
+        dB = (ah[1] - ah[0]) / (2 * h)
+        s = 1 / (1 + np.exp(-eta))
+        assert dA < 0 < dB
+        assert abs(dA * dB - (-(s ** 2) * (1 - s))) < 2e-5
+
+
+# -- structure of the recurrence --------------------------------------------------------------
+
+def test_linearity_in_v_s0_and_q():
+    T, dk, dv = 19, 6, 5
+    q, k, x, y, v = _draw(21, T, dk, dv)
+    rng = np.random.default_rng(22)
+    v2 = rng.standard_normal((T, dv)).astype(np.float32)
+    s0a = rng.standard_normal((dk, dv))
+    s0b = rng.standard_normal((dk, dv))
+    oa, sa = _fwd1(q, k, x, y, v, s0=s0a)
+    ob, sb = _fwd1(q, k, x, y, v2, s0=s0b)
+    # quantise both value tensors to multiples of 1/64 so that their float32 sum is exact
+    v = (np.round(v * 64) / 64).astype(np.float32)
+    v2 = (np.round(v2 * 64) / 64).astype(np.float32)
+    oa, sa = _fwd1(q, k, x, y, v, s0=s0a)
+    ob, sb = _fwd1(q, k, x, y, v2, s0=s0b)
+    o_v, s_v = _fwd1(q, k, x, y, (v + v2).astype(np.float32), s0=s0a + s0b)
+    assert _rel(o_v, oa + ob) < 1e-12 and _rel(s_v, sa + sb) < 1e-12
+    o3, _ = _fwd1((2 * q).astype(np.float32), k, x, y, v, s0=s0a)
+    assert _rel(o3, 2 * oa) < 1e-14
+    assert oa.shape == ob.shape and sa.shape == sb.shape
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_prefill_equals_steps_equals_split_runs(mode):
+    B, H, T, dk, dv = 2, 3, 29, 8, 6
+    rng = np.random.default_rng(31)
+    q = rng.standard_normal((B, H, T, dk)).astype(np.float32)
+    k = rng.standard_normal((B, H, T, dk)).astype(np.float32)
+    v = rng.standard_normal((B, H, T, dv)).astype(np.float32)
+    x = (rng.standard_normal((B, H, T, dk)) - 1).astype(np.float32)
+    y = rng.standard_normal((B, H, T, dk)).astype(np.float32)
+    s0 = rng.standard_normal((B, H, dk, dv))
+    o, sT = orc.ref_fwd(q, k, x, y, v, s0=s0, ingate=mode, scale=0.5)
+    # repeated decode steps
+    st = s0.copy()
+    for t in range(T):
+        ot = orc.ref_step(q[:, :, t], k[:, :, t], x[:, :, t], y[:, :, t], v[:, :, t], st,
+                          scale=0.5, ingate=mode)
+        assert _rel(ot, o[:, :, t]) < 1e-13
+    assert _rel(st, sT) < 1e-13
+    # two runs passing the state across the split
+    cut = 11
+    sl = lambda a, lo, hi: np.ascontiguousarray(a[:, :, lo:hi])
+    o1, s1 = orc.ref_fwd(sl(q, 0, cut), sl(k, 0, cut), sl(x, 0, cut), sl(y, 0, cut), sl(v, 0, cut),
+                         s0=s0, ingate=mode, scale=0.5)
+    o2, s2 = orc.ref_fwd(sl(q, cut, T), sl(k, cut, T), sl(x, cut, T), sl(y, cut, T), sl(v, cut, T),
+                         s0=s1, ingate=mode, scale=0.5)
+    assert _rel(np.concatenate([o1, o2], axis=2), o) < 1e-13 and _rel(s2, sT) < 1e-13
+
+
+def test_varlen_equals_one_by_one():
+    H, dk, dv = 2, 6, 5
+    lens = [5, 0, 13, 1, 8]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    T = int(cu[-1])
+    rng = np.random.default_rng(41)
+    q = rng.standard_normal((1, H, T, dk)).astype(np.float32)
+    k = rng.standard_normal((1, H, T, dk)).astype(np.float32)
+    v = rng.standard_normal((1, H, T, dv)).astype(np.float32)
+    x = (rng.standard_normal((1, H, T, dk)) - 1).astype(np.float32)
+    y = rng.standard_normal((1, H, T, dk)).astype(np.float32)
+    s0 = rng.standard_normal((len(lens), H, dk, dv))
+    o, sT = orc.ref_fwd(q, k, x, y, v, s0=s0, cu_seqlens=cu)
+    for n, L in enumerate(lens):
+        lo, hi = cu[n], cu[n + 1]
+        sl = lambda a: np.ascontiguousarray(a[:, :, lo:hi])
+        on, sn = orc.ref_fwd(sl(q), sl(k), sl(x), sl(y), sl(v), s0=s0[n:n + 1])
+        assert np.array_equal(on, o[:, :, lo:hi]) and np.array_equal(sn[0], sT[n])
+    # an empty sequence returns its initial state untouched
+    assert np.array_equal(sT[1], s0[1])
+    with pytest.raises(ValueError):
+        orc.ref_fwd(q, k, x, y, v, cu_seqlens=np.array([0, 9, 5, T], dtype=np.int32))
+
+
+def test_strong_decay_and_long_memory_stay_finite():
+    T, dk, dv = 64, 4, 3
+    q, k, x, y, v = _draw(51, T, dk, dv)
+    for xv, yv in ((8.0, 8.0), (-12.0, 0.0), (80.0, 80.0), (-80.0, -80.0)):
+        o, sT = _fwd1(q, k, np.full_like(x, xv), np.full_like(y, yv), v)
+        assert np.all(np.isfinite(o)) and np.all(np.isfinite(sT))
+        ref = orc.parallel_form(q, k, np.full_like(x, xv), np.full_like(y, yv), v)
+        assert _rel(o, ref) < 1e-12
