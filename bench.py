@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the DDTS hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1|cfg2|cfg4|cfg3]
+                    [--impl ours|reference]
+
+One "step" is one pass of the whole path over one batch of seeded synthetic input:
+for the prefill workloads one ``rodimus_ddts_fwd`` call (gates, in-chunk cumulative decay,
+intra-chunk scores and outputs, inter-chunk readout, state update, output and final-state
+stores); for ``cfg3`` one ``rodimus_ddts_step`` call over all sequences.  Prints ONE JSON line.
+
+With N > 1 (launched by ``torch.distributed.run``) every rank runs its own replica of the
+workload on its own GPU (independent batches: no collective on the data path) and the value
+is all ranks' tokens over the slowest rank's device time.
+
+``--impl reference`` times the fp64 CPU oracle, as it stands, on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+WORKLOADS = {"cfg1": 1, "cfg2": 2, "cfg3": 3, "cfg4": 4}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"])}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def load_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch from the committed ncu summary, if one covers this kernel/workload."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        d = json.load(f)
+    ent = d.get(f"{kernel}:{workload}")
+    return None if ent is None else ent.get("bytes_per_launch")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.samples = []
+        self.stop = threading.Event()
+        self.thread = threading.Thread(target=self._run, daemon=True)
+
+    def _once(self):
+        try:
+            out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                  "-i", str(self.idx)], capture_output=True, text=True, timeout=10).stdout
+            f = [t.strip() for t in out.strip().split(",")]
+            if len(f) >= 6:
+                self.samples.append((float(f[0]), float(f[1]), f[2:6]))
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self.stop.is_set():
+            self._once()
+            self.stop.wait(0.05)
+
+    def __enter__(self):
+        self.thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self.stop.set()
+        self.thread.join(timeout=15)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for s in self.samples for n, v in zip(names, s[2]) if v.lower().startswith("active")})
+        return {"sm_mhz": float(np.median([s[0] for s in self.samples])),
+                "sm_max_mhz": float(self.samples[0][1]), "reasons": reasons,
+                "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------------------------
+# workload description shared by both arms
+# ----------------------------------------------------------------------------------------------
+
+def describe(workload: str, p, n_gpus: int):
+    if workload == "cfg3":
+        Nseq, H, dk, dv = p.state.shape
+        return {"workload": "cfg3_decode: 256 sequences x 16 heads, one token each, fp32 state in place",
+                "Nseq_per_gpu": Nseq, "H": H, "dk": dk, "dv": dv, "ingate": "g^tau",
+                "replicas": n_gpus, "l2": "state (1.07 GB) larger than L2"}
+    B, H, T, dk, dv = p.shape
+    names = {"cfg1": "cfg1_layer_prefill: B=4 H=16 T=2048 dk=128 dv=256 bf16, zero initial state",
+             "cfg2": "cfg2_long_context: B=1 H=16 T=32768 dk=128 dv=256 bf16, nonzero initial state",
+             "cfg4": "cfg4_varlen: 64 packed sequences, lengths U[128,4096], H=16 dk=128 dv=256 bf16"}
+    return {"workload": names[workload], "B_per_gpu": B, "H": H, "T": T, "dk": dk, "dv": dv,
+            "tokens_per_gpu": p.tokens, "ingate": "g^tau", "replicas": n_gpus,
+            "l2": "inputs larger than L2, no flush"}
+
+
+def prefill_bytes(p) -> int:
+    """Algorithmic HBM bytes of one prefill call: q,k,x,y,v read, o written, states read/written."""
+    B, H, T, dk, dv = p.shape
+    el = 2 if p.dtype == "bf16" else 4
+    nseq = B if p.cu_seqlens is None else len(p.cu_seqlens) - 1
+    tok = B * H * T * (4 * dk + 2 * dv) * el
+    st = nseq * H * dk * dv * 4
+    return tok + st * (2 if p.s0 is not None else 1)
+
+
+def decode_bytes(p) -> int:
+    Nseq, H, dk, dv = p.state.shape
+    return Nseq * H * (2 * dk * dv * 4 + (4 * dk + 2 * dv) * 2)
+
+
+# ----------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle
+# ----------------------------------------------------------------------------------------------
+
+def oracle_sample_run(workload: str, p, budget_s: float = 10.0):
+    """Times the oracle on a bounded sample of the workload; returns (units, seconds, what)."""
+    from oracle import ddts_oracle as orc
+    if workload == "cfg3":
+        Nseq = min(p.state.shape[0], 64)
+        st = np.ascontiguousarray(p.state[:Nseq]).astype(np.float64)
+        sl = lambda a: np.ascontiguousarray(a[0][:Nseq])
+        args = [sl(a) for a in (p.q, p.k, p.x, p.y, p.v)]
+        t0 = time.perf_counter()
+        steps = 0
+        while steps < 64 and (time.perf_counter() - t0 < budget_s or steps < 2):
+            orc.ref_step(*args, st)
+            steps += 1
+        dt = time.perf_counter() - t0
+        per_seq = decode_bytes(p) / p.state.shape[0]
+        return per_seq * Nseq * steps, dt, f"{steps} steps over the first {Nseq} of {p.state.shape[0]} sequences"
+    B, H, T, dk, dv = p.shape
+    if p.cu_seqlens is not None:
+        heads = min(H, 2)
+        sl = lambda a: np.ascontiguousarray(a[:, :heads])
+        t0 = time.perf_counter()
+        orc.ref_fwd(sl(p.q), sl(p.k), sl(p.x), sl(p.y), sl(p.v), cu_seqlens=p.cu_seqlens, want_o=True)
+        dt = time.perf_counter() - t0
+        return p.tokens * heads / H, dt, f"{heads} of {H} heads of all {len(p.cu_seqlens) - 1} sequences"
+    heads = H if B * H * T <= 4 * 16 * 2048 else max(1, (4 * 16 * 2048) // (B * T))
+    sl = lambda a: np.ascontiguousarray(a[:, :heads])
+    s0 = None if p.s0 is None else sl(p.s0).astype(np.float64)
+    args = [sl(a) for a in (p.q, p.k, p.x, p.y, p.v)]
+    t0 = time.perf_counter()
+    reps = 0
+    while reps < 8 and (time.perf_counter() - t0 < budget_s or reps < 1):
+        orc.ref_fwd(*args, s0=s0)
+        reps += 1
+    dt = time.perf_counter() - t0
+    return p.tokens * heads / H * reps, dt, f"{reps} pass(es) over {heads} of {H} heads, all {B * T} tokens"
+
+
+def run_reference(args, workload, p):
+    from oracle import ddts_oracle as orc
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = orc.num_threads()
+    for _ in range(args.warmup):
+        oracle_sample_run(workload, p, budget_s=0.0)
+    units = secs = 0.0
+    what = ""
+    for _ in range(args.steps):
+        u, s, what = oracle_sample_run(workload, p, budget_s=max(2.0, 60.0 / max(args.steps, 1)))
+        units += u
+        secs += s
+    decode = workload == "cfg3"
+    val = units / secs / (1e9 if decode else 1.0)
+    unit = "GB/s" if decode else "tokens/s"
+    line = {
+        "impl": "reference",
+        "metric": "DDTS decode state GB/s" if decode else "DDTS prefill tokens/s",
+        "value": val, "unit": unit, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * secs / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded)",
+        "config": describe(workload, p, args.gpus),
+        "cpu_baseline": {"value": val, "unit": unit, "cores": cores, "kind": "oracle",
+                         "sample": f"each step: {what}"},
+        "e2e": {"value": val, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------------
+
+def run_ours(args, workload, p):
+    import torch
+    import torch.distributed as dist
+    import paper_2410_06577_b200 as rd
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    peaks, peak_kind = load_peaks()
+    decode = workload == "cfg3"
+    tdt = torch.bfloat16 if p.dtype == "bf16" else torch.float32
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    if decode:
+        ring = p.q.shape[0]
+        host = {n: torch.from_numpy(getattr(p, n)).to(tdt).pin_memory() for n in ("q", "k", "x", "y", "v")}
+        devt = {n: host[n].to(device) for n in host}
+        state = torch.from_numpy(p.state).to(device)
+        Nseq, H, dk, dv = p.state.shape
+        o = torch.empty((Nseq, H, dv), dtype=tdt, device=device)
+        units_per_step = decode_bytes(p) / 1e9          # GB moved per step
+        alg_bytes = decode_bytes(p)
+        kernel = "ddts_step_kernel"
+
+        def step(i):
+            s = i % ring
+            rd.ddts_step(devt["q"][s], devt["k"][s], devt["x"][s], devt["y"][s], devt["v"][s], state, out=o)
+
+        o_host = torch.empty(o.shape, dtype=tdt).pin_memory()
+        h2d = sum(host[n][0].numel() * host[n].element_size() for n in host)
+        d2h = o_host.numel() * o_host.element_size()
+        stage = {n: torch.empty_like(devt[n][0]) for n in host}
+
+        def step_e2e(i):
+            s = i % ring
+            for n in host:
+                stage[n].copy_(host[n][s], non_blocking=True)
+            rd.ddts_step(stage["q"], stage["k"], stage["x"], stage["y"], stage["v"], state, out=o)
+            o_host.copy_(o, non_blocking=True)
+    else:
+        host = {n: torch.from_numpy(getattr(p, n)).to(tdt).pin_memory() for n in ("q", "k", "x", "y", "v")}
+        devt = {n: host[n].to(device) for n in host}
+        s0 = None if p.s0 is None else torch.from_numpy(p.s0).to(device)
+        cu = None if p.cu_seqlens is None else torch.from_numpy(p.cu_seqlens).to(device)
+        cu_host = None if p.cu_seqlens is None else torch.from_numpy(p.cu_seqlens)
+        B, H, T, dk, dv = p.shape
+        nseq = B if cu is None else cu.numel() - 1
+        o = torch.empty((B, H, T, dv), dtype=tdt, device=device)
+        sT = torch.empty((nseq, H, dk, dv), dtype=torch.float32, device=device)
+        prm = rd.fwd_params(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], o, s0, sT, cu, cu_host)
+        ws = rd.new_workspace(prm, device)
+        units_per_step = p.tokens
+        alg_bytes = prefill_bytes(p)
+        kernel = "ddts_fwd_" + rd.fwd_kernel_name(prm)
+
+        def step(i):
+            rd.ddts_fwd(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], s0, cu, cu_host,
+                        out=o, final_state=sT, workspace=ws)
+
+        o_host = torch.empty(o.shape, dtype=tdt).pin_memory()
+        sT_host = torch.empty(sT.shape, dtype=torch.float32).pin_memory()
+        stage = {n: torch.empty_like(devt[n]) for n in host}
+        h2d = sum(host[n].numel() * host[n].element_size() for n in host)
+        d2h = o_host.numel() * o_host.element_size() + sT_host.numel() * 4
+
+        def step_e2e(i):
+            for n in host:
+                stage[n].copy_(host[n], non_blocking=True)
+            rd.ddts_fwd(stage["q"], stage["k"], stage["x"], stage["y"], stage["v"], s0, cu, cu_host,
+                        out=o, final_state=sT, workspace=ws)
+            o_host.copy_(o, non_blocking=True)
+            sT_host.copy_(sT, non_blocking=True)
+
+    def timed(fn, steps, warmup):
+        for i in range(warmup):
+            fn(i)
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for i in range(steps):
+            fn(warmup + i)
+        ev1.record(stream)
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    step(0)
+    torch.cuda.synchronize()
+    launches_per_step = rd.last_launch_count()
+    with ClockSampler(local) as clk:
+        ms = timed(step, args.steps, args.warmup)
+    clocks = clk.summary()
+    if not decode:
+        st = rd.device_status(ws)
+        if st != rd.OK:
+            raise SystemExit(f"device status after the timed region: {st} ({rd.status_str(st)})")
+    e2e_steps = max(1, min(args.steps, 200 if decode else 5))
+    ms_e2e = timed(step_e2e, e2e_steps, 1)
+
+    sec = ms / 1e3
+    value = units_per_step * world * args.steps / sec
+    e2e_value = units_per_step * world * e2e_steps / (ms_e2e / 1e3)
+    kern_s = sec / args.steps
+    achieved = alg_bytes / kern_s / 1e9
+    line = {
+        "metric": "DDTS decode state GB/s" if decode else "DDTS prefill tokens/s",
+        "value": value, "unit": "GB/s" if decode else "tokens/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32" if decode else ("bf16" if p.dtype == "bf16" else "f32"),
+        "data": "synthetic (seeded)", "config": describe(workload, p, world),
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "GB/s" if decode else "tokens/s",
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
+        "gpu_launches": int(launches_per_step * args.steps),
+        "roofline": {"bound": "hbm", "kernel": kernel, "achieved": achieved,
+                     "peak": peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"],
+                     "algorithmic_bytes_per_launch": int(alg_bytes),
+                     "traffic": load_traffic(kernel, workload)},
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            from oracle import ddts_oracle as orc
+            u, s, what = oracle_sample_run(workload, p, budget_s=10.0)
+            line["cpu_baseline"] = {"value": u / s / (1e9 if decode else 1.0),
+                                    "unit": "GB/s" if decode else "tokens/s",
+                                    "cores": orc.num_threads(), "kind": "oracle", "sample": what}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg1")
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    decode = args.workload == "cfg3"
+    if args.steps is None:
+        args.steps = (1000 if decode else 50) if args.impl == "ours" else 3
+    if args.warmup is None:
+        args.warmup = (10 if decode else 5) if args.impl == "ours" else 1
+    if args.impl == "ours" and args.warmup < 3:
+        args.warmup = 3
+
+    from paper_2410_06577_b200 import workloads as wl
+    rank = int(os.environ.get("RANK", "0"))
+    if args.impl == "reference" and rank != 0:
+        return
+    p = wl.config(WORKLOADS[args.workload])
+    if args.impl == "reference":
+        run_reference(args, args.workload, p)
+    else:
+        run_ours(args, args.workload, p)
+
+
+if __name__ == "__main__":
+    main()

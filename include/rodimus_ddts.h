@@ -1,0 +1,152 @@
+/*
+ * rodimus_ddts.h -- C ABI of the B200 (sm_100a) DDTS linear-attention library.
+ *
+ * The library computes the data-dependent tempered selection (DDTS) recurrence of the
+ * Rodimus block (Rodimus paper, Sec. 3.1.2 Eq. "alpha_def" and Sec. 3.1.3
+ * Eq. "rodimus_recurrent_form", with the value-side decay beta_t = 1 of Sec. 3.1.1):
+ *
+ *   g_t = softplus(x_t)      tau_t = sigmoid(y_t)              per key channel
+ *   alpha_t = exp(-g_t * tau_t)                                 decay
+ *   ahat_t  = g_t ^ tau_t            (RODIMUS_INGATE_POW_G, the paper's Eq. "alpha_def")
+ *           = (1 - exp(-g_t)) ^ tau_t   (RODIMUS_INGATE_POW_SIGMOID, alternate reading)
+ *   S_t = diag(alpha_t) S_{t-1} + (ahat_t . k_t)^T v_t          S_t is [dk, dv], fp32
+ *   o_t = scale * q_t S_t                                       state AFTER the update
+ *
+ * The projections that produce q, k, v, x, y, the value gate and the feed-through term of
+ * the full block are the caller's; v arrives already gated.
+ *
+ * Conventions shared by every entry point
+ *   - All data pointers are DEVICE pointers unless a name ends in "_host".
+ *   - The caller owns every buffer, the workspace and the stream.  The library allocates no
+ *     device memory, keeps no state between calls and never synchronises the device, except
+ *     rodimus_ddts_device_status, which waits for the stream it is given.
+ *   - Calls enqueue work on `stream` and return; outputs are valid once the stream has
+ *     reached that point.
+ *   - Every function returns a rodimus_status.  Argument errors are found on the host before
+ *     anything is launched.  Nothing aborts, throws or traps.
+ *   - Tensors are contiguous, row-major, last index fastest; pointers are 16-byte aligned.
+ *   - Inputs must be finite, with |x|, |y| <= 80.  Per-step decay factors below exp(-64) are
+ *     applied as exp(-64) by the bf16 prefill kernel (difference below 2^-92 of the state).
+ */
+#ifndef RODIMUS_DDTS_H_
+#define RODIMUS_DDTS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RODIMUS_OK = 0,
+  RODIMUS_ERR_NULL = 1,        /* a required pointer is NULL                                  */
+  RODIMUS_ERR_SHAPE = 2,       /* a size is negative, zero where it may not be, or too large  */
+  RODIMUS_ERR_DTYPE = 3,       /* dtype / ingate / struct_size not understood                 */
+  RODIMUS_ERR_ALIGN = 4,       /* a pointer is not 16-byte aligned                            */
+  RODIMUS_ERR_SEQLENS = 5,     /* cu_seqlens does not start at 0, decreases, or ends != T     */
+  RODIMUS_ERR_WORKSPACE = 6,   /* workspace missing or smaller than ..._workspace_bytes       */
+  RODIMUS_ERR_UNSUPPORTED = 7, /* valid request that no kernel here covers                    */
+  RODIMUS_ERR_CUDA = 8,        /* a CUDA runtime or driver call failed                        */
+  RODIMUS_ERR_TIMEOUT = 9      /* a bounded wait inside a kernel ran out (device status only) */
+} rodimus_status;
+
+typedef enum { RODIMUS_BF16 = 0, RODIMUS_F32 = 1 } rodimus_dtype; /* of q,k,x,y,v,o alike */
+
+typedef enum {
+  RODIMUS_INGATE_POW_G = 0,      /* ahat = g^tau              (Eq. "alpha_def")            */
+  RODIMUS_INGATE_POW_SIGMOID = 1 /* ahat = (1-exp(-g))^tau    (alternate reading)          */
+} rodimus_ingate;
+
+/*
+ * Chunked prefill over whole sequences (appendix "Chunkwise Parallel Representation of the
+ * Rodimus Block": intra-chunk masked parallel form plus inter-chunk state recurrence; the
+ * chunk length is internal and does not change the result beyond rounding).
+ *
+ * Dense:  q,k,gate_x,temp_y are [B,H,T,dk]; v,o are [B,H,T,dv]; s0,sT are [B,H,dk,dv].
+ * Varlen: cu_seqlens != NULL, B must be 1, the N sequences are packed along T
+ *         (sequence n owns rows cu_seqlens[n] .. cu_seqlens[n+1]-1 of every head),
+ *         s0,sT are [N,H,dk,dv].  Sequences of length 0 are legal (sT = s0, or zeros).
+ * s0 == NULL means a zero initial state; sT == NULL means the final state is not wanted;
+ * s0 and sT may be the same buffer.  o must not overlap any input.
+ *
+ * Kernels: dtype BF16 with dk == 128 and dv a multiple of 128 runs on the tcgen05 tensor
+ * cores; every other legal shape (dk, dv multiples of 16, at most 256) and dtype F32 run
+ * the fp32 CUDA-core kernel, which keeps all arithmetic in fp32.
+ */
+typedef struct {
+  int32_t struct_size;       /* sizeof(rodimus_ddts_fwd_params), checked                        */
+  int32_t dtype;             /* rodimus_dtype                                                   */
+  int32_t ingate;            /* rodimus_ingate                                                  */
+  int32_t B, H, T, dk, dv;   /* varlen: B = 1 and T = cu_seqlens[N]; B*H*T < 2^31               */
+  float scale;               /* multiplies o; 1.0f when q is already divided by sqrt(dk)        */
+  int32_t N;                 /* number of sequences when cu_seqlens != NULL, else ignored       */
+  const void *q, *k;         /* device [B,H,T,dk]                                               */
+  const void *gate_x;        /* device [B,H,T,dk]: pre-activation of the selection gate g       */
+  const void *temp_y;        /* device [B,H,T,dk]: pre-activation of the temperature gate tau   */
+  const void *v;             /* device [B,H,T,dv]                                               */
+  void *o;                   /* device [B,H,T,dv], written                                      */
+  const float *s0;           /* device fp32 [B|N,H,dk,dv] or NULL                               */
+  float *sT;                 /* device fp32 [B|N,H,dk,dv] or NULL, written                      */
+  const int32_t *cu_seqlens; /* device int32 [N+1] or NULL                                      */
+  const int32_t *cu_seqlens_host; /* optional host copy of cu_seqlens: checked before launch.   */
+                             /* Without it the device checks the values and reports through     */
+                             /* rodimus_ddts_device_status; bad entries are clamped, never read */
+                             /* out of bounds.                                                  */
+  void *workspace;           /* device, >= rodimus_ddts_fwd_workspace_bytes(), 256-byte aligned */
+  size_t workspace_bytes;
+  void *stream;              /* cudaStream_t of the caller (NULL = default stream)              */
+} rodimus_ddts_fwd_params;
+
+/*
+ * One decode step for Nseq independent sequences (Eq. "rodimus_recurrent_form" applied once;
+ * Sec. 3.1.3, last paragraph: O(1) time and memory per token at inference).
+ * q,k,gate_x,temp_y are [Nseq,H,dk]; v,o are [Nseq,H,dv]; state is fp32 [Nseq,H,dk,dv],
+ * read and written in place; o reads the updated state.  dk and dv are multiples of 16 with
+ * dk <= 256 and dv <= 1024.  All arithmetic is fp32.
+ */
+typedef struct {
+  int32_t struct_size; /* sizeof(rodimus_ddts_step_params) */
+  int32_t dtype;       /* rodimus_dtype of q,k,gate_x,temp_y,v,o */
+  int32_t ingate;      /* rodimus_ingate */
+  int32_t Nseq, H, dk, dv;
+  float scale;
+  const void *q, *k, *gate_x, *temp_y; /* device [Nseq,H,dk] */
+  const void *v;                       /* device [Nseq,H,dv] */
+  void *o;                             /* device [Nseq,H,dv], written */
+  float *state;                        /* device fp32 [Nseq,H,dk,dv], updated in place */
+  void *stream;
+} rodimus_ddts_step_params;
+
+/* Bytes of device workspace rodimus_ddts_fwd needs for these sizes (pointers are not read).
+ * Returns 0 if the sizes are not valid. */
+size_t rodimus_ddts_fwd_workspace_bytes(const rodimus_ddts_fwd_params *p);
+
+/* Chunked prefill; see rodimus_ddts_fwd_params. */
+int rodimus_ddts_fwd(const rodimus_ddts_fwd_params *p);
+
+/* One-token decode; see rodimus_ddts_step_params. */
+int rodimus_ddts_step(const rodimus_ddts_step_params *p);
+
+/*
+ * Waits for `stream`, then returns what the kernels of the last rodimus_ddts_fwd call that
+ * used `workspace` recorded: RODIMUS_OK, RODIMUS_ERR_SEQLENS (device-side cu_seqlens check)
+ * or RODIMUS_ERR_TIMEOUT (a bounded wait ran out; outputs are then unspecified).
+ */
+int rodimus_ddts_device_status(const void *workspace, void *stream);
+
+/* How many kernels the last successful rodimus_ddts_fwd / rodimus_ddts_step call on this host
+ * thread launched (for benchmarks that report launch counts). */
+int rodimus_ddts_last_launch_count(void);
+
+/* Name of the kernel family the given prefill request would run: "tcgen05", "simt" or
+ * "invalid".  Pointers are not read. */
+const char *rodimus_ddts_fwd_kernel_name(const rodimus_ddts_fwd_params *p);
+
+const char *rodimus_status_str(int status);
+int rodimus_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RODIMUS_DDTS_H_ */

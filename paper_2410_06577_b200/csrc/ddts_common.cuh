@@ -1,0 +1,71 @@
+// Internal declarations shared by the translation units of the DDTS library (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rodimus_ddts.h"
+
+namespace ddts {
+
+// Device-visible words at the start of the caller's workspace.
+struct WorkspaceHeader {
+  int32_t status;        // rodimus_status recorded by kernels (0 = ok); only ever raised
+  int32_t work_counter;  // next work item for persistent kernels
+  int32_t n_items;       // reserved
+  int32_t pad[61];
+};
+static_assert(sizeof(WorkspaceHeader) == 256, "workspace header is 256 bytes");
+
+constexpr int kMaxSortedSeqs = 4096;  // varlen: sequences beyond this keep their given order
+
+// Launchers: all arguments validated by the caller; they return a cudaError_t.
+cudaError_t launch_step(const rodimus_ddts_step_params& p, int* n_launches);
+cudaError_t launch_plan(const rodimus_ddts_fwd_params& p, int* n_launches);
+cudaError_t launch_fwd_simt(const rodimus_ddts_fwd_params& p, int* n_launches);
+cudaError_t launch_fwd_tc(const rodimus_ddts_fwd_params& p, int* n_launches);
+bool fwd_tc_supported(const rodimus_ddts_fwd_params& p);
+bool tc_kernel_built();
+
+// ---------------------------------------------------------------------------------------------
+// Element access for the two token dtypes.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__device__ __forceinline__ float to_f32(T v);
+template <>
+__device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T>
+__device__ __forceinline__ T from_f32(float v);
+template <>
+__device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// ---------------------------------------------------------------------------------------------
+// Gate math in full fp32 precision (Eq. "alpha_def"): natural-log decay and natural-log input
+// weight for one key channel.  Used where accuracy matters more than issue slots (decode, fp32
+// prefill).  log_alpha = -softplus(x) * sigmoid(y) <= 0;  log_ahat = sigmoid(y) * log(g) for
+// the paper's form, sigmoid(y) * log(1 - exp(-g)) = -sigmoid(y) * softplus(-x) for the other.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float softplus_f32(float x) {
+  return x > 0.f ? x + log1pf(expf(-x)) : log1pf(expf(x));
+}
+
+__device__ __forceinline__ void gate_logs_f32(float x, float y, int ingate, float& log_alpha,
+                                              float& log_ahat) {
+  const float g = softplus_f32(x);
+  const float tau = y >= 0.f ? 1.f / (1.f + expf(-y)) : expf(y) / (1.f + expf(y));
+  log_alpha = -g * tau;
+  if (ingate == RODIMUS_INGATE_POW_G) {
+    // g > 0 for every finite x >= -87; log(g) -> x as x -> -inf
+    log_ahat = tau * logf(g);
+  } else {
+    log_ahat = -tau * softplus_f32(-x);
+  }
+}
+
+}  // namespace ddts

@@ -1,0 +1,151 @@
+// One-token decode: S <- diag(alpha) S + (ahat . k)^T v in place, o = scale * q S
+// (Eq. "rodimus_recurrent_form" applied once).  Pure HBM streaming: every fp32 state element
+// is read once and written once with 16-byte accesses; nothing else is comparable in size.
+//
+// Work item = (sequence, head, tile of 128 state columns).  A CTA of 4 warps walks the dk rows
+// of its tile: warp w owns rows w, w+4, ..., lane l owns columns 4l..4l+3, so each warp-wide
+// access is one 512-byte row segment.  Rows are processed in batches of kBatch per warp with
+// all loads of a batch in flight at once; the first batch is issued before the gate math so
+// that its latency hides the token loads and the transcendental work.
+#include "ddts_common.cuh"
+
+namespace ddts {
+namespace {
+
+constexpr int kStepThreads = 128;
+constexpr int kStepWarps = kStepThreads / 32;
+constexpr int kTileCols = 128;
+constexpr int kBatch = 8;
+constexpr int kMaxDk = 256;
+
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(float4* p, const float4& v) { __stcs(p, v); }
+
+template <typename T>
+__global__ void __launch_bounds__(kStepThreads, 8)
+ddts_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ gx,
+                 const T* __restrict__ ty, const T* __restrict__ v, T* __restrict__ o,
+                 float* __restrict__ state, int n_seq_heads, int dk, int dv, float scale,
+                 int ingate) {
+  __shared__ float s_alpha[kMaxDk];
+  __shared__ float s_w[kMaxDk];   // ahat * k
+  __shared__ float s_q[kMaxDk];   // scale * q
+  __shared__ float4 s_red[kStepWarps][32];
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31;
+  const int tiles = (dv + kTileCols - 1) / kTileCols;
+  const long long n_items = (long long)n_seq_heads * tiles;
+
+  for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const long long nh = item / tiles;
+    const int col = (int)(item % tiles) * kTileCols + lane * 4;
+    const bool col_ok = col < dv;
+    float* S = state + nh * (long long)dk * dv + col;
+
+    // First batch of state rows: issued before anything else of this item.
+    float4 buf[kBatch];
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) {
+      const int r = warp + kStepWarps * j;
+      if (col_ok && r < dk) buf[j] = ld_stream(reinterpret_cast<const float4*>(S + (long long)r * dv));
+    }
+
+    // Gates of this token (fp32 throughout).
+    for (int d = tid; d < dk; d += kStepThreads) {
+      const long long i = nh * dk + d;
+      float la, lh;
+      gate_logs_f32(to_f32(gx[i]), to_f32(ty[i]), ingate, la, lh);
+      s_alpha[d] = expf(la);
+      s_w[d] = expf(lh) * to_f32(k[i]);
+      s_q[d] = scale * to_f32(q[i]);
+    }
+    float4 vv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (col_ok) {
+      const T* vp = v + nh * dv + col;
+      vv = make_float4(to_f32(vp[0]), to_f32(vp[1]), to_f32(vp[2]), to_f32(vp[3]));
+    }
+    __syncthreads();
+
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int base = 0; base < dk; base += kStepWarps * kBatch) {
+#pragma unroll
+      for (int j = 0; j < kBatch; ++j) {
+        const int r = base + warp + kStepWarps * j;
+        if (col_ok && r < dk) {
+          const float a = s_alpha[r], w = s_w[r], qq = s_q[r];
+          float4 s = buf[j];
+          s.x = fmaf(a, s.x, w * vv.x);
+          s.y = fmaf(a, s.y, w * vv.y);
+          s.z = fmaf(a, s.z, w * vv.z);
+          s.w = fmaf(a, s.w, w * vv.w);
+          acc.x = fmaf(qq, s.x, acc.x);
+          acc.y = fmaf(qq, s.y, acc.y);
+          acc.z = fmaf(qq, s.z, acc.z);
+          acc.w = fmaf(qq, s.w, acc.w);
+          st_stream(reinterpret_cast<float4*>(S + (long long)r * dv), s);
+        }
+      }
+      const int next = base + kStepWarps * kBatch;
+      if (next < dk) {
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+          const int r = next + warp + kStepWarps * j;
+          if (col_ok && r < dk)
+            buf[j] = ld_stream(reinterpret_cast<const float4*>(S + (long long)r * dv));
+        }
+      }
+    }
+
+    // o = sum over the four warps' row subsets.
+    s_red[warp][lane] = acc;
+    __syncthreads();
+    if (warp == 0 && col_ok) {
+      float4 t = s_red[0][lane];
+#pragma unroll
+      for (int w = 1; w < kStepWarps; ++w) {
+        const float4 u = s_red[w][lane];
+        t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+      }
+      T* op = o + nh * dv + col;
+      op[0] = from_f32<T>(t.x);
+      op[1] = from_f32<T>(t.y);
+      op[2] = from_f32<T>(t.z);
+      op[3] = from_f32<T>(t.w);
+    }
+    __syncthreads();  // s_alpha / s_red are rewritten by the next item
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_step(const rodimus_ddts_step_params& p, int* n_launches) {
+  *n_launches = 0;
+  const long long nh = (long long)p.Nseq * p.H;
+  if (nh == 0) return cudaSuccess;
+  const int tiles = (p.dv + kTileCols - 1) / kTileCols;
+  const long long items = nh * tiles;
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  const long long max_grid = (long long)sms * 8;
+  const int grid = (int)(items < max_grid ? items : max_grid);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
+  if (p.dtype == RODIMUS_BF16) {
+    using T = __nv_bfloat16;
+    ddts_step_kernel<T><<<grid, kStepThreads, 0, st>>>(
+        (const T*)p.q, (const T*)p.k, (const T*)p.gate_x, (const T*)p.temp_y, (const T*)p.v,
+        (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate);
+  } else {
+    using T = float;
+    ddts_step_kernel<T><<<grid, kStepThreads, 0, st>>>(
+        (const T*)p.q, (const T*)p.k, (const T*)p.gate_x, (const T*)p.temp_y, (const T*)p.v,
+        (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate);
+  }
+  *n_launches = 1;
+  return cudaGetLastError();
+}
+
+}  // namespace ddts

@@ -1,0 +1,160 @@
+// Host side of the C ABI: argument checks (before any launch), workspace sizing, kernel choice.
+#include <cstdlib>
+#include <cstring>
+
+#include "ddts_common.cuh"
+
+namespace {
+
+thread_local int t_last_launches = 0;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+size_t workspace_bytes_for(int n_seq) {
+  size_t order = (size_t)(n_seq > 0 ? n_seq : 0) * sizeof(int32_t);
+  order = (order + 255) & ~(size_t)255;
+  return sizeof(ddts::WorkspaceHeader) + order;
+}
+
+// Everything about the sizes that does not need a pointer.
+int check_fwd_sizes(const rodimus_ddts_fwd_params* p, bool varlen) {
+  if (p->struct_size != (int32_t)sizeof(rodimus_ddts_fwd_params)) return RODIMUS_ERR_DTYPE;
+  if (p->dtype != RODIMUS_BF16 && p->dtype != RODIMUS_F32) return RODIMUS_ERR_DTYPE;
+  if (p->ingate != RODIMUS_INGATE_POW_G && p->ingate != RODIMUS_INGATE_POW_SIGMOID)
+    return RODIMUS_ERR_DTYPE;
+  if (p->B < 0 || p->H < 0 || p->T < 0) return RODIMUS_ERR_SHAPE;
+  if (p->dk <= 0 || p->dv <= 0 || p->dk % 16 || p->dv % 16) return RODIMUS_ERR_SHAPE;
+  if (p->dk > 256 || p->dv > 1024) return RODIMUS_ERR_SHAPE;
+  if ((long long)p->B * p->H * p->T >= (1LL << 31)) return RODIMUS_ERR_SHAPE;
+  if (varlen) {
+    if (p->B != 1 || p->N < 0) return RODIMUS_ERR_SHAPE;
+    if ((long long)p->N * p->H >= (1LL << 31)) return RODIMUS_ERR_SHAPE;
+  }
+  return RODIMUS_OK;
+}
+
+}  // namespace
+
+namespace ddts {
+
+bool fwd_tc_supported(const rodimus_ddts_fwd_params& p) {
+  const char* force = std::getenv("RODIMUS_DDTS_FORCE_SIMT");
+  if (force && force[0] == '1') return false;
+  return tc_kernel_built() && p.dtype == RODIMUS_BF16 && p.dk == 128 && p.dv % 128 == 0;
+}
+
+}  // namespace ddts
+
+extern "C" {
+
+size_t rodimus_ddts_fwd_workspace_bytes(const rodimus_ddts_fwd_params* p) {
+  if (!p) return 0;
+  const bool varlen = p->cu_seqlens != nullptr || p->cu_seqlens_host != nullptr;
+  if (check_fwd_sizes(p, varlen) != RODIMUS_OK) return 0;
+  return workspace_bytes_for(varlen ? p->N : 0);
+}
+
+const char* rodimus_ddts_fwd_kernel_name(const rodimus_ddts_fwd_params* p) {
+  if (!p) return "invalid";
+  if (check_fwd_sizes(p, p->cu_seqlens != nullptr) != RODIMUS_OK) return "invalid";
+  return ddts::fwd_tc_supported(*p) ? "tcgen05" : "simt";
+}
+
+int rodimus_ddts_fwd(const rodimus_ddts_fwd_params* p) {
+  t_last_launches = 0;
+  if (!p) return RODIMUS_ERR_NULL;
+  const bool varlen = p->cu_seqlens != nullptr;
+  int rc = check_fwd_sizes(p, varlen);
+  if (rc != RODIMUS_OK) return rc;
+  if (!varlen && p->cu_seqlens_host) return RODIMUS_ERR_NULL;  // host copy without the device array
+  const long long rows = (long long)p->B * p->H * p->T;
+  const long long n_seq = varlen ? p->N : p->B;
+  if (rows > 0 && (!p->q || !p->k || !p->gate_x || !p->temp_y || !p->v || !p->o))
+    return RODIMUS_ERR_NULL;
+  const void* ptrs[] = {p->q, p->k, p->gate_x, p->temp_y, p->v, p->o, p->s0, p->sT, p->cu_seqlens};
+  for (const void* ptr : ptrs)
+    if (ptr && !aligned16(ptr)) return RODIMUS_ERR_ALIGN;
+  if (!p->workspace || p->workspace_bytes < workspace_bytes_for(varlen ? p->N : 0))
+    return RODIMUS_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(p->workspace) & 255u) return RODIMUS_ERR_ALIGN;
+  if (varlen && p->cu_seqlens_host) {
+    const int32_t* cu = p->cu_seqlens_host;
+    if (cu[0] != 0 || cu[p->N] != p->T) return RODIMUS_ERR_SEQLENS;
+    for (int n = 0; n < p->N; ++n)
+      if (cu[n + 1] < cu[n]) return RODIMUS_ERR_SEQLENS;
+  }
+  if (varlen && p->N == 0 && p->T != 0) return RODIMUS_ERR_SEQLENS;
+  if (n_seq * p->H == 0) return RODIMUS_OK;  // nothing to compute, nothing to write
+
+  int launches = 0, n = 0;
+  cudaError_t e = cudaSuccess;
+  if (varlen) {  // checks cu_seqlens on the device, clears the status word, orders the work
+    e = ddts::launch_plan(*p, &n);
+    launches += n;
+  }  // dense: the prefill kernel's first CTA clears the status word itself
+  if (e != cudaSuccess) return RODIMUS_ERR_CUDA;
+  if (ddts::fwd_tc_supported(*p))
+    e = ddts::launch_fwd_tc(*p, &n);
+  else
+    e = ddts::launch_fwd_simt(*p, &n);
+  launches += n;
+  if (e != cudaSuccess) return RODIMUS_ERR_CUDA;
+  t_last_launches = launches;
+  return RODIMUS_OK;
+}
+
+int rodimus_ddts_step(const rodimus_ddts_step_params* p) {
+  t_last_launches = 0;
+  if (!p) return RODIMUS_ERR_NULL;
+  if (p->struct_size != (int32_t)sizeof(rodimus_ddts_step_params)) return RODIMUS_ERR_DTYPE;
+  if (p->dtype != RODIMUS_BF16 && p->dtype != RODIMUS_F32) return RODIMUS_ERR_DTYPE;
+  if (p->ingate != RODIMUS_INGATE_POW_G && p->ingate != RODIMUS_INGATE_POW_SIGMOID)
+    return RODIMUS_ERR_DTYPE;
+  if (p->Nseq < 0 || p->H < 0) return RODIMUS_ERR_SHAPE;
+  if (p->dk <= 0 || p->dv <= 0 || p->dk % 16 || p->dv % 16) return RODIMUS_ERR_SHAPE;
+  if (p->dk > 256 || p->dv > 1024) return RODIMUS_ERR_SHAPE;
+  if ((long long)p->Nseq * p->H >= (1LL << 31) / 8) return RODIMUS_ERR_SHAPE;
+  if ((long long)p->Nseq * p->H == 0) return RODIMUS_OK;
+  if (!p->q || !p->k || !p->gate_x || !p->temp_y || !p->v || !p->o || !p->state)
+    return RODIMUS_ERR_NULL;
+  const void* ptrs[] = {p->q, p->k, p->gate_x, p->temp_y, p->v, p->o, p->state};
+  for (const void* ptr : ptrs)
+    if (!aligned16(ptr)) return RODIMUS_ERR_ALIGN;
+  int n = 0;
+  cudaError_t e = ddts::launch_step(*p, &n);
+  if (e != cudaSuccess) return RODIMUS_ERR_CUDA;
+  t_last_launches = n;
+  return RODIMUS_OK;
+}
+
+int rodimus_ddts_device_status(const void* workspace, void* stream) {
+  if (!workspace) return RODIMUS_ERR_NULL;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int32_t status = 0;
+  if (cudaMemcpyAsync(&status, workspace, sizeof(status), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return RODIMUS_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return RODIMUS_ERR_CUDA;
+  return status;
+}
+
+int rodimus_ddts_last_launch_count(void) { return t_last_launches; }
+
+const char* rodimus_status_str(int status) {
+  switch (status) {
+    case RODIMUS_OK: return "ok";
+    case RODIMUS_ERR_NULL: return "required pointer is NULL";
+    case RODIMUS_ERR_SHAPE: return "invalid shape";
+    case RODIMUS_ERR_DTYPE: return "unknown dtype, ingate or struct_size";
+    case RODIMUS_ERR_ALIGN: return "pointer not sufficiently aligned";
+    case RODIMUS_ERR_SEQLENS: return "invalid cu_seqlens";
+    case RODIMUS_ERR_WORKSPACE: return "workspace missing or too small";
+    case RODIMUS_ERR_UNSUPPORTED: return "unsupported request";
+    case RODIMUS_ERR_CUDA: return "CUDA call failed";
+    case RODIMUS_ERR_TIMEOUT: return "bounded device wait ran out";
+    default: return "unknown status";
+  }
+}
+
+int rodimus_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,327 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU oracle on the
+same seeded inputs.  Bar: max|err|/max|ref| <= 2e-2 (bf16 in, fp32 accumulate) and <= 1e-4
+(fp32 build), per output tensor (o and the final state separately)."""
+import os
+
+import numpy as np
+import pytest
+
+import paper_2410_06577_b200 as rd
+from paper_2410_06577_b200 import workloads as wl
+from oracle import ddts_oracle as orc
+from tests._util import TOL_BF16, TOL_F32, dev, host, prefill_to_device, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def _tol(dtype):
+    return TOL_BF16 if dtype == "bf16" else TOL_F32
+
+
+def _run_prefill(p, ingate=rd.INGATE_POW_G, scale=1.0, host_cu=True, want_final_state=True):
+    import torch
+    d = prefill_to_device(p)
+    o, sT = rd.ddts_fwd(d["q"], d["k"], d["x"], d["y"], d["v"], d["s0"], d["cu"],
+                        d["cu_host"] if host_cu else None, scale, ingate, want_final_state)
+    torch.cuda.synchronize()
+    return host(o), (None if sT is None else host(sT))
+
+
+def _check_prefill(p, ingate=rd.INGATE_POW_G, scale=1.0, tol=None, **kw):
+    o, sT = _run_prefill(p, ingate, scale, **kw)
+    ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0, cu_seqlens=p.cu_seqlens, scale=scale,
+                         ingate=ingate)
+    tol = tol or _tol(p.dtype)
+    eo, es = rel_err(o, ro), rel_err(sT, rs)
+    assert eo <= tol and es <= tol, (p.name, eo, es)
+    return eo, es
+
+
+# ------------------------------------------------------------------------------------------
+# decode
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype,Nseq,H,dk,dv", [
+    ("bf16", 16, 4, 128, 256),     # config 3 shrunk
+    ("f32", 3, 2, 64, 64),
+    ("bf16", 5, 3, 48, 80),        # ragged column tile, short rows
+    ("f32", 2, 1, 256, 1024),      # maximum sizes
+])
+@pytest.mark.parametrize("ingate", [rd.INGATE_POW_G, rd.INGATE_POW_SIGMOID])
+def test_decode_steps_match_oracle(dtype, Nseq, H, dk, dv, ingate):
+    import torch
+    w = wl.make_decode(3, Nseq, H, dk, dv, ring=16, dtype=dtype)
+    state = torch.from_numpy(w.state).cuda()
+    ref_state = w.state.astype(np.float64)
+    tol = _tol(dtype)
+    for s in range(16):
+        o = rd.ddts_step(dev(w.q[s], dtype), dev(w.k[s], dtype), dev(w.x[s], dtype),
+                         dev(w.y[s], dtype), dev(w.v[s], dtype), state, scale=0.5, ingate=ingate)
+        ro = orc.ref_step(w.q[s], w.k[s], w.x[s], w.y[s], w.v[s], ref_state, scale=0.5,
+                          ingate=ingate)
+        assert rel_err(host(o), ro) <= tol
+    # the fp32 state itself is held to the fp32 bar whatever the token dtype
+    assert rel_err(host(state), ref_state) <= TOL_F32
+
+
+def test_decode_full_width_many_steps():
+    """Config 3 at full width (256 sequences x 16 heads), 1000 in-place steps; the oracle follows
+    8 of the sequences."""
+    import torch
+    w = wl.config(3)
+    Nseq = w.state.shape[0]
+    pick = np.array([0, 1, 37, 100, 128, 200, 254, 255])
+    state = torch.from_numpy(w.state).cuda()
+    ref_state = np.ascontiguousarray(w.state[pick]).astype(np.float64)
+    ring = [tuple(dev(a[s], "bf16") for a in (w.q, w.k, w.x, w.y, w.v)) for s in range(16)]
+    o = torch.empty((Nseq, 16, 256), dtype=torch.bfloat16, device="cuda")
+    for step in range(1000):
+        q, k, x, y, v = ring[step % 16]
+        rd.ddts_step(q, k, x, y, v, state, out=o)
+        if step in (0, 15, 999):
+            torch.cuda.synchronize()
+        s = step % 16
+        ro = orc.ref_step(w.q[s][pick], w.k[s][pick], w.x[s][pick], w.y[s][pick], w.v[s][pick],
+                          ref_state)
+        if step in (0, 15, 999):
+            assert rel_err(host(o)[pick], ro) <= TOL_BF16, step
+    assert rel_err(host(state)[pick], ref_state) <= TOL_F32
+
+
+# ------------------------------------------------------------------------------------------
+# prefill: fp32 validation build
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("ingate", [rd.INGATE_POW_G, rd.INGATE_POW_SIGMOID])
+def test_config0_fp32(ingate):
+    p = wl.config(0)
+    _check_prefill(p, ingate)
+    # and the O(T^2) masked parallel form agrees too (zero initial state)
+    o, _ = _run_prefill(p, ingate)
+    ref = orc.parallel_form(p.q[0, 0], p.k[0, 0], p.x[0, 0], p.y[0, 0], p.v[0, 0], ingate=ingate)
+    assert rel_err(o[0, 0], ref) <= TOL_F32
+
+
+@pytest.mark.parametrize("B,H,T,dk,dv", [
+    (2, 2, 1, 64, 64),       # single token
+    (1, 3, 37, 48, 80),      # ragged everything
+    (1, 1, 131, 256, 256),   # widest keys
+    (2, 1, 16, 16, 16),      # smallest legal sizes, exactly one chunk
+])
+def test_fp32_shapes_state_and_scale(B, H, T, dk, dv):
+    p = wl.make_prefill(100 + T, B, H, T, dk, dv, "f32", gate_mean=-1.0, s0_std=0.5)
+    _check_prefill(p, scale=0.25)
+    _check_prefill(p, rd.INGATE_POW_SIGMOID, scale=3.0)
+
+
+def test_fp32_empty_sequence_returns_initial_state():
+    import torch
+    p = wl.make_prefill(7, 2, 2, 0, 64, 64, "f32", s0_std=1.0)
+    o, sT = _run_prefill(p)
+    assert o.shape == (2, 2, 0, 64)
+    assert np.array_equal(sT, p.s0.astype(np.float64))
+
+
+# ------------------------------------------------------------------------------------------
+# prefill: bf16 path (tensor-core kernel for dk = 128, dv % 128 == 0)
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("B,H,T,dv", [
+    (2, 2, 200, 256),    # several chunks and a ragged tail
+    (1, 2, 64, 128),     # exactly one chunk
+    (1, 1, 1, 256),      # one token
+    (1, 2, 65, 256),     # tail of one row
+    (3, 1, 333, 128),
+])
+@pytest.mark.parametrize("ingate", [rd.INGATE_POW_G, rd.INGATE_POW_SIGMOID])
+def test_bf16_prefill_small(B, H, T, dv, ingate):
+    p = wl.make_prefill(200 + T, B, H, T, 128, dv, "bf16", s0_std=0.1)
+    _check_prefill(p, ingate, scale=0.5)
+    p0 = wl.make_prefill(300 + T, B, H, T, 128, dv, "bf16")       # zero initial state
+    _check_prefill(p0, ingate)
+
+
+def test_bf16_other_shapes_use_cuda_core_kernel():
+    p = wl.make_prefill(11, 1, 2, 90, 64, 96, "bf16", s0_std=0.1)
+    _check_prefill(p)
+
+
+def test_bf16_output_only_and_state_aliasing():
+    import torch
+    p = wl.make_prefill(12, 1, 2, 150, 128, 256, "bf16", s0_std=0.1)
+    d = prefill_to_device(p)
+    o1, none = rd.ddts_fwd(d["q"], d["k"], d["x"], d["y"], d["v"], d["s0"], want_final_state=False)
+    assert none is None
+    s_inout = d["s0"].clone()
+    o2, sT = rd.ddts_fwd(d["q"], d["k"], d["x"], d["y"], d["v"], s_inout, final_state=s_inout)
+    torch.cuda.synchronize()
+    assert torch.equal(o1, o2)
+    ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0)
+    assert rel_err(host(o1), ro) <= TOL_BF16 and rel_err(host(s_inout), rs) <= TOL_BF16
+
+
+def test_bf16_prefill_equals_split_runs_and_decode_steps():
+    import torch
+    p = wl.make_prefill(13, 1, 2, 192, 128, 256, "bf16", s0_std=0.1)
+    d = prefill_to_device(p)
+    o, sT = rd.ddts_fwd(d["q"], d["k"], d["x"], d["y"], d["v"], d["s0"])
+    cut = 100
+    sl = lambda t, lo, hi: t[:, :, lo:hi].contiguous()
+    o1, s1 = rd.ddts_fwd(*(sl(d[n], 0, cut) for n in "qkxyv"), d["s0"])
+    o2, s2 = rd.ddts_fwd(*(sl(d[n], cut, 192) for n in "qkxyv"), s1)
+    torch.cuda.synchronize()
+    ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0)
+    assert rel_err(host(torch.cat([o1, o2], dim=2)), ro) <= TOL_BF16
+    assert rel_err(host(s2), rs) <= TOL_BF16 and rel_err(host(sT), rs) <= TOL_BF16
+    # repeated decode steps from the same initial state
+    state = d["s0"].clone()
+    outs = []
+    for t in range(192):
+        outs.append(rd.ddts_step(*(d[n][:, :, t].contiguous() for n in "qkxyv"), state))
+    torch.cuda.synchronize()
+    assert rel_err(host(torch.stack(outs, dim=2)), ro) <= TOL_BF16
+    assert rel_err(host(state), rs) <= TOL_F32
+
+
+@pytest.mark.parametrize("xv,yv", [(8.0, 8.0), (-12.0, 0.0), (3.0, -2.0)])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_strong_decay_and_long_memory(xv, yv, dtype):
+    """Adversarial gates: about 8 nats of decay per step, and almost none."""
+    p = wl.make_prefill(14, 1, 2, 150, 128, 128, dtype, s0_std=0.1)
+    p.x[...] = xv
+    p.y[...] = yv
+    _check_prefill(p)
+
+
+def test_bf16_mixed_decay_channels():
+    """Fast- and slow-decaying channels side by side inside one chunk."""
+    p = wl.make_prefill(15, 1, 2, 200, 128, 256, "bf16", s0_std=0.1)
+    p.x[..., ::2] = wl.round_to_bf16(p.x[..., ::2] + 5.0)
+    p.y[..., ::4] = 4.0
+    _check_prefill(p)
+
+
+def test_results_are_deterministic():
+    import torch
+    p = wl.make_prefill(16, 2, 2, 300, 128, 256, "bf16", s0_std=0.1)
+    d = prefill_to_device(p)
+    a = rd.ddts_fwd(d["q"], d["k"], d["x"], d["y"], d["v"], d["s0"])
+    b = rd.ddts_fwd(d["q"], d["k"], d["x"], d["y"], d["v"], d["s0"])
+    torch.cuda.synchronize()
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+# ------------------------------------------------------------------------------------------
+# varlen
+# ------------------------------------------------------------------------------------------
+
+def _varlen(seed, lens, H, dk, dv, dtype, s0_std=0.2):
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    return wl.make_prefill(seed, 1, H, int(cu[-1]), dk, dv, dtype, s0_std=s0_std, cu_seqlens=cu)
+
+
+@pytest.mark.parametrize("dtype,dk,dv", [("bf16", 128, 256), ("f32", 64, 64), ("bf16", 128, 128)])
+@pytest.mark.parametrize("host_cu", [True, False])
+def test_varlen_matches_oracle(dtype, dk, dv, host_cu):
+    lens = [5, 0, 130, 64, 1, 77, 0, 128, 63]
+    p = _varlen(20, lens, 2, dk, dv, dtype)
+    _check_prefill(p, host_cu=host_cu)
+
+
+def test_varlen_no_leak_between_sequences():
+    """Huge values in the neighbours must not reach a sequence's outputs or state."""
+    import torch
+    lens = [70, 33, 90]
+    p = _varlen(21, lens, 2, 128, 256, "bf16")
+    cu = p.cu_seqlens
+    lo, hi = int(cu[1]), int(cu[2])
+    clean_o, clean_s = _run_prefill(p)
+    for name in ("q", "k", "v"):
+        a = getattr(p, name)
+        a[:, :, :lo] = wl.round_to_bf16(a[:, :, :lo] * 64.0 + 9.0)
+        a[:, :, hi:] = wl.round_to_bf16(a[:, :, hi:] * 64.0 - 9.0)
+    p.x[:, :, :lo] = 2.0
+    p.x[:, :, hi:] = 2.0
+    o, s = _run_prefill(p)
+    assert np.array_equal(o[:, :, lo:hi], clean_o[:, :, lo:hi])
+    assert np.array_equal(s[1], clean_s[1])
+    assert not np.array_equal(s[0], clean_s[0])
+
+
+def test_varlen_bad_seqlens_reported_by_device_without_fault():
+    import torch
+    p = _varlen(22, [40, 50, 30], 2, 128, 256, "bf16")
+    d = prefill_to_device(p)
+    bad = d["cu"].clone()
+    bad[1] = 100            # decreases afterwards: 0,100,90,120
+    B, H, T, dk = d["q"].shape
+    o = torch.zeros((B, H, T, 256), dtype=torch.bfloat16, device="cuda")
+    sT = torch.zeros((3, H, dk, 256), dtype=torch.float32, device="cuda")
+    prm = rd.fwd_params(d["q"], d["k"], d["x"], d["y"], d["v"], o, d["s0"], sT, bad)
+    ws = rd.new_workspace(prm, "cuda")
+    prm.workspace, prm.workspace_bytes = ws.data_ptr(), ws.numel()
+    assert rd.fwd_raw(prm) == rd.OK            # host had nothing to check
+    assert rd.device_status(ws) == rd.ERR_SEQLENS
+    assert torch.isfinite(o.float()).all()
+    # with the host copy the same request is refused before any launch
+    bad_host = bad.cpu()
+    prm.cu_seqlens_host = bad_host.data_ptr()
+    assert rd.fwd_raw(prm) == rd.ERR_SEQLENS
+    # and a good request on the same workspace clears the device status
+    prm.cu_seqlens, prm.cu_seqlens_host = d["cu"].data_ptr(), None
+    assert rd.fwd_raw(prm) == rd.OK and rd.device_status(ws) == rd.OK
+
+
+# ------------------------------------------------------------------------------------------
+# the named configurations at full size, in the launch configuration the benchmark times
+# ------------------------------------------------------------------------------------------
+
+def test_config1_full_size():
+    p = wl.config(1)
+    assert p.shape == (4, 16, 2048, 128, 256)
+    _check_prefill(p)
+    _check_prefill(p, rd.INGATE_POW_SIGMOID)
+
+
+def test_config2_full_size_and_split_halves():
+    """T = 32768 with a nonzero initial state; the oracle follows 4 of the 16 heads, and the GPU
+    result must also equal two T = 16384 runs that pass the state across the split."""
+    import torch
+    p = wl.config(2)
+    assert p.shape == (1, 16, 32768, 128, 256)
+    d = prefill_to_device(p)
+    o, sT = rd.ddts_fwd(d["q"], d["k"], d["x"], d["y"], d["v"], d["s0"])
+    half = 16384
+    sl = lambda t, lo, hi: t[:, :, lo:hi].contiguous()
+    o1, s1 = rd.ddts_fwd(*(sl(d[n], 0, half) for n in "qkxyv"), d["s0"])
+    o2, s2 = rd.ddts_fwd(*(sl(d[n], half, 2 * half) for n in "qkxyv"), s1)
+    torch.cuda.synchronize()
+    heads = [0, 5, 10, 15]
+    pk = lambda a: np.ascontiguousarray(a[:, heads])
+    ro, rs = orc.ref_fwd(pk(p.q), pk(p.k), pk(p.x), pk(p.y), pk(p.v), s0=pk(p.s0))
+    assert rel_err(host(o)[:, heads], ro) <= TOL_BF16
+    assert rel_err(host(sT)[:, heads], rs) <= TOL_BF16
+    assert rel_err(host(torch.cat([o1, o2], dim=2))[:, heads], ro) <= TOL_BF16
+    assert rel_err(host(s2)[:, heads], rs) <= TOL_BF16
+    # the halves and the single run follow the same chunk grid, so they agree far tighter
+    assert rel_err(host(torch.cat([o1, o2], dim=2)), host(o)) <= 1e-2
+
+
+def test_config4_full_size_sampled_sequences():
+    import torch
+    p = wl.config(4)
+    cu = p.cu_seqlens
+    assert len(cu) == 65 and p.shape[1] == 16
+    d = prefill_to_device(p)
+    o, sT = rd.ddts_fwd(d["q"], d["k"], d["x"], d["y"], d["v"], None, d["cu"], d["cu_host"])
+    torch.cuda.synchronize()
+    o, sT = host(o), host(sT)
+    lens = np.diff(cu)
+    pick = sorted({0, 63, int(np.argmax(lens)), int(np.argmin(lens)), 17, 40})
+    for n in pick:
+        lo, hi = int(cu[n]), int(cu[n + 1])
+        heads = [0, 7, 15]
+        sl = lambda a: np.ascontiguousarray(a[:, heads, lo:hi])
+        ro, rs = orc.ref_fwd(sl(p.q), sl(p.k), sl(p.x), sl(p.y), sl(p.v))
+        assert rel_err(o[:, heads, lo:hi], ro) <= TOL_BF16, n
+        assert rel_err(sT[n, heads], rs[0]) <= TOL_BF16, n
