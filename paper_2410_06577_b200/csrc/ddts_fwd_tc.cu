@@ -1,6 +1,751 @@
-// placeholder until the tensor-core kernel lands
+// Chunked DDTS prefill on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), bf16 inputs,
+// dk = 128, 128 state columns per CTA.
+//
+// Chunkwise form (appendix "Chunkwise Parallel Representation of the Rodimus Block"), chunk
+// length C = 64, all decays handled in the log2 domain and anchored at the chunk start:
+//   b_r      = sum_{j<=r in chunk} log2 alpha_j                       (per key channel, <= 0)
+//   Qt_r     = q_r . 2^{b_r}                                          bf16, K-major operand
+//   Kt_i     = k_i . ahat_i . 2^{-b_i}                                bf16, K-major operand
+//   Ke_i     = k_i . ahat_i . 2^{b_C - b_i}                           bf16, MN-major operand
+//   P        = (Qt Kt^T) masked to i <= r                             [C,C]   fp32 in TMEM
+//   O        = P V + Qt S_in            (S_in = state ENTERING the chunk) [C,128] fp32 in TMEM
+//   S_out    = diag(2^{b_C}) S_in + Ke^T V                            [128,128] fp32 in TMEM
+// The fp32 state never leaves TMEM between chunks; once per chunk it makes one trip through
+// registers to be scaled by the chunk's total decay and copied, as bf16, to shared memory where
+// the readout contraction can take it as an operand.
+//
+// One CTA = 20 warps with fixed roles, connected by mbarriers (every wait is bounded):
+//   warp 0        TMA producer: q,k,x,y,v tiles of the next chunk into a 2-stage ring
+//   warp 1        tcgen05.mma issuer (one elected lane), owns the TMEM allocation
+//   warps 4-7     state group: TMEM <-> registers trip of S, initial/final state I/O
+//   warps 8-11    score/output group: P -> masked bf16 operand, O -> global memory
+//   warps 12-19   gate group: softplus/sigmoid/log/exp2 math, in-chunk scan, operand tiles
+//                 written IN PLACE over the raw q,k,x tiles (same swizzled layout)
+// Work item = (sequence, head, 128-column slice of dv), dealt round-robin to a persistent grid.
+#include <cuda.h>
+
+#include <cstring>
+
 #include "ddts_common.cuh"
+
 namespace ddts {
-bool tc_kernel_built() { return false; }
-cudaError_t launch_fwd_tc(const rodimus_ddts_fwd_params&, int* n) { *n = 0; return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kC = 64;                       // chunk rows
+constexpr int kDK = 128;                     // key channels
+constexpr int kDVS = 128;                    // value columns per CTA
+constexpr int kStages = 2;
+constexpr int kSlabBytes = kC * 128;         // [64 rows][64 bf16] = 8 KiB, 128-byte swizzled
+constexpr int kTileBytes = 2 * kSlabBytes;   // [64][128] bf16 as two slabs
+constexpr int kStageBytes = 5 * kTileBytes;  // q, k, x, y, v
+constexpr int kOffQ = 0, kOffK = kTileBytes, kOffX = 2 * kTileBytes, kOffY = 3 * kTileBytes,
+              kOffV = 4 * kTileBytes;
+constexpr int kSsSlabBytes = kDK * 128;      // [128 rows][64 bf16]
+constexpr int kOffSs = kStages * kStageBytes;            // bf16 copy of the state, 2 slabs
+constexpr int kOffD = kOffSs + 2 * kSsSlabBytes;         // float [kStages][128]: 2^{b_C}
+constexpr int kOffTot = kOffD + kStages * kDK * 4;       // float [2][8][64]: scan partials
+constexpr int kOffBar = kOffTot + 2 * 8 * 64 * 4;        // mbarriers
+constexpr int kNumBars = 16;
+constexpr int kOffMisc = kOffBar + kNumBars * 8;         // tmem base, abort flag
+constexpr int kSmemUsed = kOffMisc + 16;
+constexpr int kSmemBytes = kSmemUsed + 1024;             // slack for manual 1024-byte alignment
+
+constexpr int kThreads = 640;
+constexpr int kGateWarp0 = 12, kGateWarps = 8;
+
+// TMEM columns (fp32 words): state, output, scores
+constexpr uint32_t kColS = 0, kColO = 128, kColP = 256, kTmemCols = 512;
+
+// mbarrier indices
+enum { BAR_FULL0 = 0, BAR_FULL1, BAR_EMPTY0, BAR_EMPTY1, BAR_GATED0, BAR_GATED1, BAR_PFULL,
+       BAR_PREADY, BAR_SREADY, BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN };
+
+constexpr long long kWaitCycles = 4000000000LL;  // about two seconds: then give up, never hang
+
+struct TcArgs {
+  void* o;
+  const float* s0;
+  float* sT;
+  const int32_t* cu;
+  const int32_t* order;
+  WorkspaceHeader* hdr;
+  int H, T, dv, n_seq, slices;
+  long long n_items;
+  float scale;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.b32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag and the device status) if the
+// phase does not complete in time or another role has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          WorkspaceHeader* hdr) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+    if (mbar_try(bar, parity)) return true;
+    // a completed phase stays visible to every waiter of a group, so re-test before giving up:
+    // either all members of a group pass a given wait or none does
+    if (*abort_flag) return mbar_try(bar, parity);
+    if (clock64() - t0 > kWaitCycles) {
+      if (mbar_try(bar, parity)) return true;
+      *abort_flag = 1;
+      atomicMax(&hdr->status, (int)RODIMUS_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),
+        "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),
+        "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+        "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() {
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float lg2f(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float rcpf(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d)
+               : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle (descriptor version 1).
+//   K-major operand  [rows][64 elements]: rows 128 B apart, groups of 8 rows 1024 B apart.
+//   MN-major operand [k rows][64 elements along M or N]: k rows 128 B apart, groups of 8 k rows
+//   1024 B apart, successive 64-element groups along M/N `mn_group_bytes` apart.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3FFF) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t mn_group_bytes) {
+  return (uint64_t)((addr >> 4) & 0x3FFF) | ((uint64_t)((mn_group_bytes >> 4) & 0x3FFF) << 16) |
+         ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+struct Item {
+  long long row0;      // first global row (in the [rows, d] view) of this sequence and head
+  long long state_off; // element offset of this (sequence, head) state slice start (column 0)
+  int len;             // tokens
+  int col0;            // first value column of the slice
+};
+
+__device__ __forceinline__ Item decode_item(const TcArgs& a, long long item) {
+  Item it;
+  const int slice = (int)(item % a.slices);
+  const long long sh = item / a.slices;
+  const int h = (int)(sh % a.H);
+  long long n = sh / a.H;
+  if (a.cu) {
+    n = a.order[n];
+    int lo = a.cu[n], hi = a.cu[n + 1];
+    lo = lo < 0 ? 0 : (lo > a.T ? a.T : lo);
+    hi = hi < lo ? lo : (hi > a.T ? a.T : hi);
+    it.row0 = (long long)h * a.T + lo;
+    it.len = hi - lo;
+  } else {
+    it.row0 = (n * a.H + h) * (long long)a.T;
+    it.len = a.T;
+  }
+  it.col0 = slice * kDVS;
+  it.state_off = (n * a.H + h) * (long long)kDK * a.dv + it.col0;
+  return it;
+}
+
+// ---------------------------------------------------------------------------------------------
+// kernel
+// ---------------------------------------------------------------------------------------------
+template <int INGATE>
+__global__ void __launch_bounds__(kThreads, 1)
+ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                   const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
+                   const __grid_constant__ CUtensorMap map_v, const TcArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + kOffBar;
+  auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + kOffMisc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + kOffMisc + 4);
+  float* sD = reinterpret_cast<float*>(gbase + kOffD);
+  float* sTot = reinterpret_cast<float*>(gbase + kOffTot);
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31;
+
+  if (!a.cu && blockIdx.x == 0 && tid == 0) a.hdr->status = RODIMUS_OK;
+
+  if (tid == 0) {
+    *abort_flag = 0;
+    mbar_init(bar(BAR_FULL0), 1);
+    mbar_init(bar(BAR_FULL1), 1);
+    mbar_init(bar(BAR_EMPTY0), 1);
+    mbar_init(bar(BAR_EMPTY1), 1);
+    mbar_init(bar(BAR_GATED0), kGateWarps);
+    mbar_init(bar(BAR_GATED1), kGateWarps);
+    mbar_init(bar(BAR_PFULL), 1);
+    mbar_init(bar(BAR_PREADY), 128);
+    mbar_init(bar(BAR_SREADY), 128);
+    mbar_init(bar(BAR_SFULL), 1);
+    mbar_init(bar(BAR_OFULL), 1);
+    mbar_init(bar(BAR_OFREE), 128);
+    mbar_init(bar(BAR_GSCAN), kGateWarps);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(base + kOffMisc), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ===================================== TMA producer =====================================
+    if (lane == 0) {
+      uint32_t g = 0;
+      bool ok = true;
+      for (long long item = blockIdx.x; ok && item < a.n_items; item += gridDim.x) {
+        const Item it = decode_item(a, item);
+        const int n_chunks = (it.len + kC - 1) / kC;
+        for (int c = 0; c < n_chunks; ++c, ++g) {
+          const uint32_t s = g & 1, ph = (g >> 1) & 1;
+          if (!(ok = mbar_wait(bar(BAR_EMPTY0 + s), ph ^ 1, abort_flag, a.hdr))) break;
+          const uint32_t st = base + s * kStageBytes;
+          const uint32_t fb = bar(BAR_FULL0 + s);
+          mbar_expect_tx(fb, kStageBytes);
+          // rows beyond the tensor read as zeros; rows of the next sequence are masked later
+          const long long row = it.row0 + (long long)c * kC;
+          const int y = (int)row;
+          tma_load_2d(st + kOffQ, &map_q, 0, y, fb);
+          tma_load_2d(st + kOffQ + kSlabBytes, &map_q, 64, y, fb);
+          tma_load_2d(st + kOffK, &map_k, 0, y, fb);
+          tma_load_2d(st + kOffK + kSlabBytes, &map_k, 64, y, fb);
+          tma_load_2d(st + kOffX, &map_x, 0, y, fb);
+          tma_load_2d(st + kOffX + kSlabBytes, &map_x, 64, y, fb);
+          tma_load_2d(st + kOffY, &map_y, 0, y, fb);
+          tma_load_2d(st + kOffY + kSlabBytes, &map_y, 64, y, fb);
+          tma_load_2d(st + kOffV, &map_v, it.col0, y, fb);
+          tma_load_2d(st + kOffV + kSlabBytes, &map_v, it.col0 + 64, y, fb);
+        }
+      }
+      // Leave no bulk copy in flight: the last loads are consumed by the gate group before the
+      // other roles reach the final barrier, except after an abort, where we wait here (bounded).
+      if (*abort_flag && g > 0) {
+        const uint32_t last = g - 1;
+        const long long t0 = clock64();
+        while (!mbar_try(bar(BAR_FULL0 + (last & 1)), (last >> 1) & 1) && clock64() - t0 < kWaitCycles) {}
+        if (last > 0) {
+          const uint32_t prev = last - 1;
+          while (!mbar_try(bar(BAR_FULL0 + (prev & 1)), (prev >> 1) & 1) && clock64() - t0 < kWaitCycles) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ====================================== MMA issuer ======================================
+    if (lane == 0) {
+      constexpr uint32_t kIdescP = make_idesc(64, 64, 0, 0);
+      constexpr uint32_t kIdescO = make_idesc(64, kDVS, 0, 1);
+      constexpr uint32_t kIdescS = make_idesc(128, kDVS, 1, 1);
+      const uint32_t ss = base + kOffSs;
+      uint32_t g = 0;
+      bool ok = true;
+      for (long long item = blockIdx.x; ok && item < a.n_items; item += gridDim.x) {
+        const Item it = decode_item(a, item);
+        const int n_chunks = (it.len + kC - 1) / kC;
+        for (int c = 0; c < n_chunks; ++c, ++g) {
+          const uint32_t s = g & 1, ph = (g >> 1) & 1, ph1 = g & 1;
+          const uint32_t st = base + s * kStageBytes;
+          if (!(ok = mbar_wait(bar(BAR_GATED0 + s), ph, abort_flag, a.hdr))) break;
+          tc_fence_after();
+          // P = Qt Kt^T : M = 64 (rows r), N = 64 (rows i), K = 128 channels
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t off = (kk >> 2) * kSlabBytes + (kk & 3) * 32;
+            umma_bf16(tmem + kColP, desc_kmajor(st + kOffQ + off), desc_kmajor(st + kOffK + off),
+                      kIdescP, kk > 0);
+          }
+          umma_commit(bar(BAR_PFULL));
+          if (!(ok = mbar_wait(bar(BAR_PREADY), ph1, abort_flag, a.hdr))) break;
+          if (!(ok = mbar_wait(bar(BAR_SREADY), ph1, abort_flag, a.hdr))) break;
+          if (!(ok = mbar_wait(bar(BAR_OFREE), ph1 ^ 1, abort_flag, a.hdr))) break;
+          tc_fence_after();
+          // O = P V : M = 64, N = 128, K = 64 rows i (P operand lives in the consumed y tile)
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            umma_bf16(tmem + kColO, desc_kmajor(st + kOffY + kk * 32),
+                      desc_mnmajor(st + kOffV + kk * 2048, kSlabBytes), kIdescO, kk > 0);
+          }
+          // O += Qt S_in : K = 128 channels
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t off = (kk >> 2) * kSlabBytes + (kk & 3) * 32;
+            umma_bf16(tmem + kColO, desc_kmajor(st + kOffQ + off),
+                      desc_mnmajor(ss + kk * 2048, kSsSlabBytes), kIdescO, 1);
+          }
+          umma_commit(bar(BAR_OFULL));
+          // S = diag(D) S_in (already in TMEM) + Ke^T V : M = 128 channels, N = 128, K = 64 rows
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            umma_bf16(tmem + kColS, desc_mnmajor(st + kOffX + kk * 2048, kSlabBytes),
+                      desc_mnmajor(st + kOffV + kk * 2048, kSlabBytes), kIdescS, 1);
+          }
+          umma_commit(bar(BAR_SFULL));
+          umma_commit(bar(BAR_EMPTY0 + s));
+        }
+      }
+    }
+  } else if (warp >= 4 && warp < 8) {
+    // ====================================== state group ======================================
+    const int q4 = warp & 3;
+    const int d = q4 * 32 + lane;                         // state row (key channel) of this thread
+    const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
+    const uint32_t ss_row = base + kOffSs + d * 128;
+    uint32_t g = 0;
+    bool ok = true;
+    for (long long item = blockIdx.x; ok && item < a.n_items; item += gridDim.x) {
+      const Item it = decode_item(a, item);
+      const int n_chunks = (it.len + kC - 1) / kC;
+      const long long srow = it.state_off + (long long)d * a.dv;
+      if (n_chunks == 0) {  // empty sequence: final state = initial state
+        if (a.sT) {
+          for (int j = 0; j < kDVS / 4; ++j) {
+            float4 v4 = a.s0 ? *reinterpret_cast<const float4*>(a.s0 + srow + 4 * j)
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+            *reinterpret_cast<float4*>(a.sT + srow + 4 * j) = v4;
+          }
+        }
+        continue;
+      }
+      for (int c = 0; c < n_chunks; ++c, ++g) {
+        const uint32_t s = g & 1, ph = (g >> 1) & 1, ph1 = g & 1;
+        if (c > 0) {
+          if (!(ok = mbar_wait(bar(BAR_SFULL), ph1 ^ 1, abort_flag, a.hdr))) break;  // chunk g-1
+          tc_fence_after();
+        }
+        if (!(ok = mbar_wait(bar(BAR_GATED0 + s), ph, abort_flag, a.hdr))) break;
+        const float D = sD[s * kDK + d];
+#pragma unroll 1
+        for (int piece = 0; piece < 4; ++piece) {
+          uint32_t r[32];
+          if (c > 0) {
+            tmem_ld32(t_lane + kColS + piece * 32, r);
+            tmem_ld_wait();
+          } else if (a.s0) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float4 v4 = *reinterpret_cast<const float4*>(a.s0 + srow + piece * 32 + 4 * j);
+              r[4 * j] = __float_as_uint(v4.x);
+              r[4 * j + 1] = __float_as_uint(v4.y);
+              r[4 * j + 2] = __float_as_uint(v4.z);
+              r[4 * j + 3] = __float_as_uint(v4.w);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] = 0u;
+          }
+          // bf16 copy of S_in for the readout: MN-major, row d, 64-column slab piece/2
+          const uint32_t slab = ss_row + (piece >> 1) * kSsSlabBytes;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int chunk = (piece & 1) * 4 + j;
+            sts128(slab + ((chunk ^ (d & 7)) << 4),
+                   pack_bf16(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1])),
+                   pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3])),
+                   pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5])),
+                   pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7])));
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * D);
+          tmem_st32(t_lane + kColS + piece * 32, r);
+        }
+        tmem_st_wait();
+        fence_proxy_async();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_SREADY));
+      }
+      if (!ok) break;
+      // final state of this item (also keeps the next item's initial state from racing the MMAs)
+      {
+        const uint32_t last = g - 1;
+        if (!(ok = mbar_wait(bar(BAR_SFULL), last & 1, abort_flag, a.hdr))) break;
+        tc_fence_after();
+        if (a.sT) {
+#pragma unroll 1
+          for (int piece = 0; piece < 4; ++piece) {
+            uint32_t r[32];
+            tmem_ld32(t_lane + kColS + piece * 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              *reinterpret_cast<float4*>(a.sT + srow + piece * 32 + 4 * j) =
+                  make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                              __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+            }
+          }
+        }
+        tc_fence_before();
+      }
+    }
+  } else if (warp >= 8 && warp < 12) {
+    // ================================== score / output group ==================================
+    const int q4 = warp & 3;
+    const int r_row = q4 * 16 + lane;                     // chunk row held by lanes 0..15 (M = 64)
+    const bool has_row = lane < 16;
+    const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
+    __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(a.o);
+    uint32_t g = 0;
+    bool ok = true;
+    for (long long item = blockIdx.x; ok && item < a.n_items; item += gridDim.x) {
+      const Item it = decode_item(a, item);
+      const int n_chunks = (it.len + kC - 1) / kC;
+      for (int c = 0; c < n_chunks; ++c, ++g) {
+        const uint32_t s = g & 1, ph1 = g & 1;
+        const int nr = min(kC, it.len - c * kC);
+        const uint32_t ps_row = base + s * kStageBytes + kOffY + r_row * 128;
+        if (!(ok = mbar_wait(bar(BAR_PFULL), ph1, abort_flag, a.hdr))) break;
+        tc_fence_after();
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r[32];
+          tmem_ld32(t_lane + kColP + half * 32, r);
+          tmem_ld_wait();
+          if (has_row) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int i0 = half * 32 + 8 * j + 2 * e;
+                const float lo = (i0 <= r_row) ? __uint_as_float(r[8 * j + 2 * e]) : 0.f;
+                const float hi = (i0 + 1 <= r_row) ? __uint_as_float(r[8 * j + 2 * e + 1]) : 0.f;
+                w[e] = pack_bf16(lo, hi);
+              }
+              const int chunk = half * 4 + j;
+              sts128(ps_row + ((chunk ^ (r_row & 7)) << 4), w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_PREADY));
+        // output rows of this chunk
+        if (!(ok = mbar_wait(bar(BAR_OFULL), ph1, abort_flag, a.hdr))) break;
+        tc_fence_after();
+        __nv_bfloat16* orow = o + (it.row0 + (long long)c * kC + r_row) * a.dv + it.col0;
+#pragma unroll 1
+        for (int piece = 0; piece < 4; ++piece) {
+          uint32_t r[32];
+          tmem_ld32(t_lane + kColO + piece * 32, r);
+          tmem_ld_wait();
+          if (has_row && r_row < nr) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint4 w;
+              w.x = pack_bf16(a.scale * __uint_as_float(r[8 * j]), a.scale * __uint_as_float(r[8 * j + 1]));
+              w.y = pack_bf16(a.scale * __uint_as_float(r[8 * j + 2]), a.scale * __uint_as_float(r[8 * j + 3]));
+              w.z = pack_bf16(a.scale * __uint_as_float(r[8 * j + 4]), a.scale * __uint_as_float(r[8 * j + 5]));
+              w.w = pack_bf16(a.scale * __uint_as_float(r[8 * j + 6]), a.scale * __uint_as_float(r[8 * j + 7]));
+              *reinterpret_cast<uint4*>(orow + piece * 32 + 8 * j) = w;
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar(BAR_OFREE));
+      }
+    }
+  } else if (warp >= kGateWarp0) {
+    // ======================================= gate group =======================================
+    const int gw = warp - kGateWarp0;                     // rows 8*gw .. 8*gw+7 of the chunk
+    constexpr float kLog2e = 1.4426950408889634f;
+    constexpr float kLg2Ln2 = -0.5287663729448977f;       // log2(ln 2)
+    constexpr float kMinL2a = -64.f * kLog2e;             // per-step decay floor exp(-64)
+    uint32_t g = 0;
+    bool ok = true;
+    for (long long item = blockIdx.x; ok && item < a.n_items; item += gridDim.x) {
+      const Item it = decode_item(a, item);
+      const int n_chunks = (it.len + kC - 1) / kC;
+      for (int c = 0; c < n_chunks; ++c, ++g) {
+        const uint32_t s = g & 1, ph = (g >> 1) & 1;
+        const int nr = min(kC, it.len - c * kC);
+        const uint32_t st = base + s * kStageBytes;
+        if (!(ok = mbar_wait(bar(BAR_FULL0 + s), ph, abort_flag, a.hdr))) break;
+#pragma unroll 1
+        for (int sl = 0; sl < 2; ++sl) {
+          // element (row r, channels 64*sl + 2*lane, +1) sits at this swizzled byte offset
+          const uint32_t slab = st + sl * kSlabBytes;
+          float bq[8][2];   // inclusive in-chunk cumulative log2 decay (own rows only, so far)
+          float eh[8][2];   // log2 ahat
+          float run0 = 0.f, run1 = 0.f;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int r = gw * 8 + j;
+            const uint32_t off = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
+            const uint32_t xw = lds32(slab + kOffX + off), yw = lds32(slab + kOffY + off);
+            const float xs[2] = {__uint_as_float(xw << 16), __uint_as_float(xw & 0xFFFF0000u)};
+            const float ys[2] = {__uint_as_float(yw << 16), __uint_as_float(yw & 0xFFFF0000u)};
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const float u = ex2f(xs[e] * kLog2e);                       // e^x
+              // g * log2(e) = log2(1 + e^x); series when 1 + u would round u away
+              const float sp2 = u < 9.765625e-4f ? u * (kLog2e - 0.72134752f * u) : lg2f(1.f + u);
+              const float tau = rcpf(1.f + ex2f(-ys[e] * kLog2e));
+              float l2a = fmaxf(-sp2 * tau, kMinL2a);
+              float l2h;
+              if (INGATE == RODIMUS_INGATE_POW_G) {
+                l2h = tau * (lg2f(sp2) + kLg2Ln2);                        // tau * log2(g)
+              } else {
+                l2h = tau * (xs[e] * kLog2e - sp2);                       // tau * log2(sigmoid(x))
+              }
+              if (r >= nr) l2a = 0.f;                                     // rows past the sequence
+              if (e == 0) { run0 += l2a; bq[j][0] = run0; } else { run1 += l2a; bq[j][1] = run1; }
+              eh[j][e] = l2h;
+            }
+          }
+          // exclusive prefix over the 8 row groups, and the chunk total
+          float* tot = sTot + sl * (8 * 64);
+          *reinterpret_cast<float2*>(tot + gw * 64 + 2 * lane) = make_float2(run0, run1);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(BAR_GSCAN));
+          if (!(ok = mbar_wait(bar(BAR_GSCAN), (uint32_t)sl, abort_flag, a.hdr))) break;
+          float pre0 = 0.f, pre1 = 0.f, all0 = 0.f, all1 = 0.f;
+#pragma unroll
+          for (int w = 0; w < 8; ++w) {
+            const float2 t = *reinterpret_cast<const float2*>(tot + w * 64 + 2 * lane);
+            if (w < gw) { pre0 += t.x; pre1 += t.y; }
+            all0 += t.x; all1 += t.y;
+          }
+          if (gw == 0) {
+            *reinterpret_cast<float2*>(sD + s * kDK + sl * 64 + 2 * lane) = make_float2(ex2f(all0), ex2f(all1));
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int r = gw * 8 + j;
+            const uint32_t off = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
+            const uint32_t qw = lds32(slab + kOffQ + off), kw = lds32(slab + kOffK + off);
+            const float b0 = bq[j][0] + pre0, b1 = bq[j][1] + pre1;
+            const bool live = r < nr;
+            const float q0 = live ? __uint_as_float(qw << 16) : 0.f;
+            const float q1 = live ? __uint_as_float(qw & 0xFFFF0000u) : 0.f;
+            const float k0 = live ? __uint_as_float(kw << 16) : 0.f;
+            const float k1 = live ? __uint_as_float(kw & 0xFFFF0000u) : 0.f;
+            const uint32_t qt = pack_bf16(q0 * ex2f(b0), q1 * ex2f(b1));
+            const uint32_t kt = pack_bf16(k0 * ex2f(fminf(eh[j][0] - b0, 120.f)),
+                                          k1 * ex2f(fminf(eh[j][1] - b1, 120.f)));
+            const uint32_t ke = pack_bf16(k0 * ex2f(eh[j][0] + (all0 - b0)),
+                                          k1 * ex2f(eh[j][1] + (all1 - b1)));
+            sts32(slab + kOffQ + off, qt);
+            sts32(slab + kOffK + off, kt);
+            sts32(slab + kOffX + off, ke);
+          }
+        }
+        if (!ok) break;
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_GATED0 + s));
+      }
+    }
+  }
+
+  // ------------------------------------------ teardown ------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
+                 : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [rows, cols] bf16 row-major, box = 64 rows x 64 columns (128 bytes), 128-byte swizzle.
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)kC};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool tc_kernel_built() { return true; }
+
+cudaError_t launch_fwd_tc(const rodimus_ddts_fwd_params& p, int* n_launches) {
+  *n_launches = 0;
+  TcArgs a;
+  a.o = p.o; a.s0 = p.s0; a.sT = p.sT; a.cu = p.cu_seqlens;
+  a.hdr = reinterpret_cast<WorkspaceHeader*>(p.workspace);
+  a.order = reinterpret_cast<const int32_t*>(reinterpret_cast<const char*>(p.workspace) +
+                                             sizeof(WorkspaceHeader));
+  a.H = p.H; a.T = p.T; a.dv = p.dv;
+  a.n_seq = p.cu_seqlens ? p.N : p.B;
+  a.slices = p.dv / kDVS;
+  a.n_items = (long long)a.n_seq * p.H * a.slices;
+  a.scale = p.scale;
+  if (a.n_items == 0) return cudaSuccess;
+  const uint64_t rows = (uint64_t)p.B * p.H * p.T;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
+
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+
+  CUtensorMap mq, mk, mx, my, mv;
+  if (rows > 0) {
+    if (!make_map(&mq, p.q, rows, kDK) || !make_map(&mk, p.k, rows, kDK) ||
+        !make_map(&mx, p.gate_x, rows, kDK) || !make_map(&my, p.temp_y, rows, kDK) ||
+        !make_map(&mv, p.v, rows, (uint64_t)p.dv))
+      return cudaErrorUnknown;
+  } else {
+    memset(&mq, 0, sizeof(mq)); mk = mq; mx = mq; my = mq; mv = mq;  // never dereferenced: no chunks
+  }
+  const int grid = (int)(a.n_items < sms ? a.n_items : sms);
+  if (p.ingate == RODIMUS_INGATE_POW_G) {
+    e = cudaFuncSetAttribute(ddts_fwd_tc_kernel<RODIMUS_INGATE_POW_G>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    ddts_fwd_tc_kernel<RODIMUS_INGATE_POW_G><<<grid, kThreads, kSmemBytes, st>>>(mq, mk, mx, my, mv, a);
+  } else {
+    e = cudaFuncSetAttribute(ddts_fwd_tc_kernel<RODIMUS_INGATE_POW_SIGMOID>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    ddts_fwd_tc_kernel<RODIMUS_INGATE_POW_SIGMOID><<<grid, kThreads, kSmemBytes, st>>>(mq, mk, mx, my, mv, a);
+  }
+  *n_launches = 1;
+  return cudaGetLastError();
+}
+
+}  // namespace ddts
