@@ -25,8 +25,8 @@
  *   - Every function returns a rodimus_status.  Argument errors are found on the host before
  *     anything is launched.  Nothing aborts, throws or traps.
  *   - Tensors are contiguous, row-major, last index fastest; pointers are 16-byte aligned.
- *   - Inputs must be finite, with |x|, |y| <= 80.  Per-step decay factors below exp(-64) are
- *     applied as exp(-64) by the bf16 prefill kernel (difference below 2^-92 of the state).
+ *   - Inputs must be finite, with |x|, |y| <= 80.  Per-step decay factors below exp(-60) are
+ *     applied as exp(-60) by the bf16 prefill kernel (difference below 2^-86 of the state).
  */
 #ifndef RODIMUS_DDTS_H_
 #define RODIMUS_DDTS_H_

@@ -46,8 +46,8 @@ constexpr int kOffD = kOffSs + 2 * kSsSlabBytes;         // float [kStages][128]
 constexpr int kOffTot = kOffD + kStages * kDK * 4;       // float [2][8][64]: scan partials
 constexpr int kOffBar = kOffTot + 2 * 8 * 64 * 4;        // mbarriers
 constexpr int kNumBars = 16;
-constexpr int kOffMisc = kOffBar + kNumBars * 8;         // tmem base, abort flag
-constexpr int kSmemUsed = kOffMisc + 16;
+constexpr int kOffMisc = kOffBar + kNumBars * 8;         // control block
+constexpr int kSmemUsed = kOffMisc + 256;
 constexpr int kSmemBytes = kSmemUsed + 1024;             // slack for manual 1024-byte alignment
 
 constexpr int kThreads = 640;
@@ -262,6 +262,36 @@ __device__ __forceinline__ Item decode_item(const TcArgs& a, long long item) {
 // ---------------------------------------------------------------------------------------------
 // kernel
 // ---------------------------------------------------------------------------------------------
+// A "fill" is one 64-row tile of q,k,x,y,v brought into a stage by the producer; a "pass" is a
+// fill the gate group accepted and turned into operands.  The two differ because the chunk
+// length adapts to the data: the anchored factorisation Qt = q 2^{b}, Kt = k ahat 2^{-b} needs
+// the in-chunk decay range max_d(-b_C) to stay below kRange, so when a tile decays faster than
+// that the gate group asks for the same position again with fewer live rows (halving, then
+// doubling back), and the producer, which prefetches speculatively at a stride of 64 rows, is
+// redirected.  Every fill carries the (item, position) it was issued for; fills that no longer
+// match what the gate group expects are released unused.
+struct PassDesc {
+  int stage;      // which stage holds the operands
+  int nr;         // live rows
+  int flags;      // kPassFirst | kPassLast
+  int pad;
+  long long row;  // global row (in the [rows, d] view) of the pass's first token
+};
+constexpr int kPassFirst = 1, kPassLast = 2;
+
+struct Control {            // lives in shared memory
+  uint32_t tmem_base;
+  int abort_flag;
+  int done;                 // gate group has finished every item of this CTA
+  int redir_seq;            // bumped by the gate group after writing redir_j / redir_tpos
+  int redir_j, redir_tpos;  // where the producer must continue (CTA-local item index, token)
+  int pad[2];
+  int tag[2][2];            // per stage: (item index, token position) of the fill it holds
+  int pad2[4];
+  PassDesc pd[4];
+};
+static_assert(sizeof(Control) <= 256, "control block");
+
 template <int INGATE>
 __global__ void __launch_bounds__(kThreads, 1)
 ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -272,8 +302,8 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bars = base + kOffBar;
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + kOffMisc);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + kOffMisc + 4);
+  volatile Control* ctl = reinterpret_cast<volatile Control*>(gbase + kOffMisc);
+  volatile int* abort_flag = &ctl->abort_flag;
   float* sD = reinterpret_cast<float*>(gbase + kOffD);
   float* sTot = reinterpret_cast<float*>(gbase + kOffTot);
 
@@ -283,7 +313,9 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   if (!a.cu && blockIdx.x == 0 && tid == 0) a.hdr->status = RODIMUS_OK;
 
   if (tid == 0) {
-    *abort_flag = 0;
+    ctl->abort_flag = 0;
+    ctl->done = 0;
+    ctl->redir_seq = 0;
     mbar_init(bar(BAR_FULL0), 1);
     mbar_init(bar(BAR_FULL1), 1);
     mbar_init(bar(BAR_EMPTY0), 1);
@@ -307,47 +339,71 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem = ctl->tmem_base;
+  auto item_of = [&](int j) { return (long long)blockIdx.x + (long long)j * gridDim.x; };
 
   if (warp == 0) {
     // ===================================== TMA producer =====================================
     if (lane == 0) {
-      uint32_t g = 0;
+      uint32_t f = 0;         // fills issued
+      int j = 0, tpos = 0;    // speculative position: item index and token
+      int seen = 0;           // last redirect taken
       bool ok = true;
-      for (long long item = blockIdx.x; ok && item < a.n_items; item += gridDim.x) {
-        const Item it = decode_item(a, item);
-        const int n_chunks = (it.len + kC - 1) / kC;
-        for (int c = 0; c < n_chunks; ++c, ++g) {
-          const uint32_t s = g & 1, ph = (g >> 1) & 1;
-          if (!(ok = mbar_wait(bar(BAR_EMPTY0 + s), ph ^ 1, abort_flag, a.hdr))) break;
-          const uint32_t st = base + s * kStageBytes;
-          const uint32_t fb = bar(BAR_FULL0 + s);
-          mbar_expect_tx(fb, kStageBytes);
-          // rows beyond the tensor read as zeros; rows of the next sequence are masked later
-          const long long row = it.row0 + (long long)c * kC;
-          const int y = (int)row;
-          tma_load_2d(st + kOffQ, &map_q, 0, y, fb);
-          tma_load_2d(st + kOffQ + kSlabBytes, &map_q, 64, y, fb);
-          tma_load_2d(st + kOffK, &map_k, 0, y, fb);
-          tma_load_2d(st + kOffK + kSlabBytes, &map_k, 64, y, fb);
-          tma_load_2d(st + kOffX, &map_x, 0, y, fb);
-          tma_load_2d(st + kOffX + kSlabBytes, &map_x, 64, y, fb);
-          tma_load_2d(st + kOffY, &map_y, 0, y, fb);
-          tma_load_2d(st + kOffY + kSlabBytes, &map_y, 64, y, fb);
-          tma_load_2d(st + kOffV, &map_v, it.col0, y, fb);
-          tma_load_2d(st + kOffV + kSlabBytes, &map_v, it.col0 + 64, y, fb);
-        }
-      }
-      // Leave no bulk copy in flight: the last loads are consumed by the gate group before the
-      // other roles reach the final barrier, except after an abort, where we wait here (bounded).
-      if (*abort_flag && g > 0) {
-        const uint32_t last = g - 1;
+      while (ok) {
+        const uint32_t s = f & 1, ph = (f >> 1) & 1;
+        if (!(ok = mbar_wait(bar(BAR_EMPTY0 + s), ph ^ 1, abort_flag, a.hdr))) break;
+        Item it;
+        bool have = false;
         const long long t0 = clock64();
-        while (!mbar_try(bar(BAR_FULL0 + (last & 1)), (last >> 1) & 1) && clock64() - t0 < kWaitCycles) {}
-        if (last > 0) {
-          const uint32_t prev = last - 1;
-          while (!mbar_try(bar(BAR_FULL0 + (prev & 1)), (prev >> 1) & 1) && clock64() - t0 < kWaitCycles) {}
+        while (true) {
+          const int sq = ctl->redir_seq;
+          if (sq != seen) {
+            __threadfence_block();
+            j = ctl->redir_j;
+            tpos = ctl->redir_tpos;
+            seen = sq;
+          }
+          while (item_of(j) < a.n_items) {   // next position that has tokens left
+            it = decode_item(a, item_of(j));
+            if (tpos < it.len) { have = true; break; }
+            ++j;
+            tpos = 0;
+          }
+          if (have || ctl->done || *abort_flag) break;
+          if (clock64() - t0 > kWaitCycles) {
+            ctl->abort_flag = 1;
+            atomicMax(&a.hdr->status, (int)RODIMUS_ERR_TIMEOUT);
+            break;
+          }
+          __nanosleep(100);
         }
+        if (!have) break;
+        ctl->tag[s][0] = j;
+        ctl->tag[s][1] = tpos;
+        const uint32_t st = base + s * kStageBytes;
+        const uint32_t fb = bar(BAR_FULL0 + s);
+        mbar_expect_tx(fb, kStageBytes);
+        // rows beyond the tensor read as zeros; rows of the next sequence are masked later
+        const int y = (int)(it.row0 + tpos);
+        tma_load_2d(st + kOffQ, &map_q, 0, y, fb);
+        tma_load_2d(st + kOffQ + kSlabBytes, &map_q, 64, y, fb);
+        tma_load_2d(st + kOffK, &map_k, 0, y, fb);
+        tma_load_2d(st + kOffK + kSlabBytes, &map_k, 64, y, fb);
+        tma_load_2d(st + kOffX, &map_x, 0, y, fb);
+        tma_load_2d(st + kOffX + kSlabBytes, &map_x, 64, y, fb);
+        tma_load_2d(st + kOffY, &map_y, 0, y, fb);
+        tma_load_2d(st + kOffY + kSlabBytes, &map_y, 64, y, fb);
+        tma_load_2d(st + kOffV, &map_v, it.col0, y, fb);
+        tma_load_2d(st + kOffV + kSlabBytes, &map_v, it.col0 + 64, y, fb);
+        ++f;
+        tpos += kC;
+      }
+      // Leave no bulk copy in flight when the CTA exits: the last two fills' barriers complete
+      // by byte count, whoever consumed them.
+      const long long t1 = clock64();
+      for (uint32_t back = 1; back <= 2 && back <= f; ++back) {
+        const uint32_t ff = f - back;
+        while (!mbar_try(bar(BAR_FULL0 + (ff & 1)), (ff >> 1) & 1) && clock64() - t1 < kWaitCycles) {}
       }
     }
   } else if (warp == 1) {
@@ -359,13 +415,16 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       const uint32_t ss = base + kOffSs;
       uint32_t g = 0;
       bool ok = true;
-      for (long long item = blockIdx.x; ok && item < a.n_items; item += gridDim.x) {
-        const Item it = decode_item(a, item);
-        const int n_chunks = (it.len + kC - 1) / kC;
-        for (int c = 0; c < n_chunks; ++c, ++g) {
-          const uint32_t s = g & 1, ph = (g >> 1) & 1, ph1 = g & 1;
+      for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
+        const Item it = decode_item(a, item_of(j));
+        if (it.len == 0) continue;
+        bool last = false;
+        while (!last) {
+          const uint32_t ph1 = g & 1;
+          if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 1)), (g >> 1) & 1, abort_flag, a.hdr))) break;
+          const uint32_t s = (uint32_t)ctl->pd[g & 3].stage;
+          last = (ctl->pd[g & 3].flags & kPassLast) != 0;
           const uint32_t st = base + s * kStageBytes;
-          if (!(ok = mbar_wait(bar(BAR_GATED0 + s), ph, abort_flag, a.hdr))) break;
           tc_fence_after();
           // P = Qt Kt^T : M = 64 (rows r), N = 64 (rows i), K = 128 channels
 #pragma unroll
@@ -401,6 +460,7 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           }
           umma_commit(bar(BAR_SFULL));
           umma_commit(bar(BAR_EMPTY0 + s));
+          ++g;
         }
       }
     }
@@ -412,72 +472,76 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const uint32_t ss_row = base + kOffSs + d * 128;
     uint32_t g = 0;
     bool ok = true;
-    for (long long item = blockIdx.x; ok && item < a.n_items; item += gridDim.x) {
-      const Item it = decode_item(a, item);
-      const int n_chunks = (it.len + kC - 1) / kC;
+    for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
+      const Item it = decode_item(a, item_of(j));
       const long long srow = it.state_off + (long long)d * a.dv;
-      if (n_chunks == 0) {  // empty sequence: final state = initial state
+      if (it.len == 0) {  // empty sequence: final state = initial state
         if (a.sT) {
-          for (int j = 0; j < kDVS / 4; ++j) {
-            float4 v4 = a.s0 ? *reinterpret_cast<const float4*>(a.s0 + srow + 4 * j)
+          for (int c4 = 0; c4 < kDVS / 4; ++c4) {
+            float4 v4 = a.s0 ? *reinterpret_cast<const float4*>(a.s0 + srow + 4 * c4)
                              : make_float4(0.f, 0.f, 0.f, 0.f);
-            *reinterpret_cast<float4*>(a.sT + srow + 4 * j) = v4;
+            *reinterpret_cast<float4*>(a.sT + srow + 4 * c4) = v4;
           }
         }
         continue;
       }
-      for (int c = 0; c < n_chunks; ++c, ++g) {
-        const uint32_t s = g & 1, ph = (g >> 1) & 1, ph1 = g & 1;
-        if (c > 0) {
-          if (!(ok = mbar_wait(bar(BAR_SFULL), ph1 ^ 1, abort_flag, a.hdr))) break;  // chunk g-1
+      bool last = false, first = true;
+      while (!last) {
+        const uint32_t ph1 = g & 1;
+        if (!first) {
+          if (!(ok = mbar_wait(bar(BAR_SFULL), ph1 ^ 1, abort_flag, a.hdr))) break;  // pass g-1
           tc_fence_after();
         }
-        if (!(ok = mbar_wait(bar(BAR_GATED0 + s), ph, abort_flag, a.hdr))) break;
+        if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 1)), (g >> 1) & 1, abort_flag, a.hdr))) break;
+        const int s = ctl->pd[g & 3].stage;
+        last = (ctl->pd[g & 3].flags & kPassLast) != 0;
         const float D = sD[s * kDK + d];
 #pragma unroll 1
         for (int piece = 0; piece < 4; ++piece) {
           uint32_t r[32];
-          if (c > 0) {
+          if (!first) {
             tmem_ld32(t_lane + kColS + piece * 32, r);
             tmem_ld_wait();
           } else if (a.s0) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const float4 v4 = *reinterpret_cast<const float4*>(a.s0 + srow + piece * 32 + 4 * j);
-              r[4 * j] = __float_as_uint(v4.x);
-              r[4 * j + 1] = __float_as_uint(v4.y);
-              r[4 * j + 2] = __float_as_uint(v4.z);
-              r[4 * j + 3] = __float_as_uint(v4.w);
+            for (int c4 = 0; c4 < 8; ++c4) {
+              const float4 v4 = *reinterpret_cast<const float4*>(a.s0 + srow + piece * 32 + 4 * c4);
+              r[4 * c4] = __float_as_uint(v4.x);
+              r[4 * c4 + 1] = __float_as_uint(v4.y);
+              r[4 * c4 + 2] = __float_as_uint(v4.z);
+              r[4 * c4 + 3] = __float_as_uint(v4.w);
             }
           } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) r[j] = 0u;
+            for (int c4 = 0; c4 < 32; ++c4) r[c4] = 0u;
           }
           // bf16 copy of S_in for the readout: MN-major, row d, 64-column slab piece/2
           const uint32_t slab = ss_row + (piece >> 1) * kSsSlabBytes;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int chunk = (piece & 1) * 4 + j;
+          for (int c8 = 0; c8 < 4; ++c8) {
+            const int chunk = (piece & 1) * 4 + c8;
             sts128(slab + ((chunk ^ (d & 7)) << 4),
-                   pack_bf16(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1])),
-                   pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3])),
-                   pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5])),
-                   pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7])));
+                   pack_bf16(__uint_as_float(r[8 * c8]), __uint_as_float(r[8 * c8 + 1])),
+                   pack_bf16(__uint_as_float(r[8 * c8 + 2]), __uint_as_float(r[8 * c8 + 3])),
+                   pack_bf16(__uint_as_float(r[8 * c8 + 4]), __uint_as_float(r[8 * c8 + 5])),
+                   pack_bf16(__uint_as_float(r[8 * c8 + 6]), __uint_as_float(r[8 * c8 + 7])));
           }
 #pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * D);
+          for (int c4 = 0; c4 < 32; ++c4) r[c4] = __float_as_uint(__uint_as_float(r[c4]) * D);
           tmem_st32(t_lane + kColS + piece * 32, r);
         }
         tmem_st_wait();
         fence_proxy_async();
         tc_fence_before();
         mbar_arrive(bar(BAR_SREADY));
+        first = false;
+        ++g;
       }
       if (!ok) break;
       // final state of this item (also keeps the next item's initial state from racing the MMAs)
       {
-        const uint32_t last = g - 1;
-        if (!(ok = mbar_wait(bar(BAR_SFULL), last & 1, abort_flag, a.hdr))) break;
+        const uint32_t lastg = g - 1;
+        if (!(ok = mbar_wait(bar(BAR_SFULL), lastg & 1, abort_flag, a.hdr))) break;
         tc_fence_after();
         if (a.sT) {
 #pragma unroll 1
@@ -486,10 +550,10 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             tmem_ld32(t_lane + kColS + piece * 32, r);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              *reinterpret_cast<float4*>(a.sT + srow + piece * 32 + 4 * j) =
-                  make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                              __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+            for (int c4 = 0; c4 < 8; ++c4) {
+              *reinterpret_cast<float4*>(a.sT + srow + piece * 32 + 4 * c4) =
+                  make_float4(__uint_as_float(r[4 * c4]), __uint_as_float(r[4 * c4 + 1]),
+                              __uint_as_float(r[4 * c4 + 2]), __uint_as_float(r[4 * c4 + 3]));
             }
           }
         }
@@ -505,14 +569,18 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(a.o);
     uint32_t g = 0;
     bool ok = true;
-    for (long long item = blockIdx.x; ok && item < a.n_items; item += gridDim.x) {
-      const Item it = decode_item(a, item);
-      const int n_chunks = (it.len + kC - 1) / kC;
-      for (int c = 0; c < n_chunks; ++c, ++g) {
-        const uint32_t s = g & 1, ph1 = g & 1;
-        const int nr = min(kC, it.len - c * kC);
-        const uint32_t ps_row = base + s * kStageBytes + kOffY + r_row * 128;
+    for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
+      const Item it = decode_item(a, item_of(j));
+      if (it.len == 0) continue;
+      bool last = false;
+      while (!last) {
+        const uint32_t ph1 = g & 1;
         if (!(ok = mbar_wait(bar(BAR_PFULL), ph1, abort_flag, a.hdr))) break;
+        const int s = ctl->pd[g & 3].stage;
+        const int nr = ctl->pd[g & 3].nr;
+        const long long row = ctl->pd[g & 3].row;
+        last = (ctl->pd[g & 3].flags & kPassLast) != 0;
+        const uint32_t ps_row = base + s * kStageBytes + kOffY + r_row * 128;
         tc_fence_after();
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
@@ -521,16 +589,16 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           tmem_ld_wait();
           if (has_row) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int c8 = 0; c8 < 4; ++c8) {
               uint32_t w[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const int i0 = half * 32 + 8 * j + 2 * e;
-                const float lo = (i0 <= r_row) ? __uint_as_float(r[8 * j + 2 * e]) : 0.f;
-                const float hi = (i0 + 1 <= r_row) ? __uint_as_float(r[8 * j + 2 * e + 1]) : 0.f;
+                const int i0 = half * 32 + 8 * c8 + 2 * e;
+                const float lo = (i0 <= r_row) ? __uint_as_float(r[8 * c8 + 2 * e]) : 0.f;
+                const float hi = (i0 + 1 <= r_row) ? __uint_as_float(r[8 * c8 + 2 * e + 1]) : 0.f;
                 w[e] = pack_bf16(lo, hi);
               }
-              const int chunk = half * 4 + j;
+              const int chunk = half * 4 + c8;
               sts128(ps_row + ((chunk ^ (r_row & 7)) << 4), w[0], w[1], w[2], w[3]);
             }
           }
@@ -538,10 +606,10 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         fence_proxy_async();
         tc_fence_before();
         mbar_arrive(bar(BAR_PREADY));
-        // output rows of this chunk
+        // output rows of this pass
         if (!(ok = mbar_wait(bar(BAR_OFULL), ph1, abort_flag, a.hdr))) break;
         tc_fence_after();
-        __nv_bfloat16* orow = o + (it.row0 + (long long)c * kC + r_row) * a.dv + it.col0;
+        __nv_bfloat16* orow = o + (row + r_row) * a.dv + it.col0;
 #pragma unroll 1
         for (int piece = 0; piece < 4; ++piece) {
           uint32_t r[32];
@@ -549,36 +617,60 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           tmem_ld_wait();
           if (has_row && r_row < nr) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int c8 = 0; c8 < 4; ++c8) {
               uint4 w;
-              w.x = pack_bf16(a.scale * __uint_as_float(r[8 * j]), a.scale * __uint_as_float(r[8 * j + 1]));
-              w.y = pack_bf16(a.scale * __uint_as_float(r[8 * j + 2]), a.scale * __uint_as_float(r[8 * j + 3]));
-              w.z = pack_bf16(a.scale * __uint_as_float(r[8 * j + 4]), a.scale * __uint_as_float(r[8 * j + 5]));
-              w.w = pack_bf16(a.scale * __uint_as_float(r[8 * j + 6]), a.scale * __uint_as_float(r[8 * j + 7]));
-              *reinterpret_cast<uint4*>(orow + piece * 32 + 8 * j) = w;
+              w.x = pack_bf16(a.scale * __uint_as_float(r[8 * c8]), a.scale * __uint_as_float(r[8 * c8 + 1]));
+              w.y = pack_bf16(a.scale * __uint_as_float(r[8 * c8 + 2]), a.scale * __uint_as_float(r[8 * c8 + 3]));
+              w.z = pack_bf16(a.scale * __uint_as_float(r[8 * c8 + 4]), a.scale * __uint_as_float(r[8 * c8 + 5]));
+              w.w = pack_bf16(a.scale * __uint_as_float(r[8 * c8 + 6]), a.scale * __uint_as_float(r[8 * c8 + 7]));
+              *reinterpret_cast<uint4*>(orow + piece * 32 + 8 * c8) = w;
             }
           }
         }
         tc_fence_before();
         mbar_arrive(bar(BAR_OFREE));
+        ++g;
       }
     }
   } else if (warp >= kGateWarp0) {
     // ======================================= gate group =======================================
-    const int gw = warp - kGateWarp0;                     // rows 8*gw .. 8*gw+7 of the chunk
+    const int gw = warp - kGateWarp0;                     // rows 8*gw .. 8*gw+7 of the tile
     constexpr float kLog2e = 1.4426950408889634f;
     constexpr float kLg2Ln2 = -0.5287663729448977f;       // log2(ln 2)
-    constexpr float kMinL2a = -64.f * kLog2e;             // per-step decay floor exp(-64)
-    uint32_t g = 0;
+    constexpr float kRange = 60.f * kLog2e;               // largest in-chunk decay range, log2 units
+    uint32_t f = 0, g = 0, sc = 0;                        // fills seen, passes published, scan syncs
     bool ok = true;
-    for (long long item = blockIdx.x; ok && item < a.n_items; item += gridDim.x) {
-      const Item it = decode_item(a, item);
-      const int n_chunks = (it.len + kC - 1) / kC;
-      for (int c = 0; c < n_chunks; ++c, ++g) {
-        const uint32_t s = g & 1, ph = (g >> 1) & 1;
-        const int nr = min(kC, it.len - c * kC);
+    auto group_sync = [&]() -> bool {                     // bounded barrier over the 8 gate warps
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_GSCAN));
+      const bool r = mbar_wait(bar(BAR_GSCAN), sc & 1, abort_flag, a.hdr);
+      ++sc;
+      return r;
+    };
+    auto redirect = [&](int jj, int tt) {                 // one thread; before the stage is released
+      ctl->redir_j = jj;
+      ctl->redir_tpos = tt;
+      __threadfence_block();
+      ctl->redir_seq = ctl->redir_seq + 1;
+    };
+    for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
+      const Item it = decode_item(a, item_of(j));
+      int tpos = 0, lcap = kC;
+      bool first = true;
+      while (ok && tpos < it.len) {
+        const uint32_t s = f & 1, ph = (f >> 1) & 1;
         const uint32_t st = base + s * kStageBytes;
         if (!(ok = mbar_wait(bar(BAR_FULL0 + s), ph, abort_flag, a.hdr))) break;
+        ++f;
+        if (ctl->tag[s][0] != j || ctl->tag[s][1] != tpos) {
+          // speculative fill for a position we are not at: hand the stage back unused
+          if (!(ok = group_sync())) break;
+          if (gw == 0 && lane == 0) mbar_arrive(bar(BAR_EMPTY0 + s));
+          continue;
+        }
+        const int left = it.len - tpos;
+        const int nr = min(min(kC, left), lcap);
+        bool viol = false;
 #pragma unroll 1
         for (int sl = 0; sl < 2; ++sl) {
           // element (row r, channels 64*sl + 2*lane, +1) sits at this swizzled byte offset
@@ -587,8 +679,8 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           float eh[8][2];   // log2 ahat
           float run0 = 0.f, run1 = 0.f;
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int r = gw * 8 + j;
+          for (int i = 0; i < 8; ++i) {
+            const int r = gw * 8 + i;
             const uint32_t off = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
             const uint32_t xw = lds32(slab + kOffX + off), yw = lds32(slab + kOffY + off);
             const float xs[2] = {__uint_as_float(xw << 16), __uint_as_float(xw & 0xFFFF0000u)};
@@ -599,24 +691,22 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
               // g * log2(e) = log2(1 + e^x); series when 1 + u would round u away
               const float sp2 = u < 9.765625e-4f ? u * (kLog2e - 0.72134752f * u) : lg2f(1.f + u);
               const float tau = rcpf(1.f + ex2f(-ys[e] * kLog2e));
-              float l2a = fmaxf(-sp2 * tau, kMinL2a);
+              float l2a = fmaxf(-sp2 * tau, -kRange);                     // per-step floor exp(-60)
               float l2h;
               if (INGATE == RODIMUS_INGATE_POW_G) {
                 l2h = tau * (lg2f(sp2) + kLg2Ln2);                        // tau * log2(g)
               } else {
                 l2h = tau * (xs[e] * kLog2e - sp2);                       // tau * log2(sigmoid(x))
               }
-              if (r >= nr) l2a = 0.f;                                     // rows past the sequence
-              if (e == 0) { run0 += l2a; bq[j][0] = run0; } else { run1 += l2a; bq[j][1] = run1; }
-              eh[j][e] = l2h;
+              if (r >= nr) l2a = 0.f;                                     // rows past the pass
+              if (e == 0) { run0 += l2a; bq[i][0] = run0; } else { run1 += l2a; bq[i][1] = run1; }
+              eh[i][e] = l2h;
             }
           }
           // exclusive prefix over the 8 row groups, and the chunk total
           float* tot = sTot + sl * (8 * 64);
           *reinterpret_cast<float2*>(tot + gw * 64 + 2 * lane) = make_float2(run0, run1);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar(BAR_GSCAN));
-          if (!(ok = mbar_wait(bar(BAR_GSCAN), (uint32_t)sl, abort_flag, a.hdr))) break;
+          if (!(ok = group_sync())) break;
           float pre0 = 0.f, pre1 = 0.f, all0 = 0.f, all1 = 0.f;
 #pragma unroll
           for (int w = 0; w < 8; ++w) {
@@ -624,36 +714,57 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (w < gw) { pre0 += t.x; pre1 += t.y; }
             all0 += t.x; all1 += t.y;
           }
-          if (gw == 0) {
-            *reinterpret_cast<float2*>(sD + s * kDK + sl * 64 + 2 * lane) = make_float2(ex2f(all0), ex2f(all1));
-          }
+          // every warp sees every channel's total, so all eight reach the same verdict
+          viol = __any_sync(0xffffffffu, all0 < -kRange || all1 < -kRange) && nr > 1;
+          if (viol) break;
+          const float D0 = ex2f(all0), D1 = ex2f(all1);
+          if (gw == 0) *reinterpret_cast<float2*>(sD + s * kDK + sl * 64 + 2 * lane) = make_float2(D0, D1);
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int r = gw * 8 + j;
+          for (int i = 0; i < 8; ++i) {
+            const int r = gw * 8 + i;
             const uint32_t off = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
             const uint32_t qw = lds32(slab + kOffQ + off), kw = lds32(slab + kOffK + off);
-            const float b0 = bq[j][0] + pre0, b1 = bq[j][1] + pre1;
+            const float b0 = bq[i][0] + pre0, b1 = bq[i][1] + pre1;
             const bool live = r < nr;
             const float q0 = live ? __uint_as_float(qw << 16) : 0.f;
             const float q1 = live ? __uint_as_float(qw & 0xFFFF0000u) : 0.f;
             const float k0 = live ? __uint_as_float(kw << 16) : 0.f;
             const float k1 = live ? __uint_as_float(kw & 0xFFFF0000u) : 0.f;
-            const uint32_t qt = pack_bf16(q0 * ex2f(b0), q1 * ex2f(b1));
-            const uint32_t kt = pack_bf16(k0 * ex2f(fminf(eh[j][0] - b0, 120.f)),
-                                          k1 * ex2f(fminf(eh[j][1] - b1, 120.f)));
-            const uint32_t ke = pack_bf16(k0 * ex2f(eh[j][0] + (all0 - b0)),
-                                          k1 * ex2f(eh[j][1] + (all1 - b1)));
-            sts32(slab + kOffQ + off, qt);
-            sts32(slab + kOffK + off, kt);
-            sts32(slab + kOffX + off, ke);
+            const float kt0 = k0 * ex2f(eh[i][0] - b0), kt1 = k1 * ex2f(eh[i][1] - b1);
+            sts32(slab + kOffQ + off, pack_bf16(q0 * ex2f(b0), q1 * ex2f(b1)));
+            sts32(slab + kOffK + off, pack_bf16(kt0, kt1));
+            sts32(slab + kOffX + off, pack_bf16(kt0 * D0, kt1 * D1));       // 2^{b_C - b_i} = 2^{-b_i} D
           }
         }
         if (!ok) break;
+        if (viol) {
+          // decays too fast for 'nr' rows at once: ask for this position again, fewer rows
+          lcap = max(1, nr >> 1);
+          if (!(ok = group_sync())) break;
+          if (gw == 0 && lane == 0) {
+            redirect(j, tpos);
+            mbar_arrive(bar(BAR_EMPTY0 + s));
+          }
+          continue;
+        }
+        if (gw == 0 && lane == 0) {
+          volatile PassDesc* pd = &ctl->pd[g & 3];
+          pd->stage = (int)s;
+          pd->nr = nr;
+          pd->flags = (first ? kPassFirst : 0) | (nr == left ? kPassLast : 0);
+          pd->row = it.row0 + tpos;
+          if (nr < min(kC, left)) redirect(j, tpos + nr);   // the prefetcher assumed 64 rows
+        }
         fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_GATED0 + s));
+        if (lane == 0) mbar_arrive(bar(BAR_GATED0 + (g & 1)));
+        ++g;
+        first = false;
+        tpos += nr;
+        if (lcap < kC) lcap = min(kC, lcap * 2);
       }
     }
+    if (gw == 0 && lane == 0) ctl->done = 1;
   }
 
   // ------------------------------------------ teardown ------------------------------------------
