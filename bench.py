@@ -215,22 +215,19 @@ def run_ours(args, workload, p):
     import torch
     import torch.distributed as dist
     import paper_2410_06577_b200 as rd
+    from paper_2410_06577_b200 import dist as rdist
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = rdist.env_rank()
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=device)
+    rdist.init("nccl", device)
     peaks, peak_kind = load_peaks()
     decode = workload == "cfg3"
     tdt = torch.bfloat16 if p.dtype == "bf16" else torch.float32
     stream = torch.cuda.current_stream()
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        rdist.barrier()
         torch.cuda.synchronize()
 
     if decode:
@@ -303,12 +300,7 @@ def run_ours(args, workload, p):
             fn(warmup + i)
         ev1.record(stream)
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return rdist.max_over_ranks(ev0.elapsed_time(ev1), device)
 
     step(0)
     torch.cuda.synchronize()
