@@ -740,6 +740,7 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         if (viol) {
           // decays too fast for 'nr' rows at once: ask for this position again, fewer rows
           lcap = max(1, nr >> 1);
+          fence_proxy_async();   // slab 0 may already be rewritten; the refill is a bulk copy
           if (!(ok = group_sync())) break;
           if (gw == 0 && lane == 0) {
             redirect(j, tpos);
