@@ -25,8 +25,9 @@ cudaError_t launch_step(const rodimus_ddts_step_params& p, int* n_launches);
 cudaError_t launch_plan(const rodimus_ddts_fwd_params& p, int* n_launches);
 cudaError_t launch_fwd_simt(const rodimus_ddts_fwd_params& p, int* n_launches);
 cudaError_t launch_fwd_tc(const rodimus_ddts_fwd_params& p, int* n_launches);
+cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches);
 bool fwd_tc_supported(const rodimus_ddts_fwd_params& p);
-bool tc_kernel_built();
+bool fwd_pair_supported(const rodimus_ddts_fwd_params& p);
 
 // ---------------------------------------------------------------------------------------------
 // Element access for the two token dtypes.

@@ -1,0 +1,822 @@
+// Chunked DDTS prefill on the 5th-generation tensor cores for dv a multiple of 256: two CTAs of
+// a thread-block cluster work on one (sequence, head) and SHARE the gate math.
+//
+// Same chunk algebra as ddts_fwd_tc.cu (appendix "Chunkwise Parallel Representation of the
+// Rodimus Block"; chunk length 64, log2 domain, decays anchored at the chunk start):
+//   Qt_r = q_r 2^{b_r}     Kt_i = k_i ahat_i 2^{-b_i}     Ke_i = Kt_i 2^{b_C}
+//   P = mask(Qt Kt^T)      O = P V + Qt S_in              S_out = diag(2^{b_C}) S_in + Ke^T V
+// Every quantity that depends on the gates is per key channel and independent of the value
+// column, so the two CTAs that own the two 128-column halves of a 256-column slab of the state
+// would otherwise repeat the whole softplus / sigmoid / log / exp2 pipeline.  Here CTA c of the
+// pair loads q,k,x,y for key channels 64c..64c+63 only, turns them into Qt, Kt, Ke in place, and
+// copies those three 8 KiB slabs (plus the 64 chunk decays) into the other CTA's shared memory
+// with bulk shared-to-shared copies that complete on an mbarrier over there.  Each CTA then runs
+// the same three contractions as the single-CTA kernel on its own 128 value columns, taking
+// half of the K (or M) extent from its own slab and half from the received one.
+//
+// The pair advances in lockstep: which rows form a pass is decided from the decay totals of all
+// 128 channels, so each CTA sends its verdict along with its chunk decays and both take the OR.
+//
+// Roles in one CTA (26 warps), connected by mbarriers; every wait is bounded:
+//   warp 0        TMA producer (own channel slab of q,k,x,y and both slabs of the v slice)
+//   warp 1        tcgen05.mma issuer, owns the TMEM allocation
+//   warps 2-5     state group: TMEM <-> registers trip of S, initial / final state I/O
+//   warps 6-9     score / output group
+//   warps 10-25   gate group: 4 rows x 2 channels per thread
+#include <cuda.h>
+
+#include <cstring>
+
+#include "ddts_common.cuh"
+#include "ddts_tc_ptx.cuh"
+
+namespace ddts {
+namespace {
+
+constexpr int kC = 64;                        // chunk rows
+constexpr int kDK = 128;                      // key channels
+constexpr int kCH = 64;                       // key channels whose gates one CTA computes
+constexpr int kDVS = 128;                     // value columns per CTA
+constexpr int kSlabBytes = kC * 128;          // [64 rows][64 bf16] = 8 KiB, 128-byte swizzled
+// one stage of the TMA ring: own-channel slabs of q,k,x,y and the two slabs of v
+constexpr int kStQ = 0, kStK = kSlabBytes, kStX = 2 * kSlabBytes, kStY = 3 * kSlabBytes,
+              kStV = 4 * kSlabBytes;
+constexpr int kStageBytes = 6 * kSlabBytes;   // 48 KiB
+// one receive buffer: the partner's Qt, Kt, Ke slabs
+constexpr int kRxQ = 0, kRxK = kSlabBytes, kRxX = 2 * kSlabBytes;
+constexpr int kRxBytes = 3 * kSlabBytes;      // 24 KiB
+constexpr int kStages = 2, kRxBufs = 2;
+constexpr int kOperandBytes = kStages * kStageBytes + kRxBufs * kRxBytes;  // 144 KiB
+constexpr int kSsSlabBytes = kDK * 128;       // [128 rows][64 bf16]
+constexpr int kOffSs = kOperandBytes;                     // bf16 copy of the state, 2 slabs
+constexpr int kOffD = kOffSs + 2 * kSsSlabBytes;          // float [kStages][64]: own 2^{b_C}
+constexpr int kBlkFloats = 68;                            // 64 decays, verdict, stage, 2 pad
+constexpr int kBlkBytes = kBlkFloats * 4;                 // 272 B, a multiple of 16
+constexpr int kOffTx = kOffD + kStages * kCH * 4;         // float [2][68]: block to send
+constexpr int kOffRx = kOffTx + kRxBufs * kBlkBytes;      // float [2][68]: block received
+constexpr int kGateWarp0 = 10, kGateWarps = 16;
+constexpr int kOffTot = kOffRx + kRxBufs * kBlkBytes;     // float [2][16][64]: scan partials
+constexpr int kOffBar = kOffTot + 2 * kGateWarps * kCH * 4;
+constexpr int kNumBars = 24;
+constexpr int kOffMisc = kOffBar + kNumBars * 8;          // control block
+constexpr int kSmemUsed = kOffMisc + 256;
+constexpr int kSmemBytes = kSmemUsed + 1024;              // slack for manual 1024-byte alignment
+static_assert(kOffTx % 16 == 0 && kOffRx % 16 == 0 && kBlkBytes % 16 == 0, "bulk copy alignment");
+static_assert(kSmemBytes <= 232448, "shared memory budget");
+
+constexpr int kThreads = 32 * (kGateWarp0 + kGateWarps);  // 832
+constexpr int kStateWarp0 = 2, kScoreWarp0 = 6;
+
+// TMEM columns (fp32 words): state, output, scores
+constexpr uint32_t kColS = 0, kColO = 128, kColP = 256, kTmemCols = 512;
+
+// mbarrier indices
+enum { BAR_FULL0 = 0, BAR_FULL1,      // TMA fill landed                          (1 + bytes)
+       BAR_EMPTY0, BAR_EMPTY1,        // stage reusable: own release + partner's receipt    (2)
+       BAR_GATED0, BAR_GATED1,        // pass published by the gate group                  (16)
+       BAR_PEER0, BAR_PEER1,          // partner's three slabs landed               (1 + bytes)
+       BAR_VERD0, BAR_VERD1,          // partner's decay block landed               (1 + bytes)
+       BAR_RXFREE0, BAR_RXFREE1,      // partner is done with ITS receive buffer            (1)
+       BAR_PFULL, BAR_PREADY, BAR_SREADY, BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN };
+
+struct PairArgs {
+  void* o;
+  const float* s0;
+  float* sT;
+  const int32_t* cu;
+  const int32_t* order;
+  WorkspaceHeader* hdr;
+  int H, T, dv, n_seq, pairs;
+  long long n_items;     // (sequence, head, 256-column slab)
+  float scale;
+};
+
+struct Item {
+  long long row0;      // first global row (in the [rows, d] view) of this sequence and head
+  long long state_off; // element offset of this CTA's state slice (row 0, first own column)
+  int len;             // tokens
+  int col0;            // first value column of this CTA
+};
+
+__device__ __forceinline__ Item decode_item(const PairArgs& a, long long item, int rank) {
+  Item it;
+  const int pair = (int)(item % a.pairs);
+  const long long sh = item / a.pairs;
+  const int h = (int)(sh % a.H);
+  long long n = sh / a.H;
+  if (a.cu) {
+    n = a.order[n];
+    int lo = a.cu[n], hi = a.cu[n + 1];
+    lo = lo < 0 ? 0 : (lo > a.T ? a.T : lo);
+    hi = hi < lo ? lo : (hi > a.T ? a.T : hi);
+    it.row0 = (long long)h * a.T + lo;
+    it.len = hi - lo;
+  } else {
+    it.row0 = (n * a.H + h) * (long long)a.T;
+    it.len = a.T;
+  }
+  it.col0 = (pair * 2 + rank) * kDVS;
+  it.state_off = (n * a.H + h) * (long long)kDK * a.dv + it.col0;
+  return it;
+}
+
+// A "fill" is one 64-row tile brought into a stage by the producer; an "attempt" is a fill at
+// the position the gate group expects (the producer prefetches speculatively, so some fills are
+// not); a "pass" is an attempt both CTAs accepted.  Fill counters are private to a CTA; attempt
+// and pass counters advance identically in both, which is what the receive buffers and their
+// barriers are indexed by.
+struct PassDesc {
+  int stage;      // which stage holds the own-channel operands and v
+  int nr;         // live rows
+  int flags;      // kPassLast
+  int rx;         // which receive buffer holds the partner's operands
+  int rxph;       // parity of that buffer's barrier phase
+  int pad;
+  long long row;  // global row (in the [rows, d] view) of the pass's first token
+};
+constexpr int kPassLast = 2;
+
+struct Control {            // lives in shared memory
+  uint32_t tmem_base;
+  int abort_flag;
+  int done;                 // gate group has finished every item of this CTA
+  int redir_seq;            // bumped by the gate group after writing redir_j / redir_tpos
+  int redir_j, redir_tpos;  // where the producer must continue (CTA-local item index, token)
+  int pad[2];
+  int tag[2][2];            // per stage: (item index, token position) of the fill it holds
+  int pad2[4];
+  PassDesc pd[4];
+};
+static_assert(sizeof(Control) <= 256, "control block");
+
+template <int INGATE>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                     const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
+                     const __grid_constant__ CUtensorMap map_v, const PairArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + kOffBar;
+  auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+  volatile Control* ctl = reinterpret_cast<volatile Control*>(gbase + kOffMisc);
+  volatile int* abort_flag = &ctl->abort_flag;
+  float* sD = reinterpret_cast<float*>(gbase + kOffD);
+  volatile float* sTx = reinterpret_cast<volatile float*>(gbase + kOffTx);
+  volatile float* sRx = reinterpret_cast<volatile float*>(gbase + kOffRx);
+  float* sTot = reinterpret_cast<float*>(gbase + kOffTot);
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31;
+  const int rank = (int)cluster_ctarank();     // 0 or 1: which key-channel half and dv half
+  const int peer = rank ^ 1;
+  // The state update takes Ke for all 128 channels as ONE operand whose two 64-channel groups
+  // must sit at increasing addresses: channels 0..63 first.  So the CTA that owns the low
+  // channels keeps its stages below its receive buffers and the other CTA the opposite.
+  const uint32_t stage_base = base + (rank == 0 ? 0u : (uint32_t)(kRxBufs * kRxBytes));
+  const uint32_t rx_base = base + (rank == 0 ? (uint32_t)(kStages * kStageBytes) : 0u);
+  const uint32_t peer_rx_base = base + (peer == 0 ? (uint32_t)(kStages * kStageBytes) : 0u);
+
+  if (!a.cu && blockIdx.x == 0 && tid == 0) a.hdr->status = RODIMUS_OK;
+
+  if (tid == 0) {
+    ctl->abort_flag = 0;
+    ctl->done = 0;
+    ctl->redir_seq = 0;
+    mbar_init(bar(BAR_FULL0), 1);
+    mbar_init(bar(BAR_FULL1), 1);
+    mbar_init(bar(BAR_EMPTY0), 2);
+    mbar_init(bar(BAR_EMPTY1), 2);
+    mbar_init(bar(BAR_GATED0), kGateWarps);
+    mbar_init(bar(BAR_GATED1), kGateWarps);
+    mbar_init(bar(BAR_PEER0), 1);
+    mbar_init(bar(BAR_PEER1), 1);
+    mbar_init(bar(BAR_VERD0), 1);
+    mbar_init(bar(BAR_VERD1), 1);
+    mbar_init(bar(BAR_RXFREE0), 1);
+    mbar_init(bar(BAR_RXFREE1), 1);
+    mbar_init(bar(BAR_PFULL), 1);
+    mbar_init(bar(BAR_PREADY), 128);
+    mbar_init(bar(BAR_SREADY), 128);
+    mbar_init(bar(BAR_SFULL), 1);
+    mbar_init(bar(BAR_OFULL), 1);
+    mbar_init(bar(BAR_OFREE), 128);
+    mbar_init(bar(BAR_GSCAN), kGateWarps);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(base + kOffMisc), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  // both CTAs' barriers exist before either touches the other's shared memory
+  cluster_arrive();
+  cluster_wait();
+  const uint32_t tmem = ctl->tmem_base;
+  const long long n_pairs_grid = gridDim.x >> 1;
+  const long long pair_id = blockIdx.x >> 1;
+  auto item_of = [&](int j) { return pair_id + (long long)j * n_pairs_grid; };
+
+  if (warp == 0) {
+    // ===================================== TMA producer =====================================
+    if (lane == 0) {
+      uint32_t f = 0;         // fills issued
+      int j = 0, tpos = 0;    // speculative position: item index and token
+      int seen = 0;           // last redirect taken
+      bool ok = true;
+      while (ok) {
+        const uint32_t s = f & 1, ph = (f >> 1) & 1;
+        if (!(ok = mbar_wait_cluster(bar(BAR_EMPTY0 + s), ph ^ 1, abort_flag, a.hdr))) break;
+        Item it;
+        bool have = false;
+        const long long t0 = clock64();
+        while (true) {
+          const int sq = ctl->redir_seq;
+          if (sq != seen) {
+            __threadfence_block();
+            j = ctl->redir_j;
+            tpos = ctl->redir_tpos;
+            seen = sq;
+          }
+          while (item_of(j) < a.n_items) {   // next position that has tokens left
+            it = decode_item(a, item_of(j), rank);
+            if (tpos < it.len) { have = true; break; }
+            ++j;
+            tpos = 0;
+          }
+          if (have || ctl->done || *abort_flag) break;
+          if (clock64() - t0 > kWaitCycles) {
+            ctl->abort_flag = 1;
+            atomicMax(&a.hdr->status, (int)RODIMUS_ERR_TIMEOUT);
+            break;
+          }
+          __nanosleep(100);
+        }
+        if (!have) break;
+        ctl->tag[s][0] = j;
+        ctl->tag[s][1] = tpos;
+        const uint32_t st = stage_base + s * kStageBytes;
+        const uint32_t fb = bar(BAR_FULL0 + s);
+        mbar_expect_tx(fb, kStageBytes);
+        // rows beyond the tensor read as zeros; rows of the next sequence are masked later
+        const int y = (int)(it.row0 + tpos);
+        const int xc = rank * kCH;
+        tma_load_2d(st + kStX, &map_x, xc, y, fb);
+        tma_load_2d(st + kStY, &map_y, xc, y, fb);
+        tma_load_2d(st + kStQ, &map_q, xc, y, fb);
+        tma_load_2d(st + kStK, &map_k, xc, y, fb);
+        tma_load_2d(st + kStV, &map_v, it.col0, y, fb);
+        tma_load_2d(st + kStV + kSlabBytes, &map_v, it.col0 + 64, y, fb);
+        ++f;
+        tpos += kC;
+      }
+      // Leave no bulk copy in flight when the CTA exits: the last two fills' barriers complete
+      // by byte count, whoever consumed them.
+      const long long t1 = clock64();
+      for (uint32_t back = 1; back <= 2 && back <= f; ++back) {
+        const uint32_t ff = f - back;
+        while (!mbar_try(bar(BAR_FULL0 + (ff & 1)), (ff >> 1) & 1) && clock64() - t1 < kWaitCycles) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ====================================== MMA issuer ======================================
+    if (lane == 0) {
+      constexpr uint32_t kIdescP = make_idesc(64, 64, 0, 0);
+      constexpr uint32_t kIdescO = make_idesc(64, kDVS, 0, 1);
+      constexpr uint32_t kIdescS = make_idesc(128, kDVS, 1, 1);
+      const uint32_t ss = base + kOffSs;
+      uint32_t g = 0;
+      bool ok = true;
+      for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
+        const Item it = decode_item(a, item_of(j), rank);
+        if (it.len == 0) continue;
+        bool last = false;
+        while (!last) {
+          const uint32_t ph1 = g & 1;
+          if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 1)), (g >> 1) & 1, abort_flag, a.hdr))) break;
+          const uint32_t s = (uint32_t)ctl->pd[g & 3].stage;
+          const uint32_t rxi = (uint32_t)ctl->pd[g & 3].rx;
+          const uint32_t rxph = (uint32_t)ctl->pd[g & 3].rxph;
+          last = (ctl->pd[g & 3].flags & kPassLast) != 0;
+          if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
+          // the partner's copies out of ITS stage have all landed here: let it reuse that stage
+          {
+            const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]) & 1;
+            mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
+          }
+          const uint32_t st = stage_base + s * kStageBytes;
+          const uint32_t rx = rx_base + rxi * kRxBytes;
+          // channel slab 0 / 1 of each operand, wherever it lives in this CTA
+          const uint32_t q_sl[2] = {rank == 0 ? st + kStQ : rx + kRxQ, rank == 0 ? rx + kRxQ : st + kStQ};
+          const uint32_t k_sl[2] = {rank == 0 ? st + kStK : rx + kRxK, rank == 0 ? rx + kRxK : st + kStK};
+          const uint32_t x_lo = rank == 0 ? st + kStX : rx + kRxX;
+          const uint32_t x_hi = rank == 0 ? rx + kRxX : st + kStX;
+          tc_fence_after();
+          // P = Qt Kt^T : M = 64 (rows r), N = 64 (rows i), K = 128 channels
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t off = (kk & 3) * 32;
+            umma_bf16(tmem + kColP, desc_kmajor(q_sl[kk >> 2] + off), desc_kmajor(k_sl[kk >> 2] + off),
+                      kIdescP, kk > 0);
+          }
+          umma_commit(bar(BAR_PFULL));
+          if (!(ok = mbar_wait(bar(BAR_PREADY), ph1, abort_flag, a.hdr))) break;
+          if (!(ok = mbar_wait(bar(BAR_SREADY), ph1, abort_flag, a.hdr))) break;
+          if (!(ok = mbar_wait(bar(BAR_OFREE), ph1 ^ 1, abort_flag, a.hdr))) break;
+          tc_fence_after();
+          // O = P V : M = 64, N = 128, K = 64 rows i (P operand lives in the consumed y slab)
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            umma_bf16(tmem + kColO, desc_kmajor(st + kStY + kk * 32),
+                      desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescO, kk > 0);
+          }
+          // O += Qt S_in : K = 128 channels
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            umma_bf16(tmem + kColO, desc_kmajor(q_sl[kk >> 2] + (kk & 3) * 32),
+                      desc_mnmajor(ss + kk * 2048, kSsSlabBytes), kIdescO, 1);
+          }
+          umma_commit(bar(BAR_OFULL));
+          // S = diag(D) S_in (already in TMEM) + Ke^T V : M = 128 channels, N = 128, K = 64 rows
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            umma_bf16(tmem + kColS, desc_mnmajor(x_lo + kk * 2048, x_hi - x_lo),
+                      desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescS, 1);
+          }
+          umma_commit(bar(BAR_SFULL));
+          umma_commit(bar(BAR_EMPTY0 + s));
+          ++g;
+        }
+      }
+    }
+  } else if (warp >= kStateWarp0 && warp < kStateWarp0 + 4) {
+    // ====================================== state group ======================================
+    const int q4 = warp & 3;                              // TMEM lane quarter this warp may touch
+    const int d = q4 * 32 + lane;                         // state row (key channel) of this thread
+    const bool own_d = (d >> 6) == rank;
+    const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
+    const uint32_t ss_row = base + kOffSs + d * 128;
+    const bool signaller = warp == kStateWarp0 && lane == 0;
+    uint32_t g = 0;
+    int prev_rx = 0;
+    bool ok = true;
+    for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
+      const Item it = decode_item(a, item_of(j), rank);
+      const long long srow = it.state_off + (long long)d * a.dv;
+      if (it.len == 0) {  // empty sequence: final state = initial state
+        if (a.sT) {
+          for (int c4 = 0; c4 < kDVS / 4; ++c4) {
+            float4 v4 = a.s0 ? *reinterpret_cast<const float4*>(a.s0 + srow + 4 * c4)
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+            *reinterpret_cast<float4*>(a.sT + srow + 4 * c4) = v4;
+          }
+        }
+        continue;
+      }
+      bool last = false, first = true;
+      while (!last) {
+        const uint32_t ph1 = g & 1;
+        if (!first) {
+          if (!(ok = mbar_wait(bar(BAR_SFULL), ph1 ^ 1, abort_flag, a.hdr))) break;  // pass g-1
+          tc_fence_after();
+          // every contraction of pass g-1 has read its operands: the partner may overwrite
+          // the receive buffer that pass used
+          if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
+        }
+        if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 1)), (g >> 1) & 1, abort_flag, a.hdr))) break;
+        const int s = ctl->pd[g & 3].stage;
+        const int rxi = ctl->pd[g & 3].rx;
+        last = (ctl->pd[g & 3].flags & kPassLast) != 0;
+        prev_rx = rxi;
+        const float D = own_d ? sD[s * kCH + (d & 63)] : sRx[rxi * kBlkFloats + (d & 63)];
+#pragma unroll 1
+        for (int piece = 0; piece < 4; ++piece) {
+          uint32_t r[32];
+          if (!first) {
+            tmem_ld32(t_lane + kColS + piece * 32, r);
+            tmem_ld_wait();
+          } else if (a.s0) {
+#pragma unroll
+            for (int c4 = 0; c4 < 8; ++c4) {
+              const float4 v4 = *reinterpret_cast<const float4*>(a.s0 + srow + piece * 32 + 4 * c4);
+              r[4 * c4] = __float_as_uint(v4.x);
+              r[4 * c4 + 1] = __float_as_uint(v4.y);
+              r[4 * c4 + 2] = __float_as_uint(v4.z);
+              r[4 * c4 + 3] = __float_as_uint(v4.w);
+            }
+          } else {
+#pragma unroll
+            for (int c4 = 0; c4 < 32; ++c4) r[c4] = 0u;
+          }
+          // bf16 copy of S_in for the readout: MN-major, row d, 64-column slab piece/2
+          const uint32_t slab = ss_row + (piece >> 1) * kSsSlabBytes;
+#pragma unroll
+          for (int c8 = 0; c8 < 4; ++c8) {
+            const int chunk = (piece & 1) * 4 + c8;
+            sts128(slab + ((chunk ^ (d & 7)) << 4),
+                   pack_bf16(__uint_as_float(r[8 * c8]), __uint_as_float(r[8 * c8 + 1])),
+                   pack_bf16(__uint_as_float(r[8 * c8 + 2]), __uint_as_float(r[8 * c8 + 3])),
+                   pack_bf16(__uint_as_float(r[8 * c8 + 4]), __uint_as_float(r[8 * c8 + 5])),
+                   pack_bf16(__uint_as_float(r[8 * c8 + 6]), __uint_as_float(r[8 * c8 + 7])));
+          }
+#pragma unroll
+          for (int c4 = 0; c4 < 32; ++c4) r[c4] = __float_as_uint(__uint_as_float(r[c4]) * D);
+          tmem_st32(t_lane + kColS + piece * 32, r);
+        }
+        tmem_st_wait();
+        fence_proxy_async();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_SREADY));
+        first = false;
+        ++g;
+      }
+      if (!ok) break;
+      // final state of this item (also keeps the next item's initial state from racing the MMAs)
+      {
+        const uint32_t lastg = g - 1;
+        if (!(ok = mbar_wait(bar(BAR_SFULL), lastg & 1, abort_flag, a.hdr))) break;
+        tc_fence_after();
+        if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
+        if (a.sT) {
+#pragma unroll 1
+          for (int piece = 0; piece < 4; ++piece) {
+            uint32_t r[32];
+            tmem_ld32(t_lane + kColS + piece * 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int c4 = 0; c4 < 8; ++c4) {
+              *reinterpret_cast<float4*>(a.sT + srow + piece * 32 + 4 * c4) =
+                  make_float4(__uint_as_float(r[4 * c4]), __uint_as_float(r[4 * c4 + 1]),
+                              __uint_as_float(r[4 * c4 + 2]), __uint_as_float(r[4 * c4 + 3]));
+            }
+          }
+        }
+        tc_fence_before();
+      }
+    }
+  } else if (warp >= kScoreWarp0 && warp < kScoreWarp0 + 4) {
+    // ================================== score / output group ==================================
+    const int q4 = warp & 3;
+    const int r_row = q4 * 16 + lane;                     // chunk row held by lanes 0..15 (M = 64)
+    const bool has_row = lane < 16;
+    const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
+    __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(a.o);
+    uint32_t g = 0;
+    bool ok = true;
+    for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
+      const Item it = decode_item(a, item_of(j), rank);
+      if (it.len == 0) continue;
+      bool last = false;
+      while (!last) {
+        const uint32_t ph1 = g & 1;
+        if (!(ok = mbar_wait(bar(BAR_PFULL), ph1, abort_flag, a.hdr))) break;
+        const int s = ctl->pd[g & 3].stage;
+        const int nr = ctl->pd[g & 3].nr;
+        const long long row = ctl->pd[g & 3].row;
+        last = (ctl->pd[g & 3].flags & kPassLast) != 0;
+        const uint32_t ps_row = stage_base + s * kStageBytes + kStY + r_row * 128;
+        tc_fence_after();
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r[32];
+          tmem_ld32(t_lane + kColP + half * 32, r);
+          tmem_ld_wait();
+          if (has_row) {
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int i0 = half * 32 + 8 * c8 + 2 * e;
+                const float lo = (i0 <= r_row) ? __uint_as_float(r[8 * c8 + 2 * e]) : 0.f;
+                const float hi = (i0 + 1 <= r_row) ? __uint_as_float(r[8 * c8 + 2 * e + 1]) : 0.f;
+                w[e] = pack_bf16(lo, hi);
+              }
+              const int chunk = half * 4 + c8;
+              sts128(ps_row + ((chunk ^ (r_row & 7)) << 4), w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_PREADY));
+        // output rows of this pass
+        if (!(ok = mbar_wait(bar(BAR_OFULL), ph1, abort_flag, a.hdr))) break;
+        tc_fence_after();
+        __nv_bfloat16* orow = o + (row + r_row) * a.dv + it.col0;
+#pragma unroll 1
+        for (int piece = 0; piece < 4; ++piece) {
+          uint32_t r[32];
+          tmem_ld32(t_lane + kColO + piece * 32, r);
+          tmem_ld_wait();
+          if (has_row && r_row < nr) {
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {
+              uint4 w;
+              w.x = pack_bf16(a.scale * __uint_as_float(r[8 * c8]), a.scale * __uint_as_float(r[8 * c8 + 1]));
+              w.y = pack_bf16(a.scale * __uint_as_float(r[8 * c8 + 2]), a.scale * __uint_as_float(r[8 * c8 + 3]));
+              w.z = pack_bf16(a.scale * __uint_as_float(r[8 * c8 + 4]), a.scale * __uint_as_float(r[8 * c8 + 5]));
+              w.w = pack_bf16(a.scale * __uint_as_float(r[8 * c8 + 6]), a.scale * __uint_as_float(r[8 * c8 + 7]));
+              *reinterpret_cast<uint4*>(orow + piece * 32 + 8 * c8) = w;
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar(BAR_OFREE));
+        ++g;
+      }
+    }
+  } else if (warp >= kGateWarp0) {
+    // ======================================= gate group =======================================
+    const int gw = warp - kGateWarp0;                     // rows 4*gw .. 4*gw+3 of the tile
+    const bool leader = gw == 0 && lane == 0;
+    constexpr float kLog2e = 1.4426950408889634f;
+    constexpr float kLg2Ln2 = -0.5287663729448977f;       // log2(ln 2)
+    constexpr float kRange = 60.f * kLog2e;               // largest in-chunk decay range, log2 units
+    uint32_t f = 0, g = 0, m = 0, sc = 0;                 // fills seen, passes, attempts, scan syncs
+    bool ok = true;
+    bool armed = false;                                   // attempt m's receive barriers expect bytes
+    auto group_sync = [&]() -> bool {                     // bounded barrier over the gate warps
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_GSCAN));
+      const bool r = mbar_wait(bar(BAR_GSCAN), sc & 1, abort_flag, a.hdr);
+      ++sc;
+      return r;
+    };
+    auto redirect = [&](int jj, int tt) {                 // one thread; before the stage is released
+      ctl->redir_j = jj;
+      ctl->redir_tpos = tt;
+      __threadfence_block();
+      ctl->redir_seq = ctl->redir_seq + 1;
+    };
+    for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
+      const Item it = decode_item(a, item_of(j), rank);
+      int tpos = 0, lcap = kC;
+      while (ok && tpos < it.len) {
+        const uint32_t s = f & 1, ph = (f >> 1) & 1;
+        const uint32_t st = stage_base + s * kStageBytes;
+        if (!(ok = mbar_wait(bar(BAR_FULL0 + s), ph, abort_flag, a.hdr))) break;
+        ++f;
+        if (ctl->tag[s][0] != j || ctl->tag[s][1] != tpos) {
+          // speculative fill for a position we are not at: hand the stage back unused
+          if (!(ok = group_sync())) break;
+          if (leader) mbar_arrive_cnt(bar(BAR_EMPTY0 + s), 2);   // nothing was sent from it
+          continue;
+        }
+        // ---- attempt m: the partner's receive buffer m&1 must be free before we send into it
+        const uint32_t rxi = m & 1, rxph = (m >> 1) & 1;
+        if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
+        if (leader) {
+          mbar_expect_tx(bar(BAR_PEER0 + rxi), kRxBytes);
+          mbar_expect_tx(bar(BAR_VERD0 + rxi), kBlkBytes);
+          armed = true;
+        }
+        const int left = it.len - tpos;
+        const int nr = min(min(kC, left), lcap);
+        // element (row r, own channels 2*lane, +1) sits at this swizzled byte offset of a slab
+        float bq[4][2];   // inclusive in-chunk cumulative log2 decay (own rows only, so far)
+        float eh[4][2];   // log2 ahat
+        float run0 = 0.f, run1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int r = gw * 4 + i;
+          const uint32_t off = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
+          const uint32_t xw = lds32(st + kStX + off), yw = lds32(st + kStY + off);
+          const float xs[2] = {__uint_as_float(xw << 16), __uint_as_float(xw & 0xFFFF0000u)};
+          const float ys[2] = {__uint_as_float(yw << 16), __uint_as_float(yw & 0xFFFF0000u)};
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const float u = ex2f(xs[e] * kLog2e);                       // e^x
+            // g * log2(e) = log2(1 + e^x); series when 1 + u would round u away
+            const float sp2 = u < 9.765625e-4f ? u * (kLog2e - 0.72134752f * u) : lg2f(1.f + u);
+            const float tau = rcpf(1.f + ex2f(-ys[e] * kLog2e));
+            float l2a = fmaxf(-sp2 * tau, -kRange);                     // per-step floor exp(-60)
+            float l2h;
+            if (INGATE == RODIMUS_INGATE_POW_G) {
+              l2h = tau * (lg2f(sp2) + kLg2Ln2);                        // tau * log2(g)
+            } else {
+              l2h = tau * (xs[e] * kLog2e - sp2);                       // tau * log2(sigmoid(x))
+            }
+            if (r >= nr) l2a = 0.f;                                     // rows past the pass
+            if (e == 0) { run0 += l2a; bq[i][0] = run0; } else { run1 += l2a; bq[i][1] = run1; }
+            eh[i][e] = l2h;
+          }
+        }
+        // exclusive prefix over the 16 row groups, and the chunk total
+        float* tot = sTot + (m & 1) * (kGateWarps * kCH);
+        *reinterpret_cast<float2*>(tot + gw * kCH + 2 * lane) = make_float2(run0, run1);
+        if (!(ok = group_sync())) break;
+        float pre0 = 0.f, pre1 = 0.f, all0 = 0.f, all1 = 0.f;
+#pragma unroll
+        for (int w = 0; w < kGateWarps; ++w) {
+          const float2 t = *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane);
+          if (w < gw) { pre0 += t.x; pre1 += t.y; }
+          all0 += t.x; all1 += t.y;
+        }
+        // every warp sees all 64 own channels' totals, so all sixteen reach the same verdict
+        const bool viol_own = __any_sync(0xffffffffu, all0 < -kRange || all1 < -kRange) && nr > 1;
+        const float D0 = ex2f(all0), D1 = ex2f(all1);
+        if (gw == 0) {
+          // chunk decays of the own channels: for this CTA's state group and for the partner's
+          *reinterpret_cast<float2*>(sD + s * kCH + 2 * lane) = make_float2(D0, D1);
+          volatile float* blk = sTx + rxi * kBlkFloats;
+          blk[2 * lane] = D0;
+          blk[2 * lane + 1] = D1;
+          if (lane == 0) {
+            blk[64] = __int_as_float(viol_own ? 1 : 0);
+            blk[65] = __int_as_float((int)s);
+          }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0)
+            dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
+                            base + kOffTx + rxi * kBlkBytes, kBlkBytes,
+                            map_to_cta(bar(BAR_VERD0 + rxi), peer));
+        }
+        if (!viol_own) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int r = gw * 4 + i;
+            const uint32_t off = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
+            const uint32_t qw = lds32(st + kStQ + off), kw = lds32(st + kStK + off);
+            const float b0 = bq[i][0] + pre0, b1 = bq[i][1] + pre1;
+            const bool live = r < nr;
+            const float q0 = live ? __uint_as_float(qw << 16) : 0.f;
+            const float q1 = live ? __uint_as_float(qw & 0xFFFF0000u) : 0.f;
+            const float k0 = live ? __uint_as_float(kw << 16) : 0.f;
+            const float k1 = live ? __uint_as_float(kw & 0xFFFF0000u) : 0.f;
+            const float kt0 = k0 * ex2f(eh[i][0] - b0), kt1 = k1 * ex2f(eh[i][1] - b1);
+            sts32(st + kStQ + off, pack_bf16(q0 * ex2f(b0), q1 * ex2f(b1)));
+            sts32(st + kStK + off, pack_bf16(kt0, kt1));
+            sts32(st + kStX + off, pack_bf16(kt0 * D0, kt1 * D1));       // 2^{b_C - b_i} = 2^{-b_i} D
+          }
+        }
+        // this warp's four rows of each operand slab go to the partner (also when the attempt
+        // is about to be abandoned: the byte count the partner's barrier expects is fixed)
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          const uint32_t rows_off = gw * 512;
+          const uint32_t dst = peer_rx_base + rxi * kRxBytes + rows_off;
+          const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
+          dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, 512, pb);
+          dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK + rows_off, 512, pb);
+          dsmem_bulk_copy(map_to_cta(dst + kRxX, peer), st + kStX + rows_off, 512, pb);
+        }
+        // the partner's verdict came with its decay block
+        if (!(ok = mbar_wait_cluster(bar(BAR_VERD0 + rxi), rxph, abort_flag, a.hdr))) break;
+        const bool viol = viol_own || (__float_as_int(sRx[rxi * kBlkFloats + 64]) != 0);
+        ++m;
+        armed = false;
+        if (viol) {
+          // decays too fast for 'nr' rows at once: ask for this position again, fewer rows
+          lcap = max(1, nr >> 1);
+          if (!(ok = group_sync())) break;
+          if (leader) {
+            // whatever the partner sent for this attempt must have landed before its buffer and
+            // its stage are declared reusable
+            if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
+            const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]) & 1;
+            mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
+            mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + rxi), peer));
+            redirect(j, tpos);
+            mbar_arrive(bar(BAR_EMPTY0 + s));
+          }
+          continue;
+        }
+        if (leader) {
+          volatile PassDesc* pd = &ctl->pd[g & 3];
+          pd->stage = (int)s;
+          pd->nr = nr;
+          pd->flags = (nr == left ? kPassLast : 0);
+          pd->rx = (int)rxi;
+          pd->rxph = (int)rxph;
+          pd->row = it.row0 + tpos;
+          if (nr < min(kC, left)) redirect(j, tpos + nr);   // the prefetcher assumed 64 rows
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_GATED0 + (g & 1)));
+        ++g;
+        tpos += nr;
+        if (lcap < kC) lcap = min(kC, lcap * 2);
+      }
+    }
+    if (leader) {
+      ctl->done = 1;
+      // nothing the partner sent may still be in flight towards this CTA when it exits
+      const long long t1 = clock64();
+      for (uint32_t back = armed ? 0 : 1; back <= 2 && back <= m; ++back) {
+        const uint32_t mm = m - back;
+        while (!(mbar_try_cluster(bar(BAR_PEER0 + (mm & 1)), (mm >> 1) & 1) &&
+                 mbar_try_cluster(bar(BAR_VERD0 + (mm & 1)), (mm >> 1) & 1)) &&
+               clock64() - t1 < kWaitCycles) {}
+      }
+    }
+  }
+
+  // ------------------------------------------ teardown ------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
+                 : "memory");
+  }
+  // neither CTA leaves while the other may still signal one of its barriers
+  cluster_arrive();
+  cluster_wait();
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [rows, cols] bf16 row-major, box = 64 rows x 64 columns (128 bytes), 128-byte swizzle.
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)kC};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int INGATE>
+cudaError_t launch_pair(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mx,
+                        const CUtensorMap& my, const CUtensorMap& mv, const PairArgs& a,
+                        int max_pairs, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(ddts_fwd_pair_kernel<INGATE>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
+  const long long pairs = a.n_items < max_pairs ? a.n_items : max_pairs;
+  ddts_fwd_pair_kernel<INGATE><<<(unsigned)(2 * pairs), kThreads, kSmemBytes, st>>>(mq, mk, mx, my, mv, a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool fwd_pair_supported(const rodimus_ddts_fwd_params& p) {
+  return p.dtype == RODIMUS_BF16 && p.dk == kDK && p.dv % (2 * kDVS) == 0;
+}
+
+cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
+  *n_launches = 0;
+  PairArgs a;
+  a.o = p.o; a.s0 = p.s0; a.sT = p.sT; a.cu = p.cu_seqlens;
+  a.hdr = reinterpret_cast<WorkspaceHeader*>(p.workspace);
+  a.order = reinterpret_cast<const int32_t*>(reinterpret_cast<const char*>(p.workspace) +
+                                             sizeof(WorkspaceHeader));
+  a.H = p.H; a.T = p.T; a.dv = p.dv;
+  a.n_seq = p.cu_seqlens ? p.N : p.B;
+  a.pairs = p.dv / (2 * kDVS);
+  a.n_items = (long long)a.n_seq * p.H * a.pairs;
+  a.scale = p.scale;
+  if (a.n_items == 0) return cudaSuccess;
+  const uint64_t rows = (uint64_t)p.B * p.H * p.T;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
+
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+
+  CUtensorMap mq, mk, mx, my, mv;
+  if (rows > 0) {
+    if (!make_map(&mq, p.q, rows, kDK) || !make_map(&mk, p.k, rows, kDK) ||
+        !make_map(&mx, p.gate_x, rows, kDK) || !make_map(&my, p.temp_y, rows, kDK) ||
+        !make_map(&mv, p.v, rows, (uint64_t)p.dv))
+      return cudaErrorUnknown;
+  } else {
+    memset(&mq, 0, sizeof(mq)); mk = mq; mx = mq; my = mq; mv = mq;  // never dereferenced: no chunks
+  }
+  const int max_pairs = sms / 2 > 0 ? sms / 2 : 1;   // one CTA per SM; a pair shares a TPC
+  if (p.ingate == RODIMUS_INGATE_POW_G)
+    e = launch_pair<RODIMUS_INGATE_POW_G>(mq, mk, mx, my, mv, a, max_pairs, st);
+  else
+    e = launch_pair<RODIMUS_INGATE_POW_SIGMOID>(mq, mk, mx, my, mv, a, max_pairs, st);
+  if (e == cudaSuccess) *n_launches = 1;
+  return e;
+}
+
+}  // namespace ddts

@@ -37,10 +37,25 @@ int check_fwd_sizes(const rodimus_ddts_fwd_params* p, bool varlen) {
 
 namespace ddts {
 
+namespace {
+// RODIMUS_DDTS_KERNEL = "simt" | "single" narrows the choice of prefill kernel (for comparing
+// them); anything else, or unset, picks the fastest kernel that covers the shape.
+int kernel_override() {
+  const char* v = std::getenv("RODIMUS_DDTS_KERNEL");
+  if (!v) return 0;
+  if (!std::strcmp(v, "simt")) return 1;
+  if (!std::strcmp(v, "single")) return 2;
+  return 0;
+}
+}  // namespace
+
 bool fwd_tc_supported(const rodimus_ddts_fwd_params& p) {
-  const char* force = std::getenv("RODIMUS_DDTS_FORCE_SIMT");
-  if (force && force[0] == '1') return false;
-  return tc_kernel_built() && p.dtype == RODIMUS_BF16 && p.dk == 128 && p.dv % 128 == 0;
+  if (kernel_override() == 1) return false;
+  return p.dtype == RODIMUS_BF16 && p.dk == 128 && p.dv % 128 == 0;
+}
+
+bool fwd_pair_selected(const rodimus_ddts_fwd_params& p) {
+  return kernel_override() == 0 && fwd_pair_supported(p);
 }
 
 }  // namespace ddts
@@ -93,7 +108,9 @@ int rodimus_ddts_fwd(const rodimus_ddts_fwd_params* p) {
     launches += n;
   }  // dense: the prefill kernel's first CTA clears the status word itself
   if (e != cudaSuccess) return RODIMUS_ERR_CUDA;
-  if (ddts::fwd_tc_supported(*p))
+  if (ddts::fwd_pair_selected(*p))
+    e = ddts::launch_fwd_pair(*p, &n);
+  else if (ddts::fwd_tc_supported(*p))
     e = ddts::launch_fwd_tc(*p, &n);
   else
     e = ddts::launch_fwd_simt(*p, &n);
