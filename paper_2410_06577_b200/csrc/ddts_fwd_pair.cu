@@ -283,7 +283,9 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
   } else if (warp == 1) {
     // ====================================== MMA issuer ======================================
-    if (lane == 0) {
+    // Every lane runs the loop (waits, descriptor arithmetic stay warp-uniform); lane 0 issues.
+    {
+      const bool issuer = lane == 0;
       constexpr uint32_t kIdescP = make_idesc(64, 64, 0, 0);
       constexpr uint32_t kIdescO = make_idesc(64, kDVS, 0, 1);
       constexpr uint32_t kIdescS = make_idesc(128, kDVS, 1, 1);
@@ -302,11 +304,6 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const uint32_t rxph = (uint32_t)ctl->pd[g & 3].rxph;
           last = (ctl->pd[g & 3].flags & kPassLast) != 0;
           if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
-          // the partner's copies out of ITS stage have all landed here: let it reuse that stage
-          {
-            const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]) & 1;
-            mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
-          }
           const uint32_t st = stage_base + s * kStageBytes;
           const uint32_t rx = rx_base + rxi * kRxBytes;
           // channel slab 0 / 1 of each operand, wherever it lives in this CTA
@@ -319,10 +316,10 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk) {
             const uint32_t off = (kk & 3) * 32;
-            umma_bf16(tmem + kColP, desc_kmajor(q_sl[kk >> 2] + off), desc_kmajor(k_sl[kk >> 2] + off),
+            if (issuer) umma_bf16(tmem + kColP, desc_kmajor(q_sl[kk >> 2] + off), desc_kmajor(k_sl[kk >> 2] + off),
                       kIdescP, kk > 0);
           }
-          umma_commit(bar(BAR_PFULL));
+          if (issuer) umma_commit(bar(BAR_PFULL));
           if (!(ok = mbar_wait(bar(BAR_PREADY), ph1, abort_flag, a.hdr))) break;
           if (!(ok = mbar_wait(bar(BAR_SREADY), ph1, abort_flag, a.hdr))) break;
           if (!(ok = mbar_wait(bar(BAR_OFREE), ph1 ^ 1, abort_flag, a.hdr))) break;
@@ -330,24 +327,24 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // O = P V : M = 64, N = 128, K = 64 rows i (P operand lives in the consumed y slab)
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
-            umma_bf16(tmem + kColO, desc_kmajor(st + kStY + kk * 32),
+            if (issuer) umma_bf16(tmem + kColO, desc_kmajor(st + kStY + kk * 32),
                       desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescO, kk > 0);
           }
           // O += Qt S_in : K = 128 channels
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk) {
-            umma_bf16(tmem + kColO, desc_kmajor(q_sl[kk >> 2] + (kk & 3) * 32),
+            if (issuer) umma_bf16(tmem + kColO, desc_kmajor(q_sl[kk >> 2] + (kk & 3) * 32),
                       desc_mnmajor(ss + kk * 2048, kSsSlabBytes), kIdescO, 1);
           }
-          umma_commit(bar(BAR_OFULL));
+          if (issuer) umma_commit(bar(BAR_OFULL));
           // S = diag(D) S_in (already in TMEM) + Ke^T V : M = 128 channels, N = 128, K = 64 rows
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
-            umma_bf16(tmem + kColS, desc_mnmajor(x_lo + kk * 2048, x_hi - x_lo),
+            if (issuer) umma_bf16(tmem + kColS, desc_mnmajor(x_lo + kk * 2048, x_hi - x_lo),
                       desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescS, 1);
           }
-          umma_commit(bar(BAR_SFULL));
-          umma_commit(bar(BAR_EMPTY0 + s));
+          if (issuer) umma_commit(bar(BAR_SFULL));
+          if (issuer) umma_commit(bar(BAR_EMPTY0 + s));
           ++g;
         }
       }
@@ -479,6 +476,13 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         last = (ctl->pd[g & 3].flags & kPassLast) != 0;
         const uint32_t ps_row = stage_base + s * kStageBytes + kStY + r_row * 128;
         tc_fence_after();
+        if (warp == kScoreWarp0 && lane == 0) {
+          // P exists, so the partner's copies out of ITS stage have all landed here (the issuer
+          // waited for them): let the partner reuse that stage
+          const int rxi = ctl->pd[g & 3].rx;
+          const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]) & 1;
+          mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
+        }
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
           uint32_t r[32];

@@ -38,6 +38,20 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// try_wait that lets the hardware park the warp for up to kParkNs before it reports "not yet":
+// a parked warp takes no issue slots from the warps that are working.
+constexpr uint32_t kParkNs = 20000;
+__device__ __forceinline__ bool mbar_try_park(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+      "selp.b32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(kParkNs)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false (and raises the CTA's abort flag and the device status) if the
 // phase does not complete in time or another role has already given up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
@@ -45,7 +59,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
-    if (mbar_try(bar, parity)) return true;
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i)
+      if (mbar_try_park(bar, parity)) return true;
     // a completed phase stays visible to every waiter of a group, so re-test before giving up:
     // either all members of a group pass a given wait or none does
     if (*abort_flag) return mbar_try(bar, parity);
@@ -184,9 +200,11 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t ran
 __device__ __forceinline__ void mbar_arrive_cnt(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-// Arrive on an mbarrier of another CTA of the cluster (address from map_to_cta).
+// Arrive on an mbarrier of another CTA of the cluster (address from map_to_cta).  Relaxed: the
+// callers signal "I have finished reading / receiving", which publishes no data of their own, and
+// a cluster-scope release costs the issuing thread a couple of thousand cycles.
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar)
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar)
                : "memory");
 }
 // try_wait that acquires at cluster scope: for barriers another CTA arrives on or copies into.
@@ -201,12 +219,25 @@ __device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) 
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ bool mbar_try_park_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n"
+      "selp.b32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(kParkNs)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
                                                   volatile int* abort_flag, WorkspaceHeader* hdr) {
   if (mbar_try_cluster(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
-    if (mbar_try_cluster(bar, parity)) return true;
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i)
+      if (mbar_try_park_cluster(bar, parity)) return true;
     if (*abort_flag) return mbar_try_cluster(bar, parity);
     if (clock64() - t0 > kWaitCycles) {
       if (mbar_try_cluster(bar, parity)) return true;
