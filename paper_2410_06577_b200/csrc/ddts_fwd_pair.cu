@@ -1,18 +1,22 @@
 // Chunked DDTS prefill on the 5th-generation tensor cores for dv a multiple of 256: two CTAs of
 // a thread-block cluster work on one (sequence, head) and SHARE the gate math.
 //
-// Same chunk algebra as ddts_fwd_tc.cu (appendix "Chunkwise Parallel Representation of the
-// Rodimus Block"; chunk length 64, log2 domain, decays anchored at the chunk start):
-//   Qt_r = q_r 2^{b_r}     Kt_i = k_i ahat_i 2^{-b_i}     Ke_i = Kt_i 2^{b_C}
-//   P = mask(Qt Kt^T)      O = P V + Qt S_in              S_out = diag(2^{b_C}) S_in + Ke^T V
+// Chunk algebra (appendix "Chunkwise Parallel Representation of the Rodimus Block"; chunk length
+// 64, log2 domain, decays anchored at the chunk start, b_r = sum_{j<=r} log2 alpha_j <= 0):
+//   Qt_r = q_r 2^{b_r}            Kt_i = k_i ahat_i 2^{-b_i}          D = 2^{b_C}
+//   P = mask(Qt Kt^T)             O = P V + Qt S_in                   S_out = D . (S_in + Kt^T V)
+// The state update is written with the chunk decay OUTSIDE the bracket, so the same Kt tile
+// serves the scores (as a K-major operand) and the state update (as an MN-major operand), and
+// the row scaling by D happens when the state makes its once-per-chunk trip through registers.
+//
 // Every quantity that depends on the gates is per key channel and independent of the value
-// column, so the two CTAs that own the two 128-column halves of a 256-column slab of the state
-// would otherwise repeat the whole softplus / sigmoid / log / exp2 pipeline.  Here CTA c of the
-// pair loads q,k,x,y for key channels 64c..64c+63 only, turns them into Qt, Kt, Ke in place, and
-// copies those three 8 KiB slabs (plus the 64 chunk decays) into the other CTA's shared memory
-// with bulk shared-to-shared copies that complete on an mbarrier over there.  Each CTA then runs
-// the same three contractions as the single-CTA kernel on its own 128 value columns, taking
-// half of the K (or M) extent from its own slab and half from the received one.
+// column, so two CTAs that own the two 128-column halves of a 256-column slab of the state would
+// otherwise repeat the whole softplus / sigmoid / log / exp2 pipeline.  Here CTA c of the pair
+// loads q,k,x,y for key channels 64c..64c+63 only, turns them into Qt, Kt in place, and copies
+// those two 8 KiB slabs (plus the 64 chunk decays) into the other CTA's shared memory with bulk
+// shared-to-shared copies that complete on an mbarrier over there.  Each CTA then runs the three
+// contractions on its own 128 value columns, taking half of the K (or M) extent from its own
+// slab and half from the received one.
 //
 // The pair advances in lockstep: which rows form a pass is decided from the decay totals of all
 // 128 channels, so each CTA sends its verdict along with its chunk decays and both take the OR.
@@ -22,7 +26,7 @@
 //   warp 1        tcgen05.mma issuer, owns the TMEM allocation
 //   warps 2-5     state group: TMEM <-> registers trip of S, initial / final state I/O
 //   warps 6-9     score / output group
-//   warps 10-25   gate group: 4 rows x 2 channels per thread
+//   warps 10-25   gate group: 4 rows x 2 channels per thread, packed fp32x2 arithmetic
 #include <cuda.h>
 
 #include <cstring>
@@ -42,11 +46,11 @@ constexpr int kSlabBytes = kC * 128;          // [64 rows][64 bf16] = 8 KiB, 128
 constexpr int kStQ = 0, kStK = kSlabBytes, kStX = 2 * kSlabBytes, kStY = 3 * kSlabBytes,
               kStV = 4 * kSlabBytes;
 constexpr int kStageBytes = 6 * kSlabBytes;   // 48 KiB
-// one receive buffer: the partner's Qt, Kt, Ke slabs
-constexpr int kRxQ = 0, kRxK = kSlabBytes, kRxX = 2 * kSlabBytes;
-constexpr int kRxBytes = 3 * kSlabBytes;      // 24 KiB
-constexpr int kStages = 2, kRxBufs = 2;
-constexpr int kOperandBytes = kStages * kStageBytes + kRxBufs * kRxBytes;  // 144 KiB
+// one receive buffer: the partner's Qt, Kt slabs
+constexpr int kRxQ = 0, kRxK = kSlabBytes;
+constexpr int kRxBytes = 2 * kSlabBytes;      // 16 KiB
+constexpr int kStages = 3, kRxBufs = 2;
+constexpr int kOperandBytes = kStages * kStageBytes + kRxBufs * kRxBytes;  // 176 KiB
 constexpr int kSsSlabBytes = kDK * 128;       // [128 rows][64 bf16]
 constexpr int kOffSs = kOperandBytes;                     // bf16 copy of the state, 2 slabs
 constexpr int kOffD = kOffSs + 2 * kSsSlabBytes;          // float [kStages][64]: own 2^{b_C}
@@ -57,7 +61,7 @@ constexpr int kOffRx = kOffTx + kRxBufs * kBlkBytes;      // float [2][68]: bloc
 constexpr int kGateWarp0 = 10, kGateWarps = 16;
 constexpr int kOffTot = kOffRx + kRxBufs * kBlkBytes;     // float [2][16][64]: scan partials
 constexpr int kOffBar = kOffTot + 2 * kGateWarps * kCH * 4;
-constexpr int kNumBars = 24;
+constexpr int kNumBars = 32;
 constexpr int kOffMisc = kOffBar + kNumBars * 8;          // control block
 constexpr int kSmemUsed = kOffMisc + 256;
 constexpr int kSmemBytes = kSmemUsed + 1024;              // slack for manual 1024-byte alignment
@@ -71,13 +75,14 @@ constexpr int kStateWarp0 = 2, kScoreWarp0 = 6;
 constexpr uint32_t kColS = 0, kColO = 128, kColP = 256, kTmemCols = 512;
 
 // mbarrier indices
-enum { BAR_FULL0 = 0, BAR_FULL1,      // TMA fill landed                          (1 + bytes)
-       BAR_EMPTY0, BAR_EMPTY1,        // stage reusable: own release + partner's receipt    (2)
-       BAR_GATED0, BAR_GATED1,        // pass published by the gate group                  (16)
-       BAR_PEER0, BAR_PEER1,          // partner's three slabs landed               (1 + bytes)
-       BAR_VERD0, BAR_VERD1,          // partner's decay block landed               (1 + bytes)
+enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                      (1 + bytes)
+       BAR_EMPTY0 = 3,                // [3] stage reusable: own release + partner's receipt (2)
+       BAR_GATED0 = 6,                // [4] pass published by the gate group             (16)
+       BAR_PEER0 = 10, BAR_PEER1,     // partner's two slabs landed                 (1 + bytes)
+       BAR_VERD0, BAR_VERD1,          // own verdict written + partner's block landed (1 + bytes)
        BAR_RXFREE0, BAR_RXFREE1,      // partner is done with ITS receive buffer            (1)
        BAR_PFULL, BAR_PREADY, BAR_SREADY, BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN };
+static_assert(BAR_GSCAN < kNumBars, "barrier count");
 
 struct PairArgs {
   void* o;
@@ -142,12 +147,80 @@ struct Control {            // lives in shared memory
   int done;                 // gate group has finished every item of this CTA
   int redir_seq;            // bumped by the gate group after writing redir_j / redir_tpos
   int redir_j, redir_tpos;  // where the producer must continue (CTA-local item index, token)
+  int tag[kStages][2];      // per stage: (item index, token position) of the fill it holds
   int pad[2];
-  int tag[2][2];            // per stage: (item index, token position) of the fill it holds
-  int pad2[4];
   PassDesc pd[4];
 };
 static_assert(sizeof(Control) <= 256, "control block");
+
+// ---------------------------------------------------------------------------------------------
+// gate math on pairs of adjacent key channels (packed fp32x2 adds / multiplies / fmas)
+// ---------------------------------------------------------------------------------------------
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLg2Ln2 = -0.5287663729448977f;   // log2(ln 2)
+constexpr float kRange = 60.f * kLog2e;           // largest in-chunk decay range, log2 units
+
+__device__ __forceinline__ float2 bf16x2_to_f2(uint32_t w) {
+  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+}
+__device__ __forceinline__ float2 splat(float v) { return make_float2(v, v); }
+
+// Phase 1 for this thread's 4 rows x 2 channels: log2 decay (cumulative over the thread's own
+// rows, b) and log2 input weight (eh).  Returns the sum of the four rows' log2 decays.
+template <int INGATE, bool FULL>
+__device__ __forceinline__ float2 gate_phase1(uint32_t xs, uint32_t ys, const uint32_t (&off)[4],
+                                              int row0, int nr, float2 (&b)[4], float2 (&eh)[4]) {
+  float2 run = splat(0.f);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 x = bf16x2_to_f2(lds32(xs + off[i]));
+    const float2 y = bf16x2_to_f2(lds32(ys + off[i]));
+    const float2 xl = __fmul2_rn(x, splat(kLog2e));
+    const float2 u = make_float2(ex2f(xl.x), ex2f(xl.y));               // e^x
+    // log2(1 + e^x) = g log2(e); series where 1 + u would round u away
+    const float2 w = __fadd2_rn(u, splat(1.f));
+    const float2 ser = __fmul2_rn(u, __ffma2_rn(u, splat(-0.72134752f), splat(kLog2e)));
+    const float2 sp2 = make_float2(u.x < 9.765625e-4f ? ser.x : lg2f(w.x),
+                                   u.y < 9.765625e-4f ? ser.y : lg2f(w.y));
+    // -tau = -sigmoid(y) = 1 / (-1 - e^{-y})
+    const float2 yl = __fmul2_rn(y, splat(-kLog2e));
+    const float2 nw = __ffma2_rn(make_float2(ex2f(yl.x), ex2f(yl.y)), splat(-1.f), splat(-1.f));
+    const float2 ntau = make_float2(rcpf(nw.x), rcpf(nw.y));
+    float2 l2a = __fmul2_rn(sp2, ntau);                                 // log2 alpha <= 0
+    l2a.x = fmaxf(l2a.x, -kRange);                                      // per-step floor exp(-60)
+    l2a.y = fmaxf(l2a.y, -kRange);
+    if (INGATE == RODIMUS_INGATE_POW_G) {                               // tau * log2(g)
+      eh[i] = __fmul2_rn(ntau, __ffma2_rn(make_float2(lg2f(sp2.x), lg2f(sp2.y)), splat(-1.f),
+                                          splat(-kLg2Ln2)));
+    } else {                                                            // tau * log2(sigmoid(x))
+      eh[i] = __fmul2_rn(ntau, __ffma2_rn(xl, splat(-1.f), sp2));
+    }
+    if (!FULL && row0 + i >= nr) l2a = splat(0.f);                      // rows past the pass
+    run = __fadd2_rn(run, l2a);
+    b[i] = run;
+  }
+  return run;
+}
+
+// Phase 2: Qt = q 2^{b}, Kt = k 2^{eh - b}, written over q and k (same swizzled offsets).
+template <bool FULL>
+__device__ __forceinline__ void gate_phase2(uint32_t qs, uint32_t ks, const uint32_t (&off)[4],
+                                            int row0, int nr, float2 pre, const float2 (&b)[4],
+                                            const float2 (&eh)[4]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 q = bf16x2_to_f2(lds32(qs + off[i]));
+    float2 k = bf16x2_to_f2(lds32(ks + off[i]));
+    const float2 bb = __fadd2_rn(b[i], pre);
+    const float2 hb = __ffma2_rn(bb, splat(-1.f), eh[i]);
+    const float2 eq = make_float2(ex2f(bb.x), ex2f(bb.y));
+    const float2 ek = make_float2(ex2f(hb.x), ex2f(hb.y));
+    if (!FULL && row0 + i >= nr) { q = splat(0.f); k = splat(0.f); }
+    const float2 qt = __fmul2_rn(q, eq), kt = __fmul2_rn(k, ek);
+    sts32(qs + off[i], pack_bf16(qt.x, qt.y));
+    sts32(ks + off[i], pack_bf16(kt.x, kt.y));
+  }
+}
 
 template <int INGATE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
@@ -170,7 +243,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const int warp = tid >> 5, lane = tid & 31;
   const int rank = (int)cluster_ctarank();     // 0 or 1: which key-channel half and dv half
   const int peer = rank ^ 1;
-  // The state update takes Ke for all 128 channels as ONE operand whose two 64-channel groups
+  // The state update takes Kt for all 128 channels as ONE operand whose two 64-channel groups
   // must sit at increasing addresses: channels 0..63 first.  So the CTA that owns the low
   // channels keeps its stages below its receive buffers and the other CTA the opposite.
   const uint32_t stage_base = base + (rank == 0 ? 0u : (uint32_t)(kRxBufs * kRxBytes));
@@ -183,18 +256,16 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     ctl->abort_flag = 0;
     ctl->done = 0;
     ctl->redir_seq = 0;
-    mbar_init(bar(BAR_FULL0), 1);
-    mbar_init(bar(BAR_FULL1), 1);
-    mbar_init(bar(BAR_EMPTY0), 2);
-    mbar_init(bar(BAR_EMPTY1), 2);
-    mbar_init(bar(BAR_GATED0), kGateWarps);
-    mbar_init(bar(BAR_GATED1), kGateWarps);
-    mbar_init(bar(BAR_PEER0), 1);
-    mbar_init(bar(BAR_PEER1), 1);
-    mbar_init(bar(BAR_VERD0), 1);
-    mbar_init(bar(BAR_VERD1), 1);
-    mbar_init(bar(BAR_RXFREE0), 1);
-    mbar_init(bar(BAR_RXFREE1), 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar(BAR_FULL0 + s), 1);
+      mbar_init(bar(BAR_EMPTY0 + s), 2);
+    }
+    for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_GATED0 + i), kGateWarps);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(BAR_PEER0 + i), 1);
+      mbar_init(bar(BAR_VERD0 + i), 1);
+      mbar_init(bar(BAR_RXFREE0 + i), 1);
+    }
     mbar_init(bar(BAR_PFULL), 1);
     mbar_init(bar(BAR_PREADY), 128);
     mbar_init(bar(BAR_SREADY), 128);
@@ -224,11 +295,11 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // ===================================== TMA producer =====================================
     if (lane == 0) {
       uint32_t f = 0;         // fills issued
+      uint32_t s = 0, ph = 0; // stage and phase of fill f
       int j = 0, tpos = 0;    // speculative position: item index and token
       int seen = 0;           // last redirect taken
       bool ok = true;
       while (ok) {
-        const uint32_t s = f & 1, ph = (f >> 1) & 1;
         if (!(ok = mbar_wait_cluster(bar(BAR_EMPTY0 + s), ph ^ 1, abort_flag, a.hdr))) break;
         Item it;
         bool have = false;
@@ -271,14 +342,16 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         tma_load_2d(st + kStV, &map_v, it.col0, y, fb);
         tma_load_2d(st + kStV + kSlabBytes, &map_v, it.col0 + 64, y, fb);
         ++f;
+        if (++s == kStages) { s = 0; ph ^= 1; }
         tpos += kC;
       }
-      // Leave no bulk copy in flight when the CTA exits: the last two fills' barriers complete
-      // by byte count, whoever consumed them.
+      // Leave no bulk copy in flight when the CTA exits: the last fills' barriers complete by
+      // byte count, whoever consumed them.
       const long long t1 = clock64();
-      for (uint32_t back = 1; back <= 2 && back <= f; ++back) {
+      for (uint32_t back = 1; back <= (uint32_t)kStages && back <= f; ++back) {
         const uint32_t ff = f - back;
-        while (!mbar_try(bar(BAR_FULL0 + (ff & 1)), (ff >> 1) & 1) && clock64() - t1 < kWaitCycles) {}
+        while (!mbar_try(bar(BAR_FULL0 + ff % kStages), (ff / kStages) & 1) &&
+               clock64() - t1 < kWaitCycles) {}
       }
     }
   } else if (warp == 1) {
@@ -298,7 +371,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         bool last = false;
         while (!last) {
           const uint32_t ph1 = g & 1;
-          if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 1)), (g >> 1) & 1, abort_flag, a.hdr))) break;
+          if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 3)), (g >> 2) & 1, abort_flag, a.hdr))) break;
           const uint32_t s = (uint32_t)ctl->pd[g & 3].stage;
           const uint32_t rxi = (uint32_t)ctl->pd[g & 3].rx;
           const uint32_t rxph = (uint32_t)ctl->pd[g & 3].rxph;
@@ -309,48 +382,53 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // channel slab 0 / 1 of each operand, wherever it lives in this CTA
           const uint32_t q_sl[2] = {rank == 0 ? st + kStQ : rx + kRxQ, rank == 0 ? rx + kRxQ : st + kStQ};
           const uint32_t k_sl[2] = {rank == 0 ? st + kStK : rx + kRxK, rank == 0 ? rx + kRxK : st + kStK};
-          const uint32_t x_lo = rank == 0 ? st + kStX : rx + kRxX;
-          const uint32_t x_hi = rank == 0 ? rx + kRxX : st + kStX;
           tc_fence_after();
           // P = Qt Kt^T : M = 64 (rows r), N = 64 (rows i), K = 128 channels
+          if (issuer) {
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (kk & 3) * 32;
-            if (issuer) umma_bf16(tmem + kColP, desc_kmajor(q_sl[kk >> 2] + off), desc_kmajor(k_sl[kk >> 2] + off),
-                      kIdescP, kk > 0);
+            for (int kk = 0; kk < 8; ++kk) {
+              const uint32_t off = (kk & 3) * 32;
+              umma_bf16(tmem + kColP, desc_kmajor(q_sl[kk >> 2] + off), desc_kmajor(k_sl[kk >> 2] + off),
+                        kIdescP, kk > 0);
+            }
+            umma_commit(bar(BAR_PFULL));
           }
-          if (issuer) umma_commit(bar(BAR_PFULL));
           if (!(ok = mbar_wait(bar(BAR_PREADY), ph1, abort_flag, a.hdr))) break;
           if (!(ok = mbar_wait(bar(BAR_SREADY), ph1, abort_flag, a.hdr))) break;
           if (!(ok = mbar_wait(bar(BAR_OFREE), ph1 ^ 1, abort_flag, a.hdr))) break;
           tc_fence_after();
-          // O = P V : M = 64, N = 128, K = 64 rows i (P operand lives in the consumed y slab)
+          if (issuer) {
+            // O = P V : M = 64, N = 128, K = 64 rows i (P operand lives in the consumed y slab)
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            if (issuer) umma_bf16(tmem + kColO, desc_kmajor(st + kStY + kk * 32),
-                      desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescO, kk > 0);
-          }
-          // O += Qt S_in : K = 128 channels
+            for (int kk = 0; kk < 4; ++kk) {
+              umma_bf16(tmem + kColO, desc_kmajor(st + kStY + kk * 32),
+                        desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescO, kk > 0);
+            }
+            // O += Qt S_in : K = 128 channels
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            if (issuer) umma_bf16(tmem + kColO, desc_kmajor(q_sl[kk >> 2] + (kk & 3) * 32),
-                      desc_mnmajor(ss + kk * 2048, kSsSlabBytes), kIdescO, 1);
-          }
-          if (issuer) umma_commit(bar(BAR_OFULL));
-          // S = diag(D) S_in (already in TMEM) + Ke^T V : M = 128 channels, N = 128, K = 64 rows
+            for (int kk = 0; kk < 8; ++kk) {
+              umma_bf16(tmem + kColO, desc_kmajor(q_sl[kk >> 2] + (kk & 3) * 32),
+                        desc_mnmajor(ss + kk * 2048, kSsSlabBytes), kIdescO, 1);
+            }
+            umma_commit(bar(BAR_OFULL));
+            // S_in + Kt^T V : M = 128 channels, N = 128, K = 64 rows (S_in is already in TMEM)
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            if (issuer) umma_bf16(tmem + kColS, desc_mnmajor(x_lo + kk * 2048, x_hi - x_lo),
-                      desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescS, 1);
+            for (int kk = 0; kk < 4; ++kk) {
+              umma_bf16(tmem + kColS, desc_mnmajor(k_sl[0] + kk * 2048, k_sl[1] - k_sl[0]),
+                        desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescS, 1);
+            }
+            umma_commit(bar(BAR_SFULL));
+            umma_commit(bar(BAR_EMPTY0 + s));
           }
-          if (issuer) umma_commit(bar(BAR_SFULL));
-          if (issuer) umma_commit(bar(BAR_EMPTY0 + s));
           ++g;
         }
       }
     }
   } else if (warp >= kStateWarp0 && warp < kStateWarp0 + 4) {
     // ====================================== state group ======================================
+    // TMEM holds S_in + Kt^T V of the previous pass; the trip multiplies it by that pass's chunk
+    // decay (giving the state that enters this pass), keeps a bf16 copy for the readout and
+    // writes it back for this pass's accumulation.
     const int q4 = warp & 3;                              // TMEM lane quarter this warp may touch
     const int d = q4 * 32 + lane;                         // state row (key channel) of this thread
     const bool own_d = (d >> 6) == rank;
@@ -374,27 +452,38 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         continue;
       }
       bool last = false, first = true;
+      float Dprev = 1.f;                                  // chunk decay of the previous pass
       while (!last) {
         const uint32_t ph1 = g & 1;
         if (!first) {
           if (!(ok = mbar_wait(bar(BAR_SFULL), ph1 ^ 1, abort_flag, a.hdr))) break;  // pass g-1
           tc_fence_after();
-          // every contraction of pass g-1 has read its operands: the partner may overwrite
-          // the receive buffer that pass used
+          // every contraction of pass g-1 has read its operands: the partner may overwrite the
+          // receive buffer that pass used.  (Signalled before waiting for pass g: publishing
+          // pass g may itself need that buffer.)
           if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
         }
-        if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 1)), (g >> 1) & 1, abort_flag, a.hdr))) break;
+        // this pass's chunk decay (applied on the NEXT trip); read before this pass's
+        // contractions can start, so its stage and receive buffer are certainly still alive
+        if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 3)), (g >> 2) & 1, abort_flag, a.hdr))) break;
         const int s = ctl->pd[g & 3].stage;
         const int rxi = ctl->pd[g & 3].rx;
         last = (ctl->pd[g & 3].flags & kPassLast) != 0;
-        prev_rx = rxi;
-        const float D = own_d ? sD[s * kCH + (d & 63)] : sRx[rxi * kBlkFloats + (d & 63)];
+        const float Dcur = own_d ? sD[s * kCH + (d & 63)] : sRx[rxi * kBlkFloats + (d & 63)];
 #pragma unroll 1
         for (int piece = 0; piece < 4; ++piece) {
           uint32_t r[32];
           if (!first) {
             tmem_ld32(t_lane + kColS + piece * 32, r);
             tmem_ld_wait();
+            const float2 dd = splat(Dprev);
+#pragma unroll
+            for (int c2 = 0; c2 < 16; ++c2) {
+              const float2 t = __fmul2_rn(
+                  make_float2(__uint_as_float(r[2 * c2]), __uint_as_float(r[2 * c2 + 1])), dd);
+              r[2 * c2] = __float_as_uint(t.x);
+              r[2 * c2 + 1] = __float_as_uint(t.y);
+            }
           } else if (a.s0) {
 #pragma unroll
             for (int c4 = 0; c4 < 8; ++c4) {
@@ -419,14 +508,14 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                    pack_bf16(__uint_as_float(r[8 * c8 + 4]), __uint_as_float(r[8 * c8 + 5])),
                    pack_bf16(__uint_as_float(r[8 * c8 + 6]), __uint_as_float(r[8 * c8 + 7])));
           }
-#pragma unroll
-          for (int c4 = 0; c4 < 32; ++c4) r[c4] = __float_as_uint(__uint_as_float(r[c4]) * D);
           tmem_st32(t_lane + kColS + piece * 32, r);
         }
         tmem_st_wait();
         fence_proxy_async();
         tc_fence_before();
         mbar_arrive(bar(BAR_SREADY));
+        prev_rx = rxi;
+        Dprev = Dcur;
         first = false;
         ++g;
       }
@@ -446,8 +535,8 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 #pragma unroll
             for (int c4 = 0; c4 < 8; ++c4) {
               *reinterpret_cast<float4*>(a.sT + srow + piece * 32 + 4 * c4) =
-                  make_float4(__uint_as_float(r[4 * c4]), __uint_as_float(r[4 * c4 + 1]),
-                              __uint_as_float(r[4 * c4 + 2]), __uint_as_float(r[4 * c4 + 3]));
+                  make_float4(Dprev * __uint_as_float(r[4 * c4]), Dprev * __uint_as_float(r[4 * c4 + 1]),
+                              Dprev * __uint_as_float(r[4 * c4 + 2]), Dprev * __uint_as_float(r[4 * c4 + 3]));
             }
           }
         }
@@ -461,6 +550,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const bool has_row = lane < 16;
     const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
     __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(a.o);
+    const bool unit_scale = a.scale == 1.0f;
     uint32_t g = 0;
     bool ok = true;
     for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
@@ -480,27 +570,41 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // P exists, so the partner's copies out of ITS stage have all landed here (the issuer
           // waited for them): let the partner reuse that stage
           const int rxi = ctl->pd[g & 3].rx;
-          const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]) & 1;
+          const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]);
           mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
         }
+        // causal mask (i <= r kept).  This warp's rows are 16*q4 .. 16*q4+15, so of the two
+        // 32-column halves one is entirely kept or entirely dropped and one holds the diagonal.
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
+          const int c_lo = half * 32;
+          if (c_lo > q4 * 16 + 15) {                      // entirely above the diagonal
+            if (has_row) {
+#pragma unroll
+              for (int c8 = 0; c8 < 4; ++c8)
+                sts128(ps_row + (((half * 4 + c8) ^ (r_row & 7)) << 4), 0u, 0u, 0u, 0u);
+            }
+            continue;
+          }
           uint32_t r[32];
           tmem_ld32(t_lane + kColP + half * 32, r);
           tmem_ld_wait();
+          const bool diag = c_lo + 31 > q4 * 16;          // some column of this half exceeds a row
           if (has_row) {
 #pragma unroll
             for (int c8 = 0; c8 < 4; ++c8) {
               uint32_t w[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const int i0 = half * 32 + 8 * c8 + 2 * e;
-                const float lo = (i0 <= r_row) ? __uint_as_float(r[8 * c8 + 2 * e]) : 0.f;
-                const float hi = (i0 + 1 <= r_row) ? __uint_as_float(r[8 * c8 + 2 * e + 1]) : 0.f;
+                const int i0 = c_lo + 8 * c8 + 2 * e;
+                float lo = __uint_as_float(r[8 * c8 + 2 * e]), hi = __uint_as_float(r[8 * c8 + 2 * e + 1]);
+                if (diag) {
+                  lo = (i0 <= r_row) ? lo : 0.f;
+                  hi = (i0 + 1 <= r_row) ? hi : 0.f;
+                }
                 w[e] = pack_bf16(lo, hi);
               }
-              const int chunk = half * 4 + c8;
-              sts128(ps_row + ((chunk ^ (r_row & 7)) << 4), w[0], w[1], w[2], w[3]);
+              sts128(ps_row + (((half * 4 + c8) ^ (r_row & 7)) << 4), w[0], w[1], w[2], w[3]);
             }
           }
         }
@@ -511,6 +615,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (!(ok = mbar_wait(bar(BAR_OFULL), ph1, abort_flag, a.hdr))) break;
         tc_fence_after();
         __nv_bfloat16* orow = o + (row + r_row) * a.dv + it.col0;
+        const float2 sc2 = splat(a.scale);
 #pragma unroll 1
         for (int piece = 0; piece < 4; ++piece) {
           uint32_t r[32];
@@ -519,12 +624,14 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           if (has_row && r_row < nr) {
 #pragma unroll
             for (int c8 = 0; c8 < 4; ++c8) {
-              uint4 w;
-              w.x = pack_bf16(a.scale * __uint_as_float(r[8 * c8]), a.scale * __uint_as_float(r[8 * c8 + 1]));
-              w.y = pack_bf16(a.scale * __uint_as_float(r[8 * c8 + 2]), a.scale * __uint_as_float(r[8 * c8 + 3]));
-              w.z = pack_bf16(a.scale * __uint_as_float(r[8 * c8 + 4]), a.scale * __uint_as_float(r[8 * c8 + 5]));
-              w.w = pack_bf16(a.scale * __uint_as_float(r[8 * c8 + 6]), a.scale * __uint_as_float(r[8 * c8 + 7]));
-              *reinterpret_cast<uint4*>(orow + piece * 32 + 8 * c8) = w;
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                float2 t = make_float2(__uint_as_float(r[8 * c8 + 2 * e]), __uint_as_float(r[8 * c8 + 2 * e + 1]));
+                if (!unit_scale) t = __fmul2_rn(t, sc2);
+                w[e] = pack_bf16(t.x, t.y);
+              }
+              *reinterpret_cast<uint4*>(orow + piece * 32 + 8 * c8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
         }
@@ -536,11 +643,16 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   } else if (warp >= kGateWarp0) {
     // ======================================= gate group =======================================
     const int gw = warp - kGateWarp0;                     // rows 4*gw .. 4*gw+3 of the tile
-    const bool leader = gw == 0 && lane == 0;
-    constexpr float kLog2e = 1.4426950408889634f;
-    constexpr float kLg2Ln2 = -0.5287663729448977f;       // log2(ln 2)
-    constexpr float kRange = 60.f * kLog2e;               // largest in-chunk decay range, log2 units
-    uint32_t f = 0, g = 0, m = 0, sc = 0;                 // fills seen, passes, attempts, scan syncs
+    const bool lead_warp = gw == kGateWarps - 1;          // its running sum is the chunk total
+    const bool leader = lead_warp && lane == 0;
+    uint32_t off[4];   // swizzled byte offsets of the thread's element pairs inside a slab
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = gw * 4 + i;
+      off[i] = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
+    }
+    uint32_t fs = 0, fph = 0;                             // stage and phase of the next fill
+    uint32_t g = 0, m = 0, sc = 0;                        // passes, attempts, scan syncs
     bool ok = true;
     bool armed = false;                                   // attempt m's receive barriers expect bytes
     auto group_sync = [&]() -> bool {                     // bounded barrier over the gate warps
@@ -560,106 +672,63 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       const Item it = decode_item(a, item_of(j), rank);
       int tpos = 0, lcap = kC;
       while (ok && tpos < it.len) {
-        const uint32_t s = f & 1, ph = (f >> 1) & 1;
+        const uint32_t s = fs;
         const uint32_t st = stage_base + s * kStageBytes;
-        if (!(ok = mbar_wait(bar(BAR_FULL0 + s), ph, abort_flag, a.hdr))) break;
-        ++f;
+        if (!(ok = mbar_wait(bar(BAR_FULL0 + s), fph, abort_flag, a.hdr))) break;
+        if (++fs == kStages) { fs = 0; fph ^= 1; }
         if (ctl->tag[s][0] != j || ctl->tag[s][1] != tpos) {
           // speculative fill for a position we are not at: hand the stage back unused
           if (!(ok = group_sync())) break;
           if (leader) mbar_arrive_cnt(bar(BAR_EMPTY0 + s), 2);   // nothing was sent from it
           continue;
         }
-        // ---- attempt m: the partner's receive buffer m&1 must be free before we send into it
+        // ---- attempt m
         const uint32_t rxi = m & 1, rxph = (m >> 1) & 1;
-        if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
-        if (leader) {
-          mbar_expect_tx(bar(BAR_PEER0 + rxi), kRxBytes);
-          mbar_expect_tx(bar(BAR_VERD0 + rxi), kBlkBytes);
-          armed = true;
-        }
         const int left = it.len - tpos;
         const int nr = min(min(kC, left), lcap);
-        // element (row r, own channels 2*lane, +1) sits at this swizzled byte offset of a slab
-        float bq[4][2];   // inclusive in-chunk cumulative log2 decay (own rows only, so far)
-        float eh[4][2];   // log2 ahat
-        float run0 = 0.f, run1 = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int r = gw * 4 + i;
-          const uint32_t off = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
-          const uint32_t xw = lds32(st + kStX + off), yw = lds32(st + kStY + off);
-          const float xs[2] = {__uint_as_float(xw << 16), __uint_as_float(xw & 0xFFFF0000u)};
-          const float ys[2] = {__uint_as_float(yw << 16), __uint_as_float(yw & 0xFFFF0000u)};
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const float u = ex2f(xs[e] * kLog2e);                       // e^x
-            // g * log2(e) = log2(1 + e^x); series when 1 + u would round u away
-            const float sp2 = u < 9.765625e-4f ? u * (kLog2e - 0.72134752f * u) : lg2f(1.f + u);
-            const float tau = rcpf(1.f + ex2f(-ys[e] * kLog2e));
-            float l2a = fmaxf(-sp2 * tau, -kRange);                     // per-step floor exp(-60)
-            float l2h;
-            if (INGATE == RODIMUS_INGATE_POW_G) {
-              l2h = tau * (lg2f(sp2) + kLg2Ln2);                        // tau * log2(g)
-            } else {
-              l2h = tau * (xs[e] * kLog2e - sp2);                       // tau * log2(sigmoid(x))
-            }
-            if (r >= nr) l2a = 0.f;                                     // rows past the pass
-            if (e == 0) { run0 += l2a; bq[i][0] = run0; } else { run1 += l2a; bq[i][1] = run1; }
-            eh[i][e] = l2h;
-          }
-        }
-        // exclusive prefix over the 16 row groups, and the chunk total
+        float2 b[4], eh[4], run;
+        if (nr == kC) run = gate_phase1<INGATE, true>(st + kStX, st + kStY, off, gw * 4, nr, b, eh);
+        else          run = gate_phase1<INGATE, false>(st + kStX, st + kStY, off, gw * 4, nr, b, eh);
+        // exclusive prefix over the row groups below this warp's
         float* tot = sTot + (m & 1) * (kGateWarps * kCH);
-        *reinterpret_cast<float2*>(tot + gw * kCH + 2 * lane) = make_float2(run0, run1);
+        *reinterpret_cast<float2*>(tot + gw * kCH + 2 * lane) = run;
         if (!(ok = group_sync())) break;
-        float pre0 = 0.f, pre1 = 0.f, all0 = 0.f, all1 = 0.f;
-#pragma unroll
-        for (int w = 0; w < kGateWarps; ++w) {
-          const float2 t = *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane);
-          if (w < gw) { pre0 += t.x; pre1 += t.y; }
-          all0 += t.x; all1 += t.y;
-        }
-        // every warp sees all 64 own channels' totals, so all sixteen reach the same verdict
-        const bool viol_own = __any_sync(0xffffffffu, all0 < -kRange || all1 < -kRange) && nr > 1;
-        const float D0 = ex2f(all0), D1 = ex2f(all1);
-        if (gw == 0) {
-          // chunk decays of the own channels: for this CTA's state group and for the partner's
-          *reinterpret_cast<float2*>(sD + s * kCH + 2 * lane) = make_float2(D0, D1);
+        float2 pre = splat(0.f);
+#pragma unroll 1
+        for (int w = 0; w < gw; ++w)
+          pre = __fadd2_rn(pre, *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane));
+        // the partner's receive buffer m&1 (and this CTA's send block m&1) must be free again
+        if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
+        if (lead_warp) {
+          // chunk totals of the own 64 channels: decays for both state groups, and the verdict
+          const float2 all = __fadd2_rn(pre, run);
+          const bool viol_own = __any_sync(0xffffffffu, all.x < -kRange || all.y < -kRange) && nr > 1;
+          const float2 D = make_float2(ex2f(all.x), ex2f(all.y));
+          *reinterpret_cast<float2*>(sD + s * kCH + 2 * lane) = D;
           volatile float* blk = sTx + rxi * kBlkFloats;
-          blk[2 * lane] = D0;
-          blk[2 * lane + 1] = D1;
+          blk[2 * lane] = D.x;
+          blk[2 * lane + 1] = D.y;
           if (lane == 0) {
             blk[64] = __int_as_float(viol_own ? 1 : 0);
             blk[65] = __int_as_float((int)s);
           }
           fence_proxy_async();
           __syncwarp();
-          if (lane == 0)
-            dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
-                            base + kOffTx + rxi * kBlkBytes, kBlkBytes,
-                            map_to_cta(bar(BAR_VERD0 + rxi), peer));
         }
-        if (!viol_own) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int r = gw * 4 + i;
-            const uint32_t off = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
-            const uint32_t qw = lds32(st + kStQ + off), kw = lds32(st + kStK + off);
-            const float b0 = bq[i][0] + pre0, b1 = bq[i][1] + pre1;
-            const bool live = r < nr;
-            const float q0 = live ? __uint_as_float(qw << 16) : 0.f;
-            const float q1 = live ? __uint_as_float(qw & 0xFFFF0000u) : 0.f;
-            const float k0 = live ? __uint_as_float(kw << 16) : 0.f;
-            const float k1 = live ? __uint_as_float(kw & 0xFFFF0000u) : 0.f;
-            const float kt0 = k0 * ex2f(eh[i][0] - b0), kt1 = k1 * ex2f(eh[i][1] - b1);
-            sts32(st + kStQ + off, pack_bf16(q0 * ex2f(b0), q1 * ex2f(b1)));
-            sts32(st + kStK + off, pack_bf16(kt0, kt1));
-            sts32(st + kStX + off, pack_bf16(kt0 * D0, kt1 * D1));       // 2^{b_C - b_i} = 2^{-b_i} D
-          }
+        if (leader) {
+          // own verdict is in place (the arrive publishes it to the other gate warps); the
+          // partner's block and slabs complete the two barriers by byte count
+          mbar_expect_tx(bar(BAR_VERD0 + rxi), kBlkBytes);
+          mbar_expect_tx(bar(BAR_PEER0 + rxi), kRxBytes);
+          armed = true;
+          dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
+                          base + kOffTx + rxi * kBlkBytes, kBlkBytes,
+                          map_to_cta(bar(BAR_VERD0 + rxi), peer));
         }
+        if (nr == kC) gate_phase2<true>(st + kStQ, st + kStK, off, gw * 4, nr, pre, b, eh);
+        else          gate_phase2<false>(st + kStQ, st + kStK, off, gw * 4, nr, pre, b, eh);
         // this warp's four rows of each operand slab go to the partner (also when the attempt
-        // is about to be abandoned: the byte count the partner's barrier expects is fixed)
+        // turns out to be abandoned: the byte count the partner's barrier expects is fixed)
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) {
@@ -668,11 +737,11 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
           dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, 512, pb);
           dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK + rows_off, 512, pb);
-          dsmem_bulk_copy(map_to_cta(dst + kRxX, peer), st + kStX + rows_off, 512, pb);
         }
-        // the partner's verdict came with its decay block
+        // both verdicts: the own one (lead warp) and the partner's (came with its decay block)
         if (!(ok = mbar_wait_cluster(bar(BAR_VERD0 + rxi), rxph, abort_flag, a.hdr))) break;
-        const bool viol = viol_own || (__float_as_int(sRx[rxi * kBlkFloats + 64]) != 0);
+        const bool viol = (__float_as_int(sTx[rxi * kBlkFloats + 64]) |
+                           __float_as_int(sRx[rxi * kBlkFloats + 64])) != 0;
         ++m;
         armed = false;
         if (viol) {
@@ -683,7 +752,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             // whatever the partner sent for this attempt must have landed before its buffer and
             // its stage are declared reusable
             if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
-            const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]) & 1;
+            const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]);
             mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
             mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + rxi), peer));
             redirect(j, tpos);
@@ -702,7 +771,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           if (nr < min(kC, left)) redirect(j, tpos + nr);   // the prefetcher assumed 64 rows
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_GATED0 + (g & 1)));
+        if (lane == 0) mbar_arrive(bar(BAR_GATED0 + (g & 3)));
         ++g;
         tpos += nr;
         if (lcap < kC) lcap = min(kC, lcap * 2);
