@@ -129,6 +129,40 @@ int rodimus_ddts_fwd(const rodimus_ddts_fwd_params *p);
 int rodimus_ddts_step(const rodimus_ddts_step_params *p);
 
 /*
+ * rodimus_ddts_fwd for callers that cannot allocate device memory.  (A convenience of this
+ * library: the paper has no counterpart.)
+ *
+ * Who needs it: code that receives only input and output buffers and has no allocator to turn
+ * to -- a plug-in inside an application that distributed all device memory at start-up, a
+ * serving loop that must never hit cudaMalloc's device-wide synchronisation, a runtime that
+ * forbids allocation after initialisation.  rodimus_ddts_fwd needs a small workspace from its
+ * caller; this variant uses a fixed array inside the library's device image instead
+ * (256 + 4 * RODIMUS_NOALLOC_MAX_SEQS bytes, present on every GPU that loads the library, for
+ * the life of the process).  It allocates and frees nothing, on the device or through any
+ * library.
+ *
+ * p is read exactly as by rodimus_ddts_fwd, except that p->workspace and p->workspace_bytes are
+ * ignored.  Limit: a packed (cu_seqlens) call may hold at most RODIMUS_NOALLOC_MAX_SEQS
+ * sequences; more returns RODIMUS_ERR_WORKSPACE before anything is launched.  Every other
+ * status is that of rodimus_ddts_fwd; RODIMUS_ERR_CUDA also covers a failed look-up of the
+ * array's address.
+ *
+ * The first call on each device looks up that device's address of the array (with the device
+ * current, once, under a lock); make that first call outside any stream capture.
+ *
+ * All calls on a device share the one array, and it keeps the previous call's contents.  Nothing
+ * in it needs clearing by the caller: each call rewrites what it later reads.  But two calls
+ * whose kernels may overlap on the GPU (different streams, no dependency) race on it; order
+ * them.
+ *
+ * status_handle, if not NULL, receives a device pointer to pass as `workspace` to
+ * rodimus_ddts_device_status (NULL if the call failed); it stays valid until the next call on
+ * the same device overwrites what it points at.
+ */
+#define RODIMUS_NOALLOC_MAX_SEQS 4096
+int rodimus_ddts_fwd_noalloc(const rodimus_ddts_fwd_params *p, const void **status_handle);
+
+/*
  * Waits for `stream`, then returns what the kernels of the last rodimus_ddts_fwd call that
  * used `workspace` recorded: RODIMUS_OK, RODIMUS_ERR_SEQLENS (device-side cu_seqlens check)
  * or RODIMUS_ERR_TIMEOUT (a bounded wait ran out; outputs are then unspecified).

@@ -23,7 +23,9 @@ EXPORTED_SYMBOLS = (
     "rodimus_ddts_fwd_workspace_bytes", "rodimus_ddts_fwd", "rodimus_ddts_step",
     "rodimus_ddts_device_status", "rodimus_ddts_last_launch_count",
     "rodimus_ddts_fwd_kernel_name", "rodimus_status_str", "rodimus_version",
+    "rodimus_ddts_fwd_noalloc",
 )
+NOALLOC_MAX_SEQS = 4096
 
 
 class RodimusError(RuntimeError):
@@ -76,6 +78,9 @@ def load_library() -> ctypes.CDLL:
         lib.rodimus_ddts_fwd_workspace_bytes.restype = ctypes.c_size_t
         lib.rodimus_ddts_fwd.argtypes = [ctypes.POINTER(FwdParams)]
         lib.rodimus_ddts_fwd.restype = ctypes.c_int
+        lib.rodimus_ddts_fwd_noalloc.argtypes = [ctypes.POINTER(FwdParams),
+                                                 ctypes.POINTER(ctypes.c_void_p)]
+        lib.rodimus_ddts_fwd_noalloc.restype = ctypes.c_int
         lib.rodimus_ddts_step.argtypes = [ctypes.POINTER(StepParams)]
         lib.rodimus_ddts_step.restype = ctypes.c_int
         lib.rodimus_ddts_device_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
@@ -155,6 +160,22 @@ def fwd_kernel_name(p: FwdParams) -> str:
 def fwd_raw(p: FwdParams) -> int:
     """Calls ``rodimus_ddts_fwd`` and returns its status without raising."""
     return int(load_library().rodimus_ddts_fwd(ctypes.byref(p)))
+
+
+def fwd_noalloc_raw(p: FwdParams):
+    """Calls ``rodimus_ddts_fwd_noalloc`` (the prefill that uses the library's built-in scratch
+    array instead of a caller workspace).  Returns (status, handle); the handle is an integer
+    device address accepted by ``device_status_ptr``, or None if the call failed."""
+    h = ctypes.c_void_p()
+    rc = int(load_library().rodimus_ddts_fwd_noalloc(ctypes.byref(p), ctypes.byref(h)))
+    return rc, h.value
+
+
+def device_status_ptr(ptr: int, stream: Optional[int] = None) -> int:
+    """``rodimus_ddts_device_status`` for a raw device address (see ``fwd_noalloc_raw``)."""
+    import torch
+    st = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    return int(load_library().rodimus_ddts_device_status(ptr, st))
 
 
 def step_raw(p: StepParams) -> int:

@@ -160,3 +160,13 @@ def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(rd, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         rd.load_library()
+
+
+def test_noalloc_entry_point_argument_errors_need_no_device(lib):
+    """The checks that come before the built-in scratch array is looked up."""
+    h = ctypes.c_void_p(1)
+    assert lib.rodimus_ddts_fwd_noalloc(None, ctypes.byref(h)) == rd.ERR_NULL and h.value is None
+    p = _fwd(struct_size=8)
+    assert rd.fwd_noalloc_raw(p) == (rd.ERR_DTYPE, None)
+    p = _fwd(B=1, N=rd.NOALLOC_MAX_SEQS + 1, cu_seqlens=FAKE)
+    assert rd.fwd_noalloc_raw(p) == (rd.ERR_WORKSPACE, None)
