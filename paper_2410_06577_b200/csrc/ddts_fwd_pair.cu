@@ -21,12 +21,20 @@
 // The pair advances in lockstep: which rows form a pass is decided from the decay totals of all
 // 128 channels, so each CTA sends its verdict along with its chunk decays and both take the OR.
 //
-// Roles in one CTA (26 warps), connected by mbarriers; every wait is bounded:
+// Roles in one CTA (27 warps), connected by mbarriers; every wait is bounded:
 //   warp 0        TMA producer (own channel slab of q,k,x,y and both slabs of the v slice)
 //   warp 1        tcgen05.mma issuer, owns the TMEM allocation
 //   warps 2-5     state group: TMEM <-> registers trip of S, initial / final state I/O
 //   warps 6-9     score / output group
 //   warps 10-25   gate group: 4 rows x 2 channels per thread, packed fp32x2 arithmetic
+//   warp 26       gate control: chunk totals, verdict exchange with the partner, publishing
+//
+// The loop-carried chain is  state update of pass g -> rescaling of S -> state update of pass
+// g+1 , so the issuer puts the state update of a pass BEFORE its output contractions, and the
+// state lives in TWO TMEM buffers used alternately: the state group reads S_in + Kt^T V of the
+// previous pass from one, writes D times it into the other (which frees the next state update
+// at once), and afterwards, off the chain, reads the old buffer again to make the bf16 copy
+// that the readout takes as an operand.
 #include <cuda.h>
 
 #include <cstring>
@@ -68,20 +76,23 @@ constexpr int kSmemBytes = kSmemUsed + 1024;              // slack for manual 10
 static_assert(kOffTx % 16 == 0 && kOffRx % 16 == 0 && kBlkBytes % 16 == 0, "bulk copy alignment");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
-constexpr int kThreads = 32 * (kGateWarp0 + kGateWarps);  // 832
+constexpr int kThreads = 32 * (kGateWarp0 + kGateWarps + 1);  // 864: 16 gate warps + control
 constexpr int kStateWarp0 = 2, kScoreWarp0 = 6;
 
-// TMEM columns (fp32 words): state, output, scores
-constexpr uint32_t kColS = 0, kColO = 128, kColP = 256, kTmemCols = 512;
+// TMEM columns (fp32 words): two state buffers, output, scores
+constexpr uint32_t kColS = 0, kColO = 256, kColP = 384, kTmemCols = 512;
 
 // mbarrier indices
 enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                      (1 + bytes)
        BAR_EMPTY0 = 3,                // [3] stage reusable: own release + partner's receipt (2)
-       BAR_GATED0 = 6,                // [4] pass published by the gate group             (16)
+       BAR_GATED0 = 6,                // [4] pass published by the gate group             (17)
        BAR_PEER0 = 10, BAR_PEER1,     // partner's two slabs landed                 (1 + bytes)
        BAR_VERD0, BAR_VERD1,          // own verdict written + partner's block landed (1 + bytes)
        BAR_RXFREE0, BAR_RXFREE1,      // partner is done with ITS receive buffer            (1)
-       BAR_PFULL, BAR_PREADY, BAR_SREADY, BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN };
+       BAR_PFULL, BAR_PREADY,
+       BAR_SREADY_S,                  // S rescaled in TMEM: the state update may accumulate (128)
+       BAR_SREADY_O,                  // bf16 copy of S_in in shared memory: the readout may run (128)
+       BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN };
 static_assert(BAR_GSCAN < kNumBars, "barrier count");
 
 struct PairArgs {
@@ -167,7 +178,7 @@ __device__ __forceinline__ float2 splat(float v) { return make_float2(v, v); }
 
 // Phase 1 for this thread's 4 rows x 2 channels: log2 decay (cumulative over the thread's own
 // rows, b) and log2 input weight (eh).  Returns the sum of the four rows' log2 decays.
-template <int INGATE, bool FULL>
+template <int INGATE>
 __device__ __forceinline__ float2 gate_phase1(uint32_t xs, uint32_t ys, const uint32_t (&off)[4],
                                               int row0, int nr, float2 (&b)[4], float2 (&eh)[4]) {
   float2 run = splat(0.f);
@@ -195,7 +206,7 @@ __device__ __forceinline__ float2 gate_phase1(uint32_t xs, uint32_t ys, const ui
     } else {                                                            // tau * log2(sigmoid(x))
       eh[i] = __fmul2_rn(ntau, __ffma2_rn(xl, splat(-1.f), sp2));
     }
-    if (!FULL && row0 + i >= nr) l2a = splat(0.f);                      // rows past the pass
+    if (row0 + i >= nr) l2a = splat(0.f);                               // rows past the pass
     run = __fadd2_rn(run, l2a);
     b[i] = run;
   }
@@ -203,7 +214,6 @@ __device__ __forceinline__ float2 gate_phase1(uint32_t xs, uint32_t ys, const ui
 }
 
 // Phase 2: Qt = q 2^{b}, Kt = k 2^{eh - b}, written over q and k (same swizzled offsets).
-template <bool FULL>
 __device__ __forceinline__ void gate_phase2(uint32_t qs, uint32_t ks, const uint32_t (&off)[4],
                                             int row0, int nr, float2 pre, const float2 (&b)[4],
                                             const float2 (&eh)[4]) {
@@ -215,7 +225,7 @@ __device__ __forceinline__ void gate_phase2(uint32_t qs, uint32_t ks, const uint
     const float2 hb = __ffma2_rn(bb, splat(-1.f), eh[i]);
     const float2 eq = make_float2(ex2f(bb.x), ex2f(bb.y));
     const float2 ek = make_float2(ex2f(hb.x), ex2f(hb.y));
-    if (!FULL && row0 + i >= nr) { q = splat(0.f); k = splat(0.f); }
+    if (row0 + i >= nr) { q = splat(0.f); k = splat(0.f); }
     const float2 qt = __fmul2_rn(q, eq), kt = __fmul2_rn(k, ek);
     sts32(qs + off[i], pack_bf16(qt.x, qt.y));
     sts32(ks + off[i], pack_bf16(kt.x, kt.y));
@@ -260,7 +270,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       mbar_init(bar(BAR_FULL0 + s), 1);
       mbar_init(bar(BAR_EMPTY0 + s), 2);
     }
-    for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_GATED0 + i), kGateWarps);
+    for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_GATED0 + i), kGateWarps + 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(BAR_PEER0 + i), 1);
       mbar_init(bar(BAR_VERD0 + i), 1);
@@ -268,11 +278,12 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
     mbar_init(bar(BAR_PFULL), 1);
     mbar_init(bar(BAR_PREADY), 128);
-    mbar_init(bar(BAR_SREADY), 128);
+    mbar_init(bar(BAR_SREADY_S), 128);
+    mbar_init(bar(BAR_SREADY_O), 128);
     mbar_init(bar(BAR_SFULL), 1);
     mbar_init(bar(BAR_OFULL), 1);
     mbar_init(bar(BAR_OFREE), 128);
-    mbar_init(bar(BAR_GSCAN), kGateWarps);
+    mbar_init(bar(BAR_GSCAN), kGateWarps + 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -393,8 +404,19 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             }
             umma_commit(bar(BAR_PFULL));
           }
+          if (!(ok = mbar_wait(bar(BAR_SREADY_S), ph1, abort_flag, a.hdr))) break;
+          tc_fence_after();
+          if (issuer) {
+            // S_in + Kt^T V : M = 128 channels, N = 128, K = 64 rows (S_in sits in buffer g & 1)
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              umma_bf16(tmem + kColS + (g & 1) * 128, desc_mnmajor(k_sl[0] + kk * 2048, k_sl[1] - k_sl[0]),
+                        desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescS, 1);
+            }
+            umma_commit(bar(BAR_SFULL));
+          }
           if (!(ok = mbar_wait(bar(BAR_PREADY), ph1, abort_flag, a.hdr))) break;
-          if (!(ok = mbar_wait(bar(BAR_SREADY), ph1, abort_flag, a.hdr))) break;
+          if (!(ok = mbar_wait(bar(BAR_SREADY_O), ph1, abort_flag, a.hdr))) break;
           if (!(ok = mbar_wait(bar(BAR_OFREE), ph1 ^ 1, abort_flag, a.hdr))) break;
           tc_fence_after();
           if (issuer) {
@@ -411,14 +433,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                         desc_mnmajor(ss + kk * 2048, kSsSlabBytes), kIdescO, 1);
             }
             umma_commit(bar(BAR_OFULL));
-            // S_in + Kt^T V : M = 128 channels, N = 128, K = 64 rows (S_in is already in TMEM)
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              umma_bf16(tmem + kColS, desc_mnmajor(k_sl[0] + kk * 2048, k_sl[1] - k_sl[0]),
-                        desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescS, 1);
-            }
-            umma_commit(bar(BAR_SFULL));
-            umma_commit(bar(BAR_EMPTY0 + s));
+            umma_commit(bar(BAR_EMPTY0 + s));   // every contraction of the pass has read its operands
           }
           ++g;
         }
@@ -426,13 +441,16 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
   } else if (warp >= kStateWarp0 && warp < kStateWarp0 + 4) {
     // ====================================== state group ======================================
-    // TMEM holds S_in + Kt^T V of the previous pass; the trip multiplies it by that pass's chunk
-    // decay (giving the state that enters this pass), keeps a bf16 copy for the readout and
-    // writes it back for this pass's accumulation.
+    // Pass g accumulates its state update in TMEM buffer g & 1.  Each thread owns one state row
+    // (key channel).  Step 1 reads S_in + Kt^T V of pass g-1 from the other buffer, multiplies
+    // by that pass's chunk decay and writes the result, the state entering pass g, into buffer
+    // g & 1: the state update of pass g may start.  Step 2 reads the old buffer again and stores
+    // the same product as bf16 in shared memory for the readout, once the readout of pass g-1
+    // has finished with the previous copy.
     const int q4 = warp & 3;                              // TMEM lane quarter this warp may touch
     const int d = q4 * 32 + lane;                         // state row (key channel) of this thread
     const bool own_d = (d >> 6) == rank;
-    const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
+    const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16) + kColS;
     const uint32_t ss_row = base + kOffSs + d * 128;
     const bool signaller = warp == kStateWarp0 && lane == 0;
     uint32_t g = 0;
@@ -453,51 +471,71 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
       bool last = false, first = true;
       float Dprev = 1.f;                                  // chunk decay of the previous pass
+      // 32 columns of the state entering the pass: D_prev times the previous buffer, or the
+      // caller's initial state for the first pass of a sequence
+      auto load_piece = [&](uint32_t (&r)[32], uint32_t t_prev, int piece) {
+        if (!first) {
+          tmem_ld32(t_prev + piece * 32, r);
+          tmem_ld_wait();
+          const float2 dd = splat(Dprev);
+#pragma unroll
+          for (int c2 = 0; c2 < 16; ++c2) {
+            const float2 t = __fmul2_rn(
+                make_float2(__uint_as_float(r[2 * c2]), __uint_as_float(r[2 * c2 + 1])), dd);
+            r[2 * c2] = __float_as_uint(t.x);
+            r[2 * c2 + 1] = __float_as_uint(t.y);
+          }
+        } else if (a.s0) {
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4) {
+            const float4 v4 = *reinterpret_cast<const float4*>(a.s0 + srow + piece * 32 + 4 * c4);
+            r[4 * c4] = __float_as_uint(v4.x);
+            r[4 * c4 + 1] = __float_as_uint(v4.y);
+            r[4 * c4 + 2] = __float_as_uint(v4.z);
+            r[4 * c4 + 3] = __float_as_uint(v4.w);
+          }
+        } else {
+#pragma unroll
+          for (int c4 = 0; c4 < 32; ++c4) r[c4] = 0u;
+        }
+      };
       while (!last) {
         const uint32_t ph1 = g & 1;
+        const uint32_t t_cur = t_lane + (g & 1) * 128, t_prev = t_lane + ((g & 1) ^ 1) * 128;
         if (!first) {
           if (!(ok = mbar_wait(bar(BAR_SFULL), ph1 ^ 1, abort_flag, a.hdr))) break;  // pass g-1
           tc_fence_after();
-          // every contraction of pass g-1 has read its operands: the partner may overwrite the
-          // receive buffer that pass used.  (Signalled before waiting for pass g: publishing
-          // pass g may itself need that buffer.)
+        }
+        // step 1: the state entering this pass, into this pass's buffer
+#pragma unroll 1
+        for (int piece = 0; piece < 4; ++piece) {
+          uint32_t r[32];
+          load_piece(r, t_prev, piece);
+          tmem_st32(t_cur + piece * 32, r);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_SREADY_S));
+        if (!first) {
+          // the previous pass's readout has finished with the old copy (and, with its state
+          // update, with every operand of that pass: the partner may reuse the receive buffer).
+          // Signalled before waiting for pass g: publishing pass g may itself need that buffer.
+          if (!(ok = mbar_wait(bar(BAR_OFULL), ph1 ^ 1, abort_flag, a.hdr))) break;
           if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
         }
-        // this pass's chunk decay (applied on the NEXT trip); read before this pass's
-        // contractions can start, so its stage and receive buffer are certainly still alive
+        // this pass's chunk decay (applied on the NEXT trip); read before this pass's readout
+        // can be issued, so its stage and receive buffer are certainly still alive
         if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 3)), (g >> 2) & 1, abort_flag, a.hdr))) break;
         const int s = ctl->pd[g & 3].stage;
         const int rxi = ctl->pd[g & 3].rx;
         last = (ctl->pd[g & 3].flags & kPassLast) != 0;
         const float Dcur = own_d ? sD[s * kCH + (d & 63)] : sRx[rxi * kBlkFloats + (d & 63)];
+        // step 2: bf16 copy of the same state for the readout: MN-major, row d, two 64-column
+        // slabs.  (The old buffer is untouched until the NEXT pass's step 1.)
 #pragma unroll 1
         for (int piece = 0; piece < 4; ++piece) {
           uint32_t r[32];
-          if (!first) {
-            tmem_ld32(t_lane + kColS + piece * 32, r);
-            tmem_ld_wait();
-            const float2 dd = splat(Dprev);
-#pragma unroll
-            for (int c2 = 0; c2 < 16; ++c2) {
-              const float2 t = __fmul2_rn(
-                  make_float2(__uint_as_float(r[2 * c2]), __uint_as_float(r[2 * c2 + 1])), dd);
-              r[2 * c2] = __float_as_uint(t.x);
-              r[2 * c2 + 1] = __float_as_uint(t.y);
-            }
-          } else if (a.s0) {
-#pragma unroll
-            for (int c4 = 0; c4 < 8; ++c4) {
-              const float4 v4 = *reinterpret_cast<const float4*>(a.s0 + srow + piece * 32 + 4 * c4);
-              r[4 * c4] = __float_as_uint(v4.x);
-              r[4 * c4 + 1] = __float_as_uint(v4.y);
-              r[4 * c4 + 2] = __float_as_uint(v4.z);
-              r[4 * c4 + 3] = __float_as_uint(v4.w);
-            }
-          } else {
-#pragma unroll
-            for (int c4 = 0; c4 < 32; ++c4) r[c4] = 0u;
-          }
-          // bf16 copy of S_in for the readout: MN-major, row d, 64-column slab piece/2
+          load_piece(r, t_prev, piece);
           const uint32_t slab = ss_row + (piece >> 1) * kSsSlabBytes;
 #pragma unroll
           for (int c8 = 0; c8 < 4; ++c8) {
@@ -508,12 +546,9 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                    pack_bf16(__uint_as_float(r[8 * c8 + 4]), __uint_as_float(r[8 * c8 + 5])),
                    pack_bf16(__uint_as_float(r[8 * c8 + 6]), __uint_as_float(r[8 * c8 + 7])));
           }
-          tmem_st32(t_lane + kColS + piece * 32, r);
         }
-        tmem_st_wait();
         fence_proxy_async();
-        tc_fence_before();
-        mbar_arrive(bar(BAR_SREADY));
+        mbar_arrive(bar(BAR_SREADY_O));
         prev_rx = rxi;
         Dprev = Dcur;
         first = false;
@@ -524,13 +559,15 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       {
         const uint32_t lastg = g - 1;
         if (!(ok = mbar_wait(bar(BAR_SFULL), lastg & 1, abort_flag, a.hdr))) break;
+        if (!(ok = mbar_wait(bar(BAR_OFULL), lastg & 1, abort_flag, a.hdr))) break;
         tc_fence_after();
         if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
         if (a.sT) {
+          const uint32_t t_fin = t_lane + (lastg & 1) * 128;
 #pragma unroll 1
           for (int piece = 0; piece < 4; ++piece) {
             uint32_t r[32];
-            tmem_ld32(t_lane + kColS + piece * 32, r);
+            tmem_ld32(t_fin + piece * 32, r);
             tmem_ld_wait();
 #pragma unroll
             for (int c4 = 0; c4 < 8; ++c4) {
@@ -641,10 +678,13 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
     }
   } else if (warp >= kGateWarp0) {
-    // ======================================= gate group =======================================
+    // ============================== gate group and its control warp ==============================
+    // The sixteen gate warps do the per-element work; the control warp does everything that is
+    // serial (chunk totals, decays, verdict, the block for the partner, publishing the pass), so
+    // that none of it sits between the two phases of a gate warp.
     const int gw = warp - kGateWarp0;                     // rows 4*gw .. 4*gw+3 of the tile
-    const bool lead_warp = gw == kGateWarps - 1;          // its running sum is the chunk total
-    const bool leader = lead_warp && lane == 0;
+    const bool is_ctl = gw == kGateWarps;
+    const bool leader = is_ctl && lane == 0;
     uint32_t off[4];   // swizzled byte offsets of the thread's element pairs inside a slab
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -655,7 +695,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     uint32_t g = 0, m = 0, sc = 0;                        // passes, attempts, scan syncs
     bool ok = true;
     bool armed = false;                                   // attempt m's receive barriers expect bytes
-    auto group_sync = [&]() -> bool {                     // bounded barrier over the gate warps
+    auto group_sync = [&]() -> bool {                     // bounded barrier over the 17 warps
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_GSCAN));
       const bool r = mbar_wait(bar(BAR_GSCAN), sc & 1, abort_flag, a.hdr);
@@ -686,25 +726,45 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const uint32_t rxi = m & 1, rxph = (m >> 1) & 1;
         const int left = it.len - tpos;
         const int nr = min(min(kC, left), lcap);
-        float2 b[4], eh[4], run;
-        if (nr == kC) run = gate_phase1<INGATE, true>(st + kStX, st + kStY, off, gw * 4, nr, b, eh);
-        else          run = gate_phase1<INGATE, false>(st + kStX, st + kStY, off, gw * 4, nr, b, eh);
-        // exclusive prefix over the row groups below this warp's
         float* tot = sTot + (m & 1) * (kGateWarps * kCH);
-        *reinterpret_cast<float2*>(tot + gw * kCH + 2 * lane) = run;
-        if (!(ok = group_sync())) break;
-        float2 pre = splat(0.f);
-#pragma unroll 1
-        for (int w = 0; w < gw; ++w)
-          pre = __fadd2_rn(pre, *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane));
-        // the partner's receive buffer m&1 (and this CTA's send block m&1) must be free again
-        if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
-        if (lead_warp) {
+        if (!is_ctl) {
+          float2 b[4], eh[4];
+          const float2 run = gate_phase1<INGATE>(st + kStX, st + kStY, off, gw * 4, nr, b, eh);
+          *reinterpret_cast<float2*>(tot + gw * kCH + 2 * lane) = run;
+          if (!(ok = group_sync())) break;
+          // exclusive prefix over the row groups below this warp's
+          float2 pre = splat(0.f);
+#pragma unroll
+          for (int w = 0; w < kGateWarps - 1; ++w) {        // all loads in flight at once
+            const float2 t = *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane);
+            if (w < gw) pre = __fadd2_rn(pre, t);
+          }
+          gate_phase2(st + kStQ, st + kStK, off, gw * 4, nr, pre, b, eh);
+          // this warp's four rows of each operand slab go to the partner (also when the attempt
+          // turns out to be abandoned: the byte count the partner's barrier expects is fixed),
+          // once the partner's receive buffer m&1 is free again
+          fence_proxy_async();
+          if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
+          __syncwarp();
+          if (lane == 0) {
+            const uint32_t rows_off = gw * 512;
+            const uint32_t dst = peer_rx_base + rxi * kRxBytes + rows_off;
+            const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
+            dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, 512, pb);
+            dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK + rows_off, 512, pb);
+          }
+        } else {
+          if (!(ok = group_sync())) break;
           // chunk totals of the own 64 channels: decays for both state groups, and the verdict
-          const float2 all = __fadd2_rn(pre, run);
+          float2 all = splat(0.f);
+#pragma unroll
+          for (int w = 0; w < kGateWarps; ++w)
+            all = __fadd2_rn(all, *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane));
           const bool viol_own = __any_sync(0xffffffffu, all.x < -kRange || all.y < -kRange) && nr > 1;
           const float2 D = make_float2(ex2f(all.x), ex2f(all.y));
           *reinterpret_cast<float2*>(sD + s * kCH + 2 * lane) = D;
+          // the send block m&1 (like the partner's receive buffer m&1) must be free again
+          if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
           volatile float* blk = sTx + rxi * kBlkFloats;
           blk[2 * lane] = D.x;
           blk[2 * lane + 1] = D.y;
@@ -714,31 +774,18 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           }
           fence_proxy_async();
           __syncwarp();
+          if (lane == 0) {
+            // own verdict is in place (the arrive publishes it to the gate warps); the partner's
+            // block and slabs complete the two barriers by byte count
+            mbar_expect_tx(bar(BAR_VERD0 + rxi), kBlkBytes);
+            mbar_expect_tx(bar(BAR_PEER0 + rxi), kRxBytes);
+            armed = true;
+            dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
+                            base + kOffTx + rxi * kBlkBytes, kBlkBytes,
+                            map_to_cta(bar(BAR_VERD0 + rxi), peer));
+          }
         }
-        if (leader) {
-          // own verdict is in place (the arrive publishes it to the other gate warps); the
-          // partner's block and slabs complete the two barriers by byte count
-          mbar_expect_tx(bar(BAR_VERD0 + rxi), kBlkBytes);
-          mbar_expect_tx(bar(BAR_PEER0 + rxi), kRxBytes);
-          armed = true;
-          dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
-                          base + kOffTx + rxi * kBlkBytes, kBlkBytes,
-                          map_to_cta(bar(BAR_VERD0 + rxi), peer));
-        }
-        if (nr == kC) gate_phase2<true>(st + kStQ, st + kStK, off, gw * 4, nr, pre, b, eh);
-        else          gate_phase2<false>(st + kStQ, st + kStK, off, gw * 4, nr, pre, b, eh);
-        // this warp's four rows of each operand slab go to the partner (also when the attempt
-        // turns out to be abandoned: the byte count the partner's barrier expects is fixed)
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) {
-          const uint32_t rows_off = gw * 512;
-          const uint32_t dst = peer_rx_base + rxi * kRxBytes + rows_off;
-          const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
-          dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, 512, pb);
-          dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK + rows_off, 512, pb);
-        }
-        // both verdicts: the own one (lead warp) and the partner's (came with its decay block)
+        // both verdicts: the own one and the partner's (came with its decay block)
         if (!(ok = mbar_wait_cluster(bar(BAR_VERD0 + rxi), rxph, abort_flag, a.hdr))) break;
         const bool viol = (__float_as_int(sTx[rxi * kBlkFloats + 64]) |
                            __float_as_int(sRx[rxi * kBlkFloats + 64])) != 0;

@@ -53,10 +53,10 @@ __device__ __forceinline__ bool mbar_try_park(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false (and raises the CTA's abort flag and the device status) if the
-// phase does not complete in time or another role has already given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          WorkspaceHeader* hdr) {
-  if (mbar_try(bar, parity)) return true;
+// phase does not complete in time or another role has already given up.  The polling loop is
+// kept out of line: it is cold, and dozens of inlined copies would crowd the instruction cache.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            WorkspaceHeader* hdr) {
   const long long t0 = clock64();
   while (true) {
 #pragma unroll 1
@@ -72,6 +72,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       return false;
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          WorkspaceHeader* hdr) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, hdr);
 }
 __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -230,9 +235,8 @@ __device__ __forceinline__ bool mbar_try_park_cluster(uint32_t bar, uint32_t par
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
-                                                  volatile int* abort_flag, WorkspaceHeader* hdr) {
-  if (mbar_try_cluster(bar, parity)) return true;
+__device__ __noinline__ bool mbar_wait_cluster_slow(uint32_t bar, uint32_t parity,
+                                                    volatile int* abort_flag, WorkspaceHeader* hdr) {
   const long long t0 = clock64();
   while (true) {
 #pragma unroll 1
@@ -246,6 +250,11 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
       return false;
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
+                                                  volatile int* abort_flag, WorkspaceHeader* hdr) {
+  if (mbar_try_cluster(bar, parity)) return true;
+  return mbar_wait_cluster_slow(bar, parity, abort_flag, hdr);
 }
 // Bulk copy from this CTA's shared memory into another CTA's; completes (by byte count) on an
 // mbarrier of the destination CTA.  Addresses and size are multiples of 16 bytes.
