@@ -21,13 +21,13 @@
 // The pair advances in lockstep: which rows form a pass is decided from the decay totals of all
 // 128 channels, so each CTA sends its verdict along with its chunk decays and both take the OR.
 //
-// Roles in one CTA (27 warps), connected by mbarriers; every wait is bounded:
+// Roles in one CTA (19 warps), connected by mbarriers; every wait is bounded:
 //   warp 0        TMA producer (own channel slab of q,k,x,y and both slabs of the v slice)
 //   warp 1        tcgen05.mma issuer, owns the TMEM allocation
 //   warps 2-5     state group: TMEM <-> registers trip of S, initial / final state I/O
 //   warps 6-9     score / output group
-//   warps 10-25   gate group: 4 rows x 2 channels per thread, packed fp32x2 arithmetic
-//   warp 26       gate control: chunk totals, verdict exchange with the partner, publishing
+//   warps 10-17   gate group: 8 rows x 2 channels per thread, packed fp32x2 arithmetic
+//   warp 18       gate control: chunk totals, verdict exchange with the partner, publishing
 //
 // The loop-carried chain is  state update of pass g -> rescaling of S -> state update of pass
 // g+1 , so the issuer puts the state update of a pass BEFORE its output contractions, and the
@@ -66,8 +66,9 @@ constexpr int kBlkFloats = 68;                            // 64 decays, verdict,
 constexpr int kBlkBytes = kBlkFloats * 4;                 // 272 B, a multiple of 16
 constexpr int kOffTx = kOffD + kStages * kCH * 4;         // float [2][68]: block to send
 constexpr int kOffRx = kOffTx + kRxBufs * kBlkBytes;      // float [2][68]: block received
-constexpr int kGateWarp0 = 10, kGateWarps = 16;
-constexpr int kOffTot = kOffRx + kRxBufs * kBlkBytes;     // float [2][16][64]: scan partials
+constexpr int kGateWarp0 = 10, kGateWarps = 8;
+constexpr int kGR = kC / kGateWarps;                       // rows per gate thread
+constexpr int kOffTot = kOffRx + kRxBufs * kBlkBytes;     // float [2][8][64]: scan partials
 constexpr int kOffBar = kOffTot + 2 * kGateWarps * kCH * 4;
 constexpr int kNumBars = 32;
 constexpr int kOffMisc = kOffBar + kNumBars * 8;          // control block
@@ -76,7 +77,7 @@ constexpr int kSmemBytes = kSmemUsed + 1024;              // slack for manual 10
 static_assert(kOffTx % 16 == 0 && kOffRx % 16 == 0 && kBlkBytes % 16 == 0, "bulk copy alignment");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
-constexpr int kThreads = 32 * (kGateWarp0 + kGateWarps + 1);  // 864: 16 gate warps + control
+constexpr int kThreads = 32 * (kGateWarp0 + kGateWarps + 1);  // 608: 8 gate warps + control
 constexpr int kStateWarp0 = 2, kScoreWarp0 = 6;
 
 // TMEM columns (fp32 words): two state buffers, output, scores
@@ -85,7 +86,7 @@ constexpr uint32_t kColS = 0, kColO = 256, kColP = 384, kTmemCols = 512;
 // mbarrier indices
 enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                      (1 + bytes)
        BAR_EMPTY0 = 3,                // [3] stage reusable: own release + partner's receipt (2)
-       BAR_GATED0 = 6,                // [4] pass published by the gate group             (17)
+       BAR_GATED0 = 6,                // [4] pass published by gate warps + control        (9)
        BAR_PEER0 = 10, BAR_PEER1,     // partner's two slabs landed                 (1 + bytes)
        BAR_VERD0, BAR_VERD1,          // own verdict written + partner's block landed (1 + bytes)
        BAR_RXFREE0, BAR_RXFREE1,      // partner is done with ITS receive buffer            (1)
@@ -179,11 +180,11 @@ __device__ __forceinline__ float2 splat(float v) { return make_float2(v, v); }
 // Phase 1 for this thread's 4 rows x 2 channels: log2 decay (cumulative over the thread's own
 // rows, b) and log2 input weight (eh).  Returns the sum of the four rows' log2 decays.
 template <int INGATE>
-__device__ __forceinline__ float2 gate_phase1(uint32_t xs, uint32_t ys, const uint32_t (&off)[4],
-                                              int row0, int nr, float2 (&b)[4], float2 (&eh)[4]) {
+__device__ __forceinline__ float2 gate_phase1(uint32_t xs, uint32_t ys, const uint32_t (&off)[kGR],
+                                              int row0, int nr, float2 (&b)[kGR], float2 (&eh)[kGR]) {
   float2 run = splat(0.f);
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < kGR; ++i) {
     const float2 x = bf16x2_to_f2(lds32(xs + off[i]));
     const float2 y = bf16x2_to_f2(lds32(ys + off[i]));
     const float2 xl = __fmul2_rn(x, splat(kLog2e));
@@ -214,11 +215,11 @@ __device__ __forceinline__ float2 gate_phase1(uint32_t xs, uint32_t ys, const ui
 }
 
 // Phase 2: Qt = q 2^{b}, Kt = k 2^{eh - b}, written over q and k (same swizzled offsets).
-__device__ __forceinline__ void gate_phase2(uint32_t qs, uint32_t ks, const uint32_t (&off)[4],
-                                            int row0, int nr, float2 pre, const float2 (&b)[4],
-                                            const float2 (&eh)[4]) {
+__device__ __forceinline__ void gate_phase2(uint32_t qs, uint32_t ks, const uint32_t (&off)[kGR],
+                                            int row0, int nr, float2 pre, const float2 (&b)[kGR],
+                                            const float2 (&eh)[kGR]) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < kGR; ++i) {
     float2 q = bf16x2_to_f2(lds32(qs + off[i]));
     float2 k = bf16x2_to_f2(lds32(ks + off[i]));
     const float2 bb = __fadd2_rn(b[i], pre);
@@ -685,17 +686,17 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int gw = warp - kGateWarp0;                     // rows 4*gw .. 4*gw+3 of the tile
     const bool is_ctl = gw == kGateWarps;
     const bool leader = is_ctl && lane == 0;
-    uint32_t off[4];   // swizzled byte offsets of the thread's element pairs inside a slab
+    uint32_t off[kGR]; // swizzled byte offsets of the thread's element pairs inside a slab
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int r = gw * 4 + i;
+    for (int i = 0; i < kGR; ++i) {
+      const int r = gw * kGR + i;
       off[i] = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
     }
     uint32_t fs = 0, fph = 0;                             // stage and phase of the next fill
     uint32_t g = 0, m = 0, sc = 0;                        // passes, attempts, scan syncs
     bool ok = true;
     bool armed = false;                                   // attempt m's receive barriers expect bytes
-    auto group_sync = [&]() -> bool {                     // bounded barrier over the 17 warps
+    auto group_sync = [&]() -> bool {                     // bounded barrier over gate warps + control
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_GSCAN));
       const bool r = mbar_wait(bar(BAR_GSCAN), sc & 1, abort_flag, a.hdr);
@@ -728,8 +729,8 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int nr = min(min(kC, left), lcap);
         float* tot = sTot + (m & 1) * (kGateWarps * kCH);
         if (!is_ctl) {
-          float2 b[4], eh[4];
-          const float2 run = gate_phase1<INGATE>(st + kStX, st + kStY, off, gw * 4, nr, b, eh);
+          float2 b[kGR], eh[kGR];
+          const float2 run = gate_phase1<INGATE>(st + kStX, st + kStY, off, gw * kGR, nr, b, eh);
           *reinterpret_cast<float2*>(tot + gw * kCH + 2 * lane) = run;
           if (!(ok = group_sync())) break;
           // exclusive prefix over the row groups below this warp's
@@ -739,7 +740,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const float2 t = *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane);
             if (w < gw) pre = __fadd2_rn(pre, t);
           }
-          gate_phase2(st + kStQ, st + kStK, off, gw * 4, nr, pre, b, eh);
+          gate_phase2(st + kStQ, st + kStK, off, gw * kGR, nr, pre, b, eh);
           // this warp's four rows of each operand slab go to the partner (also when the attempt
           // turns out to be abandoned: the byte count the partner's barrier expects is fixed),
           // once the partner's receive buffer m&1 is free again
@@ -747,11 +748,11 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
           __syncwarp();
           if (lane == 0) {
-            const uint32_t rows_off = gw * 512;
+            const uint32_t rows_off = gw * (kGR * 128);
             const uint32_t dst = peer_rx_base + rxi * kRxBytes + rows_off;
             const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
-            dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, 512, pb);
-            dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK + rows_off, 512, pb);
+            dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, kGR * 128, pb);
+            dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK + rows_off, kGR * 128, pb);
           }
         } else {
           if (!(ok = group_sync())) break;
