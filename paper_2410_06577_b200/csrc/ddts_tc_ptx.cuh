@@ -212,12 +212,15 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar) {
   asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar)
                : "memory");
 }
-// try_wait that acquires at cluster scope: for barriers another CTA arrives on or copies into.
+// Wait on a barrier that another CTA of the cluster arrives on or bulk-copies into.  Same
+// instruction as the local wait: completion by byte count already makes the copied data visible
+// to the waiter, the plain remote arrivals carry no data, and a cluster-scope acquire costs
+// several hundred cycles per wait.
 __device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
       "selp.b32 %0, 1, 0, p;\n}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
@@ -228,7 +231,7 @@ __device__ __forceinline__ bool mbar_try_park_cluster(uint32_t bar, uint32_t par
   uint32_t ok;
   asm volatile(
       "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
       "selp.b32 %0, 1, 0, p;\n}"
       : "=r"(ok)
       : "r"(bar), "r"(parity), "r"(kParkNs)
