@@ -391,18 +391,25 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
           const uint32_t st = stage_base + s * kStageBytes;
           const uint32_t rx = rx_base + rxi * kRxBytes;
-          // channel slab 0 / 1 of each operand, wherever it lives in this CTA
-          const uint32_t q_sl[2] = {rank == 0 ? st + kStQ : rx + kRxQ, rank == 0 ? rx + kRxQ : st + kStQ};
-          const uint32_t k_sl[2] = {rank == 0 ? st + kStK : rx + kRxK, rank == 0 ? rx + kRxK : st + kStK};
+          // Low descriptor halves of the pass's operands (channel slab 0 / 1 of Qt and Kt sit in
+          // the stage or in the receive buffer depending on the rank); stepping K is one add.
+          const uint32_t q_own = st + kStQ, q_rx = rx + kRxQ, k_own = st + kStK, k_rx = rx + kRxK;
+          const uint32_t k_lo_addr = rank == 0 ? k_own : k_rx, k_hi_addr = rank == 0 ? k_rx : k_own;
+          const uint32_t dq0 = desc_lo_kmajor(rank == 0 ? q_own : q_rx);
+          const uint32_t dq1 = desc_lo_kmajor(rank == 0 ? q_rx : q_own);
+          const uint32_t dk0 = desc_lo_kmajor(k_lo_addr), dk1 = desc_lo_kmajor(k_hi_addr);
+          const uint32_t dkt = desc_lo_mnmajor(k_lo_addr, k_hi_addr - k_lo_addr);  // Kt^T, 128 channels
+          const uint32_t dv = desc_lo_mnmajor(st + kStV, kSlabBytes);
+          const uint32_t dp = desc_lo_kmajor(st + kStY);
+          const uint32_t dss = desc_lo_mnmajor(ss, kSsSlabBytes);
           tc_fence_after();
           // P = Qt Kt^T : M = 64 (rows r), N = 64 (rows i), K = 128 channels
           if (issuer) {
+            umma_bf16_lo<false>(tmem + kColP, dq0, dk0, kIdescP);
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-              const uint32_t off = (kk & 3) * 32;
-              umma_bf16(tmem + kColP, desc_kmajor(q_sl[kk >> 2] + off), desc_kmajor(k_sl[kk >> 2] + off),
-                        kIdescP, kk > 0);
-            }
+            for (int kk = 1; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColP, dq0 + 2 * kk, dk0 + 2 * kk, kIdescP);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColP, dq1 + 2 * kk, dk1 + 2 * kk, kIdescP);
             umma_commit(bar(BAR_PFULL));
           }
           if (!(ok = mbar_wait(bar(BAR_SREADY_S), ph1, abort_flag, a.hdr))) break;
@@ -410,10 +417,8 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           if (issuer) {
             // S_in + Kt^T V : M = 128 channels, N = 128, K = 64 rows (S_in sits in buffer g & 1)
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              umma_bf16(tmem + kColS + (g & 1) * 128, desc_mnmajor(k_sl[0] + kk * 2048, k_sl[1] - k_sl[0]),
-                        desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescS, 1);
-            }
+            for (int kk = 0; kk < 4; ++kk)
+              umma_bf16_lo<true>(tmem + kColS + (g & 1) * 128, dkt + 128 * kk, dv + 128 * kk, kIdescS);
             umma_commit(bar(BAR_SFULL));
           }
           if (!(ok = mbar_wait(bar(BAR_PREADY), ph1, abort_flag, a.hdr))) break;
@@ -422,17 +427,14 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           tc_fence_after();
           if (issuer) {
             // O = P V : M = 64, N = 128, K = 64 rows i (P operand lives in the consumed y slab)
+            umma_bf16_lo<false>(tmem + kColO, dp, dv, kIdescO);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              umma_bf16(tmem + kColO, desc_kmajor(st + kStY + kk * 32),
-                        desc_mnmajor(st + kStV + kk * 2048, kSlabBytes), kIdescO, kk > 0);
-            }
+            for (int kk = 1; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColO, dp + 2 * kk, dv + 128 * kk, kIdescO);
             // O += Qt S_in : K = 128 channels
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-              umma_bf16(tmem + kColO, desc_kmajor(q_sl[kk >> 2] + (kk & 3) * 32),
-                        desc_mnmajor(ss + kk * 2048, kSsSlabBytes), kIdescO, 1);
-            }
+            for (int kk = 0; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColO, dq0 + 2 * kk, dss + 128 * kk, kIdescO);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColO, dq1 + 2 * kk, dss + 128 * (kk + 4), kIdescO);
             umma_commit(bar(BAR_OFULL));
             umma_commit(bar(BAR_EMPTY0 + s));   // every contraction of the pass has read its operands
           }

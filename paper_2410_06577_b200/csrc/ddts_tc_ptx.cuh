@@ -182,6 +182,28 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t mn_grou
   return (uint64_t)((addr >> 4) & 0x3FFF) | ((uint64_t)((mn_group_bytes >> 4) & 0x3FFF) << 16) |
          ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
+// The same descriptors as two 32-bit halves.  The high half is one constant for every 128-byte
+// swizzled operand; the low half holds the address (and, for MN-major, the group stride), so
+// stepping along K is one 32-bit add: +2 per 32 bytes (K-major), +128 per 2048 bytes (MN-major).
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo_kmajor(uint32_t addr) {
+  return ((addr >> 4) & 0x3FFFu) | (1u << 16);
+}
+__device__ __forceinline__ uint32_t desc_lo_mnmajor(uint32_t addr, uint32_t mn_group_bytes) {
+  return ((addr >> 4) & 0x3FFFu) | (((mn_group_bytes >> 4) & 0x3FFFu) << 16);
+}
+template <bool ACC>
+__device__ __forceinline__ void umma_bf16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
+                                             uint32_t idesc) {
+  asm volatile(
+      "{\n.reg .pred p;\n.reg .b64 da, db;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "mov.b64 da, {%1, %5};\n"
+      "mov.b64 db, {%2, %5};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(ACC ? 1u : 0u), "r"(kDescHi)
+      : "memory");
+}
 // Instruction descriptor: bf16 x bf16 -> fp32.
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn, int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
