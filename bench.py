@@ -56,31 +56,58 @@ def load_traffic(kernel: str, workload: str):
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML (read-only queries) while the timed region
+    runs; falls back to ``nvidia-smi`` if the NVML binding is unavailable."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index: int):
         self.idx = gpu_index
-        self.samples = []
+        self.samples = []          # (sm_mhz, max_mhz, [active reason names])
         self.stop = threading.Event()
         self.thread = threading.Thread(target=self._run, daemon=True)
+        self.nvml = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            # NVML numbers devices in PCI order; honour CUDA_VISIBLE_DEVICES when it holds indices
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            ids = [t for t in vis.split(",") if t.strip().isdigit()]
+            phys = int(ids[gpu_index]) if gpu_index < len(ids) else gpu_index
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self.masks = {
+                "hw_slowdown": pynvml.nvmlClocksEventReasonHwSlowdown,
+                "hw_thermal_slowdown": pynvml.nvmlClocksEventReasonHwThermalSlowdown,
+                "sw_thermal_slowdown": pynvml.nvmlClocksEventReasonSwThermalSlowdown,
+                "sw_power_cap": pynvml.nvmlClocksEventReasonSwPowerCap,
+            }
+            self.nvml = pynvml
+        except Exception:
+            self.nvml = None
 
     def _once(self):
         try:
+            if self.nvml is not None:
+                mhz = float(self.nvml.nvmlDeviceGetClockInfo(self.handle, self.nvml.NVML_CLOCK_SM))
+                bits = int(self.nvml.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                self.samples.append((mhz, self.max_mhz, [n for n, m in self.masks.items() if bits & m]))
+                return
             out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
                                   "-i", str(self.idx)], capture_output=True, text=True, timeout=10).stdout
             f = [t.strip() for t in out.strip().split(",")]
             if len(f) >= 6:
-                self.samples.append((float(f[0]), float(f[1]), f[2:6]))
+                act = [n for n, v in zip(self.NAMES, f[2:6]) if v.lower().startswith("active")]
+                self.samples.append((float(f[0]), float(f[1]), act))
         except Exception:
             pass
 
     def _run(self):
         while not self.stop.is_set():
             self._once()
-            self.stop.wait(0.05)
+            self.stop.wait(0.002 if self.nvml is not None else 0.05)
 
     def __enter__(self):
         self.thread.start()
@@ -93,11 +120,10 @@ class ClockSampler:
     def summary(self):
         if not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = sorted({n for s in self.samples for n, v in zip(names, s[2]) if v.lower().startswith("active")})
+        reasons = sorted({n for s in self.samples for n in s[2]})
         return {"sm_mhz": float(np.median([s[0] for s in self.samples])),
                 "sm_max_mhz": float(self.samples[0][1]), "reasons": reasons,
-                "samples": len(self.samples)}
+                "samples": len(self.samples), "source": "nvml" if self.nvml is not None else "nvidia-smi"}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -360,9 +386,9 @@ def main():
     args = ap.parse_args()
     decode = args.workload == "cfg3"
     if args.steps is None:
-        args.steps = (1000 if decode else 50) if args.impl == "ours" else 3
+        args.steps = (1000 if decode else {"cfg1": 2000, "cfg2": 200, "cfg4": 200}[args.workload]) if args.impl == "ours" else 3
     if args.warmup is None:
-        args.warmup = (10 if decode else 5) if args.impl == "ours" else 1
+        args.warmup = (10 if decode else 20) if args.impl == "ours" else 1
     if args.impl == "ours" and args.warmup < 3:
         args.warmup = 3
 

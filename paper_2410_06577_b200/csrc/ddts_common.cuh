@@ -28,6 +28,8 @@ cudaError_t launch_fwd_tc(const rodimus_ddts_fwd_params& p, int* n_launches);
 cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches);
 bool fwd_tc_supported(const rodimus_ddts_fwd_params& p);
 bool fwd_pair_supported(const rodimus_ddts_fwd_params& p);
+// Workspace a dense call needs if its sequences are to be split along time (0: no split).
+size_t fwd_pair_split_workspace_bytes(const rodimus_ddts_fwd_params& p);
 
 // ---------------------------------------------------------------------------------------------
 // Element access for the two token dtypes.

@@ -106,13 +106,17 @@ struct PairArgs {
   int H, T, dv, n_seq, pairs;
   long long n_items;     // (sequence, head, 256-column slab)
   float scale;
+  float* dtot;           // optional [n_seq, H, dk]: product of all chunk decays of each sequence
+  int sT_only;           // >= 0: only this sequence's final state is stored, as if it were number 0
 };
 
 struct Item {
   long long row0;      // first global row (in the [rows, d] view) of this sequence and head
   long long state_off; // element offset of this CTA's state slice (row 0, first own column)
+  long long seq_head;  // sequence * H + head
   int len;             // tokens
   int col0;            // first value column of this CTA
+  int seq;             // sequence number (after the longest-first reordering)
 };
 
 __device__ __forceinline__ Item decode_item(const PairArgs& a, long long item, int rank) {
@@ -133,7 +137,9 @@ __device__ __forceinline__ Item decode_item(const PairArgs& a, long long item, i
     it.len = a.T;
   }
   it.col0 = (pair * 2 + rank) * kDVS;
-  it.state_off = (n * a.H + h) * (long long)kDK * a.dv + it.col0;
+  it.seq_head = n * a.H + h;
+  it.seq = (int)n;
+  it.state_off = it.seq_head * (long long)kDK * a.dv + it.col0;
   return it;
 }
 
@@ -474,6 +480,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
       bool last = false, first = true;
       float Dprev = 1.f;                                  // chunk decay of the previous pass
+      float Dall = 1.f;                                   // product of the chunk decays so far
       // 32 columns of the state entering the pass: D_prev times the previous buffer, or the
       // caller's initial state for the first pass of a sequence
       auto load_piece = [&](uint32_t (&r)[32], uint32_t t_prev, int piece) {
@@ -554,10 +561,12 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         mbar_arrive(bar(BAR_SREADY_O));
         prev_rx = rxi;
         Dprev = Dcur;
+        Dall *= Dcur;
         first = false;
         ++g;
       }
       if (!ok) break;
+      if (a.dtot && it.col0 == 0) a.dtot[it.seq_head * kDK + d] = Dall;
       // final state of this item (also keeps the next item's initial state from racing the MMAs)
       {
         const uint32_t lastg = g - 1;
@@ -565,7 +574,8 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (!(ok = mbar_wait(bar(BAR_OFULL), lastg & 1, abort_flag, a.hdr))) break;
         tc_fence_after();
         if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
-        if (a.sT) {
+        if (a.sT && (a.sT_only < 0 || it.seq == a.sT_only)) {
+          const long long frow = a.sT_only < 0 ? srow : srow - (long long)a.sT_only * a.H * kDK * a.dv;
           const uint32_t t_fin = t_lane + (lastg & 1) * 128;
 #pragma unroll 1
           for (int piece = 0; piece < 4; ++piece) {
@@ -574,7 +584,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             tmem_ld_wait();
 #pragma unroll
             for (int c4 = 0; c4 < 8; ++c4) {
-              *reinterpret_cast<float4*>(a.sT + srow + piece * 32 + 4 * c4) =
+              *reinterpret_cast<float4*>(a.sT + frow + piece * 32 + 4 * c4) =
                   make_float4(Dprev * __uint_as_float(r[4 * c4]), Dprev * __uint_as_float(r[4 * c4 + 1]),
                               Dprev * __uint_as_float(r[4 * c4 + 2]), Dprev * __uint_as_float(r[4 * c4 + 3]));
             }
@@ -902,19 +912,95 @@ bool fwd_pair_supported(const rodimus_ddts_fwd_params& p) {
   return p.dtype == RODIMUS_BF16 && p.dk == kDK && p.dv % (2 * kDVS) == 0;
 }
 
+namespace {
+
+// ---------------------------------------------------------------------------------------------
+// Long sequences, few heads: split along time
+// ---------------------------------------------------------------------------------------------
+// The state recurrence is linear, S_end = D_seg . S_start + dS_seg, where dS_seg is the segment's
+// final state from a zero start and D_seg the product of its decays.  When a dense call has fewer
+// (sequence, head, 256-column) items than the device has CTA pairs, the sequence is cut into G
+// segments that run as separate packed "sequences":
+//   launch A  segments 0..G-2 from a zero state: dS_seg and D_seg (their outputs are provisional)
+//   combine   S_start(k) = D(k-1) . S_start(k-1) + dS(k-1), k = 1..G-1 (elementwise, tiny)
+//   launch C  all G segments from their true initial states: final outputs, final state
+// which trades about (2G-1)/G of the work for G times the parallelism.
+struct SplitPlan {
+  int G = 0;            // segments (0: do not split)
+  int L = 0;            // rows per segment (multiple of the chunk length)
+  size_t off_order = 0, off_cu = 0, off_dtot = 0, off_ds = 0, off_start = 0, bytes = 0;
+};
+
+constexpr int kMinSegmentRows = 2048;
+constexpr int kMaxSegments = 16;
+
+SplitPlan make_split_plan(const rodimus_ddts_fwd_params& p) {
+  SplitPlan sp;
+  if (p.cu_seqlens || p.cu_seqlens_host || !fwd_pair_supported(p)) return sp;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return sp;
+  }
+  const long long items = (long long)p.B * p.H * (p.dv / (2 * kDVS));
+  if (items <= 0 || p.T < 2 * kMinSegmentRows) return sp;
+  long long g = (sms / 2) / items;
+  if (g > p.T / kMinSegmentRows) g = p.T / kMinSegmentRows;
+  if (g > kMaxSegments) g = kMaxSegments;
+  if (g < 2) return sp;
+  const int L = (int)(((p.T + g - 1) / g + kC - 1) / kC * kC);
+  const int G = (p.T + L - 1) / L;
+  if (G < 2) return sp;
+  auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+  const size_t state = (size_t)p.B * p.H * kDK * p.dv * sizeof(float);
+  sp.G = G; sp.L = L;
+  sp.off_order = sizeof(WorkspaceHeader);
+  sp.off_cu = sp.off_order + up((size_t)G * 4);
+  sp.off_dtot = sp.off_cu + up((size_t)(G + 1) * 4);
+  sp.off_ds = sp.off_dtot + up((size_t)(G - 1) * p.B * p.H * kDK * 4);
+  sp.off_start = sp.off_ds + (size_t)(G - 1) * state;
+  sp.bytes = sp.off_start + (size_t)G * state;
+  return sp;
+}
+
+// cu_seqlens and the (identity) order of the G segments; clears the status word.
+__global__ void ddts_segments_kernel(WorkspaceHeader* hdr, int32_t* order, int32_t* cu, int G, int L, int T) {
+  const int i = threadIdx.x;
+  if (i == 0) { hdr->status = RODIMUS_OK; hdr->work_counter = 0; hdr->n_items = G; }
+  if (i < G) order[i] = i;
+  if (i <= G) cu[i] = min(i * L, T);
+}
+
+// S_start(0) = s0 (or zero); S_start(k) = D(k-1) . S_start(k-1) + dS(k-1).  One thread per four
+// state columns of one (batch, head, channel) row; BHD = B*H*dk rows of dv columns.
+__global__ void ddts_combine_kernel(const float* __restrict__ s0, const float* __restrict__ ds,
+                                    const float* __restrict__ dtot, float* __restrict__ start,
+                                    int G, long long BHD, int dv) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int v4 = dv / 4;
+  if (idx >= BHD * v4) return;
+  const long long row = idx / v4;
+  const long long e = row * dv + (idx % v4) * 4;
+  const long long seg = BHD * dv;
+  float4 s = s0 ? *reinterpret_cast<const float4*>(s0 + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+  *reinterpret_cast<float4*>(start + e) = s;
+  for (int k = 1; k < G; ++k) {
+    const float d = dtot[(long long)(k - 1) * BHD + row];
+    const float4 t = *reinterpret_cast<const float4*>(ds + (long long)(k - 1) * seg + e);
+    s = make_float4(fmaf(d, s.x, t.x), fmaf(d, s.y, t.y), fmaf(d, s.z, t.z), fmaf(d, s.w, t.w));
+    *reinterpret_cast<float4*>(start + (long long)k * seg + e) = s;
+  }
+}
+
+}  // namespace
+
+size_t fwd_pair_split_workspace_bytes(const rodimus_ddts_fwd_params& p) { return make_split_plan(p).bytes; }
+
 cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   *n_launches = 0;
-  PairArgs a;
-  a.o = p.o; a.s0 = p.s0; a.sT = p.sT; a.cu = p.cu_seqlens;
-  a.hdr = reinterpret_cast<WorkspaceHeader*>(p.workspace);
-  a.order = reinterpret_cast<const int32_t*>(reinterpret_cast<const char*>(p.workspace) +
-                                             sizeof(WorkspaceHeader));
-  a.H = p.H; a.T = p.T; a.dv = p.dv;
-  a.n_seq = p.cu_seqlens ? p.N : p.B;
-  a.pairs = p.dv / (2 * kDVS);
-  a.n_items = (long long)a.n_seq * p.H * a.pairs;
-  a.scale = p.scale;
-  if (a.n_items == 0) return cudaSuccess;
+  const long long n_seq0 = p.cu_seqlens ? p.N : p.B;
+  if (n_seq0 * p.H == 0) return cudaSuccess;
   const uint64_t rows = (uint64_t)p.B * p.H * p.T;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
 
@@ -934,12 +1020,59 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
     memset(&mq, 0, sizeof(mq)); mk = mq; mx = mq; my = mq; mv = mq;  // never dereferenced: no chunks
   }
   const int max_pairs = sms / 2 > 0 ? sms / 2 : 1;   // one CTA per SM; a pair shares a TPC
-  if (p.ingate == RODIMUS_INGATE_POW_G)
-    e = launch_pair<RODIMUS_INGATE_POW_G>(mq, mk, mx, my, mv, a, max_pairs, st);
-  else
-    e = launch_pair<RODIMUS_INGATE_POW_SIGMOID>(mq, mk, mx, my, mv, a, max_pairs, st);
-  if (e == cudaSuccess) *n_launches = 1;
-  return e;
+  auto run = [&](const PairArgs& a) {
+    return p.ingate == RODIMUS_INGATE_POW_G
+               ? launch_pair<RODIMUS_INGATE_POW_G>(mq, mk, mx, my, mv, a, max_pairs, st)
+               : launch_pair<RODIMUS_INGATE_POW_SIGMOID>(mq, mk, mx, my, mv, a, max_pairs, st);
+  };
+  char* ws = reinterpret_cast<char*>(p.workspace);
+  PairArgs a;
+  a.o = p.o; a.s0 = p.s0; a.sT = p.sT; a.cu = p.cu_seqlens;
+  a.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+  a.order = reinterpret_cast<const int32_t*>(ws + sizeof(WorkspaceHeader));
+  a.H = p.H; a.T = p.T; a.dv = p.dv;
+  a.n_seq = (int)n_seq0;
+  a.pairs = p.dv / (2 * kDVS);
+  a.n_items = n_seq0 * p.H * a.pairs;
+  a.scale = p.scale;
+  a.dtot = nullptr;
+  a.sT_only = -1;
+
+  const SplitPlan sp = make_split_plan(p);
+  if (sp.G < 2 || p.workspace_bytes < sp.bytes) {   // one launch over whole sequences
+    e = run(a);
+    if (e == cudaSuccess) *n_launches = 1;
+    return e;
+  }
+  // ---- split along time: the (batch, head) pairs act as heads of G packed sequences
+  int32_t* order = reinterpret_cast<int32_t*>(ws + sp.off_order);
+  int32_t* cu = reinterpret_cast<int32_t*>(ws + sp.off_cu);
+  float* dtot = reinterpret_cast<float*>(ws + sp.off_dtot);
+  float* ds = reinterpret_cast<float*>(ws + sp.off_ds);
+  float* start = reinterpret_cast<float*>(ws + sp.off_start);
+  const int BH = p.B * p.H;
+  ddts_segments_kernel<<<1, 32, 0, st>>>(a.hdr, order, cu, sp.G, sp.L, p.T);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  a.cu = cu; a.order = order; a.H = BH;
+  // A: local final states and decay products of all but the last segment
+  a.n_seq = sp.G - 1;
+  a.n_items = (long long)a.n_seq * BH * a.pairs;
+  a.s0 = nullptr; a.sT = ds; a.dtot = dtot;
+  if ((e = run(a)) != cudaSuccess) return e;
+  // combine
+  {
+    const long long BHD = (long long)BH * kDK;
+    const long long threads = BHD * (p.dv / 4);
+    ddts_combine_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(p.s0, ds, dtot, start, sp.G, BHD, p.dv);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  // C: every segment from its true initial state
+  a.n_seq = sp.G;
+  a.n_items = (long long)a.n_seq * BH * a.pairs;
+  a.s0 = start; a.sT = p.sT; a.dtot = nullptr; a.sT_only = sp.G - 1;
+  if ((e = run(a)) != cudaSuccess) return e;
+  *n_launches = 4;
+  return cudaSuccess;
 }
 
 }  // namespace ddts

@@ -66,7 +66,11 @@ size_t rodimus_ddts_fwd_workspace_bytes(const rodimus_ddts_fwd_params* p) {
   if (!p) return 0;
   const bool varlen = p->cu_seqlens != nullptr || p->cu_seqlens_host != nullptr;
   if (check_fwd_sizes(p, varlen) != RODIMUS_OK) return 0;
-  return workspace_bytes_for(varlen ? p->N : 0);
+  const size_t base = workspace_bytes_for(varlen ? p->N : 0);
+  // long dense sequences with few heads run faster split along time, given room for the
+  // segments' states; a caller that passes only the base size still gets the unsplit path
+  const size_t split = ddts::fwd_pair_selected(*p) ? ddts::fwd_pair_split_workspace_bytes(*p) : 0;
+  return split > base ? split : base;
 }
 
 const char* rodimus_ddts_fwd_kernel_name(const rodimus_ddts_fwd_params* p) {
