@@ -15,14 +15,14 @@ namespace {
 constexpr int kStepThreads = 128;
 constexpr int kStepWarps = kStepThreads / 32;
 constexpr int kTileCols = 128;
-constexpr int kBatch = 8;
+constexpr int kBatch = 16;
 constexpr int kMaxDk = 256;
 
 __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(float4* p, const float4& v) { __stcs(p, v); }
 
 template <typename T>
-__global__ void __launch_bounds__(kStepThreads, 8)
+__global__ void __launch_bounds__(kStepThreads, 4)
 ddts_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ gx,
                  const T* __restrict__ ty, const T* __restrict__ v, T* __restrict__ o,
                  float* __restrict__ state, int n_seq_heads, int dk, int dv, float scale,
@@ -130,7 +130,11 @@ cudaError_t launch_step(const rodimus_ddts_step_params& p, int* n_launches) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  const long long max_grid = (long long)sms * 8;
+  // One CTA per item: measured 6 % faster than a persistent grid of 8 CTAs per SM (the hardware
+  // block scheduler balances the tail better than a fixed stride does).  The in-kernel loop only
+  // matters beyond the grid-size limit.
+  const long long max_grid = items < 0x7fffffffLL ? items : 0x7fffffffLL;
+  (void)sms;
   const int grid = (int)(items < max_grid ? items : max_grid);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
   if (p.dtype == RODIMUS_BF16) {
