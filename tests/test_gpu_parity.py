@@ -307,6 +307,44 @@ def test_config2_full_size_and_split_halves():
     assert rel_err(host(torch.cat([o1, o2], dim=2)), host(o)) <= 1e-2
 
 
+@pytest.mark.parametrize("B,H,T,dv,with_s0", [
+    (1, 2, 4096 + 100, 256, True),     # two segments, ragged second segment
+    (2, 3, 6500, 256, False),          # six (batch, head) pairs, three segments
+    (1, 1, 9000, 512, True),           # two 256-column slabs per head, four segments
+])
+def test_long_sequences_split_along_time(B, H, T, dv, with_s0):
+    """Dense calls with fewer heads than CTA pairs are cut into time segments joined through the
+    linear state recurrence; outputs and final state must still match the sequential oracle, and
+    must agree with the unsplit kernel (base-size workspace) far more tightly."""
+    import torch
+    p = wl.make_prefill(31 + T, B, H, T, 128, dv, "bf16", s0_std=0.2 if with_s0 else None)
+    d = prefill_to_device(p)
+    o = torch.empty((B, H, T, dv), dtype=torch.bfloat16, device="cuda")
+    sT = torch.empty((B, H, 128, dv), dtype=torch.float32, device="cuda")
+    prm = rd.fwd_params(d["q"], d["k"], d["x"], d["y"], d["v"], o, d["s0"], sT, scale=0.5)
+    need = rd.fwd_workspace_bytes(prm)
+    assert need > 4096, "this shape should ask for the segments' state workspace"
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    prm.workspace, prm.workspace_bytes = ws.data_ptr(), need
+    assert rd.fwd_raw(prm) == rd.OK and rd.last_launch_count() == 4
+    assert rd.device_status(ws) == rd.OK
+    ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0, scale=0.5)
+    assert rel_err(host(o), ro) <= TOL_BF16 and rel_err(host(sT), rs) <= TOL_BF16
+    # same request with only the base workspace: one launch, no split
+    o1, s1 = torch.empty_like(o), torch.empty_like(sT)
+    prm1 = rd.fwd_params(d["q"], d["k"], d["x"], d["y"], d["v"], o1, d["s0"], s1, scale=0.5)
+    ws1 = torch.empty(256, dtype=torch.uint8, device="cuda")
+    prm1.workspace, prm1.workspace_bytes = ws1.data_ptr(), 256
+    assert rd.fwd_raw(prm1) == rd.OK and rd.last_launch_count() == 1
+    torch.cuda.synchronize()
+    assert rel_err(host(o), host(o1)) <= 1e-2 and rel_err(host(sT), host(s1)) <= 1e-2
+    # output only (no final state wanted)
+    prm.sT = None
+    assert rd.fwd_raw(prm) == rd.OK
+    torch.cuda.synchronize()
+    assert rel_err(host(o), ro) <= TOL_BF16
+
+
 def test_config4_full_size_sampled_sequences():
     import torch
     p = wl.config(4)
