@@ -108,6 +108,7 @@ struct PairArgs {
   float scale;
   float* dtot;           // optional [n_seq, H, dk]: product of all chunk decays of each sequence
   int sT_only;           // >= 0: only this sequence's final state is stored, as if it were number 0
+  int state_only;        // 1: only final states and decay products are wanted (no q, scores, outputs)
 };
 
 struct Item {
@@ -221,21 +222,27 @@ __device__ __forceinline__ float2 gate_phase1(uint32_t xs, uint32_t ys, const ui
 }
 
 // Phase 2: Qt = q 2^{b}, Kt = k 2^{eh - b}, written over q and k (same swizzled offsets).
+// STATE_ONLY: the pass only updates the state, so Qt is not needed.
+template <bool STATE_ONLY>
 __device__ __forceinline__ void gate_phase2(uint32_t qs, uint32_t ks, const uint32_t (&off)[kGR],
                                             int row0, int nr, float2 pre, const float2 (&b)[kGR],
                                             const float2 (&eh)[kGR]) {
 #pragma unroll
   for (int i = 0; i < kGR; ++i) {
-    float2 q = bf16x2_to_f2(lds32(qs + off[i]));
     float2 k = bf16x2_to_f2(lds32(ks + off[i]));
     const float2 bb = __fadd2_rn(b[i], pre);
     const float2 hb = __ffma2_rn(bb, splat(-1.f), eh[i]);
-    const float2 eq = make_float2(ex2f(bb.x), ex2f(bb.y));
     const float2 ek = make_float2(ex2f(hb.x), ex2f(hb.y));
-    if (row0 + i >= nr) { q = splat(0.f); k = splat(0.f); }
-    const float2 qt = __fmul2_rn(q, eq), kt = __fmul2_rn(k, ek);
-    sts32(qs + off[i], pack_bf16(qt.x, qt.y));
+    if (row0 + i >= nr) k = splat(0.f);
+    const float2 kt = __fmul2_rn(k, ek);
     sts32(ks + off[i], pack_bf16(kt.x, kt.y));
+    if (!STATE_ONLY) {
+      float2 q = bf16x2_to_f2(lds32(qs + off[i]));
+      const float2 eq = make_float2(ex2f(bb.x), ex2f(bb.y));
+      if (row0 + i >= nr) q = splat(0.f);
+      const float2 qt = __fmul2_rn(q, eq);
+      sts32(qs + off[i], pack_bf16(qt.x, qt.y));
+    }
   }
 }
 
@@ -349,13 +356,13 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         ctl->tag[s][1] = tpos;
         const uint32_t st = stage_base + s * kStageBytes;
         const uint32_t fb = bar(BAR_FULL0 + s);
-        mbar_expect_tx(fb, kStageBytes);
+        mbar_expect_tx(fb, a.state_only ? kStageBytes - kSlabBytes : kStageBytes);
         // rows beyond the tensor read as zeros; rows of the next sequence are masked later
         const int y = (int)(it.row0 + tpos);
         const int xc = rank * kCH;
         tma_load_2d(st + kStX, &map_x, xc, y, fb);
         tma_load_2d(st + kStY, &map_y, xc, y, fb);
-        tma_load_2d(st + kStQ, &map_q, xc, y, fb);
+        if (!a.state_only) tma_load_2d(st + kStQ, &map_q, xc, y, fb);
         tma_load_2d(st + kStK, &map_k, xc, y, fb);
         tma_load_2d(st + kStV, &map_v, it.col0, y, fb);
         tma_load_2d(st + kStV + kSlabBytes, &map_v, it.col0 + 64, y, fb);
@@ -410,7 +417,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const uint32_t dss = desc_lo_mnmajor(ss, kSsSlabBytes);
           tc_fence_after();
           // P = Qt Kt^T : M = 64 (rows r), N = 64 (rows i), K = 128 channels
-          if (issuer) {
+          if (issuer && !a.state_only) {
             umma_bf16_lo<false>(tmem + kColP, dq0, dk0, kIdescP);
 #pragma unroll
             for (int kk = 1; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColP, dq0 + 2 * kk, dk0 + 2 * kk, kIdescP);
@@ -426,7 +433,9 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             for (int kk = 0; kk < 4; ++kk)
               umma_bf16_lo<true>(tmem + kColS + (g & 1) * 128, dkt + 128 * kk, dv + 128 * kk, kIdescS);
             umma_commit(bar(BAR_SFULL));
+            if (a.state_only) umma_commit(bar(BAR_EMPTY0 + s));
           }
+          if (a.state_only) { ++g; continue; }             // no scores, no outputs
           if (!(ok = mbar_wait(bar(BAR_PREADY), ph1, abort_flag, a.hdr))) break;
           if (!(ok = mbar_wait(bar(BAR_SREADY_O), ph1, abort_flag, a.hdr))) break;
           if (!(ok = mbar_wait(bar(BAR_OFREE), ph1 ^ 1, abort_flag, a.hdr))) break;
@@ -530,7 +539,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // the previous pass's readout has finished with the old copy (and, with its state
           // update, with every operand of that pass: the partner may reuse the receive buffer).
           // Signalled before waiting for pass g: publishing pass g may itself need that buffer.
-          if (!(ok = mbar_wait(bar(BAR_OFULL), ph1 ^ 1, abort_flag, a.hdr))) break;
+          if (!a.state_only && !(ok = mbar_wait(bar(BAR_OFULL), ph1 ^ 1, abort_flag, a.hdr))) break;
           if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
         }
         // this pass's chunk decay (applied on the NEXT trip); read before this pass's readout
@@ -543,7 +552,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // step 2: bf16 copy of the same state for the readout: MN-major, row d, two 64-column
         // slabs.  (The old buffer is untouched until the NEXT pass's step 1.)
 #pragma unroll 1
-        for (int piece = 0; piece < 4; ++piece) {
+        for (int piece = 0; piece < (a.state_only ? 0 : 4); ++piece) {
           uint32_t r[32];
           load_piece(r, t_prev, piece);
           const uint32_t slab = ss_row + (piece >> 1) * kSsSlabBytes;
@@ -571,7 +580,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       {
         const uint32_t lastg = g - 1;
         if (!(ok = mbar_wait(bar(BAR_SFULL), lastg & 1, abort_flag, a.hdr))) break;
-        if (!(ok = mbar_wait(bar(BAR_OFULL), lastg & 1, abort_flag, a.hdr))) break;
+        if (!a.state_only && !(ok = mbar_wait(bar(BAR_OFULL), lastg & 1, abort_flag, a.hdr))) break;
         tc_fence_after();
         if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
         if (a.sT && (a.sT_only < 0 || it.seq == a.sT_only)) {
@@ -609,6 +618,20 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       bool last = false;
       while (!last) {
         const uint32_t ph1 = g & 1;
+        if (a.state_only) {
+          // nothing to mask or store: only the partner's stage is handed back, once its slab has
+          // landed here
+          if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 3)), (g >> 2) & 1, abort_flag, a.hdr))) break;
+          const int rxi = ctl->pd[g & 3].rx;
+          last = (ctl->pd[g & 3].flags & kPassLast) != 0;
+          if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), (uint32_t)ctl->pd[g & 3].rxph, abort_flag, a.hdr))) break;
+          if (warp == kScoreWarp0 && lane == 0) {
+            const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]);
+            mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
+          }
+          ++g;
+          continue;
+        }
         if (!(ok = mbar_wait(bar(BAR_PFULL), ph1, abort_flag, a.hdr))) break;
         const int s = ctl->pd[g & 3].stage;
         const int nr = ctl->pd[g & 3].nr;
@@ -752,7 +775,8 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const float2 t = *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane);
             if (w < gw) pre = __fadd2_rn(pre, t);
           }
-          gate_phase2(st + kStQ, st + kStK, off, gw * kGR, nr, pre, b, eh);
+          if (a.state_only) gate_phase2<true>(st + kStQ, st + kStK, off, gw * kGR, nr, pre, b, eh);
+          else              gate_phase2<false>(st + kStQ, st + kStK, off, gw * kGR, nr, pre, b, eh);
           // this warp's four rows of each operand slab go to the partner (also when the attempt
           // turns out to be abandoned: the byte count the partner's barrier expects is fixed),
           // once the partner's receive buffer m&1 is free again
@@ -763,7 +787,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const uint32_t rows_off = gw * (kGR * 128);
             const uint32_t dst = peer_rx_base + rxi * kRxBytes + rows_off;
             const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
-            dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, kGR * 128, pb);
+            if (!a.state_only) dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, kGR * 128, pb);
             dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK + rows_off, kGR * 128, pb);
           }
         } else {
@@ -791,7 +815,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             // own verdict is in place (the arrive publishes it to the gate warps); the partner's
             // block and slabs complete the two barriers by byte count
             mbar_expect_tx(bar(BAR_VERD0 + rxi), kBlkBytes);
-            mbar_expect_tx(bar(BAR_PEER0 + rxi), kRxBytes);
+            mbar_expect_tx(bar(BAR_PEER0 + rxi), a.state_only ? kRxBytes - kSlabBytes : kRxBytes);
             armed = true;
             dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
                             base + kOffTx + rxi * kBlkBytes, kBlkBytes,
@@ -921,7 +945,7 @@ namespace {
 // final state from a zero start and D_seg the product of its decays.  When a dense call has fewer
 // (sequence, head, 256-column) items than the device has CTA pairs, the sequence is cut into G
 // segments that run as separate packed "sequences":
-//   launch A  segments 0..G-2 from a zero state: dS_seg and D_seg (their outputs are provisional)
+//   launch A  segments 0..G-2 from a zero state, state only: dS_seg and D_seg (no q, scores, outputs)
 //   combine   S_start(k) = D(k-1) . S_start(k-1) + dS(k-1), k = 1..G-1 (elementwise, tiny)
 //   launch C  all G segments from their true initial states: final outputs, final state
 // which trades about (2G-1)/G of the work for G times the parallelism.
@@ -1037,6 +1061,7 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   a.scale = p.scale;
   a.dtot = nullptr;
   a.sT_only = -1;
+  a.state_only = 0;
 
   const SplitPlan sp = make_split_plan(p);
   if (sp.G < 2 || p.workspace_bytes < sp.bytes) {   // one launch over whole sequences
@@ -1057,7 +1082,7 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   // A: local final states and decay products of all but the last segment
   a.n_seq = sp.G - 1;
   a.n_items = (long long)a.n_seq * BH * a.pairs;
-  a.s0 = nullptr; a.sT = ds; a.dtot = dtot;
+  a.s0 = nullptr; a.sT = ds; a.dtot = dtot; a.state_only = 1;
   if ((e = run(a)) != cudaSuccess) return e;
   // combine
   {
@@ -1069,7 +1094,7 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   // C: every segment from its true initial state
   a.n_seq = sp.G;
   a.n_items = (long long)a.n_seq * BH * a.pairs;
-  a.s0 = start; a.sT = p.sT; a.dtot = nullptr; a.sT_only = sp.G - 1;
+  a.s0 = start; a.sT = p.sT; a.dtot = nullptr; a.sT_only = sp.G - 1; a.state_only = 0;
   if ((e = run(a)) != cudaSuccess) return e;
   *n_launches = 4;
   return cudaSuccess;
