@@ -108,7 +108,7 @@ struct PairArgs {
   float scale;
   float* dtot;           // optional [n_seq, H, dk]: product of all chunk decays of each sequence
   int sT_only;           // >= 0: only this sequence's final state is stored, as if it were number 0
-  int state_only;        // 1: only final states and decay products are wanted (no q, scores, outputs)
+  int state_only;        // 1: launch the state-only instantiation of the kernel
 };
 
 struct Item {
@@ -246,7 +246,9 @@ __device__ __forceinline__ void gate_phase2(uint32_t qs, uint32_t ks, const uint
   }
 }
 
-template <int INGATE>
+// STATE_ONLY: only final states and decay products are wanted (no q, scores, outputs); a
+// compile-time switch so that the full kernel carries none of its branches.
+template <int INGATE, bool STATE_ONLY>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
@@ -356,13 +358,13 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         ctl->tag[s][1] = tpos;
         const uint32_t st = stage_base + s * kStageBytes;
         const uint32_t fb = bar(BAR_FULL0 + s);
-        mbar_expect_tx(fb, a.state_only ? kStageBytes - kSlabBytes : kStageBytes);
+        mbar_expect_tx(fb, STATE_ONLY ? kStageBytes - kSlabBytes : kStageBytes);
         // rows beyond the tensor read as zeros; rows of the next sequence are masked later
         const int y = (int)(it.row0 + tpos);
         const int xc = rank * kCH;
         tma_load_2d(st + kStX, &map_x, xc, y, fb);
         tma_load_2d(st + kStY, &map_y, xc, y, fb);
-        if (!a.state_only) tma_load_2d(st + kStQ, &map_q, xc, y, fb);
+        if (!STATE_ONLY) tma_load_2d(st + kStQ, &map_q, xc, y, fb);
         tma_load_2d(st + kStK, &map_k, xc, y, fb);
         tma_load_2d(st + kStV, &map_v, it.col0, y, fb);
         tma_load_2d(st + kStV + kSlabBytes, &map_v, it.col0 + 64, y, fb);
@@ -417,7 +419,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const uint32_t dss = desc_lo_mnmajor(ss, kSsSlabBytes);
           tc_fence_after();
           // P = Qt Kt^T : M = 64 (rows r), N = 64 (rows i), K = 128 channels
-          if (issuer && !a.state_only) {
+          if (issuer && !STATE_ONLY) {
             umma_bf16_lo<false>(tmem + kColP, dq0, dk0, kIdescP);
 #pragma unroll
             for (int kk = 1; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColP, dq0 + 2 * kk, dk0 + 2 * kk, kIdescP);
@@ -433,9 +435,9 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             for (int kk = 0; kk < 4; ++kk)
               umma_bf16_lo<true>(tmem + kColS + (g & 1) * 128, dkt + 128 * kk, dv + 128 * kk, kIdescS);
             umma_commit(bar(BAR_SFULL));
-            if (a.state_only) umma_commit(bar(BAR_EMPTY0 + s));
+            if (STATE_ONLY) umma_commit(bar(BAR_EMPTY0 + s));
           }
-          if (a.state_only) { ++g; continue; }             // no scores, no outputs
+          if (STATE_ONLY) { ++g; continue; }             // no scores, no outputs
           if (!(ok = mbar_wait(bar(BAR_PREADY), ph1, abort_flag, a.hdr))) break;
           if (!(ok = mbar_wait(bar(BAR_SREADY_O), ph1, abort_flag, a.hdr))) break;
           if (!(ok = mbar_wait(bar(BAR_OFREE), ph1 ^ 1, abort_flag, a.hdr))) break;
@@ -539,7 +541,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // the previous pass's readout has finished with the old copy (and, with its state
           // update, with every operand of that pass: the partner may reuse the receive buffer).
           // Signalled before waiting for pass g: publishing pass g may itself need that buffer.
-          if (!a.state_only && !(ok = mbar_wait(bar(BAR_OFULL), ph1 ^ 1, abort_flag, a.hdr))) break;
+          if (!STATE_ONLY && !(ok = mbar_wait(bar(BAR_OFULL), ph1 ^ 1, abort_flag, a.hdr))) break;
           if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
         }
         // this pass's chunk decay (applied on the NEXT trip); read before this pass's readout
@@ -552,7 +554,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // step 2: bf16 copy of the same state for the readout: MN-major, row d, two 64-column
         // slabs.  (The old buffer is untouched until the NEXT pass's step 1.)
 #pragma unroll 1
-        for (int piece = 0; piece < (a.state_only ? 0 : 4); ++piece) {
+        for (int piece = 0; piece < (STATE_ONLY ? 0 : 4); ++piece) {
           uint32_t r[32];
           load_piece(r, t_prev, piece);
           const uint32_t slab = ss_row + (piece >> 1) * kSsSlabBytes;
@@ -580,7 +582,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       {
         const uint32_t lastg = g - 1;
         if (!(ok = mbar_wait(bar(BAR_SFULL), lastg & 1, abort_flag, a.hdr))) break;
-        if (!a.state_only && !(ok = mbar_wait(bar(BAR_OFULL), lastg & 1, abort_flag, a.hdr))) break;
+        if (!STATE_ONLY && !(ok = mbar_wait(bar(BAR_OFULL), lastg & 1, abort_flag, a.hdr))) break;
         tc_fence_after();
         if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
         if (a.sT && (a.sT_only < 0 || it.seq == a.sT_only)) {
@@ -618,7 +620,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       bool last = false;
       while (!last) {
         const uint32_t ph1 = g & 1;
-        if (a.state_only) {
+        if (STATE_ONLY) {
           // nothing to mask or store: only the partner's stage is handed back, once its slab has
           // landed here
           if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 3)), (g >> 2) & 1, abort_flag, a.hdr))) break;
@@ -775,8 +777,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const float2 t = *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane);
             if (w < gw) pre = __fadd2_rn(pre, t);
           }
-          if (a.state_only) gate_phase2<true>(st + kStQ, st + kStK, off, gw * kGR, nr, pre, b, eh);
-          else              gate_phase2<false>(st + kStQ, st + kStK, off, gw * kGR, nr, pre, b, eh);
+          gate_phase2<STATE_ONLY>(st + kStQ, st + kStK, off, gw * kGR, nr, pre, b, eh);
           // this warp's four rows of each operand slab go to the partner (also when the attempt
           // turns out to be abandoned: the byte count the partner's barrier expects is fixed),
           // once the partner's receive buffer m&1 is free again
@@ -787,7 +788,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const uint32_t rows_off = gw * (kGR * 128);
             const uint32_t dst = peer_rx_base + rxi * kRxBytes + rows_off;
             const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
-            if (!a.state_only) dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, kGR * 128, pb);
+            if (!STATE_ONLY) dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, kGR * 128, pb);
             dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK + rows_off, kGR * 128, pb);
           }
         } else {
@@ -815,7 +816,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             // own verdict is in place (the arrive publishes it to the gate warps); the partner's
             // block and slabs complete the two barriers by byte count
             mbar_expect_tx(bar(BAR_VERD0 + rxi), kBlkBytes);
-            mbar_expect_tx(bar(BAR_PEER0 + rxi), a.state_only ? kRxBytes - kSlabBytes : kRxBytes);
+            mbar_expect_tx(bar(BAR_PEER0 + rxi), STATE_ONLY ? kRxBytes - kSlabBytes : kRxBytes);
             armed = true;
             dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
                             base + kOffTx + rxi * kBlkBytes, kBlkBytes,
@@ -918,15 +919,15 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int INGATE>
+template <int INGATE, bool STATE_ONLY>
 cudaError_t launch_pair(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mx,
                         const CUtensorMap& my, const CUtensorMap& mv, const PairArgs& a,
                         int max_pairs, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(ddts_fwd_pair_kernel<INGATE>,
+  cudaError_t e = cudaFuncSetAttribute(ddts_fwd_pair_kernel<INGATE, STATE_ONLY>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
   const long long pairs = a.n_items < max_pairs ? a.n_items : max_pairs;
-  ddts_fwd_pair_kernel<INGATE><<<(unsigned)(2 * pairs), kThreads, kSmemBytes, st>>>(mq, mk, mx, my, mv, a);
+  ddts_fwd_pair_kernel<INGATE, STATE_ONLY><<<(unsigned)(2 * pairs), kThreads, kSmemBytes, st>>>(mq, mk, mx, my, mv, a);
   return cudaGetLastError();
 }
 
@@ -1045,9 +1046,13 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   }
   const int max_pairs = sms / 2 > 0 ? sms / 2 : 1;   // one CTA per SM; a pair shares a TPC
   auto run = [&](const PairArgs& a) {
+    if (a.state_only)
+      return p.ingate == RODIMUS_INGATE_POW_G
+                 ? launch_pair<RODIMUS_INGATE_POW_G, true>(mq, mk, mx, my, mv, a, max_pairs, st)
+                 : launch_pair<RODIMUS_INGATE_POW_SIGMOID, true>(mq, mk, mx, my, mv, a, max_pairs, st);
     return p.ingate == RODIMUS_INGATE_POW_G
-               ? launch_pair<RODIMUS_INGATE_POW_G>(mq, mk, mx, my, mv, a, max_pairs, st)
-               : launch_pair<RODIMUS_INGATE_POW_SIGMOID>(mq, mk, mx, my, mv, a, max_pairs, st);
+               ? launch_pair<RODIMUS_INGATE_POW_G, false>(mq, mk, mx, my, mv, a, max_pairs, st)
+               : launch_pair<RODIMUS_INGATE_POW_SIGMOID, false>(mq, mk, mx, my, mv, a, max_pairs, st);
   };
   char* ws = reinterpret_cast<char*>(p.workspace);
   PairArgs a;
