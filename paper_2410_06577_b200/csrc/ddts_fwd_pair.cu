@@ -38,6 +38,7 @@
 #include <cuda.h>
 
 #include <cstring>
+#include <mutex>
 
 #include "ddts_common.cuh"
 #include "ddts_tc_ptx.cuh"
@@ -944,20 +945,24 @@ namespace {
 // ---------------------------------------------------------------------------------------------
 // The state recurrence is linear, S_end = D_seg . S_start + dS_seg, where dS_seg is the segment's
 // final state from a zero start and D_seg the product of its decays.  When a dense call has fewer
-// (sequence, head, 256-column) items than the device has CTA pairs, the sequence is cut into G
-// segments that run as separate packed "sequences":
-//   launch A  segments 0..G-2 from a zero state, state only: dS_seg and D_seg (no q, scores, outputs)
-//   combine   S_start(k) = D(k-1) . S_start(k-1) + dS(k-1), k = 1..G-1 (elementwise, tiny)
-//   launch C  all G segments from their true initial states: final outputs, final state
-// which trades about (2G-1)/G of the work for G times the parallelism.
+// (sequence, head, 256-column) items than the device has CTA pairs, the sequence is cut into a
+// short head segment 0 and G equal segments 1..G that run as separate packed "sequences":
+//   launch A   segments 1..G-1 from a zero state, state only: dS_seg and D_seg      } side by side,
+//   launch C0  segment 0 from the caller's initial state: outputs, S_start(1)       } two streams
+//   combine    S_start(k+1) = D(k) . S_start(k) + dS(k), k = 1..G-1 (elementwise, tiny)
+//   launch C   segments 1..G from their true initial states: outputs, final state
+// Segment 0 is shorter by the ratio of a state-only pass to a full pass, so that A and C0 end
+// together; the whole trades about (2G - 0.3)/(G + 0.7) of the work for G times the parallelism.
 struct SplitPlan {
-  int G = 0;            // segments (0: do not split)
-  int L = 0;            // rows per segment (multiple of the chunk length)
+  int G = 0;            // segments after the head segment (0: do not split)
+  int L0 = 0;           // rows of the head segment (multiple of the chunk length)
+  int L = 0;            // rows of each later segment (multiple of the chunk length)
   size_t off_order = 0, off_cu = 0, off_dtot = 0, off_ds = 0, off_start = 0, bytes = 0;
 };
 
 constexpr int kMinSegmentRows = 2048;
 constexpr int kMaxSegments = 16;
+constexpr double kStateOnlyCost = 0.7;   // head segment length relative to the others (state-only pass / full pass; best of a sweep)
 
 SplitPlan make_split_plan(const rodimus_ddts_fwd_params& p) {
   SplitPlan sp;
@@ -974,48 +979,75 @@ SplitPlan make_split_plan(const rodimus_ddts_fwd_params& p) {
   if (g > p.T / kMinSegmentRows) g = p.T / kMinSegmentRows;
   if (g > kMaxSegments) g = kMaxSegments;
   if (g < 2) return sp;
-  const int L = (int)(((p.T + g - 1) / g + kC - 1) / kC * kC);
-  const int G = (p.T + L - 1) / L;
-  if (G < 2) return sp;
+  int L = (int)((long long)(p.T / (g + kStateOnlyCost)) + kC - 1) / kC * kC;
+  if ((long long)g * L >= p.T) L = (int)((p.T / (g + 1)) / kC * kC);   // keep a head segment
+  const int L0 = p.T - (int)g * L;
+  if (L <= 0 || L0 <= 0) return sp;
   auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
   const size_t state = (size_t)p.B * p.H * kDK * p.dv * sizeof(float);
-  sp.G = G; sp.L = L;
+  sp.G = (int)g; sp.L0 = L0; sp.L = L;
   sp.off_order = sizeof(WorkspaceHeader);
-  sp.off_cu = sp.off_order + up((size_t)G * 4);
-  sp.off_dtot = sp.off_cu + up((size_t)(G + 1) * 4);
-  sp.off_ds = sp.off_dtot + up((size_t)(G - 1) * p.B * p.H * kDK * 4);
-  sp.off_start = sp.off_ds + (size_t)(G - 1) * state;
-  sp.bytes = sp.off_start + (size_t)G * state;
+  sp.off_cu = sp.off_order + up((size_t)(g + 1) * 4);
+  sp.off_dtot = sp.off_cu + up((size_t)(g + 2) * 4);
+  sp.off_ds = sp.off_dtot + up((size_t)(g - 1) * p.B * p.H * kDK * 4);
+  sp.off_start = sp.off_ds + (size_t)(g - 1) * state;
+  sp.bytes = sp.off_start + (size_t)g * state;
   return sp;
 }
 
-// cu_seqlens and the (identity) order of the G segments; clears the status word.
-__global__ void ddts_segments_kernel(WorkspaceHeader* hdr, int32_t* order, int32_t* cu, int G, int L, int T) {
+// cu_seqlens of the head segment and the G later ones, and an identity order; clears the status word.
+__global__ void ddts_segments_kernel(WorkspaceHeader* hdr, int32_t* order, int32_t* cu, int G, int L0,
+                                     int L, int T) {
   const int i = threadIdx.x;
-  if (i == 0) { hdr->status = RODIMUS_OK; hdr->work_counter = 0; hdr->n_items = G; }
-  if (i < G) order[i] = i;
-  if (i <= G) cu[i] = min(i * L, T);
+  if (i == 0) { hdr->status = RODIMUS_OK; hdr->work_counter = 0; hdr->n_items = G + 1; }
+  if (i <= G) order[i] = i;
+  if (i <= G + 1) cu[i] = i == 0 ? 0 : min(L0 + (i - 1) * L, T);
 }
 
-// S_start(0) = s0 (or zero); S_start(k) = D(k-1) . S_start(k-1) + dS(k-1).  One thread per four
+// start[0] = S_start(1) is given (final state of the head segment); start[k] = D(k) . start[k-1]
+// + dS(k) for k = 1..n, with ds / dtot entry k-1 belonging to segment k.  One thread per four
 // state columns of one (batch, head, channel) row; BHD = B*H*dk rows of dv columns.
-__global__ void ddts_combine_kernel(const float* __restrict__ s0, const float* __restrict__ ds,
-                                    const float* __restrict__ dtot, float* __restrict__ start,
-                                    int G, long long BHD, int dv) {
+__global__ void ddts_combine_kernel(const float* __restrict__ ds, const float* __restrict__ dtot,
+                                    float* __restrict__ start, int n, long long BHD, int dv) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int v4 = dv / 4;
   if (idx >= BHD * v4) return;
   const long long row = idx / v4;
   const long long e = row * dv + (idx % v4) * 4;
   const long long seg = BHD * dv;
-  float4 s = s0 ? *reinterpret_cast<const float4*>(s0 + e) : make_float4(0.f, 0.f, 0.f, 0.f);
-  *reinterpret_cast<float4*>(start + e) = s;
-  for (int k = 1; k < G; ++k) {
+  float4 s = *reinterpret_cast<const float4*>(start + e);
+  for (int k = 1; k <= n; ++k) {
     const float d = dtot[(long long)(k - 1) * BHD + row];
     const float4 t = *reinterpret_cast<const float4*>(ds + (long long)(k - 1) * seg + e);
     s = make_float4(fmaf(d, s.x, t.x), fmaf(d, s.y, t.y), fmaf(d, s.z, t.z), fmaf(d, s.w, t.w));
     *reinterpret_cast<float4*>(start + (long long)k * seg + e) = s;
   }
+}
+
+// A second stream and two events per device, so that the two independent launches of the time
+// split can run side by side.  Created on first use; if that fails the launches simply follow
+// each other on the caller's stream.
+struct SideStream {
+  bool tried = false, ok = false;
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+constexpr int kMaxDevices = 64;
+SideStream g_side[kMaxDevices];
+std::mutex g_side_mutex;
+
+SideStream* side_stream(int dev) {
+  if (dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_side_mutex);
+  SideStream& s = g_side[dev];
+  if (!s.tried) {
+    s.tried = true;
+    s.ok = cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) == cudaSuccess &&
+           cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) == cudaSuccess;
+    if (!s.ok) cudaGetLastError();
+  }
+  return s.ok ? &s : nullptr;
 }
 
 }  // namespace
@@ -1045,7 +1077,7 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
     memset(&mq, 0, sizeof(mq)); mk = mq; mx = mq; my = mq; mv = mq;  // never dereferenced: no chunks
   }
   const int max_pairs = sms / 2 > 0 ? sms / 2 : 1;   // one CTA per SM; a pair shares a TPC
-  auto run = [&](const PairArgs& a) {
+  auto run = [&](const PairArgs& a, cudaStream_t st) {
     if (a.state_only)
       return p.ingate == RODIMUS_INGATE_POW_G
                  ? launch_pair<RODIMUS_INGATE_POW_G, true>(mq, mk, mx, my, mv, a, max_pairs, st)
@@ -1070,38 +1102,61 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
 
   const SplitPlan sp = make_split_plan(p);
   if (sp.G < 2 || p.workspace_bytes < sp.bytes) {   // one launch over whole sequences
-    e = run(a);
+    e = run(a, st);
     if (e == cudaSuccess) *n_launches = 1;
     return e;
   }
-  // ---- split along time: the (batch, head) pairs act as heads of G packed sequences
+  // ---- split along time: the (batch, head) pairs act as heads of packed sequences
   int32_t* order = reinterpret_cast<int32_t*>(ws + sp.off_order);
   int32_t* cu = reinterpret_cast<int32_t*>(ws + sp.off_cu);
   float* dtot = reinterpret_cast<float*>(ws + sp.off_dtot);
   float* ds = reinterpret_cast<float*>(ws + sp.off_ds);
   float* start = reinterpret_cast<float*>(ws + sp.off_start);
   const int BH = p.B * p.H;
-  ddts_segments_kernel<<<1, 32, 0, st>>>(a.hdr, order, cu, sp.G, sp.L, p.T);
+  ddts_segments_kernel<<<1, 32, 0, st>>>(a.hdr, order, cu, sp.G, sp.L0, sp.L, p.T);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  a.cu = cu; a.order = order; a.H = BH;
-  // A: local final states and decay products of all but the last segment
+  SideStream* side = side_stream(dev);
+  cudaStream_t st0 = st;                             // stream of launch C0
+  if (side) {
+    if (cudaEventRecord(side->fork, st) == cudaSuccess &&
+        cudaStreamWaitEvent(side->stream, side->fork, 0) == cudaSuccess) {
+      st0 = side->stream;
+    } else {
+      cudaGetLastError();
+      side = nullptr;
+    }
+  }
+  a.order = order; a.H = BH;
+  // A: local final states and decay products of segments 1..G-1
+  a.cu = cu + 1;
   a.n_seq = sp.G - 1;
   a.n_items = (long long)a.n_seq * BH * a.pairs;
   a.s0 = nullptr; a.sT = ds; a.dtot = dtot; a.state_only = 1;
-  if ((e = run(a)) != cudaSuccess) return e;
+  if ((e = run(a, st)) != cudaSuccess) return e;
+  // C0: the head segment from the caller's initial state; its final state starts segment 1
+  a.cu = cu;
+  a.n_seq = 1;
+  a.n_items = (long long)BH * a.pairs;
+  a.s0 = p.s0; a.sT = start; a.dtot = nullptr; a.state_only = 0;
+  if ((e = run(a, st0)) != cudaSuccess) return e;
+  if (side) {
+    if ((e = cudaEventRecord(side->join, st0)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(st, side->join, 0)) != cudaSuccess) return e;
+  }
   // combine
   {
     const long long BHD = (long long)BH * kDK;
     const long long threads = BHD * (p.dv / 4);
-    ddts_combine_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(p.s0, ds, dtot, start, sp.G, BHD, p.dv);
+    ddts_combine_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(ds, dtot, start, sp.G - 1, BHD, p.dv);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
-  // C: every segment from its true initial state
+  // C: segments 1..G from their true initial states
+  a.cu = cu + 1;
   a.n_seq = sp.G;
   a.n_items = (long long)a.n_seq * BH * a.pairs;
   a.s0 = start; a.sT = p.sT; a.dtot = nullptr; a.sT_only = sp.G - 1; a.state_only = 0;
-  if ((e = run(a)) != cudaSuccess) return e;
-  *n_launches = 4;
+  if ((e = run(a, st)) != cudaSuccess) return e;
+  *n_launches = 5;
   return cudaSuccess;
 }
 

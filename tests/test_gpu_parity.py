@@ -308,14 +308,15 @@ def test_config2_full_size_and_split_halves():
 
 
 @pytest.mark.parametrize("B,H,T,dv,with_s0", [
-    (1, 2, 4096 + 100, 256, True),     # two segments, ragged second segment
-    (2, 3, 6500, 256, False),          # six (batch, head) pairs, three segments
-    (1, 1, 9000, 512, True),           # two 256-column slabs per head, four segments
+    (1, 2, 4096 + 100, 256, True),     # head segment + two segments, ragged last segment
+    (2, 3, 6500, 256, False),          # six (batch, head) pairs, head segment + three segments
+    (1, 1, 9000, 512, True),           # two 256-column slabs per head, head segment + four segments
 ])
 def test_long_sequences_split_along_time(B, H, T, dv, with_s0):
     """Dense calls with fewer heads than CTA pairs are cut into time segments joined through the
-    linear state recurrence; outputs and final state must still match the sequential oracle, and
-    must agree with the unsplit kernel (base-size workspace) far more tightly."""
+    linear state recurrence (five launches: segment table, state-only pass and head segment side
+    by side, combine, full pass); outputs and final state must still match the sequential oracle,
+    and must agree with the unsplit kernel (base-size workspace) far more tightly."""
     import torch
     p = wl.make_prefill(31 + T, B, H, T, 128, dv, "bf16", s0_std=0.2 if with_s0 else None)
     d = prefill_to_device(p)
@@ -326,7 +327,7 @@ def test_long_sequences_split_along_time(B, H, T, dv, with_s0):
     assert need > 4096, "this shape should ask for the segments' state workspace"
     ws = torch.empty(need, dtype=torch.uint8, device="cuda")
     prm.workspace, prm.workspace_bytes = ws.data_ptr(), need
-    assert rd.fwd_raw(prm) == rd.OK and rd.last_launch_count() == 4
+    assert rd.fwd_raw(prm) == rd.OK and rd.last_launch_count() == 5
     assert rd.device_status(ws) == rd.OK
     ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0, scale=0.5)
     assert rel_err(host(o), ro) <= TOL_BF16 and rel_err(host(sT), rs) <= TOL_BF16
