@@ -27,7 +27,9 @@
 //   warps 2-5     state group: TMEM <-> registers trip of S, initial / final state I/O
 //   warps 6-9     score / output group
 //   warps 10-17   gate group: 8 rows x 2 channels per thread, packed fp32x2 arithmetic
-//   warp 18       gate control: chunk totals, verdict exchange with the partner, publishing
+//   warp 18       gate control: chunk totals, verdict exchange with the partner, the two slab
+//                 copies (one thread: sixteen small copies issued by the gate warps took them
+//                 ~1400 cycles per pass), publishing
 //
 // The loop-carried chain is  state update of pass g -> rescaling of S -> state update of pass
 // g+1 , so the issuer puts the state update of a pass BEFORE its output contractions, and the
@@ -94,8 +96,9 @@ enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                    
        BAR_PFULL, BAR_PREADY,
        BAR_SREADY_S,                  // S rescaled in TMEM: the state update may accumulate (128)
        BAR_SREADY_O,                  // bf16 copy of S_in in shared memory: the readout may run (128)
-       BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN };
-static_assert(BAR_GSCAN < kNumBars, "barrier count");
+       BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN,
+       BAR_ROWS };                    // every gate warp has rewritten its rows of the pass (16)
+static_assert(BAR_ROWS < kNumBars, "barrier count");
 
 struct PairArgs {
   void* o;
@@ -301,6 +304,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     mbar_init(bar(BAR_OFULL), 1);
     mbar_init(bar(BAR_OFREE), 128);
     mbar_init(bar(BAR_GSCAN), kGateWarps + 1);
+    mbar_init(bar(BAR_ROWS), kGateWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -779,19 +783,11 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (w < gw) pre = __fadd2_rn(pre, t);
           }
           gate_phase2<STATE_ONLY>(st + kStQ, st + kStK, off, gw * kGR, nr, pre, b, eh);
-          // this warp's four rows of each operand slab go to the partner (also when the attempt
-          // turns out to be abandoned: the byte count the partner's barrier expects is fixed),
-          // once the partner's receive buffer m&1 is free again
+          // the rewritten rows are visible to the bulk-copy engine and to the tensor core; the
+          // control warp sends the whole slabs to the partner once every gate warp has said so
           fence_proxy_async();
-          if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
           __syncwarp();
-          if (lane == 0) {
-            const uint32_t rows_off = gw * (kGR * 128);
-            const uint32_t dst = peer_rx_base + rxi * kRxBytes + rows_off;
-            const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
-            if (!STATE_ONLY) dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ + rows_off, kGR * 128, pb);
-            dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK + rows_off, kGR * 128, pb);
-          }
+          if (lane == 0) mbar_arrive(bar(BAR_ROWS));
         } else {
           if (!(ok = group_sync())) break;
           // chunk totals of the own 64 channels: decays for both state groups, and the verdict
@@ -822,6 +818,16 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
                             base + kOffTx + rxi * kBlkBytes, kBlkBytes,
                             map_to_cta(bar(BAR_VERD0 + rxi), peer));
+          }
+          // both operand slabs of the attempt go to the partner in one copy each (also when the
+          // attempt turns out to be abandoned: the byte count the partner's barrier expects is
+          // fixed); the partner's receive buffer m&1 is free, see above
+          if (!(ok = mbar_wait(bar(BAR_ROWS), m & 1, abort_flag, a.hdr))) break;
+          if (lane == 0) {
+            const uint32_t dst = peer_rx_base + rxi * kRxBytes;
+            const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
+            if (!STATE_ONLY) dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ, kSlabBytes, pb);
+            dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK, kSlabBytes, pb);
           }
         }
         // both verdicts: the own one and the partner's (came with its decay block)
