@@ -89,7 +89,7 @@ constexpr uint32_t kColS = 0, kColO = 256, kColP = 384, kTmemCols = 512;
 // mbarrier indices
 enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                      (1 + bytes)
        BAR_EMPTY0 = 3,                // [3] stage reusable: own release + partner's receipt (2)
-       BAR_GATED0 = 6,                // [4] pass published by gate warps + control        (9)
+       BAR_GATED0 = 6,                // [4] pass published by the control warp              (1)
        BAR_PEER0 = 10, BAR_PEER1,     // partner's two slabs landed                 (1 + bytes)
        BAR_VERD0, BAR_VERD1,          // own verdict written + partner's block landed (1 + bytes)
        BAR_RXFREE0, BAR_RXFREE1,      // partner is done with ITS receive buffer            (1)
@@ -290,7 +290,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       mbar_init(bar(BAR_FULL0 + s), 1);
       mbar_init(bar(BAR_EMPTY0 + s), 2);
     }
-    for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_GATED0 + i), kGateWarps + 1);
+    for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_GATED0 + i), 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(BAR_PEER0 + i), 1);
       mbar_init(bar(BAR_VERD0 + i), 1);
@@ -819,6 +819,17 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                             base + kOffTx + rxi * kBlkBytes, kBlkBytes,
                             map_to_cta(bar(BAR_VERD0 + rxi), peer));
           }
+          // the descriptor of the pass this attempt becomes if both CTAs accept it (slot g & 3 is
+          // not read before its barrier completes; a refused attempt's entry is overwritten)
+          if (lane == 0) {
+            volatile PassDesc* pd = &ctl->pd[g & 3];
+            pd->stage = (int)s;
+            pd->nr = nr;
+            pd->flags = (nr == left ? kPassLast : 0);
+            pd->rx = (int)rxi;
+            pd->rxph = (int)rxph;
+            pd->row = it.row0 + tpos;
+          }
           // both operand slabs of the attempt go to the partner in one copy each (also when the
           // attempt turns out to be abandoned: the byte count the partner's barrier expects is
           // fixed); the partner's receive buffer m&1 is free, see above
@@ -852,18 +863,12 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           }
           continue;
         }
+        // the control warp alone publishes the pass (its descriptor is already written): it has
+        // seen every gate warp's rows through BAR_ROWS
         if (leader) {
-          volatile PassDesc* pd = &ctl->pd[g & 3];
-          pd->stage = (int)s;
-          pd->nr = nr;
-          pd->flags = (nr == left ? kPassLast : 0);
-          pd->rx = (int)rxi;
-          pd->rxph = (int)rxph;
-          pd->row = it.row0 + tpos;
           if (nr < min(kC, left)) redirect(j, tpos + nr);   // the prefetcher assumed 64 rows
+          mbar_arrive(bar(BAR_GATED0 + (g & 3)));
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_GATED0 + (g & 3)));
         ++g;
         tpos += nr;
         if (lcap < kC) lcap = min(kC, lcap * 2);
