@@ -307,6 +307,36 @@ def test_config2_full_size_and_split_halves():
     assert rel_err(host(torch.cat([o1, o2], dim=2)), host(o)) <= 1e-2
 
 
+@pytest.mark.gpu
+def test_time_split_on_a_user_stream_back_to_back():
+    """The time split forks to a second stream and joins again: on a non-default user stream,
+    with calls issued back to back into the same buffers' successors and read on that stream
+    without any device-wide synchronisation, every call must see its own complete result."""
+    import torch
+    B, H, T, dv = 1, 2, 5000, 256
+    ps = [wl.make_prefill(700 + i, B, H, T, 128, dv, "bf16", s0_std=0.1) for i in range(3)]
+    side = torch.cuda.Stream()
+    outs = []
+    with torch.cuda.stream(side):
+        ds = [prefill_to_device(p) for p in ps]
+        for d in ds:
+            o = torch.empty((B, H, T, dv), dtype=torch.bfloat16, device="cuda")
+            sT = torch.empty((B, H, 128, dv), dtype=torch.float32, device="cuda")
+            prm = rd.fwd_params(d["q"], d["k"], d["x"], d["y"], d["v"], o, d["s0"], sT)
+            need = rd.fwd_workspace_bytes(prm)
+            ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+            prm.workspace, prm.workspace_bytes = ws.data_ptr(), need
+            assert rd.fwd_raw(prm) == rd.OK and rd.last_launch_count() == 5
+            # consumers on the same stream, queued right behind the call
+            outs.append((o.float().sum(dim=-1), sT.clone(), o, ws))
+        side.synchronize()
+    for p, (osum, sT, o, ws) in zip(ps, outs):
+        assert rd.device_status(ws) == rd.OK
+        ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0)
+        assert rel_err(host(o), ro) <= TOL_BF16 and rel_err(host(sT), rs) <= TOL_BF16
+        assert rel_err(host(osum), np.asarray(host(o), dtype=np.float64).sum(axis=-1)) <= 1e-2
+
+
 @pytest.mark.parametrize("B,H,T,dv,with_s0", [
     (1, 2, 4096 + 100, 256, True),     # head segment + two segments, ragged last segment
     (2, 3, 6500, 256, False),          # six (batch, head) pairs, head segment + three segments
