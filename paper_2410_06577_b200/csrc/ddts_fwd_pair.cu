@@ -963,7 +963,7 @@ namespace {
 //   combine    S_start(k+1) = D(k) . S_start(k) + dS(k), k = 1..G-1 (elementwise, tiny)
 //   launch C   segments 1..G from their true initial states: outputs, final state
 // Segment 0 is shorter by the ratio of a state-only pass to a full pass, so that A and C0 end
-// together; the whole trades about (2G - 0.3)/(G + 0.7) of the work for G times the parallelism.
+// together; the whole trades about (2G - 0.35)/(G + 0.65) of the work for G times the parallelism.
 struct SplitPlan {
   int G = 0;            // segments after the head segment (0: do not split)
   int L0 = 0;           // rows of the head segment (multiple of the chunk length)
@@ -973,7 +973,7 @@ struct SplitPlan {
 
 constexpr int kMinSegmentRows = 2048;
 constexpr int kMaxSegments = 16;
-constexpr double kStateOnlyCost = 0.7;   // head segment length relative to the others (state-only pass / full pass; best of a sweep)
+constexpr double kStateOnlyCost = 0.65;  // head segment length relative to the others (state-only pass / full pass; best of a sweep)
 
 SplitPlan make_split_plan(const rodimus_ddts_fwd_params& p) {
   SplitPlan sp;
