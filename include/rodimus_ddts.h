@@ -18,8 +18,11 @@
  * Conventions shared by every entry point
  *   - All data pointers are DEVICE pointers unless a name ends in "_host".
  *   - The caller owns every buffer, the workspace and the stream.  The library allocates no
- *     device memory, keeps no state between calls and never synchronises the device, except
- *     rodimus_ddts_device_status, which waits for the stream it is given.
+ *     device memory and never synchronises the device, except rodimus_ddts_device_status,
+ *     which waits for the stream it is given.  The only state it keeps between calls is, per
+ *     device, one extra stream and two events, created the first time a call is split along
+ *     time (see rodimus_ddts_fwd_workspace_bytes); if they cannot be created the split runs
+ *     on the caller's stream alone.
  *   - Calls enqueue work on `stream` and return; outputs are valid once the stream has
  *     reached that point.
  *   - Every function returns a rodimus_status.  Argument errors are found on the host before
@@ -119,7 +122,15 @@ typedef struct {
 } rodimus_ddts_step_params;
 
 /* Bytes of device workspace rodimus_ddts_fwd needs for these sizes (pointers are not read).
- * Returns 0 if the sizes are not valid. */
+ * Returns 0 if the sizes are not valid.
+ * For a dense bf16 call with long sequences and fewer (sequence, head) units than the device
+ * has SM pairs, the size includes room for per-segment states: given that much, the call cuts
+ * the sequences into time segments that run side by side (the state recurrence is linear in
+ * the state, so segments are joined exactly up to rounding) and part of the work is enqueued
+ * on the library's own second stream, forked from and joined back into `stream` with events, so
+ * the call still behaves as one piece of work on `stream`.  A caller that passes less (never
+ * less than 256 bytes plus 4 bytes per packed sequence, rounded up to 256) gets the same
+ * result from a single launch. */
 size_t rodimus_ddts_fwd_workspace_bytes(const rodimus_ddts_fwd_params *p);
 
 /* Chunked prefill; see rodimus_ddts_fwd_params. */
