@@ -308,6 +308,27 @@ def test_config2_full_size_and_split_halves():
 
 
 @pytest.mark.gpu
+def test_time_split_with_the_alternate_input_gate_and_fast_decay():
+    """The split's state-only instantiation exists per input-gate mode, and a segment's decay
+    product can underflow to zero (strong decay): both must still give the sequential result."""
+    import torch
+    B, H, T, dv = 1, 3, 4500, 256
+    for ingate, gate_mean in ((rd.INGATE_POW_SIGMOID, -3.0), (rd.INGATE_POW_G, 1.5)):
+        p = wl.make_prefill(900 + ingate, B, H, T, 128, dv, "bf16", gate_mean=gate_mean, s0_std=0.3)
+        d = prefill_to_device(p)
+        o = torch.empty((B, H, T, dv), dtype=torch.bfloat16, device="cuda")
+        sT = torch.empty((B, H, 128, dv), dtype=torch.float32, device="cuda")
+        prm = rd.fwd_params(d["q"], d["k"], d["x"], d["y"], d["v"], o, d["s0"], sT, ingate=ingate)
+        need = rd.fwd_workspace_bytes(prm)
+        ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        prm.workspace, prm.workspace_bytes = ws.data_ptr(), need
+        assert rd.fwd_raw(prm) == rd.OK and rd.last_launch_count() == 5
+        assert rd.device_status(ws) == rd.OK
+        ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0, ingate=ingate)
+        assert rel_err(host(o), ro) <= TOL_BF16 and rel_err(host(sT), rs) <= TOL_BF16
+
+
+@pytest.mark.gpu
 def test_time_split_on_a_user_stream_back_to_back():
     """The time split forks to a second stream and joins again: on a non-default user stream,
     with calls issued back to back into the same buffers' successors and read on that stream
