@@ -97,7 +97,7 @@ enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                    
        BAR_SREADY_S,                  // S rescaled in TMEM: the state update may accumulate (128)
        BAR_SREADY_O,                  // bf16 copy of S_in in shared memory: the readout may run (128)
        BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN,
-       BAR_ROWS };                    // every gate warp has rewritten its rows of the pass (16)
+       BAR_ROWS };                    // every gate warp has rewritten its rows of the pass (8)
 static_assert(BAR_ROWS < kNumBars, "barrier count");
 
 struct PairArgs {
