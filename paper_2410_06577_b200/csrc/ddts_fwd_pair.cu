@@ -188,8 +188,8 @@ __device__ __forceinline__ float2 bf16x2_to_f2(uint32_t w) {
 }
 __device__ __forceinline__ float2 splat(float v) { return make_float2(v, v); }
 
-// Phase 1 for this thread's 4 rows x 2 channels: log2 decay (cumulative over the thread's own
-// rows, b) and log2 input weight (eh).  Returns the sum of the four rows' log2 decays.
+// Phase 1 for this thread's kGR rows x 2 channels: log2 decay (cumulative over the thread's own
+// rows, b) and log2 input weight (eh).  Returns the sum of those rows' log2 decays.
 template <int INGATE>
 __device__ __forceinline__ float2 gate_phase1(uint32_t xs, uint32_t ys, const uint32_t (&off)[kGR],
                                               int row0, int nr, float2 (&b)[kGR], float2 (&eh)[kGR]) {
@@ -722,10 +722,10 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
   } else if (warp >= kGateWarp0) {
     // ============================== gate group and its control warp ==============================
-    // The sixteen gate warps do the per-element work; the control warp does everything that is
+    // The gate warps do the per-element work; the control warp does everything that is
     // serial (chunk totals, decays, verdict, the block for the partner, publishing the pass), so
     // that none of it sits between the two phases of a gate warp.
-    const int gw = warp - kGateWarp0;                     // rows 4*gw .. 4*gw+3 of the tile
+    const int gw = warp - kGateWarp0;                     // rows kGR*gw .. kGR*gw+kGR-1 of the tile
     const bool is_ctl = gw == kGateWarps;
     const bool leader = is_ctl && lane == 0;
     uint32_t off[kGR]; // swizzled byte offsets of the thread's element pairs inside a slab
