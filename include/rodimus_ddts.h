@@ -22,7 +22,9 @@
  *     which waits for the stream it is given.  The only state it keeps between calls is, per
  *     device, one extra stream and two events, created the first time a call is split along
  *     time (see rodimus_ddts_fwd_workspace_bytes); if they cannot be created the split runs
- *     on the caller's stream alone.
+ *     on the caller's stream alone.  Calls from several host threads are allowed (each with
+ *     its own buffers, workspace and stream); the enqueueing of split calls is serialised
+ *     inside the library.
  *   - Calls enqueue work on `stream` and return; outputs are valid once the stream has
  *     reached that point.
  *   - Every function returns a rodimus_status.  Argument errors are found on the host before

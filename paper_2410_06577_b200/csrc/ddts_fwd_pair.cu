@@ -1045,7 +1045,9 @@ struct SideStream {
 };
 constexpr int kMaxDevices = 64;
 SideStream g_side[kMaxDevices];
-std::mutex g_side_mutex;
+std::mutex g_side_mutex;        // creation of the entries
+std::mutex g_side_use_mutex;    // the fork ... join sequence: an event holds the LAST record only, so
+                                // two host threads must not interleave their records and waits
 
 SideStream* side_stream(int dev) {
   if (dev < 0 || dev >= kMaxDevices) return nullptr;
@@ -1128,6 +1130,8 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   SideStream* side = side_stream(dev);
   cudaStream_t st0 = st;                             // stream of launch C0
+  std::unique_lock<std::mutex> side_use(g_side_use_mutex, std::defer_lock);
+  if (side) side_use.lock();
   if (side) {
     if (cudaEventRecord(side->fork, st) == cudaSuccess &&
         cudaStreamWaitEvent(side->stream, side->fork, 0) == cudaSuccess) {
@@ -1153,6 +1157,7 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   if (side) {
     if ((e = cudaEventRecord(side->join, st0)) != cudaSuccess) return e;
     if ((e = cudaStreamWaitEvent(st, side->join, 0)) != cudaSuccess) return e;
+    side_use.unlock();
   }
   // combine
   {

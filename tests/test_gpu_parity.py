@@ -329,6 +329,45 @@ def test_time_split_with_the_alternate_input_gate_and_fast_decay():
 
 
 @pytest.mark.gpu
+def test_time_split_from_two_host_threads():
+    """Two host threads, each on its own stream, issue split calls at the same time (the C call
+    runs without the interpreter lock): the library's one extra stream per device is shared, so
+    the fork and join of one call must not pick up the other call's events."""
+    import threading
+    import torch
+    B, H, T, dv = 1, 2, 4300, 256
+    results = {}
+
+    def worker(tag):
+        torch.cuda.set_device(0)
+        stream = torch.cuda.Stream()
+        outs = []
+        with torch.cuda.stream(stream):
+            for i in range(4):
+                p = wl.make_prefill(1200 + 10 * tag + i, B, H, T, 128, dv, "bf16", s0_std=0.1)
+                d = prefill_to_device(p)
+                o = torch.empty((B, H, T, dv), dtype=torch.bfloat16, device="cuda")
+                sT = torch.empty((B, H, 128, dv), dtype=torch.float32, device="cuda")
+                prm = rd.fwd_params(d["q"], d["k"], d["x"], d["y"], d["v"], o, d["s0"], sT)
+                need = rd.fwd_workspace_bytes(prm)
+                ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+                prm.workspace, prm.workspace_bytes = ws.data_ptr(), need
+                rc = rd.fwd_raw(prm)
+                outs.append((rc, p, o, sT, ws, d))
+            stream.synchronize()
+        results[tag] = outs
+
+    threads = [threading.Thread(target=worker, args=(t,)) for t in (0, 1)]
+    for t in threads: t.start()
+    for t in threads: t.join()
+    for tag in (0, 1):
+        for rc, p, o, sT, ws, _ in results[tag]:
+            assert rc == rd.OK and rd.device_status(ws) == rd.OK
+            ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0)
+            assert rel_err(host(o), ro) <= TOL_BF16 and rel_err(host(sT), rs) <= TOL_BF16
+
+
+@pytest.mark.gpu
 def test_time_split_on_a_user_stream_back_to_back():
     """The time split forks to a second stream and joins again: on a non-default user stream,
     with calls issued back to back into the same buffers' successors and read on that stream
