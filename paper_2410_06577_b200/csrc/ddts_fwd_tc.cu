@@ -628,15 +628,18 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
+  // looked up once (initialisation of a function-local static is thread-safe); a failed lookup
+  // leaves nullptr and the callers report an error
+  static const EncodeTiledFn fn = []() -> EncodeTiledFn {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
+        qres != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
       return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
+    }
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
   return fn;
 }
 
