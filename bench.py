@@ -237,17 +237,46 @@ def run_reference(args, workload, p):
 # our arm
 # ----------------------------------------------------------------------------------------------
 
-def run_ours(args, workload, p):
+# Work per token-head behind the three bound times printed beside every prefill roofline
+# (dk = 128, dv = 256): tensor flops of the chunkwise form at chunk length 64 (state update and
+# readout 2*dk*dv each, causal intra-chunk (C+1)(dk+dv)) and special-function approximations of
+# the gate math (7 per key channel with the paper's input gate: softplus 2, sigmoid 2, log g 1,
+# the two operand exponentials 2).
+DATASHEET = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+
+
+def work_per_token_head(dk: int, dv: int, chunk: int = 64):
+    return {"tensor_flops": 4 * dk * dv + (chunk + 1) * (dk + dv), "sfu_ops": 7 * dk}
+
+
+def measure_sfu_rate(rd, torch, device):
+    """Special-function approximations per second of the whole device (CUDA events around the
+    library's probe launch, best of 5 after a warm-up)."""
+    sink = torch.zeros(1, dtype=torch.float32, device=device)
+    stream = torch.cuda.current_stream()
+    best = None
+    for it in range(6):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        ops = rd.sfu_probe(4096, sink)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if it:
+            rate = ops / (e0.elapsed_time(e1) / 1e3)
+            best = rate if best is None else max(best, rate)
+    return best
+
+
+def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sfu_rate,
+            min_region_ms=60.0, with_e2e=True):
+    """Times `steps` calls of the workload (regions of exactly `steps` calls, repeated back to
+    back until the clock sampler has had at least `min_region_ms` to look at; the median region
+    is reported) and returns the record with value, roofline, clocks, e2e and launch count."""
     import torch
-    import torch.distributed as dist
     import paper_2410_06577_b200 as rd
     from paper_2410_06577_b200 import dist as rdist
 
-    rank, world, local = rdist.env_rank()
-    torch.cuda.set_device(local)
     device = torch.device("cuda", local)
-    rdist.init("nccl", device)
-    peaks, peak_kind = load_peaks()
     decode = workload == "cfg3"
     tdt = torch.bfloat16 if p.dtype == "bf16" else torch.float32
     stream = torch.cuda.current_stream()
@@ -256,16 +285,18 @@ def run_ours(args, workload, p):
         rdist.barrier()
         torch.cuda.synchronize()
 
+    host = {n: torch.from_numpy(getattr(p, n)).to(tdt).pin_memory() for n in ("q", "k", "x", "y", "v")}
+    devt = {n: host[n].to(device) for n in host}
     if decode:
         ring = p.q.shape[0]
-        host = {n: torch.from_numpy(getattr(p, n)).to(tdt).pin_memory() for n in ("q", "k", "x", "y", "v")}
-        devt = {n: host[n].to(device) for n in host}
         state = torch.from_numpy(p.state).to(device)
         Nseq, H, dk, dv = p.state.shape
         o = torch.empty((Nseq, H, dv), dtype=tdt, device=device)
         units_per_step = decode_bytes(p) / 1e9          # GB moved per step
         alg_bytes = decode_bytes(p)
         kernel = "ddts_step_kernel"
+        token_heads = Nseq * H
+        ws = None
 
         def step(i):
             s = i % ring
@@ -283,8 +314,6 @@ def run_ours(args, workload, p):
             rd.ddts_step(stage["q"], stage["k"], stage["x"], stage["y"], stage["v"], state, out=o)
             o_host.copy_(o, non_blocking=True)
     else:
-        host = {n: torch.from_numpy(getattr(p, n)).to(tdt).pin_memory() for n in ("q", "k", "x", "y", "v")}
-        devt = {n: host[n].to(device) for n in host}
         s0 = None if p.s0 is None else torch.from_numpy(p.s0).to(device)
         cu = None if p.cu_seqlens is None else torch.from_numpy(p.cu_seqlens).to(device)
         cu_host = None if p.cu_seqlens is None else torch.from_numpy(p.cu_seqlens)
@@ -297,6 +326,7 @@ def run_ours(args, workload, p):
         units_per_step = p.tokens
         alg_bytes = prefill_bytes(p)
         kernel = "ddts_fwd_" + rd.fwd_kernel_name(prm)
+        token_heads = B * H * T
 
         def step(i):
             rd.ddts_fwd(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], s0, cu, cu_host,
@@ -304,72 +334,135 @@ def run_ours(args, workload, p):
 
         o_host = torch.empty(o.shape, dtype=tdt).pin_memory()
         sT_host = torch.empty(sT.shape, dtype=torch.float32).pin_memory()
-        stage = {n: torch.empty_like(devt[n]) for n in host}
         h2d = sum(host[n].numel() * host[n].element_size() for n in host)
         d2h = o_host.numel() * o_host.element_size() + sT_host.numel() * 4
 
         def step_e2e(i):
+            # the stage buffers ARE the resident inputs: every step overwrites them from the host
             for n in host:
-                stage[n].copy_(host[n], non_blocking=True)
-            rd.ddts_fwd(stage["q"], stage["k"], stage["x"], stage["y"], stage["v"], s0, cu, cu_host,
+                devt[n].copy_(host[n], non_blocking=True)
+            rd.ddts_fwd(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], s0, cu, cu_host,
                         out=o, final_state=sT, workspace=ws)
             o_host.copy_(o, non_blocking=True)
             sT_host.copy_(sT, non_blocking=True)
 
-    def timed(fn, steps, warmup):
+    def timed_regions(fn, steps, warmup, min_ms):
+        """Regions of exactly `steps` calls, event-bracketed, back to back; returns their times
+        (ms, max over ranks each)."""
         for i in range(warmup):
             fn(i)
         barrier()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record(stream)
-        for i in range(steps):
-            fn(warmup + i)
-        ev1.record(stream)
-        barrier()
-        return rdist.max_over_ranks(ev0.elapsed_time(ev1), device)
+        times = []
+        n = warmup
+        total = 0.0
+        while True:
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record(stream)
+            for i in range(steps):
+                fn(n + i)
+            ev1.record(stream)
+            barrier()
+            t = rdist.max_over_ranks(ev0.elapsed_time(ev1), device)
+            times.append(t)
+            total += t
+            n += steps
+            if total >= min_ms or len(times) >= 200:
+                return times
 
     step(0)
     torch.cuda.synchronize()
     launches_per_step = rd.last_launch_count()
     with ClockSampler(local) as clk:
-        ms = timed(step, args.steps, args.warmup)
+        regions = timed_regions(step, steps, warmup, min_region_ms)
     clocks = clk.summary()
-    if not decode:
+    if ws is not None:
         st = rd.device_status(ws)
         if st != rd.OK:
             raise SystemExit(f"device status after the timed region: {st} ({rd.status_str(st)})")
-    e2e_steps = max(1, min(args.steps, 200 if decode else 5))
-    ms_e2e = timed(step_e2e, e2e_steps, 1)
-
+    ms = float(np.median(regions))
     sec = ms / 1e3
-    value = units_per_step * world * args.steps / sec
-    e2e_value = units_per_step * world * e2e_steps / (ms_e2e / 1e3)
-    kern_s = sec / args.steps
+    value = units_per_step * world * steps / sec
+    kern_s = sec / steps
     achieved = alg_bytes / kern_s / 1e9
-    line = {
+    rec = {
         "metric": "DDTS decode state GB/s" if decode else "DDTS prefill tokens/s",
         "value": value, "unit": "GB/s" if decode else "tokens/s",
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32" if decode else ("bf16" if p.dtype == "bf16" else "f32"),
         "data": "synthetic (seeded)", "config": describe(workload, p, world),
+        "timed_regions": {"count": len(regions), "steps_each": steps, "reported": "median",
+                          "ms_min": float(min(regions)), "ms_median": ms, "ms_max": float(max(regions))},
         "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": "GB/s" if decode else "tokens/s",
-                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
-        "gpu_launches": int(launches_per_step * args.steps),
-        "roofline": {"bound": "hbm", "kernel": kernel, "achieved": achieved,
-                     "peak": peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"],
-                     "algorithmic_bytes_per_launch": int(alg_bytes),
-                     "traffic": load_traffic(kernel, workload)},
+        "gpu_launches": int(launches_per_step * steps),
     }
+    wk = work_per_token_head(128, 256)
+    bounds = {"hbm_us": alg_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6}
+    if not decode:
+        bounds["tensor_us"] = token_heads * wk["tensor_flops"] / (peaks["bf16_tflops"] * 1e12) * 1e6
+        bounds["sfu_us"] = (token_heads * wk["sfu_ops"] / sfu_rate * 1e6) if sfu_rate else "unmeasured"
+        bounds["sfu_rate_gops"] = (sfu_rate / 1e9) if sfu_rate else "unmeasured"
+    rec["roofline"] = {"bound": "hbm", "kernel": kernel, "achieved": achieved,
+                       "peak": peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                       "frac": achieved / peaks["hbm_gbs"],
+                       "frac_of_datasheet_peak": achieved / DATASHEET["hbm_gbs"],
+                       "datasheet_peak": DATASHEET["hbm_gbs"],
+                       "algorithmic_bytes_per_launch": int(alg_bytes),
+                       "bound_times": bounds,
+                       "traffic": load_traffic(kernel, workload)}
+    if with_e2e:
+        e2e_steps = max(1, min(steps, 200 if decode else 5))
+        e2e_regions = timed_regions(step_e2e, e2e_steps, 1, 0.0)
+        rec["e2e"] = {"value": units_per_step * world * e2e_steps / (e2e_regions[0] / 1e3),
+                      "unit": "GB/s" if decode else "tokens/s",
+                      "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps}
+    return rec
+
+
+SUB_DEFAULTS = {"cfg1": (500, 5), "cfg2": (100, 5), "cfg4": (40, 5), "cfg3": (1000, 10)}
+
+
+def run_ours(args, workload, p):
+    import torch
+    import torch.distributed as dist
+    import paper_2410_06577_b200 as rd
+    from paper_2410_06577_b200 import dist as rdist
+    from paper_2410_06577_b200 import workloads as wl
+
+    rank, world, local = rdist.env_rank()
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    rdist.init("nccl", device)
+    peaks, peak_kind = load_peaks()
+    sfu_rate = measure_sfu_rate(rd, torch, device)
+
+    line = measure(workload, p, args.steps, args.warmup, world, rank, local, peaks, peak_kind, sfu_rate)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import ddts_oracle as orc
+        decode = workload == "cfg3"
+        u, s, what = oracle_sample_run(workload, p, budget_s=10.0)
+        line["cpu_baseline"] = {"value": u / s / (1e9 if decode else 1.0),
+                                "unit": "GB/s" if decode else "tokens/s",
+                                "cores": orc.num_threads(), "kind": "oracle", "sample": what}
+    # The metric has a prefill half and a decode half, and the prefill bar holds on the long and
+    # the packed workloads too: at one GPU the other named workloads ride along as sub-records,
+    # each timed with its own step count (the top-level fields stay those of `workload`).
+    if world == 1 and not args.no_extra:
+        del p
+        extra = {}
+        for name in ("cfg1", "cfg2", "cfg3", "cfg4"):
+            if name == workload and args.steps >= SUB_DEFAULTS[name][0]:
+                continue
+            torch.cuda.empty_cache()
+            pw = wl.config(WORKLOADS[name])
+            k, w = SUB_DEFAULTS[name]
+            r = measure(name, pw, k, w, world, rank, local, peaks, peak_kind, sfu_rate, with_e2e=False)
+            extra[name] = {key: r[key] for key in ("metric", "value", "unit", "steps", "warmup", "ms_per_step",
+                                                   "dtype", "config", "timed_regions", "clocks",
+                                                   "gpu_launches", "roofline")}
+            del pw
+        line["workloads"] = extra
     if rank == 0:
-        if world == 1 and not args.no_cpu_baseline:
-            from oracle import ddts_oracle as orc
-            u, s, what = oracle_sample_run(workload, p, budget_s=10.0)
-            line["cpu_baseline"] = {"value": u / s / (1e9 if decode else 1.0),
-                                    "unit": "GB/s" if decode else "tokens/s",
-                                    "cores": orc.num_threads(), "kind": "oracle", "sample": what}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -383,10 +476,12 @@ def main():
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg1")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="only the workload named by --workload, no sub-records for the others")
     args = ap.parse_args()
     decode = args.workload == "cfg3"
     if args.steps is None:
-        args.steps = (1000 if decode else {"cfg1": 2000, "cfg2": 200, "cfg4": 200}[args.workload]) if args.impl == "ours" else 3
+        args.steps = SUB_DEFAULTS[args.workload][0] if args.impl == "ours" else 3
     if args.warmup is None:
         args.warmup = (10 if decode else 20) if args.impl == "ours" else 1
     if args.impl == "ours" and args.warmup < 3:

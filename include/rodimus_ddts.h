@@ -190,6 +190,14 @@ int rodimus_ddts_last_launch_count(void);
  * "invalid".  Pointers are not read. */
 const char *rodimus_ddts_fwd_kernel_name(const rodimus_ddts_fwd_params *p);
 
+/* Diagnostic for benchmarks (the paper has no counterpart): enqueues on `stream` one launch that
+ * does nothing but special-function-unit approximations (ex2), `iters` rounds of 8 per thread
+ * on a grid that fills the device, and stores in *ops (host) how many it will execute.  The
+ * caller times the launch with events: ops / time is the rate that bounds the gate math
+ * (softplus, sigmoid, logarithms and exponentials of Eq. "alpha_def") of the prefill kernels.
+ * `sink` is one device float (written only in a case that does not occur).  iters in 1 .. 2^24. */
+int rodimus_ddts_sfu_probe(int iters, float *sink, void *stream, long long *ops);
+
 const char *rodimus_status_str(int status);
 int rodimus_version(void);
 

@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = (
     "rodimus_ddts_fwd_workspace_bytes", "rodimus_ddts_fwd", "rodimus_ddts_step",
     "rodimus_ddts_device_status", "rodimus_ddts_last_launch_count",
     "rodimus_ddts_fwd_kernel_name", "rodimus_status_str", "rodimus_version",
-    "rodimus_ddts_fwd_noalloc",
+    "rodimus_ddts_fwd_noalloc", "rodimus_ddts_sfu_probe",
 )
 NOALLOC_MAX_SEQS = 4096
 
@@ -88,6 +88,9 @@ def load_library() -> ctypes.CDLL:
         lib.rodimus_ddts_last_launch_count.restype = ctypes.c_int
         lib.rodimus_ddts_fwd_kernel_name.argtypes = [ctypes.POINTER(FwdParams)]
         lib.rodimus_ddts_fwd_kernel_name.restype = ctypes.c_char_p
+        lib.rodimus_ddts_sfu_probe.argtypes = [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                               ctypes.POINTER(ctypes.c_longlong)]
+        lib.rodimus_ddts_sfu_probe.restype = ctypes.c_int
         lib.rodimus_status_str.argtypes = [ctypes.c_int]
         lib.rodimus_status_str.restype = ctypes.c_char_p
         lib.rodimus_version.restype = ctypes.c_int
@@ -176,6 +179,18 @@ def device_status_ptr(ptr: int, stream: Optional[int] = None) -> int:
     import torch
     st = torch.cuda.current_stream().cuda_stream if stream is None else stream
     return int(load_library().rodimus_ddts_device_status(ptr, st))
+
+
+def sfu_probe(iters: int, sink, stream: Optional[int] = None) -> int:
+    """Enqueues the special-function-unit probe (``rodimus_ddts_sfu_probe``) on the current
+    stream and returns the number of approximations it executes; the caller times it."""
+    import torch
+    st = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    ops = ctypes.c_longlong(0)
+    rc = int(load_library().rodimus_ddts_sfu_probe(int(iters), sink.data_ptr(), st, ctypes.byref(ops)))
+    if rc != OK:
+        raise RodimusError(rc, "rodimus_ddts_sfu_probe")
+    return int(ops.value)
 
 
 def step_raw(p: StepParams) -> int:

@@ -6,7 +6,7 @@ an application that gave away all device memory at start-up, or in a serving loo
 supply the small workspace ``rodimus_ddts_fwd`` asks for, so the library carries one of fixed
 size in its own device image.  These tests call that variant through the C ABI, twice in a row
 (the built-in array keeps whatever the previous call left in it), and require the same outputs
-as the ordinary entry point, which is itself held to the oracle elsewhere.
+as the ordinary entry point and, like it, agreement with the CPU oracle.
 
 This file sorts last on purpose: a run that stops at the first failure has then already been
 through every other test.
@@ -18,6 +18,7 @@ import pytest
 
 import paper_2410_06577_b200 as rd
 from paper_2410_06577_b200 import workloads as wl
+from oracle import ddts_oracle as orc
 from tests._util import TOL_BF16, TOL_F32, host, prefill_to_device, rel_err
 
 
@@ -42,6 +43,8 @@ def _both_ways(p_in, tol):
     p.workspace, p.workspace_bytes = ws.data_ptr(), ws.numel()
     assert rd.fwd_raw(p) == rd.OK
     assert rd.device_status(ws) == rd.OK
+    ro, rs = orc.ref_fwd(p_in.q, p_in.k, p_in.x, p_in.y, p_in.v, s0=p_in.s0,
+                         cu_seqlens=p_in.cu_seqlens, scale=0.5)
     # the variant without a workspace, two calls in a row
     for _ in range(2):
         o, s = new_o(), new_s()
@@ -52,6 +55,15 @@ def _both_ways(p_in, tol):
         torch.cuda.synchronize()
         assert rel_err(host(o), host(o_ref)) <= tol
         assert rel_err(host(s), host(s_ref)) <= tol
+        # and directly against the oracle, sequence by sequence for packed inputs
+        cu = p_in.cu_seqlens if p_in.cu_seqlens is not None else [0, T]
+        for n in range(len(cu) - 1):
+            lo, hi = int(cu[n]), int(cu[n + 1])
+            so = np.s_[:, :, lo:hi] if p_in.cu_seqlens is not None else np.s_[...]
+            ss = np.s_[n] if p_in.cu_seqlens is not None else np.s_[...]
+            if hi > lo:
+                assert rel_err(host(o)[so], ro[so]) <= tol, n
+            assert rel_err(host(s)[ss], rs[ss]) <= tol, n
 
 
 @pytest.mark.gpu
