@@ -6,8 +6,19 @@
 //   Qt_r = q_r 2^{b_r}            Kt_i = k_i ahat_i 2^{-b_i}          D = 2^{b_C}
 //   P = mask(Qt Kt^T)             O = P V + Qt S_in                   S_out = D . (S_in + Kt^T V)
 // The state update is written with the chunk decay OUTSIDE the bracket, so the same Kt tile
-// serves the scores (as a K-major operand) and the state update (as an MN-major operand), and
-// the row scaling by D happens when the state makes its once-per-chunk trip through registers.
+// serves the scores and the state update, and the scaling by D happens when the state makes its
+// once-per-chunk trip through registers.
+//
+// Everything that involves the value columns is computed TRANSPOSED, with the value column as
+// the M extent of the tensor-core instruction (tensor-memory lane = value column):
+//   S^T += V^T Kt            [128 value columns x 128 channels]   A = V^T (smem), B = Kt (smem)
+//   O^T  = V^T P^T + Sb Qt^T [128 value columns x 64 rows]        A = V^T (smem) / Sb (TENSOR
+//                                                                  MEMORY), B = P, Qt (smem)
+// so every one of these instructions runs at M = 128 (an M = 64 instruction uses half of the
+// datapath), and the bf16 copy Sb of the state that the readout contracts with is an A operand
+// in tensor memory: it never goes through shared memory, which is the resource the roles of
+// this kernel compete for.  With lane = value column, a warp's accesses to the initial and
+// final states in global memory are 128 contiguous bytes per key channel.
 //
 // Every quantity that depends on the gates is per key channel and independent of the value
 // column, so two CTAs that own the two 128-column halves of a 256-column slab of the state would
@@ -24,7 +35,7 @@
 // Roles in one CTA (19 warps), connected by mbarriers; every wait is bounded:
 //   warp 0        TMA producer (own channel slab of q,k,x,y and both slabs of the v slice)
 //   warp 1        tcgen05.mma issuer, owns the TMEM allocation
-//   warps 2-5     state group: TMEM <-> registers trip of S, initial / final state I/O
+//   warps 2-5     state group: TMEM <-> registers trip of S^T, initial / final state I/O
 //   warps 6-9     score / output group
 //   warps 10-17   gate group: 8 rows x 2 channels per thread, packed fp32x2 arithmetic
 //   warp 18       gate control: chunk totals, verdict exchange with the partner, the two slab
@@ -34,9 +45,8 @@
 // The loop-carried chain is  state update of pass g -> rescaling of S -> state update of pass
 // g+1 , so the issuer puts the state update of a pass BEFORE its output contractions, and the
 // state lives in TWO TMEM buffers used alternately: the state group reads S_in + Kt^T V of the
-// previous pass from one, writes D times it into the other (which frees the next state update
-// at once), and afterwards, off the chain, reads the old buffer again to make the bf16 copy
-// that the readout takes as an operand.
+// previous pass from one and writes D times it into the other, as fp32 for the next state update
+// and as packed bf16 (also double-buffered) for the readout.
 #include <cuda.h>
 
 #include <cstring>
@@ -62,14 +72,16 @@ constexpr int kRxQ = 0, kRxK = kSlabBytes;
 constexpr int kRxBytes = 2 * kSlabBytes;      // 16 KiB
 constexpr int kStages = 3, kRxBufs = 2;
 constexpr int kOperandBytes = kStages * kStageBytes + kRxBufs * kRxBytes;  // 176 KiB
-constexpr int kSsSlabBytes = kDK * 128;       // [128 rows][64 bf16]
-constexpr int kOffSs = kOperandBytes;                     // bf16 copy of the state, 2 slabs
-constexpr int kOffD = kOffSs + 2 * kSsSlabBytes;          // float [kStages][64]: own 2^{b_C}
+constexpr int kOtRowBytes = kDVS * 2;                     // one output row of this CTA: 256 B
+constexpr int kOtBytes = kC * kOtRowBytes;                // output tile [64 rows][128 bf16], 16 KiB
+constexpr int kOffOt = kOperandBytes;                     // two output tiles (pass parity)
+constexpr int kOffDp = kOffOt + 2 * kOtBytes;             // float [4][128]: chunk decays of all
+                                                          // channels, per published pass (g & 3)
 constexpr int kBlkFloats = 68;                            // 64 decays, verdict, stage, 2 pad
 constexpr int kBlkBytes = kBlkFloats * 4;                 // 272 B, a multiple of 16
-constexpr int kOffTx = kOffD + kStages * kCH * 4;         // float [2][68]: block to send
+constexpr int kOffTx = kOffDp + 4 * kDK * 4;              // float [2][68]: block to send
 constexpr int kOffRx = kOffTx + kRxBufs * kBlkBytes;      // float [2][68]: block received
-constexpr int kGateWarp0 = 10, kGateWarps = 8;
+constexpr int kGateWarp0 = 10, kGateWarps = 16;
 constexpr int kGR = kC / kGateWarps;                       // rows per gate thread
 constexpr int kOffTot = kOffRx + kRxBufs * kBlkBytes;     // float [2][8][64]: scan partials
 constexpr int kOffBar = kOffTot + 2 * kGateWarps * kCH * 4;
@@ -83,8 +95,10 @@ static_assert(kSmemBytes <= 232448, "shared memory budget");
 constexpr int kThreads = 32 * (kGateWarp0 + kGateWarps + 1);  // 608: 8 gate warps + control
 constexpr int kStateWarp0 = 2, kScoreWarp0 = 6;
 
-// TMEM columns (fp32 words): two state buffers, output, scores
-constexpr uint32_t kColS = 0, kColO = 256, kColP = 384, kTmemCols = 512;
+// TMEM columns (32-bit words): two state buffers S^T [lane = value column][128 channels], output
+// O^T [lane = value column][64 rows], scores P [64 rows in 16-lane groups][64], and two buffers
+// of the bf16 state copy Sb [lane = value column][64 columns = 128 channels, two per word]
+constexpr uint32_t kColS = 0, kColO = 256, kColP = 320, kColSb = 384, kTmemCols = 512;
 
 // mbarrier indices
 enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                      (1 + bytes)
@@ -94,9 +108,10 @@ enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                    
        BAR_VERD0, BAR_VERD1,          // own verdict written + partner's block landed (1 + bytes)
        BAR_RXFREE0, BAR_RXFREE1,      // partner is done with ITS receive buffer            (1)
        BAR_PFULL, BAR_PREADY,
-       BAR_SREADY_S,                  // S rescaled in TMEM: the state update may accumulate (128)
-       BAR_SREADY_O,                  // bf16 copy of S_in in shared memory: the readout may run (128)
+       BAR_SREADY,                    // state entering the pass is in TMEM, fp32 and bf16 (128)
        BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN,
+       BAR_OTFULL0, BAR_OTFULL1,      // output tile written by the whole score group        (128)
+       BAR_OTFREE0, BAR_OTFREE1,      // output tile's copies to global have read it            (1)
        BAR_ROWS };                    // every gate warp has rewritten its rows of the pass (8)
 static_assert(BAR_ROWS < kNumBars, "barrier count");
 
@@ -256,7 +271,8 @@ template <int INGATE, bool STATE_ONLY>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
-                     const __grid_constant__ CUtensorMap map_v, const PairArgs a) {
+                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
+                     const PairArgs a) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
@@ -264,7 +280,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   volatile Control* ctl = reinterpret_cast<volatile Control*>(gbase + kOffMisc);
   volatile int* abort_flag = &ctl->abort_flag;
-  float* sD = reinterpret_cast<float*>(gbase + kOffD);
+  float* sDp = reinterpret_cast<float*>(gbase + kOffDp);
   volatile float* sTx = reinterpret_cast<volatile float*>(gbase + kOffTx);
   volatile float* sRx = reinterpret_cast<volatile float*>(gbase + kOffRx);
   float* sTot = reinterpret_cast<float*>(gbase + kOffTot);
@@ -298,14 +314,59 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
     mbar_init(bar(BAR_PFULL), 1);
     mbar_init(bar(BAR_PREADY), 128);
-    mbar_init(bar(BAR_SREADY_S), 128);
-    mbar_init(bar(BAR_SREADY_O), 128);
+    mbar_init(bar(BAR_SREADY), 128);
     mbar_init(bar(BAR_SFULL), 1);
     mbar_init(bar(BAR_OFULL), 1);
     mbar_init(bar(BAR_OFREE), 128);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(BAR_OTFULL0 + i), 128);
+      mbar_init(bar(BAR_OTFREE0 + i), 1);
+    }
     mbar_init(bar(BAR_GSCAN), kGateWarps + 1);
     mbar_init(bar(BAR_ROWS), kGateWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // One 64-row tile of this CTA's operands into stage s (this thread is the producer).
+  auto issue_fill = [&](uint32_t s, const Item& it, int j, int tpos) {
+    ctl->tag[s][0] = j;
+    ctl->tag[s][1] = tpos;
+    const uint32_t st = stage_base + s * kStageBytes;
+    const uint32_t fb = bar(BAR_FULL0 + s);
+    mbar_expect_tx(fb, STATE_ONLY ? kStageBytes - kSlabBytes : kStageBytes);
+    // rows beyond the tensor read as zeros; rows of the next sequence are masked later
+    const int y = (int)(it.row0 + tpos);
+    const int xc = rank * kCH;
+    tma_load_2d(st + kStX, &map_x, xc, y, fb);
+    tma_load_2d(st + kStY, &map_y, xc, y, fb);
+    if (!STATE_ONLY) tma_load_2d(st + kStQ, &map_q, xc, y, fb);
+    tma_load_2d(st + kStK, &map_k, xc, y, fb);
+    tma_load_2d(st + kStV, &map_v, it.col0, y, fb);
+    tma_load_2d(st + kStV + kSlabBytes, &map_v, it.col0 + 64, y, fb);
+    // The tile that will go into this stage NEXT time is asked into L2 now: a stage is refilled
+    // only when its pass has been consumed, so the fill's latency is on the critical cycle of
+    // the ring, and from L2 it is less than half of what it is from HBM.
+    const int yp = y + kStages * kC;
+    if (tpos + kStages * kC < it.len) {
+      tma_prefetch_2d(&map_x, xc, yp);
+      tma_prefetch_2d(&map_y, xc, yp);
+      if (!STATE_ONLY) tma_prefetch_2d(&map_q, xc, yp);
+      tma_prefetch_2d(&map_k, xc, yp);
+      tma_prefetch_2d(&map_v, it.col0, yp);
+      tma_prefetch_2d(&map_v, it.col0 + 64, yp);
+    }
+  };
+  // The first fill touches only this CTA's own barriers and shared memory, so it goes out
+  // before the tensor-memory allocation and the cluster handshake instead of after them.
+  uint32_t early_fills = 0;
+  if (tid == 0) {
+    const long long item0 = (long long)(blockIdx.x >> 1);
+    if (item0 < a.n_items) {
+      const Item it = decode_item(a, item0, rank);
+      if (it.len > 0) {
+        issue_fill(0, it, 0, 0);
+        early_fills = 1;
+      }
+    }
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -326,9 +387,9 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   if (warp == 0) {
     // ===================================== TMA producer =====================================
     if (lane == 0) {
-      uint32_t f = 0;         // fills issued
-      uint32_t s = 0, ph = 0; // stage and phase of fill f
-      int j = 0, tpos = 0;    // speculative position: item index and token
+      uint32_t f = early_fills;            // fills issued
+      uint32_t s = early_fills, ph = 0;    // stage and phase of fill f
+      int j = 0, tpos = early_fills * kC;  // speculative position: item index and token
       int seen = 0;           // last redirect taken
       bool ok = true;
       while (ok) {
@@ -359,20 +420,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           __nanosleep(100);
         }
         if (!have) break;
-        ctl->tag[s][0] = j;
-        ctl->tag[s][1] = tpos;
-        const uint32_t st = stage_base + s * kStageBytes;
-        const uint32_t fb = bar(BAR_FULL0 + s);
-        mbar_expect_tx(fb, STATE_ONLY ? kStageBytes - kSlabBytes : kStageBytes);
-        // rows beyond the tensor read as zeros; rows of the next sequence are masked later
-        const int y = (int)(it.row0 + tpos);
-        const int xc = rank * kCH;
-        tma_load_2d(st + kStX, &map_x, xc, y, fb);
-        tma_load_2d(st + kStY, &map_y, xc, y, fb);
-        if (!STATE_ONLY) tma_load_2d(st + kStQ, &map_q, xc, y, fb);
-        tma_load_2d(st + kStK, &map_k, xc, y, fb);
-        tma_load_2d(st + kStV, &map_v, it.col0, y, fb);
-        tma_load_2d(st + kStV + kSlabBytes, &map_v, it.col0 + 64, y, fb);
+        issue_fill(s, it, j, tpos);
         ++f;
         if (++s == kStages) { s = 0; ph ^= 1; }
         tpos += kC;
@@ -391,10 +439,10 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // Every lane runs the loop (waits, descriptor arithmetic stay warp-uniform); lane 0 issues.
     {
       const bool issuer = lane == 0;
-      constexpr uint32_t kIdescP = make_idesc(64, 64, 0, 0);
-      constexpr uint32_t kIdescO = make_idesc(64, kDVS, 0, 1);
-      constexpr uint32_t kIdescS = make_idesc(128, kDVS, 1, 1);
-      const uint32_t ss = base + kOffSs;
+      constexpr uint32_t kIdescP = make_idesc(64, 64, 0, 0);       // P = Qt Kt^T
+      constexpr uint32_t kIdescS = make_idesc(kDVS, kDK, 1, 1);    // S^T += V^T Kt
+      constexpr uint32_t kIdescOv = make_idesc(kDVS, kC, 1, 0);    // O^T  = V^T P^T
+      constexpr uint32_t kIdescOs = make_idesc(kDVS, kC, 0, 0);    // O^T += Sb Qt^T, A in TMEM
       uint32_t g = 0;
       bool ok = true;
       for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
@@ -418,10 +466,12 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const uint32_t dq0 = desc_lo_kmajor(rank == 0 ? q_own : q_rx);
           const uint32_t dq1 = desc_lo_kmajor(rank == 0 ? q_rx : q_own);
           const uint32_t dk0 = desc_lo_kmajor(k_lo_addr), dk1 = desc_lo_kmajor(k_hi_addr);
-          const uint32_t dkt = desc_lo_mnmajor(k_lo_addr, k_hi_addr - k_lo_addr);  // Kt^T, 128 channels
+          // Kt as [rows][128 channels], channels 0..63 and 64..127 in two slabs
+          const uint32_t dkt = desc_lo_mnmajor(k_lo_addr, k_hi_addr - k_lo_addr);
+          // V as [rows][128 value columns], two 64-column slabs
           const uint32_t dv = desc_lo_mnmajor(st + kStV, kSlabBytes);
           const uint32_t dp = desc_lo_kmajor(st + kStY);
-          const uint32_t dss = desc_lo_mnmajor(ss, kSsSlabBytes);
+          const uint32_t t_sb = tmem + kColSb + (g & 1) * 64;
           tc_fence_after();
           // P = Qt Kt^T : M = 64 (rows r), N = 64 (rows i), K = 128 channels
           if (issuer && !STATE_ONLY) {
@@ -432,31 +482,32 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             for (int kk = 0; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColP, dq1 + 2 * kk, dk1 + 2 * kk, kIdescP);
             umma_commit(bar(BAR_PFULL));
           }
-          if (!(ok = mbar_wait(bar(BAR_SREADY_S), ph1, abort_flag, a.hdr))) break;
+          if (!(ok = mbar_wait(bar(BAR_SREADY), ph1, abort_flag, a.hdr))) break;
           tc_fence_after();
           if (issuer) {
-            // S_in + Kt^T V : M = 128 channels, N = 128, K = 64 rows (S_in sits in buffer g & 1)
+            // S_in^T + V^T Kt : M = 128 value columns, N = 128 channels, K = 64 rows (S_in^T sits
+            // in buffer g & 1)
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              umma_bf16_lo<true>(tmem + kColS + (g & 1) * 128, dkt + 128 * kk, dv + 128 * kk, kIdescS);
+              umma_bf16_lo<true>(tmem + kColS + (g & 1) * 128, dv + 128 * kk, dkt + 128 * kk, kIdescS);
             umma_commit(bar(BAR_SFULL));
             if (STATE_ONLY) umma_commit(bar(BAR_EMPTY0 + s));
           }
           if (STATE_ONLY) { ++g; continue; }             // no scores, no outputs
           if (!(ok = mbar_wait(bar(BAR_PREADY), ph1, abort_flag, a.hdr))) break;
-          if (!(ok = mbar_wait(bar(BAR_SREADY_O), ph1, abort_flag, a.hdr))) break;
           if (!(ok = mbar_wait(bar(BAR_OFREE), ph1 ^ 1, abort_flag, a.hdr))) break;
           tc_fence_after();
           if (issuer) {
-            // O = P V : M = 64, N = 128, K = 64 rows i (P operand lives in the consumed y slab)
-            umma_bf16_lo<false>(tmem + kColO, dp, dv, kIdescO);
+            // O^T = V^T P^T : M = 128 value columns, N = 64 rows r, K = 64 rows i (the masked
+            // scores P[r][i] live in the consumed y slab)
+            umma_bf16_lo<false>(tmem + kColO, dv, dp, kIdescOv);
 #pragma unroll
-            for (int kk = 1; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColO, dp + 2 * kk, dv + 128 * kk, kIdescO);
-            // O += Qt S_in : K = 128 channels
+            for (int kk = 1; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColO, dv + 128 * kk, dp + 2 * kk, kIdescOv);
+            // O^T += Sb Qt^T : K = 128 channels; Sb (bf16 copy of S_in^T) is read from TMEM
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColO, dq0 + 2 * kk, dss + 128 * kk, kIdescO);
+            for (int kk = 0; kk < 4; ++kk) umma_bf16_atmem<true>(tmem + kColO, t_sb + 8 * kk, dq0 + 2 * kk, kIdescOs);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColO, dq1 + 2 * kk, dss + 128 * (kk + 4), kIdescO);
+            for (int kk = 0; kk < 4; ++kk) umma_bf16_atmem<true>(tmem + kColO, t_sb + 8 * (kk + 4), dq1 + 2 * kk, kIdescOs);
             umma_commit(bar(BAR_OFULL));
             umma_commit(bar(BAR_EMPTY0 + s));   // every contraction of the pass has read its operands
           }
@@ -466,123 +517,104 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
   } else if (warp >= kStateWarp0 && warp < kStateWarp0 + 4) {
     // ====================================== state group ======================================
-    // Pass g accumulates its state update in TMEM buffer g & 1.  Each thread owns one state row
-    // (key channel).  Step 1 reads S_in + Kt^T V of pass g-1 from the other buffer, multiplies
-    // by that pass's chunk decay and writes the result, the state entering pass g, into buffer
-    // g & 1: the state update of pass g may start.  Step 2 reads the old buffer again and stores
-    // the same product as bf16 in shared memory for the readout, once the readout of pass g-1
-    // has finished with the previous copy.
+    // Each thread owns one value column of the CTA's slice (= one TMEM lane of S^T); the 128
+    // key channels are its TMEM columns.  Pass g accumulates its state update in buffer g & 1.
+    // Once per pass the group reads S_in^T + V^T Kt of pass g-1 from the other buffer, scales
+    // channel d by that pass's chunk decay D[d], and writes the result - the state entering
+    // pass g - twice: as fp32 into buffer g & 1 (the state update of pass g accumulates onto
+    // it) and as packed bf16 into Sb buffer g & 1 (the A operand of pass g's readout).  Both
+    // targets are free: the tensor pipe runs in order, so the state update of pass g-1 having
+    // completed means the readout of pass g-2, the last reader of either, has completed too.
     const int q4 = warp & 3;                              // TMEM lane quarter this warp may touch
-    const int d = q4 * 32 + lane;                         // state row (key channel) of this thread
-    const bool own_d = (d >> 6) == rank;
-    const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16) + kColS;
-    const uint32_t ss_row = base + kOffSs + d * 128;
+    const int c = q4 * 32 + lane;                         // value column (TMEM lane) of this thread
+    const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
     const bool signaller = warp == kStateWarp0 && lane == 0;
     uint32_t g = 0;
     int prev_rx = 0;
     bool ok = true;
     for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
       const Item it = decode_item(a, item_of(j), rank);
-      const long long srow = it.state_off + (long long)d * a.dv;
+      // element (channel d, own column) of the state: soff + d * dv; a warp covers 32
+      // consecutive columns, 128 contiguous bytes per channel
+      const long long soff = it.state_off + c;
       if (it.len == 0) {  // empty sequence: final state = initial state
         if (a.sT) {
-          for (int c4 = 0; c4 < kDVS / 4; ++c4) {
-            float4 v4 = a.s0 ? *reinterpret_cast<const float4*>(a.s0 + srow + 4 * c4)
-                             : make_float4(0.f, 0.f, 0.f, 0.f);
-            *reinterpret_cast<float4*>(a.sT + srow + 4 * c4) = v4;
-          }
+#pragma unroll 4
+          for (int d = 0; d < kDK; ++d)
+            a.sT[soff + (long long)d * a.dv] = a.s0 ? a.s0[soff + (long long)d * a.dv] : 0.f;
         }
         continue;
       }
       bool last = false, first = true;
-      float Dprev = 1.f;                                  // chunk decay of the previous pass
-      float Dall = 1.f;                                   // product of the chunk decays so far
-      // 32 columns of the state entering the pass: D_prev times the previous buffer, or the
-      // caller's initial state for the first pass of a sequence
-      auto load_piece = [&](uint32_t (&r)[32], uint32_t t_prev, int piece) {
+      float Dall = 1.f;          // product of the chunk decays of channel c so far (for dtot)
+      // 32 channels of the state entering the pass: D of the previous pass times the previous
+      // buffer, or the caller's initial state for the first pass of a sequence
+      auto load_piece = [&](uint32_t (&r)[32], uint32_t t_prev, const float* dprev, int piece) {
         if (!first) {
           tmem_ld32(t_prev + piece * 32, r);
           tmem_ld_wait();
-          const float2 dd = splat(Dprev);
 #pragma unroll
-          for (int c2 = 0; c2 < 16; ++c2) {
-            const float2 t = __fmul2_rn(
-                make_float2(__uint_as_float(r[2 * c2]), __uint_as_float(r[2 * c2 + 1])), dd);
-            r[2 * c2] = __float_as_uint(t.x);
-            r[2 * c2 + 1] = __float_as_uint(t.y);
+          for (int c4 = 0; c4 < 8; ++c4) {
+            const float4 dd = *reinterpret_cast<const float4*>(dprev + piece * 32 + 4 * c4);  // broadcast
+            const float2 lo = __fmul2_rn(make_float2(__uint_as_float(r[4 * c4]), __uint_as_float(r[4 * c4 + 1])),
+                                         make_float2(dd.x, dd.y));
+            const float2 hi = __fmul2_rn(make_float2(__uint_as_float(r[4 * c4 + 2]), __uint_as_float(r[4 * c4 + 3])),
+                                         make_float2(dd.z, dd.w));
+            r[4 * c4] = __float_as_uint(lo.x);
+            r[4 * c4 + 1] = __float_as_uint(lo.y);
+            r[4 * c4 + 2] = __float_as_uint(hi.x);
+            r[4 * c4 + 3] = __float_as_uint(hi.y);
           }
         } else if (a.s0) {
 #pragma unroll
-          for (int c4 = 0; c4 < 8; ++c4) {
-            const float4 v4 = *reinterpret_cast<const float4*>(a.s0 + srow + piece * 32 + 4 * c4);
-            r[4 * c4] = __float_as_uint(v4.x);
-            r[4 * c4 + 1] = __float_as_uint(v4.y);
-            r[4 * c4 + 2] = __float_as_uint(v4.z);
-            r[4 * c4 + 3] = __float_as_uint(v4.w);
-          }
+          for (int i = 0; i < 32; ++i)
+            r[i] = __float_as_uint(a.s0[soff + (long long)(piece * 32 + i) * a.dv]);
         } else {
 #pragma unroll
-          for (int c4 = 0; c4 < 32; ++c4) r[c4] = 0u;
+          for (int i = 0; i < 32; ++i) r[i] = 0u;
         }
       };
       while (!last) {
         const uint32_t ph1 = g & 1;
-        const uint32_t t_cur = t_lane + (g & 1) * 128, t_prev = t_lane + ((g & 1) ^ 1) * 128;
+        const uint32_t t_cur = t_lane + kColS + (g & 1) * 128, t_prev = t_lane + kColS + ((g & 1) ^ 1) * 128;
+        const uint32_t t_sb = t_lane + kColSb + (g & 1) * 64;
+        const float* dprev = sDp + ((g - 1) & 3) * kDK;
         if (!first) {
           if (!(ok = mbar_wait(bar(BAR_SFULL), ph1 ^ 1, abort_flag, a.hdr))) break;  // pass g-1
           tc_fence_after();
         }
-        // step 1: the state entering this pass, into this pass's buffer
 #pragma unroll 1
         for (int piece = 0; piece < 4; ++piece) {
           uint32_t r[32];
-          load_piece(r, t_prev, piece);
+          load_piece(r, t_prev, dprev, piece);
           tmem_st32(t_cur + piece * 32, r);
+          if (!STATE_ONLY) {
+            uint32_t w[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              w[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+            tmem_st16(t_sb + piece * 16, w);
+          }
         }
         tmem_st_wait();
         tc_fence_before();
-        mbar_arrive(bar(BAR_SREADY_S));
+        mbar_arrive(bar(BAR_SREADY));
         if (!first) {
-          // the previous pass's readout has finished with the old copy (and, with its state
-          // update, with every operand of that pass: the partner may reuse the receive buffer).
-          // Signalled before waiting for pass g: publishing pass g may itself need that buffer.
+          // the previous pass's contractions have all read their operands: the partner may reuse
+          // the receive buffer.  Signalled before waiting for pass g: publishing pass g may
+          // itself need that buffer.
           if (!STATE_ONLY && !(ok = mbar_wait(bar(BAR_OFULL), ph1 ^ 1, abort_flag, a.hdr))) break;
           if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
         }
-        // this pass's chunk decay (applied on the NEXT trip); read before this pass's readout
-        // can be issued, so its stage and receive buffer are certainly still alive
         if (!(ok = mbar_wait(bar(BAR_GATED0 + (g & 3)), (g >> 2) & 1, abort_flag, a.hdr))) break;
-        const int s = ctl->pd[g & 3].stage;
-        const int rxi = ctl->pd[g & 3].rx;
+        prev_rx = ctl->pd[g & 3].rx;
         last = (ctl->pd[g & 3].flags & kPassLast) != 0;
-        const float Dcur = own_d ? sD[s * kCH + (d & 63)] : sRx[rxi * kBlkFloats + (d & 63)];
-        // step 2: bf16 copy of the same state for the readout: MN-major, row d, two 64-column
-        // slabs.  (The old buffer is untouched until the NEXT pass's step 1.)
-#pragma unroll 1
-        for (int piece = 0; piece < (STATE_ONLY ? 0 : 4); ++piece) {
-          uint32_t r[32];
-          load_piece(r, t_prev, piece);
-          const uint32_t slab = ss_row + (piece >> 1) * kSsSlabBytes;
-#pragma unroll
-          for (int c8 = 0; c8 < 4; ++c8) {
-            const int chunk = (piece & 1) * 4 + c8;
-            sts128(slab + ((chunk ^ (d & 7)) << 4),
-                   pack_bf16(__uint_as_float(r[8 * c8]), __uint_as_float(r[8 * c8 + 1])),
-                   pack_bf16(__uint_as_float(r[8 * c8 + 2]), __uint_as_float(r[8 * c8 + 3])),
-                   pack_bf16(__uint_as_float(r[8 * c8 + 4]), __uint_as_float(r[8 * c8 + 5])),
-                   pack_bf16(__uint_as_float(r[8 * c8 + 6]), __uint_as_float(r[8 * c8 + 7])));
-          }
-        }
-        fence_proxy_async();
-        mbar_arrive(bar(BAR_SREADY_O));
-        prev_rx = rxi;
-        Dprev = Dcur;
-        Dall *= Dcur;
+        Dall *= sDp[(g & 3) * kDK + c];                   // thread c follows channel c
         first = false;
         ++g;
       }
       if (!ok) break;
-      if (a.dtot && it.col0 == 0) a.dtot[it.seq_head * kDK + d] = Dall;
+      if (a.dtot && it.col0 == 0) a.dtot[it.seq_head * kDK + c] = Dall;
       // final state of this item (also keeps the next item's initial state from racing the MMAs)
       {
         const uint32_t lastg = g - 1;
@@ -591,19 +623,17 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         tc_fence_after();
         if (signaller) mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + prev_rx), peer));
         if (a.sT && (a.sT_only < 0 || it.seq == a.sT_only)) {
-          const long long frow = a.sT_only < 0 ? srow : srow - (long long)a.sT_only * a.H * kDK * a.dv;
-          const uint32_t t_fin = t_lane + (lastg & 1) * 128;
+          const long long foff = a.sT_only < 0 ? soff : soff - (long long)a.sT_only * a.H * kDK * a.dv;
+          const uint32_t t_fin = t_lane + kColS + (lastg & 1) * 128;
+          const float* dlast = sDp + (lastg & 3) * kDK;
 #pragma unroll 1
           for (int piece = 0; piece < 4; ++piece) {
             uint32_t r[32];
             tmem_ld32(t_fin + piece * 32, r);
             tmem_ld_wait();
 #pragma unroll
-            for (int c4 = 0; c4 < 8; ++c4) {
-              *reinterpret_cast<float4*>(a.sT + frow + piece * 32 + 4 * c4) =
-                  make_float4(Dprev * __uint_as_float(r[4 * c4]), Dprev * __uint_as_float(r[4 * c4 + 1]),
-                              Dprev * __uint_as_float(r[4 * c4 + 2]), Dprev * __uint_as_float(r[4 * c4 + 3]));
-            }
+            for (int i = 0; i < 32; ++i)
+              a.sT[foff + (long long)(piece * 32 + i) * a.dv] = dlast[piece * 32 + i] * __uint_as_float(r[i]);
           }
         }
         tc_fence_before();
@@ -614,6 +644,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int q4 = warp & 3;
     const int r_row = q4 * 16 + lane;                     // chunk row held by lanes 0..15 (M = 64)
     const bool has_row = lane < 16;
+    const int c_out = q4 * 32 + lane;                     // value column of this thread (O^T lane)
     const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
     __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(a.o);
     const bool unit_scale = a.scale == 1.0f;
@@ -691,35 +722,57 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         fence_proxy_async();
         tc_fence_before();
         mbar_arrive(bar(BAR_PREADY));
-        // output rows of this pass
+        // Outputs of this pass.  O^T has the CTA's value column c_out in TMEM lane c_out and the
+        // pass's rows in its columns; the tile is transposed through shared memory (a warp
+        // writes 32 adjacent bf16 of one row per instruction) and leaves as bulk copies of half a
+        // row (128 contiguous bytes) per thread, live rows only.  Two tiles alternate, so the
+        // copies of a pass are still reading while the next pass is written.
         if (!(ok = mbar_wait(bar(BAR_OFULL), ph1, abort_flag, a.hdr))) break;
         tc_fence_after();
-        __nv_bfloat16* orow = o + (row + r_row) * a.dv + it.col0;
-        const float2 sc2 = splat(a.scale);
+        // the copies that read this tile two passes ago have finished reading
+        if (!(ok = mbar_wait(bar(BAR_OTFREE0 + ph1), ((g >> 1) & 1) ^ 1, abort_flag, a.hdr))) break;
+        const uint32_t ot = base + kOffOt + ph1 * kOtBytes;
 #pragma unroll 1
-        for (int piece = 0; piece < 4; ++piece) {
+        for (int piece = 0; piece < 2; ++piece) {
           uint32_t r[32];
           tmem_ld32(t_lane + kColO + piece * 32, r);
           tmem_ld_wait();
-          if (has_row && r_row < nr) {
+          if (piece == 1) {                               // the accumulator is free again
+            tc_fence_before();
+            mbar_arrive(bar(BAR_OFREE));
+          }
+          const uint32_t dst = ot + piece * 32 * kOtRowBytes + c_out * 2;
 #pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {
-              uint32_t w[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                float2 t = make_float2(__uint_as_float(r[8 * c8 + 2 * e]), __uint_as_float(r[8 * c8 + 2 * e + 1]));
-                if (!unit_scale) t = __fmul2_rn(t, sc2);
-                w[e] = pack_bf16(t.x, t.y);
-              }
-              *reinterpret_cast<uint4*>(orow + piece * 32 + 8 * c8) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
+          for (int i = 0; i < 32; ++i) {
+            float t = __uint_as_float(r[i]);
+            if (!unit_scale) t *= a.scale;
+            sts16(dst + i * kOtRowBytes, __bfloat16_as_ushort(__float2bfloat16_rn(t)));
           }
         }
-        tc_fence_before();
-        mbar_arrive(bar(BAR_OFREE));
+        fence_proxy_async();
+        mbar_arrive(bar(BAR_OTFULL0 + ph1));
+        if (q4 == 0) {
+          // One warp sends the tile: a full tile as ONE tensor copy (the copy engine takes its
+          // requests one after another, and a hundred small ones per pass cost more than the
+          // pass), a ragged last tile of a sequence row by row so that nothing is written into
+          // the rows of the next sequence.
+          if (!(ok = mbar_wait(bar(BAR_OTFULL0 + ph1), (g >> 1) & 1, abort_flag, a.hdr))) break;
+          if (nr == kC) {
+            if (lane == 0) tma_store_2d(&map_o, it.col0, (int)row, ot);
+          } else {
+            for (int rr = lane; rr < nr; rr += 32)
+              bulk_store(o + (row + rr) * a.dv + it.col0, ot + rr * kOtRowBytes, kOtRowBytes);
+          }
+          bulk_commit();
+          // the previous pass's copies (the other tile) have finished reading
+          bulk_wait_read<1>();
+          __syncwarp();
+          if (g > 0 && lane == 0) mbar_arrive(bar(BAR_OTFREE0 + (ph1 ^ 1)));
+        }
         ++g;
       }
     }
+    bulk_wait<0>();   // this thread's output copies are complete before the CTA may exit
   } else if (warp >= kGateWarp0) {
     // ============================== gate group and its control warp ==============================
     // The gate warps do the per-element work; the control warp does everything that is
@@ -770,6 +823,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int left = it.len - tpos;
         const int nr = min(min(kC, left), lcap);
         float* tot = sTot + (m & 1) * (kGateWarps * kCH);
+        float2 Down = splat(1.f);                         // control warp: own chunk decays
         if (!is_ctl) {
           float2 b[kGR], eh[kGR];
           const float2 run = gate_phase1<INGATE>(st + kStX, st + kStY, off, gw * kGR, nr, b, eh);
@@ -797,7 +851,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             all = __fadd2_rn(all, *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane));
           const bool viol_own = __any_sync(0xffffffffu, all.x < -kRange || all.y < -kRange) && nr > 1;
           const float2 D = make_float2(ex2f(all.x), ex2f(all.y));
-          *reinterpret_cast<float2*>(sD + s * kCH + 2 * lane) = D;
+          Down = D;
           // the send block m&1 (like the partner's receive buffer m&1) must be free again
           if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
           volatile float* blk = sTx + rxi * kBlkFloats;
@@ -864,7 +918,16 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           continue;
         }
         // the control warp alone publishes the pass (its descriptor is already written): it has
-        // seen every gate warp's rows through BAR_ROWS
+        // seen every gate warp's rows through BAR_ROWS.  With the pass go the chunk decays of all
+        // 128 channels (own half from registers, the partner's from its block) for the state
+        // group, in a slot of their own: the stage and the block are recycled sooner.
+        if (is_ctl) {
+          float* dp = sDp + (g & 3) * kDK;
+          *reinterpret_cast<float2*>(dp + rank * kCH + 2 * lane) = Down;
+          *reinterpret_cast<float2*>(dp + peer * kCH + 2 * lane) =
+              make_float2(sRx[rxi * kBlkFloats + 2 * lane], sRx[rxi * kBlkFloats + 2 * lane + 1]);
+          __syncwarp();
+        }
         if (leader) {
           if (nr < min(kC, left)) redirect(j, tpos + nr);   // the prefetcher assumed 64 rows
           mbar_arrive(bar(BAR_GATED0 + (g & 3)));
@@ -921,28 +984,29 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// [rows, cols] bf16 row-major, box = 64 rows x 64 columns (128 bytes), 128-byte swizzle.
-bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
+// [rows, cols] bf16 row-major.  Operand maps: box = 64 rows x 64 columns (128 bytes), 128-byte
+// swizzle.  Output map: box = 64 rows x 128 columns, dense (the layout of the output tile).
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, bool output = false) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {cols * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)kC};
+  const cuuint32_t box[2] = {output ? (cuuint32_t)kDVS : 64u, (cuuint32_t)kC};
   const cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, output ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int INGATE, bool STATE_ONLY>
 cudaError_t launch_pair(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mx,
-                        const CUtensorMap& my, const CUtensorMap& mv, const PairArgs& a,
-                        int max_pairs, cudaStream_t st) {
+                        const CUtensorMap& my, const CUtensorMap& mv, const CUtensorMap& mo,
+                        const PairArgs& a, int max_pairs, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(ddts_fwd_pair_kernel<INGATE, STATE_ONLY>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
   const long long pairs = a.n_items < max_pairs ? a.n_items : max_pairs;
-  ddts_fwd_pair_kernel<INGATE, STATE_ONLY><<<(unsigned)(2 * pairs), kThreads, kSmemBytes, st>>>(mq, mk, mx, my, mv, a);
+  ddts_fwd_pair_kernel<INGATE, STATE_ONLY><<<(unsigned)(2 * pairs), kThreads, kSmemBytes, st>>>(mq, mk, mx, my, mv, mo, a);
   return cudaGetLastError();
 }
 
@@ -1083,24 +1147,24 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
 
-  CUtensorMap mq, mk, mx, my, mv;
+  CUtensorMap mq, mk, mx, my, mv, mo;
   if (rows > 0) {
     if (!make_map(&mq, p.q, rows, kDK) || !make_map(&mk, p.k, rows, kDK) ||
         !make_map(&mx, p.gate_x, rows, kDK) || !make_map(&my, p.temp_y, rows, kDK) ||
-        !make_map(&mv, p.v, rows, (uint64_t)p.dv))
+        !make_map(&mv, p.v, rows, (uint64_t)p.dv) || !make_map(&mo, p.o, rows, (uint64_t)p.dv, true))
       return cudaErrorUnknown;
   } else {
-    memset(&mq, 0, sizeof(mq)); mk = mq; mx = mq; my = mq; mv = mq;  // never dereferenced: no chunks
+    memset(&mq, 0, sizeof(mq)); mk = mq; mx = mq; my = mq; mv = mq; mo = mq;  // never dereferenced: no chunks
   }
   const int max_pairs = sms / 2 > 0 ? sms / 2 : 1;   // one CTA per SM; a pair shares a TPC
   auto run = [&](const PairArgs& a, cudaStream_t st) {
     if (a.state_only)
       return p.ingate == RODIMUS_INGATE_POW_G
-                 ? launch_pair<RODIMUS_INGATE_POW_G, true>(mq, mk, mx, my, mv, a, max_pairs, st)
-                 : launch_pair<RODIMUS_INGATE_POW_SIGMOID, true>(mq, mk, mx, my, mv, a, max_pairs, st);
+                 ? launch_pair<RODIMUS_INGATE_POW_G, true>(mq, mk, mx, my, mv, mo, a, max_pairs, st)
+                 : launch_pair<RODIMUS_INGATE_POW_SIGMOID, true>(mq, mk, mx, my, mv, mo, a, max_pairs, st);
     return p.ingate == RODIMUS_INGATE_POW_G
-               ? launch_pair<RODIMUS_INGATE_POW_G, false>(mq, mk, mx, my, mv, a, max_pairs, st)
-               : launch_pair<RODIMUS_INGATE_POW_SIGMOID, false>(mq, mk, mx, my, mv, a, max_pairs, st);
+               ? launch_pair<RODIMUS_INGATE_POW_G, false>(mq, mk, mx, my, mv, mo, a, max_pairs, st)
+               : launch_pair<RODIMUS_INGATE_POW_SIGMOID, false>(mq, mk, mx, my, mv, mo, a, max_pairs, st);
   };
   char* ws = reinterpret_cast<char*>(p.workspace);
   PairArgs a;
