@@ -642,8 +642,13 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   } else if (warp >= kScoreWarp0 && warp < kScoreWarp0 + 4) {
     // ================================== score / output group ==================================
     const int q4 = warp & 3;
-    const int r_row = q4 * 16 + lane;                     // chunk row held by lanes 0..15 (M = 64)
-    const bool has_row = lane < 16;
+    // stmatrix roles of this thread: it addresses row mat_k of matrix lane/8 of each x4 group;
+    // matrices 0,1 are the low / high 8 rows of one 8-column block, 2,3 those of the next block
+    const int mat_k = lane & 7, mat_h = (lane >> 3) & 1, mat_j = lane >> 4;
+    // diagonal block: element (row t/4, columns 2(t%4) + e) is kept iff the column does not
+    // exceed the row
+    const uint32_t mask_diag = (2 * (lane & 3) <= (lane >> 2) ? 0x0000FFFFu : 0u) |
+                               (2 * (lane & 3) + 1 <= (lane >> 2) ? 0xFFFF0000u : 0u);
     const int c_out = q4 * 32 + lane;                     // value column of this thread (O^T lane)
     const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
     __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(a.o);
@@ -675,7 +680,9 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int nr = ctl->pd[g & 3].nr;
         const long long row = ctl->pd[g & 3].row;
         last = (ctl->pd[g & 3].flags & kPassLast) != 0;
-        const uint32_t ps_row = stage_base + s * kStageBytes + kStY + r_row * 128;
+        // row of the P tile ([r][i], 128-byte rows, 16-byte chunks swizzled by r & 7) whose
+        // address this thread supplies to stmatrix: row block mat_h, row mat_k within it
+        const uint32_t ps_mat = stage_base + s * kStageBytes + kStY + (q4 * 16 + mat_h * 8 + mat_k) * 128;
         tc_fence_after();
         if (warp == kScoreWarp0 && lane == 0) {
           // P exists, so the partner's copies out of ITS stage have all landed here (the issuer
@@ -684,40 +691,32 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]);
           mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
         }
-        // causal mask (i <= r kept).  This warp's rows are 16*q4 .. 16*q4+15, so of the two
-        // 32-column halves one is entirely kept or entirely dropped and one holds the diagonal.
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-          const int c_lo = half * 32;
-          if (c_lo > q4 * 16 + 15) {                      // entirely above the diagonal
-            if (has_row) {
+        // Causal mask (i <= r kept) and conversion to bf16.  The M = 64 accumulator keeps this
+        // warp's rows 16*q4 .. 16*q4+15 in the first 16 lanes of its TMEM quarter; the 16x256b
+        // load hands them out in 8x8-matrix fragments (all 32 threads busy: thread t holds rows
+        // t/4 and t/4 + 8 of the warp's 16, two adjacent columns per 8-column block), so a pair
+        // of columns packs into one word and four blocks go to shared memory per stmatrix.  Of
+        // the four 16-column groups, those left of the diagonal are kept whole, the one on the
+        // diagonal is masked with a per-thread constant, those right of it are zeros that are
+        // not even read.
 #pragma unroll
-              for (int c8 = 0; c8 < 4; ++c8)
-                sts128(ps_row + (((half * 4 + c8) ^ (r_row & 7)) << 4), 0u, 0u, 0u, 0u);
-            }
-            continue;
-          }
-          uint32_t r[32];
-          tmem_ld32(t_lane + kColP + half * 32, r);
-          tmem_ld_wait();
-          const bool diag = c_lo + 31 > q4 * 16;          // some column of this half exceeds a row
-          if (has_row) {
-#pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {
-              uint32_t w[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int i0 = c_lo + 8 * c8 + 2 * e;
-                float lo = __uint_as_float(r[8 * c8 + 2 * e]), hi = __uint_as_float(r[8 * c8 + 2 * e + 1]);
-                if (diag) {
-                  lo = (i0 <= r_row) ? lo : 0.f;
-                  hi = (i0 + 1 <= r_row) ? hi : 0.f;
-                }
-                w[e] = pack_bf16(lo, hi);
-              }
-              sts128(ps_row + (((half * 4 + c8) ^ (r_row & 7)) << 4), w[0], w[1], w[2], w[3]);
+        for (int jp = 0; jp < 4; ++jp) {
+          uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;   // (rows lo, cols j0) (hi, j0) (lo, j1) (hi, j1)
+          if (jp <= q4) {
+            uint32_t r[8];
+            tmem_ld_16x256b_x2(t_lane + kColP + 16 * jp, r);
+            tmem_ld_wait();
+            m0 = pack_bf16(__uint_as_float(r[0]), __uint_as_float(r[1]));
+            m1 = pack_bf16(__uint_as_float(r[2]), __uint_as_float(r[3]));
+            m2 = pack_bf16(__uint_as_float(r[4]), __uint_as_float(r[5]));
+            m3 = pack_bf16(__uint_as_float(r[6]), __uint_as_float(r[7]));
+            if (jp == q4) {   // columns 16*q4 .. 16*q4+15 against rows 16*q4 + t/4 (+ 8)
+              m0 &= mask_diag;
+              m2 = 0u;
+              m3 &= mask_diag;
             }
           }
+          stmatrix_x4(ps_mat + (((uint32_t)(2 * jp + mat_j) ^ (uint32_t)mat_k) << 4), m0, m1, m2, m3);
         }
         fence_proxy_async();
         tc_fence_before();
