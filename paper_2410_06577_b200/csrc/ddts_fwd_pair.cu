@@ -72,8 +72,7 @@ constexpr int kRxQ = 0, kRxK = kSlabBytes;
 constexpr int kRxBytes = 2 * kSlabBytes;      // 16 KiB
 constexpr int kStages = 3, kRxBufs = 2;
 constexpr int kOperandBytes = kStages * kStageBytes + kRxBufs * kRxBytes;  // 176 KiB
-constexpr int kOtRowBytes = kDVS * 2;                     // one output row of this CTA: 256 B
-constexpr int kOtBytes = kC * kOtRowBytes;                // output tile [64 rows][128 bf16], 16 KiB
+constexpr int kOtBytes = 2 * kSlabBytes;                  // output tile: two [64 rows][64 bf16] slabs
 constexpr int kOffOt = kOperandBytes;                     // two output tiles (pass parity)
 constexpr int kOffDp = kOffOt + 2 * kOtBytes;             // float [4][128]: chunk decays of all
                                                           // channels, per published pass (g & 3)
@@ -272,6 +271,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
+                     const __grid_constant__ CUtensorMap map_o8, const __grid_constant__ CUtensorMap map_o1,
                      const PairArgs a) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -649,9 +649,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // exceed the row
     const uint32_t mask_diag = (2 * (lane & 3) <= (lane >> 2) ? 0x0000FFFFu : 0u) |
                                (2 * (lane & 3) + 1 <= (lane >> 2) ? 0xFFFF0000u : 0u);
-    const int c_out = q4 * 32 + lane;                     // value column of this thread (O^T lane)
     const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
-    __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(a.o);
     const bool unit_scale = a.scale == 1.0f;
     uint32_t g = 0;
     bool ok = true;
@@ -721,46 +719,64 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         fence_proxy_async();
         tc_fence_before();
         mbar_arrive(bar(BAR_PREADY));
-        // Outputs of this pass.  O^T has the CTA's value column c_out in TMEM lane c_out and the
-        // pass's rows in its columns; the tile is transposed through shared memory (a warp
-        // writes 32 adjacent bf16 of one row per instruction) and leaves as bulk copies of half a
-        // row (128 contiguous bytes) per thread, live rows only.  Two tiles alternate, so the
-        // copies of a pass are still reading while the next pass is written.
+        // Outputs of this pass.  O^T has the CTA's value columns in the TMEM lanes and the pass's
+        // rows in its columns.  The 16x256b load hands out 8x8 fragments [value column][row];
+        // stmatrix.trans writes each transposed, 16 bytes (8 value columns) of one output row at
+        // a time, into a tile of two 64-column slabs laid out like the operand tiles (128-byte
+        // rows, 16-byte chunks swizzled by row & 7: conflict-free), and the tile leaves through
+        // tensor copies that undo the swizzle.  Two tiles alternate, so the copies of a pass are
+        // still reading while the next pass is written.
         if (!(ok = mbar_wait(bar(BAR_OFULL), ph1, abort_flag, a.hdr))) break;
         tc_fence_after();
         // the copies that read this tile two passes ago have finished reading
         if (!(ok = mbar_wait(bar(BAR_OTFREE0 + ph1), ((g >> 1) & 1) ^ 1, abort_flag, a.hdr))) break;
         const uint32_t ot = base + kOffOt + ph1 * kOtBytes;
+        // this thread addresses output row 8 * (2 jp + mat_j) + mat_k of column block mat_h
+        const uint32_t ot_mat = ot + (q4 >> 1) * kSlabBytes + (mat_j * 8 + mat_k) * 128;
 #pragma unroll 1
-        for (int piece = 0; piece < 2; ++piece) {
+        for (int hv = 0; hv < 2; ++hv) {                  // lanes 0..15 / 16..31 of the TMEM quarter
           uint32_t r[32];
-          tmem_ld32(t_lane + kColO + piece * 32, r);
+          tmem_ld_16x256b_x8(t_lane + ((uint32_t)(16 * hv) << 16) + kColO, r);
           tmem_ld_wait();
-          if (piece == 1) {                               // the accumulator is free again
+          if (hv == 1) {                                  // the accumulator is free again
             tc_fence_before();
             mbar_arrive(bar(BAR_OFREE));
           }
-          const uint32_t dst = ot + piece * 32 * kOtRowBytes + c_out * 2;
+          if (!unit_scale) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            float t = __uint_as_float(r[i]);
-            if (!unit_scale) t *= a.scale;
-            sts16(dst + i * kOtRowBytes, __bfloat16_as_ushort(__float2bfloat16_rn(t)));
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * a.scale);
+          }
+          // 16-byte chunk (8 value columns) of this thread's matrices within the slab
+          const uint32_t chunk = (uint32_t)(4 * (q4 & 1) + 2 * hv + mat_h);
+          const uint32_t dst = ot_mat + ((chunk ^ (uint32_t)mat_k) << 4);
+#pragma unroll
+          for (int jp = 0; jp < 4; ++jp) {                // output rows 16 jp .. 16 jp + 15
+            const int j0 = 2 * jp, j1 = 2 * jp + 1;
+            stmatrix_x4_trans(dst + jp * 16 * 128,
+                              pack_bf16(__uint_as_float(r[4 * j0]), __uint_as_float(r[4 * j0 + 1])),
+                              pack_bf16(__uint_as_float(r[4 * j0 + 2]), __uint_as_float(r[4 * j0 + 3])),
+                              pack_bf16(__uint_as_float(r[4 * j1]), __uint_as_float(r[4 * j1 + 1])),
+                              pack_bf16(__uint_as_float(r[4 * j1 + 2]), __uint_as_float(r[4 * j1 + 3])));
           }
         }
         fence_proxy_async();
         mbar_arrive(bar(BAR_OTFULL0 + ph1));
         if (q4 == 0) {
-          // One warp sends the tile: a full tile as ONE tensor copy (the copy engine takes its
-          // requests one after another, and a hundred small ones per pass cost more than the
-          // pass), a ragged last tile of a sequence row by row so that nothing is written into
-          // the rows of the next sequence.
+          // One warp sends the tile.  A full tile is two tensor copies (one per slab; the copy
+          // engine takes its requests one after another, so few large ones).  A ragged last tile
+          // of a sequence goes in boxes of 8 rows and of 1 row, one per lane, so that nothing is
+          // written into the rows of the next sequence.
           if (!(ok = mbar_wait(bar(BAR_OTFULL0 + ph1), (g >> 1) & 1, abort_flag, a.hdr))) break;
           if (nr == kC) {
-            if (lane == 0) tma_store_2d(&map_o, it.col0, (int)row, ot);
+            if (lane < 2) tma_store_2d(&map_o, it.col0 + 64 * lane, (int)row, ot + lane * kSlabBytes);
           } else {
-            for (int rr = lane; rr < nr; rr += 32)
-              bulk_store(o + (row + rr) * a.dv + it.col0, ot + rr * kOtRowBytes, kOtRowBytes);
+            const int n8 = nr >> 3, n1 = nr & 7;          // at most 7 + 7 boxes per slab
+            const int slab = lane & 1, v = lane >> 1;
+            if (v < n8)
+              tma_store_2d(&map_o8, it.col0 + 64 * slab, (int)row + 8 * v, ot + slab * kSlabBytes + 8 * v * 128);
+            else if (v < n8 + n1)
+              tma_store_2d(&map_o1, it.col0 + 64 * slab, (int)row + 8 * n8 + (v - n8),
+                           ot + slab * kSlabBytes + (8 * n8 + (v - n8)) * 128);
           }
           bulk_commit();
           // the previous pass's copies (the other tile) have finished reading
@@ -983,29 +999,31 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// [rows, cols] bf16 row-major.  Operand maps: box = 64 rows x 64 columns (128 bytes), 128-byte
-// swizzle.  Output map: box = 64 rows x 128 columns, dense (the layout of the output tile).
-bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, bool output = false) {
+// [rows, cols] bf16 row-major; box = box_rows rows x 64 columns (128 bytes), 128-byte swizzle.
+// Operands and full output tiles use 64-row boxes; ragged output tiles 8-row and 1-row boxes.
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows = kC) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {cols * 2};
-  const cuuint32_t box[2] = {output ? (cuuint32_t)kDVS : 64u, (cuuint32_t)kC};
+  const cuuint32_t box[2] = {64u, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, output ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+struct PairMaps {
+  CUtensorMap q, k, x, y, v, o, o8, o1;
+};
+
 template <int INGATE, bool STATE_ONLY>
-cudaError_t launch_pair(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mx,
-                        const CUtensorMap& my, const CUtensorMap& mv, const CUtensorMap& mo,
-                        const PairArgs& a, int max_pairs, cudaStream_t st) {
+cudaError_t launch_pair(const PairMaps& m, const PairArgs& a, int max_pairs, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(ddts_fwd_pair_kernel<INGATE, STATE_ONLY>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
   const long long pairs = a.n_items < max_pairs ? a.n_items : max_pairs;
-  ddts_fwd_pair_kernel<INGATE, STATE_ONLY><<<(unsigned)(2 * pairs), kThreads, kSmemBytes, st>>>(mq, mk, mx, my, mv, mo, a);
+  ddts_fwd_pair_kernel<INGATE, STATE_ONLY><<<(unsigned)(2 * pairs), kThreads, kSmemBytes, st>>>(m.q, m.k, m.x, m.y, m.v, m.o, m.o8, m.o1, a);
   return cudaGetLastError();
 }
 
@@ -1146,24 +1164,26 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
 
-  CUtensorMap mq, mk, mx, my, mv, mo;
+  PairMaps m;
   if (rows > 0) {
-    if (!make_map(&mq, p.q, rows, kDK) || !make_map(&mk, p.k, rows, kDK) ||
-        !make_map(&mx, p.gate_x, rows, kDK) || !make_map(&my, p.temp_y, rows, kDK) ||
-        !make_map(&mv, p.v, rows, (uint64_t)p.dv) || !make_map(&mo, p.o, rows, (uint64_t)p.dv, true))
+    const uint64_t dv = (uint64_t)p.dv;
+    if (!make_map(&m.q, p.q, rows, kDK) || !make_map(&m.k, p.k, rows, kDK) ||
+        !make_map(&m.x, p.gate_x, rows, kDK) || !make_map(&m.y, p.temp_y, rows, kDK) ||
+        !make_map(&m.v, p.v, rows, dv) || !make_map(&m.o, p.o, rows, dv) ||
+        !make_map(&m.o8, p.o, rows, dv, 8) || !make_map(&m.o1, p.o, rows, dv, 1))
       return cudaErrorUnknown;
   } else {
-    memset(&mq, 0, sizeof(mq)); mk = mq; mx = mq; my = mq; mv = mq; mo = mq;  // never dereferenced: no chunks
+    memset(&m, 0, sizeof(m));   // never dereferenced: no chunks
   }
   const int max_pairs = sms / 2 > 0 ? sms / 2 : 1;   // one CTA per SM; a pair shares a TPC
   auto run = [&](const PairArgs& a, cudaStream_t st) {
     if (a.state_only)
       return p.ingate == RODIMUS_INGATE_POW_G
-                 ? launch_pair<RODIMUS_INGATE_POW_G, true>(mq, mk, mx, my, mv, mo, a, max_pairs, st)
-                 : launch_pair<RODIMUS_INGATE_POW_SIGMOID, true>(mq, mk, mx, my, mv, mo, a, max_pairs, st);
+                 ? launch_pair<RODIMUS_INGATE_POW_G, true>(m, a, max_pairs, st)
+                 : launch_pair<RODIMUS_INGATE_POW_SIGMOID, true>(m, a, max_pairs, st);
     return p.ingate == RODIMUS_INGATE_POW_G
-               ? launch_pair<RODIMUS_INGATE_POW_G, false>(mq, mk, mx, my, mv, mo, a, max_pairs, st)
-               : launch_pair<RODIMUS_INGATE_POW_SIGMOID, false>(mq, mk, mx, my, mv, mo, a, max_pairs, st);
+               ? launch_pair<RODIMUS_INGATE_POW_G, false>(m, a, max_pairs, st)
+               : launch_pair<RODIMUS_INGATE_POW_SIGMOID, false>(m, a, max_pairs, st);
   };
   char* ws = reinterpret_cast<char*>(p.workspace);
   PairArgs a;
