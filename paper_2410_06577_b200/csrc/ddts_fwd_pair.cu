@@ -111,7 +111,9 @@ enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                    
        BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN,
        BAR_OTFULL0, BAR_OTFULL1,      // output tile written by the whole score group        (128)
        BAR_OTFREE0, BAR_OTFREE1,      // output tile's copies to global have read it            (1)
-       BAR_ROWS };                    // every gate warp has rewritten its rows of the pass (8)
+       BAR_GO0, BAR_GO1,              // an order for the gate warps is in its slot              (1)
+       BAR_PRE,                       // the row groups' prefixes are in place                   (1)
+       BAR_ROWS };                    // every gate warp has rewritten its rows of the pass
 static_assert(BAR_ROWS < kNumBars, "barrier count");
 
 struct PairArgs {
@@ -187,6 +189,7 @@ struct Control {            // lives in shared memory
   int tag[kStages][2];      // per stage: (item index, token position) of the fill it holds
   int pad[2];
   PassDesc pd[4];
+  struct { int stage, nr; } ord[2];   // orders of the control warp to the gate warps (stage < 0: leave)
 };
 static_assert(sizeof(Control) <= 256, "control block");
 
@@ -322,7 +325,10 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       mbar_init(bar(BAR_OTFULL0 + i), 128);
       mbar_init(bar(BAR_OTFREE0 + i), 1);
     }
-    mbar_init(bar(BAR_GSCAN), kGateWarps + 1);
+    mbar_init(bar(BAR_GSCAN), kGateWarps);
+    mbar_init(bar(BAR_GO0), 1);
+    mbar_init(bar(BAR_GO1), 1);
+    mbar_init(bar(BAR_PRE), 1);
     mbar_init(bar(BAR_ROWS), kGateWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -790,107 +796,119 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     bulk_wait<0>();   // this thread's output copies are complete before the CTA may exit
   } else if (warp >= kGateWarp0) {
     // ============================== gate group and its control warp ==============================
-    // The gate warps do the per-element work; the control warp does everything that is
-    // serial (chunk totals, decays, verdict, the block for the partner, publishing the pass), so
-    // that none of it sits between the two phases of a gate warp.
+    // The gate warps are workers: for every order of the control warp (a stage and a row count)
+    // they run phase 1 on their rows, hand in the column sums, wait for their prefix, run phase
+    // 2 and report.  Everything serial or rare lives in the control warp: which fill is an
+    // attempt, the scan over the 16 row groups, decays, verdict exchange, the copies to the
+    // partner, refusals and redirects, publishing the pass.
     const int gw = warp - kGateWarp0;                     // rows kGR*gw .. kGR*gw+kGR-1 of the tile
     const bool is_ctl = gw == kGateWarps;
-    const bool leader = is_ctl && lane == 0;
-    uint32_t off[kGR]; // swizzled byte offsets of the thread's element pairs inside a slab
-#pragma unroll
-    for (int i = 0; i < kGR; ++i) {
-      const int r = gw * kGR + i;
-      off[i] = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
-    }
-    uint32_t fs = 0, fph = 0;                             // stage and phase of the next fill
-    uint32_t g = 0, m = 0, sc = 0;                        // passes, attempts, scan syncs
     bool ok = true;
-    bool armed = false;                                   // attempt m's receive barriers expect bytes
-    auto group_sync = [&]() -> bool {                     // bounded barrier over gate warps + control
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_GSCAN));
-      const bool r = mbar_wait(bar(BAR_GSCAN), sc & 1, abort_flag, a.hdr);
-      ++sc;
-      return r;
-    };
-    auto redirect = [&](int jj, int tt) {                 // one thread; before the stage is released
-      ctl->redir_j = jj;
-      ctl->redir_tpos = tt;
-      __threadfence_block();
-      ctl->redir_seq = ctl->redir_seq + 1;
-    };
-    for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
-      const Item it = decode_item(a, item_of(j), rank);
-      int tpos = 0, lcap = kC;
-      while (ok && tpos < it.len) {
-        const uint32_t s = fs;
-        const uint32_t st = stage_base + s * kStageBytes;
-        if (!(ok = mbar_wait(bar(BAR_FULL0 + s), fph, abort_flag, a.hdr))) break;
-        if (++fs == kStages) { fs = 0; fph ^= 1; }
-        if (ctl->tag[s][0] != j || ctl->tag[s][1] != tpos) {
-          // speculative fill for a position we are not at: hand the stage back unused
-          if (!(ok = group_sync())) break;
-          if (leader) mbar_arrive_cnt(bar(BAR_EMPTY0 + s), 2);   // nothing was sent from it
-          continue;
+    if (!is_ctl) {
+      uint32_t off[kGR]; // swizzled byte offsets of the thread's element pairs inside a slab
+#pragma unroll
+      for (int i = 0; i < kGR; ++i) {
+        const int r = gw * kGR + i;
+        off[i] = r * 128 + ((((uint32_t)lane >> 2) ^ (r & 7)) << 4) + ((lane & 3) << 2);
+      }
+      for (uint32_t oc = 0;; ++oc) {                      // order counter
+        if (!mbar_wait(bar(BAR_GO0 + (oc & 1)), (oc >> 1) & 1, abort_flag, a.hdr)) break;
+        const int s = ctl->ord[oc & 1].stage;
+        const int nr = ctl->ord[oc & 1].nr;
+        if (s < 0) break;                                 // no more work
+        const uint32_t st = stage_base + (uint32_t)s * kStageBytes;
+        float* tot = sTot + (oc & 1) * (kGateWarps * kCH) + gw * kCH + 2 * lane;
+        float2 b[kGR], eh[kGR];
+        const float2 run = gate_phase1<INGATE>(st + kStX, st + kStY, off, gw * kGR, nr, b, eh);
+        *reinterpret_cast<float2*>(tot) = run;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_GSCAN));
+        // the control warp replaces each row group's sum by the sum of the groups before it
+        if (!mbar_wait(bar(BAR_PRE), oc & 1, abort_flag, a.hdr)) break;
+        const float2 pre = *reinterpret_cast<const float2*>(tot);
+        gate_phase2<STATE_ONLY>(st + kStQ, st + kStK, off, gw * kGR, nr, pre, b, eh);
+        // the rewritten rows are visible to the bulk-copy engine and to the tensor core; the
+        // control warp sends the whole slabs to the partner once every gate warp has said so
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_ROWS));
+      }
+    } else {
+      const bool leader = lane == 0;
+      uint32_t fs = 0, fph = 0;                           // stage and phase of the next fill
+      uint32_t g = 0, m = 0;                              // passes, attempts (= orders)
+      bool armed = false;                                 // attempt m's receive barriers expect bytes
+      auto redirect = [&](int jj, int tt) {               // one thread; before the stage is released
+        ctl->redir_j = jj;
+        ctl->redir_tpos = tt;
+        __threadfence_block();
+        ctl->redir_seq = ctl->redir_seq + 1;
+      };
+      auto give_order = [&](int stage, int nr) {          // slot m & 1: the workers read order m-2
+        if (leader) {                                     // before they reported on order m-1
+          ctl->ord[m & 1].stage = stage;
+          ctl->ord[m & 1].nr = nr;
+          mbar_arrive(bar(BAR_GO0 + (m & 1)));
         }
-        // ---- attempt m
-        const uint32_t rxi = m & 1, rxph = (m >> 1) & 1;
-        const int left = it.len - tpos;
-        const int nr = min(min(kC, left), lcap);
-        float* tot = sTot + (m & 1) * (kGateWarps * kCH);
-        float2 Down = splat(1.f);                         // control warp: own chunk decays
-        if (!is_ctl) {
-          float2 b[kGR], eh[kGR];
-          const float2 run = gate_phase1<INGATE>(st + kStX, st + kStY, off, gw * kGR, nr, b, eh);
-          *reinterpret_cast<float2*>(tot + gw * kCH + 2 * lane) = run;
-          if (!(ok = group_sync())) break;
-          // exclusive prefix over the row groups below this warp's
-          float2 pre = splat(0.f);
-#pragma unroll
-          for (int w = 0; w < kGateWarps - 1; ++w) {        // all loads in flight at once
-            const float2 t = *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane);
-            if (w < gw) pre = __fadd2_rn(pre, t);
+      };
+      for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
+        const Item it = decode_item(a, item_of(j), rank);
+        int tpos = 0, lcap = kC;
+        while (ok && tpos < it.len) {
+          const uint32_t s = fs;
+          const uint32_t st = stage_base + s * kStageBytes;
+          if (!(ok = mbar_wait(bar(BAR_FULL0 + s), fph, abort_flag, a.hdr))) break;
+          if (++fs == kStages) { fs = 0; fph ^= 1; }
+          if (ctl->tag[s][0] != j || ctl->tag[s][1] != tpos) {
+            // speculative fill for a position we are not at: hand the stage back unused
+            if (leader) mbar_arrive_cnt(bar(BAR_EMPTY0 + s), 2);   // nothing was sent from it
+            continue;
           }
-          gate_phase2<STATE_ONLY>(st + kStQ, st + kStK, off, gw * kGR, nr, pre, b, eh);
-          // the rewritten rows are visible to the bulk-copy engine and to the tensor core; the
-          // control warp sends the whole slabs to the partner once every gate warp has said so
-          fence_proxy_async();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar(BAR_ROWS));
-        } else {
-          if (!(ok = group_sync())) break;
-          // chunk totals of the own 64 channels: decays for both state groups, and the verdict
+          // ---- attempt m
+          const uint32_t rxi = m & 1, rxph = (m >> 1) & 1;
+          const int left = it.len - tpos;
+          const int nr = min(min(kC, left), lcap);
+          give_order((int)s, nr);
+          float* tot = sTot + (m & 1) * (kGateWarps * kCH) + 2 * lane;
+          if (!(ok = mbar_wait(bar(BAR_GSCAN), m & 1, abort_flag, a.hdr))) break;
+          // scan over the row groups (this lane: two channels): each group's sum becomes the sum
+          // of the groups before it; the total gives the chunk decays and the verdict
           float2 all = splat(0.f);
+          {
+            float2 t[kGateWarps];
 #pragma unroll
-          for (int w = 0; w < kGateWarps; ++w)
-            all = __fadd2_rn(all, *reinterpret_cast<const float2*>(tot + w * kCH + 2 * lane));
+            for (int w = 0; w < kGateWarps; ++w) t[w] = *reinterpret_cast<const float2*>(tot + w * kCH);
+#pragma unroll
+            for (int w = 0; w < kGateWarps; ++w) {
+              *reinterpret_cast<float2*>(tot + w * kCH) = all;
+              all = __fadd2_rn(all, t[w]);
+            }
+          }
+          __syncwarp();
+          if (leader) mbar_arrive(bar(BAR_PRE));
           const bool viol_own = __any_sync(0xffffffffu, all.x < -kRange || all.y < -kRange) && nr > 1;
           const float2 D = make_float2(ex2f(all.x), ex2f(all.y));
-          Down = D;
           // the send block m&1 (like the partner's receive buffer m&1) must be free again
           if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
           volatile float* blk = sTx + rxi * kBlkFloats;
           blk[2 * lane] = D.x;
           blk[2 * lane + 1] = D.y;
-          if (lane == 0) {
+          if (leader) {
             blk[64] = __int_as_float(viol_own ? 1 : 0);
             blk[65] = __int_as_float((int)s);
           }
           fence_proxy_async();
           __syncwarp();
-          if (lane == 0) {
-            // own verdict is in place (the arrive publishes it to the gate warps); the partner's
-            // block and slabs complete the two barriers by byte count
+          if (leader) {
+            // the partner's block and slabs complete the two barriers by byte count
             mbar_expect_tx(bar(BAR_VERD0 + rxi), kBlkBytes);
             mbar_expect_tx(bar(BAR_PEER0 + rxi), STATE_ONLY ? kRxBytes - kSlabBytes : kRxBytes);
             armed = true;
             dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
                             base + kOffTx + rxi * kBlkBytes, kBlkBytes,
                             map_to_cta(bar(BAR_VERD0 + rxi), peer));
-          }
-          // the descriptor of the pass this attempt becomes if both CTAs accept it (slot g & 3 is
-          // not read before its barrier completes; a refused attempt's entry is overwritten)
-          if (lane == 0) {
+            // the descriptor of the pass this attempt becomes if both CTAs accept it (slot g & 3
+            // is not read before its barrier completes; a refused attempt's entry is overwritten)
             volatile PassDesc* pd = &ctl->pd[g & 3];
             pd->stage = (int)s;
             pd->nr = nr;
@@ -903,64 +921,63 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // attempt turns out to be abandoned: the byte count the partner's barrier expects is
           // fixed); the partner's receive buffer m&1 is free, see above
           if (!(ok = mbar_wait(bar(BAR_ROWS), m & 1, abort_flag, a.hdr))) break;
-          if (lane == 0) {
+          if (leader) {
             const uint32_t dst = peer_rx_base + rxi * kRxBytes;
             const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
             if (!STATE_ONLY) dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ, kSlabBytes, pb);
             dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK, kSlabBytes, pb);
           }
-        }
-        // both verdicts: the own one and the partner's (came with its decay block)
-        if (!(ok = mbar_wait_cluster(bar(BAR_VERD0 + rxi), rxph, abort_flag, a.hdr))) break;
-        const bool viol = (__float_as_int(sTx[rxi * kBlkFloats + 64]) |
-                           __float_as_int(sRx[rxi * kBlkFloats + 64])) != 0;
-        ++m;
-        armed = false;
-        if (viol) {
-          // decays too fast for 'nr' rows at once: ask for this position again, fewer rows
-          lcap = max(1, nr >> 1);
-          if (!(ok = group_sync())) break;
-          if (leader) {
-            // whatever the partner sent for this attempt must have landed before its buffer and
-            // its stage are declared reusable
-            if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
-            const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]);
-            mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
-            mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + rxi), peer));
-            redirect(j, tpos);
-            mbar_arrive(bar(BAR_EMPTY0 + s));
+          // both verdicts: the own one and the partner's (came with its decay block)
+          if (!(ok = mbar_wait_cluster(bar(BAR_VERD0 + rxi), rxph, abort_flag, a.hdr))) break;
+          const bool viol = viol_own || __float_as_int(sRx[rxi * kBlkFloats + 64]) != 0;
+          ++m;
+          armed = false;
+          if (viol) {
+            // decays too fast for 'nr' rows at once: ask for this position again, fewer rows
+            lcap = max(1, nr >> 1);
+            if (leader) {
+              // whatever the partner sent for this attempt must have landed before its buffer
+              // and its stage are declared reusable
+              if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
+              const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]);
+              mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
+              mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + rxi), peer));
+              redirect(j, tpos);
+              mbar_arrive(bar(BAR_EMPTY0 + s));
+            }
+            continue;
           }
-          continue;
+          // Publish the pass (its descriptor is already written; every gate warp's rows were seen
+          // through BAR_ROWS).  With it go the chunk decays of all 128 channels (own half from
+          // registers, the partner's from its block) for the state group, in a slot of their
+          // own: the stage and the block are recycled sooner.
+          {
+            float* dp = sDp + (g & 3) * kDK;
+            *reinterpret_cast<float2*>(dp + rank * kCH + 2 * lane) = D;
+            *reinterpret_cast<float2*>(dp + peer * kCH + 2 * lane) =
+                make_float2(sRx[rxi * kBlkFloats + 2 * lane], sRx[rxi * kBlkFloats + 2 * lane + 1]);
+            __syncwarp();
+          }
+          if (leader) {
+            if (nr < min(kC, left)) redirect(j, tpos + nr);   // the prefetcher assumed 64 rows
+            mbar_arrive(bar(BAR_GATED0 + (g & 3)));
+          }
+          ++g;
+          tpos += nr;
+          if (lcap < kC) lcap = min(kC, lcap * 2);
         }
-        // the control warp alone publishes the pass (its descriptor is already written): it has
-        // seen every gate warp's rows through BAR_ROWS.  With the pass go the chunk decays of all
-        // 128 channels (own half from registers, the partner's from its block) for the state
-        // group, in a slot of their own: the stage and the block are recycled sooner.
-        if (is_ctl) {
-          float* dp = sDp + (g & 3) * kDK;
-          *reinterpret_cast<float2*>(dp + rank * kCH + 2 * lane) = Down;
-          *reinterpret_cast<float2*>(dp + peer * kCH + 2 * lane) =
-              make_float2(sRx[rxi * kBlkFloats + 2 * lane], sRx[rxi * kBlkFloats + 2 * lane + 1]);
-          __syncwarp();
-        }
-        if (leader) {
-          if (nr < min(kC, left)) redirect(j, tpos + nr);   // the prefetcher assumed 64 rows
-          mbar_arrive(bar(BAR_GATED0 + (g & 3)));
-        }
-        ++g;
-        tpos += nr;
-        if (lcap < kC) lcap = min(kC, lcap * 2);
       }
-    }
-    if (leader) {
-      ctl->done = 1;
-      // nothing the partner sent may still be in flight towards this CTA when it exits
-      const long long t1 = clock64();
-      for (uint32_t back = armed ? 0 : 1; back <= 2 && back <= m; ++back) {
-        const uint32_t mm = m - back;
-        while (!(mbar_try_cluster(bar(BAR_PEER0 + (mm & 1)), (mm >> 1) & 1) &&
-                 mbar_try_cluster(bar(BAR_VERD0 + (mm & 1)), (mm >> 1) & 1)) &&
-               clock64() - t1 < kWaitCycles) {}
+      give_order(-1, 0);                                  // the workers leave (also after a failed wait)
+      if (leader) {
+        ctl->done = 1;
+        // nothing the partner sent may still be in flight towards this CTA when it exits
+        const long long t1 = clock64();
+        for (uint32_t back = armed ? 0 : 1; back <= 2 && back <= m; ++back) {
+          const uint32_t mm = m - back;
+          while (!(mbar_try_cluster(bar(BAR_PEER0 + (mm & 1)), (mm >> 1) & 1) &&
+                   mbar_try_cluster(bar(BAR_VERD0 + (mm & 1)), (mm >> 1) & 1)) &&
+                 clock64() - t1 < kWaitCycles) {}
+        }
       }
     }
   }
