@@ -836,7 +836,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     } else {
       const bool leader = lane == 0;
       uint32_t fs = 0, fph = 0;                           // stage and phase of the next fill
-      uint32_t g = 0, m = 0;                              // passes, attempts (= orders)
+      uint32_t g = 0, m = 0, oc = 0;                      // passes, exchanged attempts, orders given
       bool armed = false;                                 // attempt m's receive barriers expect bytes
       auto redirect = [&](int jj, int tt) {               // one thread; before the stage is released
         ctl->redir_j = jj;
@@ -844,19 +844,47 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         __threadfence_block();
         ctl->redir_seq = ctl->redir_seq + 1;
       };
-      auto give_order = [&](int stage, int nr) {          // slot m & 1: the workers read order m-2
-        if (leader) {                                     // before they reported on order m-1
-          ctl->ord[m & 1].stage = stage;
-          ctl->ord[m & 1].nr = nr;
-          mbar_arrive(bar(BAR_GO0 + (m & 1)));
+      // Order number oc goes into slot oc & 1.  The workers read order oc-2 before they reported
+      // on it, and at most two orders are outstanding.
+      auto give_order = [&](int stage, int nr) {
+        if (leader) {
+          ctl->ord[oc & 1].stage = stage;
+          ctl->ord[oc & 1].nr = nr;
+          mbar_arrive(bar(BAR_GO0 + (oc & 1)));
         }
+        ++oc;
       };
-      for (int j = 0; ok && item_of(j) < a.n_items; ++j) {
-        const Item it = decode_item(a, item_of(j), rank);
-        int tpos = 0, lcap = kC;
-        while (ok && tpos < it.len) {
-          const uint32_t s = fs;
-          const uint32_t st = stage_base + s * kStageBytes;
+      // position of the attempt at hand: CTA-local item index, the item, token, row cap
+      int j = 0, tpos = 0, lcap = kC;
+      Item it;
+      auto seek = [&](int& jj, Item& ii, int& tt) {       // first position at or after (jj, tt) with tokens
+        while (item_of(jj) < a.n_items) {
+          ii = decode_item(a, item_of(jj), rank);
+          if (tt < ii.len) return true;
+          ++jj;
+          tt = 0;
+        }
+        return false;
+      };
+      bool have = seek(j, it, tpos);
+      // An order given ahead of time: while the workers are in phase 2 of an attempt, the next
+      // fill - if it has landed and is the tile that follows when the attempt is accepted - is
+      // ordered at once, so that the workers never wait for the control warp's serial tail
+      // (copies to the partner, verdict, publishing).  If the attempt is then refused, the
+      // order ahead is carried through (the workers are on it) and its stage handed back unused.
+      bool ahead = false;
+      uint32_t ahead_s = 0;
+      int ahead_nr = 0;
+      while (ok && have) {
+        uint32_t s;
+        int nr;
+        const int left = it.len - tpos;
+        if (ahead) {
+          s = ahead_s;
+          nr = ahead_nr;
+          ahead = false;
+        } else {
+          s = fs;
           if (!(ok = mbar_wait(bar(BAR_FULL0 + s), fph, abort_flag, a.hdr))) break;
           if (++fs == kStages) { fs = 0; fph ^= 1; }
           if (ctl->tag[s][0] != j || ctl->tag[s][1] != tpos) {
@@ -864,108 +892,132 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (leader) mbar_arrive_cnt(bar(BAR_EMPTY0 + s), 2);   // nothing was sent from it
             continue;
           }
-          // ---- attempt m
-          const uint32_t rxi = m & 1, rxph = (m >> 1) & 1;
-          const int left = it.len - tpos;
-          const int nr = min(min(kC, left), lcap);
+          nr = min(min(kC, left), lcap);
           give_order((int)s, nr);
-          float* tot = sTot + (m & 1) * (kGateWarps * kCH) + 2 * lane;
-          if (!(ok = mbar_wait(bar(BAR_GSCAN), m & 1, abort_flag, a.hdr))) break;
-          // scan over the row groups (this lane: two channels): each group's sum becomes the sum
-          // of the groups before it; the total gives the chunk decays and the verdict
-          float2 all = splat(0.f);
-          {
-            float2 t[kGateWarps];
-#pragma unroll
-            for (int w = 0; w < kGateWarps; ++w) t[w] = *reinterpret_cast<const float2*>(tot + w * kCH);
-#pragma unroll
-            for (int w = 0; w < kGateWarps; ++w) {
-              *reinterpret_cast<float2*>(tot + w * kCH) = all;
-              all = __fadd2_rn(all, t[w]);
-            }
-          }
-          __syncwarp();
-          if (leader) mbar_arrive(bar(BAR_PRE));
-          const bool viol_own = __any_sync(0xffffffffu, all.x < -kRange || all.y < -kRange) && nr > 1;
-          const float2 D = make_float2(ex2f(all.x), ex2f(all.y));
-          // the send block m&1 (like the partner's receive buffer m&1) must be free again
-          if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
-          volatile float* blk = sTx + rxi * kBlkFloats;
-          blk[2 * lane] = D.x;
-          blk[2 * lane + 1] = D.y;
-          if (leader) {
-            blk[64] = __int_as_float(viol_own ? 1 : 0);
-            blk[65] = __int_as_float((int)s);
-          }
-          fence_proxy_async();
-          __syncwarp();
-          if (leader) {
-            // the partner's block and slabs complete the two barriers by byte count
-            mbar_expect_tx(bar(BAR_VERD0 + rxi), kBlkBytes);
-            mbar_expect_tx(bar(BAR_PEER0 + rxi), STATE_ONLY ? kRxBytes - kSlabBytes : kRxBytes);
-            armed = true;
-            dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
-                            base + kOffTx + rxi * kBlkBytes, kBlkBytes,
-                            map_to_cta(bar(BAR_VERD0 + rxi), peer));
-            // the descriptor of the pass this attempt becomes if both CTAs accept it (slot g & 3
-            // is not read before its barrier completes; a refused attempt's entry is overwritten)
-            volatile PassDesc* pd = &ctl->pd[g & 3];
-            pd->stage = (int)s;
-            pd->nr = nr;
-            pd->flags = (nr == left ? kPassLast : 0);
-            pd->rx = (int)rxi;
-            pd->rxph = (int)rxph;
-            pd->row = it.row0 + tpos;
-          }
-          // both operand slabs of the attempt go to the partner in one copy each (also when the
-          // attempt turns out to be abandoned: the byte count the partner's barrier expects is
-          // fixed); the partner's receive buffer m&1 is free, see above
-          if (!(ok = mbar_wait(bar(BAR_ROWS), m & 1, abort_flag, a.hdr))) break;
-          if (leader) {
-            const uint32_t dst = peer_rx_base + rxi * kRxBytes;
-            const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
-            if (!STATE_ONLY) dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ, kSlabBytes, pb);
-            dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK, kSlabBytes, pb);
-          }
-          // both verdicts: the own one and the partner's (came with its decay block)
-          if (!(ok = mbar_wait_cluster(bar(BAR_VERD0 + rxi), rxph, abort_flag, a.hdr))) break;
-          const bool viol = viol_own || __float_as_int(sRx[rxi * kBlkFloats + 64]) != 0;
-          ++m;
-          armed = false;
-          if (viol) {
-            // decays too fast for 'nr' rows at once: ask for this position again, fewer rows
-            lcap = max(1, nr >> 1);
-            if (leader) {
-              // whatever the partner sent for this attempt must have landed before its buffer
-              // and its stage are declared reusable
-              if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
-              const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]);
-              mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
-              mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + rxi), peer));
-              redirect(j, tpos);
-              mbar_arrive(bar(BAR_EMPTY0 + s));
-            }
-            continue;
-          }
-          // Publish the pass (its descriptor is already written; every gate warp's rows were seen
-          // through BAR_ROWS).  With it go the chunk decays of all 128 channels (own half from
-          // registers, the partner's from its block) for the state group, in a slot of their
-          // own: the stage and the block are recycled sooner.
-          {
-            float* dp = sDp + (g & 3) * kDK;
-            *reinterpret_cast<float2*>(dp + rank * kCH + 2 * lane) = D;
-            *reinterpret_cast<float2*>(dp + peer * kCH + 2 * lane) =
-                make_float2(sRx[rxi * kBlkFloats + 2 * lane], sRx[rxi * kBlkFloats + 2 * lane + 1]);
-            __syncwarp();
-          }
-          if (leader) {
-            if (nr < min(kC, left)) redirect(j, tpos + nr);   // the prefetcher assumed 64 rows
-            mbar_arrive(bar(BAR_GATED0 + (g & 3)));
-          }
-          ++g;
-          tpos += nr;
-          if (lcap < kC) lcap = min(kC, lcap * 2);
         }
+        const uint32_t st = stage_base + s * kStageBytes;
+        const uint32_t ocur = oc - 1;                     // the order of this attempt
+        // ---- attempt m
+        const uint32_t rxi = m & 1, rxph = (m >> 1) & 1;
+        float* tot = sTot + (ocur & 1) * (kGateWarps * kCH) + 2 * lane;
+        if (!(ok = mbar_wait(bar(BAR_GSCAN), ocur & 1, abort_flag, a.hdr))) break;
+        // scan over the row groups (this lane: two channels): each group's sum becomes the sum
+        // of the groups before it; the total gives the chunk decays and the verdict
+        float2 all = splat(0.f);
+        {
+          float2 t[kGateWarps];
+#pragma unroll
+          for (int w = 0; w < kGateWarps; ++w) t[w] = *reinterpret_cast<const float2*>(tot + w * kCH);
+#pragma unroll
+          for (int w = 0; w < kGateWarps; ++w) {
+            *reinterpret_cast<float2*>(tot + w * kCH) = all;
+            all = __fadd2_rn(all, t[w]);
+          }
+        }
+        __syncwarp();
+        if (leader) mbar_arrive(bar(BAR_PRE));
+        // ---- the position that follows if this attempt is accepted, and the order ahead
+        int nj = j, ntpos = tpos + nr, nlcap = lcap < kC ? min(kC, lcap * 2) : kC;
+        Item nit = it;
+        const bool nhave = ntpos < it.len ? true : seek(nj, nit, ntpos);
+        if (nhave && mbar_try(bar(BAR_FULL0 + fs), fph) && ctl->tag[fs][0] == nj && ctl->tag[fs][1] == ntpos) {
+          ahead = true;
+          ahead_s = fs;
+          ahead_nr = min(min(kC, nit.len - ntpos), nlcap);
+          if (++fs == kStages) { fs = 0; fph ^= 1; }
+          give_order((int)ahead_s, ahead_nr);
+        }
+        const bool viol_own = __any_sync(0xffffffffu, all.x < -kRange || all.y < -kRange) && nr > 1;
+        const float2 D = make_float2(ex2f(all.x), ex2f(all.y));
+        // the send block m&1 (like the partner's receive buffer m&1) must be free again
+        if (!(ok = mbar_wait_cluster(bar(BAR_RXFREE0 + rxi), rxph ^ 1, abort_flag, a.hdr))) break;
+        volatile float* blk = sTx + rxi * kBlkFloats;
+        blk[2 * lane] = D.x;
+        blk[2 * lane + 1] = D.y;
+        if (leader) {
+          blk[64] = __int_as_float(viol_own ? 1 : 0);
+          blk[65] = __int_as_float((int)s);
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (leader) {
+          // the partner's block and slabs complete the two barriers by byte count
+          mbar_expect_tx(bar(BAR_VERD0 + rxi), kBlkBytes);
+          mbar_expect_tx(bar(BAR_PEER0 + rxi), STATE_ONLY ? kRxBytes - kSlabBytes : kRxBytes);
+          armed = true;
+          dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
+                          base + kOffTx + rxi * kBlkBytes, kBlkBytes,
+                          map_to_cta(bar(BAR_VERD0 + rxi), peer));
+          // the descriptor of the pass this attempt becomes if both CTAs accept it (slot g & 3
+          // is not read before its barrier completes; a refused attempt's entry is overwritten)
+          volatile PassDesc* pd = &ctl->pd[g & 3];
+          pd->stage = (int)s;
+          pd->nr = nr;
+          pd->flags = (nr == left ? kPassLast : 0);
+          pd->rx = (int)rxi;
+          pd->rxph = (int)rxph;
+          pd->row = it.row0 + tpos;
+        }
+        // both operand slabs of the attempt go to the partner in one copy each (also when the
+        // attempt turns out to be abandoned: the byte count the partner's barrier expects is
+        // fixed); the partner's receive buffer m&1 is free, see above
+        if (!(ok = mbar_wait(bar(BAR_ROWS), ocur & 1, abort_flag, a.hdr))) break;
+        if (leader) {
+          const uint32_t dst = peer_rx_base + rxi * kRxBytes;
+          const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
+          if (!STATE_ONLY) dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ, kSlabBytes, pb);
+          dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK, kSlabBytes, pb);
+        }
+        // both verdicts: the own one and the partner's (came with its decay block)
+        if (!(ok = mbar_wait_cluster(bar(BAR_VERD0 + rxi), rxph, abort_flag, a.hdr))) break;
+        const bool viol = viol_own || __float_as_int(sRx[rxi * kBlkFloats + 64]) != 0;
+        ++m;
+        armed = false;
+        if (viol) {
+          // decays too fast for 'nr' rows at once: ask for this position again, fewer rows
+          lcap = max(1, nr >> 1);
+          if (ahead) {
+            // carry the order ahead through with the workers, then drop it
+            const uint32_t oa = oc - 1;
+            if (!(ok = mbar_wait(bar(BAR_GSCAN), oa & 1, abort_flag, a.hdr))) break;
+            if (leader) mbar_arrive(bar(BAR_PRE));
+            if (!(ok = mbar_wait(bar(BAR_ROWS), oa & 1, abort_flag, a.hdr))) break;
+            if (leader) mbar_arrive_cnt(bar(BAR_EMPTY0 + ahead_s), 2);
+            ahead = false;
+          }
+          if (leader) {
+            // whatever the partner sent for this attempt must have landed before its buffer
+            // and its stage are declared reusable
+            if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
+            const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]);
+            mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
+            mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + rxi), peer));
+            redirect(j, tpos);
+            mbar_arrive(bar(BAR_EMPTY0 + s));
+          }
+          continue;
+        }
+        // Publish the pass (its descriptor is already written; every gate warp's rows were seen
+        // through BAR_ROWS).  With it go the chunk decays of all 128 channels (own half from
+        // registers, the partner's from its block) for the state group, in a slot of their
+        // own: the stage and the block are recycled sooner.
+        {
+          float* dp = sDp + (g & 3) * kDK;
+          *reinterpret_cast<float2*>(dp + rank * kCH + 2 * lane) = D;
+          *reinterpret_cast<float2*>(dp + peer * kCH + 2 * lane) =
+              make_float2(sRx[rxi * kBlkFloats + 2 * lane], sRx[rxi * kBlkFloats + 2 * lane + 1]);
+          __syncwarp();
+        }
+        if (leader) {
+          if (nr < min(kC, left)) redirect(j, tpos + nr);   // the prefetcher assumed 64 rows
+          mbar_arrive(bar(BAR_GATED0 + (g & 3)));
+        }
+        ++g;
+        j = nj;
+        it = nit;
+        tpos = ntpos;
+        lcap = nlcap;
+        have = nhave;
       }
       give_order(-1, 0);                                  // the workers leave (also after a failed wait)
       if (leader) {
