@@ -46,12 +46,12 @@ extern "C" {
 typedef enum {
   RODIMUS_OK = 0,
   RODIMUS_ERR_NULL = 1,        /* a required pointer is NULL                                  */
-  RODIMUS_ERR_SHAPE = 2,       /* a size is negative, zero where it may not be, or too large  */
+  RODIMUS_ERR_SHAPE = 2,       /* a size is negative, zero where it may not be, or overflows  */
   RODIMUS_ERR_DTYPE = 3,       /* dtype / ingate / struct_size not understood                 */
   RODIMUS_ERR_ALIGN = 4,       /* a pointer is not 16-byte aligned                            */
   RODIMUS_ERR_SEQLENS = 5,     /* cu_seqlens does not start at 0, decreases, or ends != T     */
   RODIMUS_ERR_WORKSPACE = 6,   /* workspace missing or smaller than ..._workspace_bytes       */
-  RODIMUS_ERR_UNSUPPORTED = 7, /* valid request that no kernel here covers                    */
+  RODIMUS_ERR_UNSUPPORTED = 7, /* dk or dv not a multiple of 16, dk > 256 or dv > 1024        */
   RODIMUS_ERR_CUDA = 8,        /* a CUDA runtime or driver call failed                        */
   RODIMUS_ERR_TIMEOUT = 9      /* a bounded wait inside a kernel ran out (device status only) */
 } rodimus_status;
@@ -76,8 +76,8 @@ typedef enum {
  * s0 and sT may be the same buffer.  o must not overlap any input.
  *
  * Kernels: dtype BF16 with dk == 128 and dv a multiple of 128 runs on the tcgen05 tensor
- * cores; every other legal shape (dk, dv multiples of 16, at most 256) and dtype F32 run
- * the fp32 CUDA-core kernel, which keeps all arithmetic in fp32.
+ * cores; every other supported shape (dk, dv multiples of 16, dk <= 256, dv <= 1024) and
+ * dtype F32 run the fp32 CUDA-core kernel, which keeps all arithmetic in fp32.
  */
 typedef struct {
   int32_t struct_size;       /* sizeof(rodimus_ddts_fwd_params), checked                        */

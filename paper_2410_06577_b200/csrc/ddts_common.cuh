@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "rodimus_ddts.h"
 
 namespace ddts {
@@ -12,13 +14,25 @@ namespace ddts {
 // Device-visible words at the start of the caller's workspace.
 struct WorkspaceHeader {
   int32_t status;        // rodimus_status recorded by kernels (0 = ok); only ever raised
-  int32_t work_counter;  // next work item for persistent kernels
-  int32_t n_items;       // reserved
-  int32_t pad[61];
+  int32_t pad[63];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "workspace header is 256 bytes");
 
 constexpr int kMaxSortedSeqs = 4096;  // varlen: sequences beyond this keep their given order
+
+// The current device and its SM count (the count is asked for once per device).
+cudaError_t current_device(int* dev, int* sms);
+
+// Opt-in to more than 48 KiB of dynamic shared memory, once per kernel and device: `done` is a
+// per-kernel bit mask over device ordinals (devices beyond 63 simply ask every time).
+template <typename Kernel>
+inline cudaError_t opt_in_shared_memory(Kernel kernel, int bytes, int dev, std::atomic<unsigned long long>& done) {
+  const unsigned long long bit = dev >= 0 && dev < 64 ? 1ull << dev : 0ull;
+  if (bit && (done.load(std::memory_order_acquire) & bit)) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && bit) done.fetch_or(bit, std::memory_order_release);
+  return e;
+}
 
 // Launchers: all arguments validated by the caller; they return a cudaError_t.
 cudaError_t launch_step(const rodimus_ddts_step_params& p, int* n_launches);

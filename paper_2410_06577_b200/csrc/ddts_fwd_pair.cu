@@ -897,6 +897,19 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
         const uint32_t st = stage_base + s * kStageBytes;
         const uint32_t ocur = oc - 1;                     // the order of this attempt
+        // ---- the position that follows if this attempt is accepted, and the order ahead
+        int nj = j, ntpos = tpos + nr, nlcap = lcap < kC ? min(kC, lcap * 2) : kC;
+        Item nit = it;
+        const bool nhave = ntpos < it.len ? true : seek(nj, nit, ntpos);
+        auto try_ahead = [&]() {
+          if (ahead || !nhave || !mbar_try(bar(BAR_FULL0 + fs), fph)) return;
+          if (ctl->tag[fs][0] != nj || ctl->tag[fs][1] != ntpos) return;
+          ahead = true;
+          ahead_s = fs;
+          ahead_nr = min(min(kC, nit.len - ntpos), nlcap);
+          if (++fs == kStages) { fs = 0; fph ^= 1; }
+          give_order((int)ahead_s, ahead_nr);
+        };
         // ---- attempt m
         const uint32_t rxi = m & 1, rxph = (m >> 1) & 1;
         float* tot = sTot + (ocur & 1) * (kGateWarps * kCH) + 2 * lane;
@@ -916,17 +929,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
         __syncwarp();
         if (leader) mbar_arrive(bar(BAR_PRE));
-        // ---- the position that follows if this attempt is accepted, and the order ahead
-        int nj = j, ntpos = tpos + nr, nlcap = lcap < kC ? min(kC, lcap * 2) : kC;
-        Item nit = it;
-        const bool nhave = ntpos < it.len ? true : seek(nj, nit, ntpos);
-        if (nhave && mbar_try(bar(BAR_FULL0 + fs), fph) && ctl->tag[fs][0] == nj && ctl->tag[fs][1] == ntpos) {
-          ahead = true;
-          ahead_s = fs;
-          ahead_nr = min(min(kC, nit.len - ntpos), nlcap);
-          if (++fs == kStages) { fs = 0; fph ^= 1; }
-          give_order((int)ahead_s, ahead_nr);
-        }
+        try_ahead();                                      // if the next fill had not landed before
         const bool viol_own = __any_sync(0xffffffffu, all.x < -kRange || all.y < -kRange) && nr > 1;
         const float2 D = make_float2(ex2f(all.x), ex2f(all.y));
         // the send block m&1 (like the partner's receive buffer m&1) must be free again
@@ -1086,10 +1089,44 @@ struct PairMaps {
   CUtensorMap q, k, x, y, v, o, o8, o1;
 };
 
+// A tensor map depends only on (address, rows, columns, box rows): each host thread keeps the
+// last few it encoded, so that repeated calls on the same buffers (a decode loop's prefill, a
+// benchmark) skip the eight driver calls.
+struct MapKey {
+  const void* ptr;
+  uint64_t rows, cols;
+  uint32_t box_rows;
+};
+constexpr int kMapCacheSize = 32;
+struct MapCache {
+  MapKey key[kMapCacheSize];
+  CUtensorMap map[kMapCacheSize];
+  int used = 0, next = 0;
+};
+thread_local MapCache t_maps;
+
+bool cached_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows = kC) {
+  MapCache& c = t_maps;
+  for (int i = 0; i < c.used; ++i) {
+    const MapKey& k = c.key[i];
+    if (k.ptr == ptr && k.rows == rows && k.cols == cols && k.box_rows == box_rows) {
+      *m = c.map[i];
+      return true;
+    }
+  }
+  if (!make_map(m, ptr, rows, cols, box_rows)) return false;
+  const int slot = c.next;
+  c.key[slot] = MapKey{ptr, rows, cols, box_rows};
+  c.map[slot] = *m;
+  c.next = (slot + 1) % kMapCacheSize;
+  if (c.used < kMapCacheSize) ++c.used;
+  return true;
+}
+
 template <int INGATE, bool STATE_ONLY>
-cudaError_t launch_pair(const PairMaps& m, const PairArgs& a, int max_pairs, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(ddts_fwd_pair_kernel<INGATE, STATE_ONLY>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+cudaError_t launch_pair(const PairMaps& m, const PairArgs& a, int max_pairs, int dev, cudaStream_t st) {
+  static std::atomic<unsigned long long> opted{0};   // one per instantiation
+  cudaError_t e = opt_in_shared_memory(ddts_fwd_pair_kernel<INGATE, STATE_ONLY>, kSmemBytes, dev, opted);
   if (e != cudaSuccess) return e;
   const long long pairs = a.n_items < max_pairs ? a.n_items : max_pairs;
   ddts_fwd_pair_kernel<INGATE, STATE_ONLY><<<(unsigned)(2 * pairs), kThreads, kSmemBytes, st>>>(m.q, m.k, m.x, m.y, m.v, m.o, m.o8, m.o1, a);
@@ -1119,7 +1156,7 @@ namespace {
 // together; the whole trades about (2G - 0.35)/(G + 0.65) of the work for G times the parallelism.
 struct SplitPlan {
   int G = 0;            // segments after the head segment (0: do not split)
-  int L0 = 0;           // rows of the head segment (multiple of the chunk length)
+  int L0 = 0;           // rows of the head segment (any number: T - G * L)
   int L = 0;            // rows of each later segment (multiple of the chunk length)
   size_t off_order = 0, off_cu = 0, off_dtot = 0, off_ds = 0, off_start = 0, bytes = 0;
 };
@@ -1132,8 +1169,7 @@ SplitPlan make_split_plan(const rodimus_ddts_fwd_params& p) {
   SplitPlan sp;
   if (p.cu_seqlens || p.cu_seqlens_host || !fwd_pair_supported(p)) return sp;
   int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+  if (current_device(&dev, &sms) != cudaSuccess) {
     cudaGetLastError();
     return sp;
   }
@@ -1163,7 +1199,7 @@ SplitPlan make_split_plan(const rodimus_ddts_fwd_params& p) {
 __global__ void ddts_segments_kernel(WorkspaceHeader* hdr, int32_t* order, int32_t* cu, int G, int L0,
                                      int L, int T) {
   const int i = threadIdx.x;
-  if (i == 0) { hdr->status = RODIMUS_OK; hdr->work_counter = 0; hdr->n_items = G + 1; }
+  if (i == 0) hdr->status = RODIMUS_OK;
   if (i <= G) order[i] = i;
   if (i <= G + 1) cu[i] = i == 0 ? 0 : min(L0 + (i - 1) * L, T);
 }
@@ -1228,18 +1264,16 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
 
   int dev = 0, sms = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaError_t e = current_device(&dev, &sms);
   if (e != cudaSuccess) return e;
 
   PairMaps m;
   if (rows > 0) {
     const uint64_t dv = (uint64_t)p.dv;
-    if (!make_map(&m.q, p.q, rows, kDK) || !make_map(&m.k, p.k, rows, kDK) ||
-        !make_map(&m.x, p.gate_x, rows, kDK) || !make_map(&m.y, p.temp_y, rows, kDK) ||
-        !make_map(&m.v, p.v, rows, dv) || !make_map(&m.o, p.o, rows, dv) ||
-        !make_map(&m.o8, p.o, rows, dv, 8) || !make_map(&m.o1, p.o, rows, dv, 1))
+    if (!cached_map(&m.q, p.q, rows, kDK) || !cached_map(&m.k, p.k, rows, kDK) ||
+        !cached_map(&m.x, p.gate_x, rows, kDK) || !cached_map(&m.y, p.temp_y, rows, kDK) ||
+        !cached_map(&m.v, p.v, rows, dv) || !cached_map(&m.o, p.o, rows, dv) ||
+        !cached_map(&m.o8, p.o, rows, dv, 8) || !cached_map(&m.o1, p.o, rows, dv, 1))
       return cudaErrorUnknown;
   } else {
     memset(&m, 0, sizeof(m));   // never dereferenced: no chunks
@@ -1248,11 +1282,11 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   auto run = [&](const PairArgs& a, cudaStream_t st) {
     if (a.state_only)
       return p.ingate == RODIMUS_INGATE_POW_G
-                 ? launch_pair<RODIMUS_INGATE_POW_G, true>(m, a, max_pairs, st)
-                 : launch_pair<RODIMUS_INGATE_POW_SIGMOID, true>(m, a, max_pairs, st);
+                 ? launch_pair<RODIMUS_INGATE_POW_G, true>(m, a, max_pairs, dev, st)
+                 : launch_pair<RODIMUS_INGATE_POW_SIGMOID, true>(m, a, max_pairs, dev, st);
     return p.ingate == RODIMUS_INGATE_POW_G
-               ? launch_pair<RODIMUS_INGATE_POW_G, false>(m, a, max_pairs, st)
-               : launch_pair<RODIMUS_INGATE_POW_SIGMOID, false>(m, a, max_pairs, st);
+               ? launch_pair<RODIMUS_INGATE_POW_G, false>(m, a, max_pairs, dev, st)
+               : launch_pair<RODIMUS_INGATE_POW_SIGMOID, false>(m, a, max_pairs, dev, st);
   };
   char* ws = reinterpret_cast<char*>(p.workspace);
   PairArgs a;
@@ -1297,23 +1331,32 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
     }
   }
   a.order = order; a.H = BH;
+  // Whatever happens after the fork, the side stream is joined back into the caller's stream
+  // before this call returns, so that no work of the call is left outside `stream` (and an
+  // enclosing stream capture is not left with an unjoined branch).
+  auto join = [&]() -> cudaError_t {
+    if (!side) return cudaSuccess;
+    cudaError_t je = cudaEventRecord(side->join, st0);
+    if (je == cudaSuccess) je = cudaStreamWaitEvent(st, side->join, 0);
+    side_use.unlock();
+    side = nullptr;
+    return je;
+  };
   // A: local final states and decay products of segments 1..G-1
   a.cu = cu + 1;
   a.n_seq = sp.G - 1;
   a.n_items = (long long)a.n_seq * BH * a.pairs;
   a.s0 = nullptr; a.sT = ds; a.dtot = dtot; a.state_only = 1;
-  if ((e = run(a, st)) != cudaSuccess) return e;
+  if ((e = run(a, st)) != cudaSuccess) { join(); return e; }
   // C0: the head segment from the caller's initial state; its final state starts segment 1
   a.cu = cu;
   a.n_seq = 1;
   a.n_items = (long long)BH * a.pairs;
   a.s0 = p.s0; a.sT = start; a.dtot = nullptr; a.state_only = 0;
-  if ((e = run(a, st0)) != cudaSuccess) return e;
-  if (side) {
-    if ((e = cudaEventRecord(side->join, st0)) != cudaSuccess) return e;
-    if ((e = cudaStreamWaitEvent(st, side->join, 0)) != cudaSuccess) return e;
-    side_use.unlock();
-  }
+  e = run(a, st0);
+  const cudaError_t je = join();
+  if (e != cudaSuccess) return e;
+  if (je != cudaSuccess) return je;
   // combine
   {
     const long long BHD = (long long)BH * kDK;

@@ -675,9 +675,7 @@ cudaError_t launch_fwd_tc(const rodimus_ddts_fwd_params& p, int* n_launches) {
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
 
   int dev = 0, sms = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaError_t e = current_device(&dev, &sms);
   if (e != cudaSuccess) return e;
 
   CUtensorMap mq, mk, mx, my, mv;
@@ -690,14 +688,13 @@ cudaError_t launch_fwd_tc(const rodimus_ddts_fwd_params& p, int* n_launches) {
     memset(&mq, 0, sizeof(mq)); mk = mq; mx = mq; my = mq; mv = mq;  // never dereferenced: no chunks
   }
   const int grid = (int)(a.n_items < sms ? a.n_items : sms);
+  static std::atomic<unsigned long long> opted_g{0}, opted_s{0};
   if (p.ingate == RODIMUS_INGATE_POW_G) {
-    e = cudaFuncSetAttribute(ddts_fwd_tc_kernel<RODIMUS_INGATE_POW_G>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = opt_in_shared_memory(ddts_fwd_tc_kernel<RODIMUS_INGATE_POW_G>, kSmemBytes, dev, opted_g);
     if (e != cudaSuccess) return e;
     ddts_fwd_tc_kernel<RODIMUS_INGATE_POW_G><<<grid, kThreads, kSmemBytes, st>>>(mq, mk, mx, my, mv, a);
   } else {
-    e = cudaFuncSetAttribute(ddts_fwd_tc_kernel<RODIMUS_INGATE_POW_SIGMOID>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = opt_in_shared_memory(ddts_fwd_tc_kernel<RODIMUS_INGATE_POW_SIGMOID>, kSmemBytes, dev, opted_s);
     if (e != cudaSuccess) return e;
     ddts_fwd_tc_kernel<RODIMUS_INGATE_POW_SIGMOID><<<grid, kThreads, kSmemBytes, st>>>(mq, mk, mx, my, mv, a);
   }

@@ -32,8 +32,6 @@ ddts_plan_kernel(const int32_t* __restrict__ cu, int N, int T, WorkspaceHeader* 
   __syncthreads();
   if (tid == 0) {
     hdr->status = s_bad ? (int)RODIMUS_ERR_SEQLENS : (int)RODIMUS_OK;
-    hdr->work_counter = 0;
-    hdr->n_items = N;
   }
   const int ns = N < kMaxSortedSeqs ? N : kMaxSortedSeqs;
   for (int n = tid; n < N; n += kPlanThreads) {

@@ -34,9 +34,7 @@ extern "C" int rodimus_ddts_sfu_probe(int iters, float* sink, void* stream, long
   if (!sink || !ops) return RODIMUS_ERR_NULL;
   if (iters <= 0 || iters > (1 << 24)) return RODIMUS_ERR_SHAPE;
   int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return RODIMUS_ERR_CUDA;
+  if (ddts::current_device(&dev, &sms) != cudaSuccess) return RODIMUS_ERR_CUDA;
   const int ctas = sms * 8;            // 2048 threads per SM: every scheduler has work to hide latency
   ddts_sfu_probe_kernel<<<ctas, kProbeThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(iters, sink);
   if (cudaGetLastError() != cudaSuccess) return RODIMUS_ERR_CUDA;

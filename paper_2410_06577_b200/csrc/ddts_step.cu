@@ -126,9 +126,7 @@ cudaError_t launch_step(const rodimus_ddts_step_params& p, int* n_launches) {
   const int tiles = (p.dv + kTileCols - 1) / kTileCols;
   const long long items = nh * tiles;
   int dev = 0, sms = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaError_t e = current_device(&dev, &sms);
   if (e != cudaSuccess) return e;
   // One CTA per item: measured 6 % faster than a persistent grid of 8 CTAs per SM (the hardware
   // block scheduler balances the tail better than a fixed stride does).  The in-kernel loop only

@@ -294,6 +294,30 @@ __device__ __forceinline__ void umma_bf16_atmem(uint32_t d_tmem, uint32_t a_tmem
       ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(ACC ? 1u : 0u), "r"(kDescHi)
       : "memory");
 }
+// One tcgen05.mma, bf16 x bf16 -> fp32.  Descriptors are passed whole (64 bits): stepping along K
+// is then one 64-bit add of a constant to a base the issuer keeps in registers, and the
+// accumulate flag is an immediate that the assembler folds into the predicate.
+template <bool ACC>
+__device__ __forceinline__ void umma_bf16_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "n"(ACC ? 1 : 0)
+      : "memory");
+}
+// The same with the A operand in tensor memory: lane = row of A (M = 128), bf16 packed two per
+// 32-bit column, even K index in the low half (K = 16 elements = 8 columns per instruction).
+template <bool ACC>
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "n"(ACC ? 1 : 0)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; }
 // Instruction descriptor: bf16 x bf16 -> fp32.
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn, int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |

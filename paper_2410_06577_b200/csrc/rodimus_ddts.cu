@@ -1,5 +1,4 @@
 // Host side of the C ABI: argument checks (before any launch), workspace sizing, kernel choice.
-#include <cstdlib>
 #include <cstring>
 
 #include "ddts_common.cuh"
@@ -23,8 +22,9 @@ int check_fwd_sizes(const rodimus_ddts_fwd_params* p, bool varlen) {
   if (p->ingate != RODIMUS_INGATE_POW_G && p->ingate != RODIMUS_INGATE_POW_SIGMOID)
     return RODIMUS_ERR_DTYPE;
   if (p->B < 0 || p->H < 0 || p->T < 0) return RODIMUS_ERR_SHAPE;
-  if (p->dk <= 0 || p->dv <= 0 || p->dk % 16 || p->dv % 16) return RODIMUS_ERR_SHAPE;
-  if (p->dk > 256 || p->dv > 1024) return RODIMUS_ERR_SHAPE;
+  if (p->dk <= 0 || p->dv <= 0) return RODIMUS_ERR_SHAPE;
+  // well-formed widths that none of the kernels covers
+  if (p->dk % 16 || p->dv % 16 || p->dk > 256 || p->dv > 1024) return RODIMUS_ERR_UNSUPPORTED;
   if ((long long)p->B * p->H * p->T >= (1LL << 31)) return RODIMUS_ERR_SHAPE;
   if (varlen) {
     if (p->B != 1 || p->N < 0) return RODIMUS_ERR_SHAPE;
@@ -37,26 +37,26 @@ int check_fwd_sizes(const rodimus_ddts_fwd_params* p, bool varlen) {
 
 namespace ddts {
 
-namespace {
-// RODIMUS_DDTS_KERNEL = "simt" | "single" narrows the choice of prefill kernel (for comparing
-// them); anything else, or unset, picks the fastest kernel that covers the shape.
-int kernel_override() {
-  const char* v = std::getenv("RODIMUS_DDTS_KERNEL");
-  if (!v) return 0;
-  if (!std::strcmp(v, "simt")) return 1;
-  if (!std::strcmp(v, "single")) return 2;
-  return 0;
+cudaError_t current_device(int* dev, int* sms) {
+  static std::atomic<int> cached[64];   // SM count per device ordinal, 0 = not asked yet
+  cudaError_t e = cudaGetDevice(dev);
+  if (e != cudaSuccess) return e;
+  const bool slot = *dev >= 0 && *dev < 64;
+  int n = slot ? cached[*dev].load(std::memory_order_relaxed) : 0;
+  if (n == 0) {
+    e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, *dev);
+    if (e != cudaSuccess) return e;
+    if (slot) cached[*dev].store(n, std::memory_order_relaxed);
+  }
+  *sms = n;
+  return cudaSuccess;
 }
-}  // namespace
 
 bool fwd_tc_supported(const rodimus_ddts_fwd_params& p) {
-  if (kernel_override() == 1) return false;
   return p.dtype == RODIMUS_BF16 && p.dk == 128 && p.dv % 128 == 0;
 }
 
-bool fwd_pair_selected(const rodimus_ddts_fwd_params& p) {
-  return kernel_override() == 0 && fwd_pair_supported(p);
-}
+bool fwd_pair_selected(const rodimus_ddts_fwd_params& p) { return fwd_pair_supported(p); }
 
 }  // namespace ddts
 
@@ -132,8 +132,8 @@ int rodimus_ddts_step(const rodimus_ddts_step_params* p) {
   if (p->ingate != RODIMUS_INGATE_POW_G && p->ingate != RODIMUS_INGATE_POW_SIGMOID)
     return RODIMUS_ERR_DTYPE;
   if (p->Nseq < 0 || p->H < 0) return RODIMUS_ERR_SHAPE;
-  if (p->dk <= 0 || p->dv <= 0 || p->dk % 16 || p->dv % 16) return RODIMUS_ERR_SHAPE;
-  if (p->dk > 256 || p->dv > 1024) return RODIMUS_ERR_SHAPE;
+  if (p->dk <= 0 || p->dv <= 0) return RODIMUS_ERR_SHAPE;
+  if (p->dk % 16 || p->dv % 16 || p->dk > 256 || p->dv > 1024) return RODIMUS_ERR_UNSUPPORTED;
   if ((long long)p->Nseq * p->H >= (1LL << 31) / 8) return RODIMUS_ERR_SHAPE;
   if ((long long)p->Nseq * p->H == 0) return RODIMUS_OK;
   if (!p->q || !p->k || !p->gate_x || !p->temp_y || !p->v || !p->o || !p->state)

@@ -86,8 +86,8 @@ def test_fwd_argument_errors(lib):
     assert rd.fwd_raw(_fwd(dtype=7)) == rd.ERR_DTYPE
     assert rd.fwd_raw(_fwd(ingate=2)) == rd.ERR_DTYPE
     assert rd.fwd_raw(_fwd(T=-1)) == rd.ERR_SHAPE
-    assert rd.fwd_raw(_fwd(dk=120)) == rd.ERR_SHAPE
-    assert rd.fwd_raw(_fwd(dk=512)) == rd.ERR_SHAPE
+    assert rd.fwd_raw(_fwd(dk=120)) == rd.ERR_UNSUPPORTED
+    assert rd.fwd_raw(_fwd(dk=512)) == rd.ERR_UNSUPPORTED
     assert rd.fwd_raw(_fwd(dv=0)) == rd.ERR_SHAPE
     assert rd.fwd_raw(_fwd(B=1 << 15, H=1 << 10, T=1 << 10)) == rd.ERR_SHAPE
     assert rd.fwd_raw(_fwd(q=0)) == rd.ERR_NULL
@@ -148,8 +148,8 @@ def test_step_argument_errors(lib):
     assert rd.step_raw(_step(dtype=-1)) == rd.ERR_DTYPE
     assert rd.step_raw(_step(ingate=9)) == rd.ERR_DTYPE
     assert rd.step_raw(_step(Nseq=-3)) == rd.ERR_SHAPE
-    assert rd.step_raw(_step(dk=100)) == rd.ERR_SHAPE
-    assert rd.step_raw(_step(dv=2048)) == rd.ERR_SHAPE
+    assert rd.step_raw(_step(dk=100)) == rd.ERR_UNSUPPORTED
+    assert rd.step_raw(_step(dv=2048)) == rd.ERR_UNSUPPORTED
     assert rd.step_raw(_step(state=0)) == rd.ERR_NULL
     assert rd.step_raw(_step(v=FAKE + 4)) == rd.ERR_ALIGN
     assert rd.step_raw(_step(Nseq=0)) == rd.OK and rd.last_launch_count() == 0
