@@ -198,6 +198,15 @@ const char *rodimus_ddts_fwd_kernel_name(const rodimus_ddts_fwd_params *p);
  * `sink` is one device float (written only in a case that does not occur).  iters in 1 .. 2^24. */
 int rodimus_ddts_sfu_probe(int iters, float *sink, void *stream, long long *ops);
 
+/* Test hook (the paper has no counterpart).  Every wait inside the tensor-core prefill kernels is
+ * bounded: when one runs out, the kernel stops early, frees what it holds and records
+ * RODIMUS_ERR_TIMEOUT in the workspace status word (outputs are then unspecified, the device
+ * stays usable).  The bound is a launch argument of about two seconds' worth of clock cycles;
+ * this call replaces it, process-wide, for the launches that follow: 0 makes the first wait that
+ * is not satisfied at once run out, which is how the tests reach that path without hanging
+ * anything; a negative value restores the default.  Not for production use. */
+int rodimus_ddts_test_set_wait_limit(long long cycles);
+
 const char *rodimus_status_str(int status);
 int rodimus_version(void);
 

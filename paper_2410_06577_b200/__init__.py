@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = (
     "rodimus_ddts_fwd_workspace_bytes", "rodimus_ddts_fwd", "rodimus_ddts_step",
     "rodimus_ddts_device_status", "rodimus_ddts_last_launch_count",
     "rodimus_ddts_fwd_kernel_name", "rodimus_status_str", "rodimus_version",
-    "rodimus_ddts_fwd_noalloc", "rodimus_ddts_sfu_probe",
+    "rodimus_ddts_fwd_noalloc", "rodimus_ddts_sfu_probe", "rodimus_ddts_test_set_wait_limit",
 )
 NOALLOC_MAX_SEQS = 4096
 
@@ -91,6 +91,8 @@ def load_library() -> ctypes.CDLL:
         lib.rodimus_ddts_sfu_probe.argtypes = [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
                                                ctypes.POINTER(ctypes.c_longlong)]
         lib.rodimus_ddts_sfu_probe.restype = ctypes.c_int
+        lib.rodimus_ddts_test_set_wait_limit.argtypes = [ctypes.c_longlong]
+        lib.rodimus_ddts_test_set_wait_limit.restype = ctypes.c_int
         lib.rodimus_status_str.argtypes = [ctypes.c_int]
         lib.rodimus_status_str.restype = ctypes.c_char_p
         lib.rodimus_version.restype = ctypes.c_int
@@ -191,6 +193,16 @@ def sfu_probe(iters: int, sink, stream: Optional[int] = None) -> int:
     if rc != OK:
         raise RodimusError(rc, "rodimus_ddts_sfu_probe")
     return int(ops.value)
+
+
+def test_set_wait_limit(cycles: int) -> None:
+    """Test hook (``rodimus_ddts_test_set_wait_limit``): bound of the kernels' main-loop waits in
+    clock cycles for the launches that follow; 0 = the first unsatisfied wait times out, negative =
+    back to the default."""
+    load_library().rodimus_ddts_test_set_wait_limit(int(cycles))
+
+
+test_set_wait_limit.__test__ = False   # not a pytest test
 
 
 def step_raw(p: StepParams) -> int:

@@ -34,6 +34,10 @@ inline cudaError_t opt_in_shared_memory(Kernel kernel, int bytes, int dev, std::
   return e;
 }
 
+// Limit, in clock cycles, that the tensor-core prefill kernels give each of their main-loop
+// waits (see rodimus_ddts_test_set_wait_limit).
+long long main_loop_wait_cycles();
+
 // Launchers: all arguments validated by the caller; they return a cudaError_t.
 cudaError_t launch_step(const rodimus_ddts_step_params& p, int* n_launches);
 cudaError_t launch_plan(const rodimus_ddts_fwd_params& p, int* n_launches);

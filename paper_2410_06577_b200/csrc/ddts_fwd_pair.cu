@@ -80,7 +80,9 @@ constexpr int kBlkFloats = 68;                            // 64 decays, verdict,
 constexpr int kBlkBytes = kBlkFloats * 4;                 // 272 B, a multiple of 16
 constexpr int kOffTx = kOffDp + 4 * kDK * 4;              // float [2][68]: block to send
 constexpr int kOffRx = kOffTx + kRxBufs * kBlkBytes;      // float [2][68]: block received
-constexpr int kGateWarp0 = 10, kGateWarps = 16;
+constexpr int kCtlWarp = 2;                             // low warp numbers for the single-warp roles:
+                                                      // among ready warps the scheduler favours the oldest
+constexpr int kGateWarp0 = 12, kGateWarps = 16;
 constexpr int kGR = kC / kGateWarps;                       // rows per gate thread
 constexpr int kOffTot = kOffRx + kRxBufs * kBlkBytes;     // float [2][8][64]: scan partials
 constexpr int kOffBar = kOffTot + 2 * kGateWarps * kCH * 4;
@@ -91,8 +93,8 @@ constexpr int kSmemBytes = kSmemUsed + 1024;              // slack for manual 10
 static_assert(kOffTx % 16 == 0 && kOffRx % 16 == 0 && kBlkBytes % 16 == 0, "bulk copy alignment");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
-constexpr int kThreads = 32 * (kGateWarp0 + kGateWarps + 1);  // 608: 8 gate warps + control
-constexpr int kStateWarp0 = 2, kScoreWarp0 = 6;
+constexpr int kThreads = 32 * (kGateWarp0 + kGateWarps);   // 896 (warp 3 has no role)
+constexpr int kStateWarp0 = 4, kScoreWarp0 = 8;
 
 // TMEM columns (32-bit words): two state buffers S^T [lane = value column][128 channels], output
 // O^T [lane = value column][64 rows], scores P [64 rows in 16-lane groups][64], and two buffers
@@ -113,8 +115,9 @@ enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                    
        BAR_OTFREE0, BAR_OTFREE1,      // output tile's copies to global have read it            (1)
        BAR_GO0, BAR_GO1,              // an order for the gate warps is in its slot              (1)
        BAR_PRE,                       // the row groups' prefixes are in place                   (1)
-       BAR_ROWS };                    // every gate warp has rewritten its rows of the pass
-static_assert(BAR_ROWS < kNumBars, "barrier count");
+       BAR_ROWS,                      // every gate warp has rewritten its rows of the pass
+       BAR_DRAIN };                   // teardown after a timeout: issued contractions are done  (1)
+static_assert(BAR_DRAIN < kNumBars, "barrier count");
 
 struct PairArgs {
   void* o;
@@ -126,6 +129,7 @@ struct PairArgs {
   int H, T, dv, n_seq, pairs;
   long long n_items;     // (sequence, head, 256-column slab)
   float scale;
+  long long wait_cycles; // limit of one main-loop wait (clock cycles)
   float* dtot;           // optional [n_seq, H, dk]: product of all chunk decays of each sequence
   int sT_only;           // >= 0: only this sequence's final state is stored, as if it were number 0
   int state_only;        // 1: launch the state-only instantiation of the kernel
@@ -182,8 +186,13 @@ constexpr int kPassLast = 2;
 
 struct Control {            // lives in shared memory
   uint32_t tmem_base;
-  int abort_flag;
   int done;                 // gate group has finished every item of this CTA
+  WaitCtl wait;             // abort flag and limit shared by every bounded wait of the CTA
+  // teardown handshake of the pair: how many attempts' decay blocks / operand slabs this CTA
+  // has copied to the partner and for how many it has armed its own receive barriers; and what
+  // the partner says about itself (written by the partner before the first closing barrier)
+  int sent_blk, sent_slab, armed_cnt;
+  int peer_abort, peer_sent_blk, peer_sent_slab;
   int redir_seq;            // bumped by the gate group after writing redir_j / redir_tpos
   int redir_j, redir_tpos;  // where the producer must continue (CTA-local item index, token)
   int tag[kStages][2];      // per stage: (item index, token position) of the fill it holds
@@ -282,7 +291,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const uint32_t bars = base + kOffBar;
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   volatile Control* ctl = reinterpret_cast<volatile Control*>(gbase + kOffMisc);
-  volatile int* abort_flag = &ctl->abort_flag;
+  volatile WaitCtl* abort_flag = &ctl->wait;
   float* sDp = reinterpret_cast<float*>(gbase + kOffDp);
   volatile float* sTx = reinterpret_cast<volatile float*>(gbase + kOffTx);
   volatile float* sRx = reinterpret_cast<volatile float*>(gbase + kOffRx);
@@ -302,7 +311,10 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   if (!a.cu && blockIdx.x == 0 && tid == 0) a.hdr->status = RODIMUS_OK;
 
   if (tid == 0) {
-    ctl->abort_flag = 0;
+    ctl->wait.abort_flag = 0;
+    ctl->wait.limit = a.wait_cycles;
+    ctl->sent_blk = ctl->sent_slab = ctl->armed_cnt = 0;
+    ctl->peer_abort = ctl->peer_sent_blk = ctl->peer_sent_slab = 0;
     ctl->done = 0;
     ctl->redir_seq = 0;
     for (int s = 0; s < kStages; ++s) {
@@ -329,6 +341,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     mbar_init(bar(BAR_GO0), 1);
     mbar_init(bar(BAR_GO1), 1);
     mbar_init(bar(BAR_PRE), 1);
+    mbar_init(bar(BAR_DRAIN), 1);
     mbar_init(bar(BAR_ROWS), kGateWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -417,9 +430,9 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ++j;
             tpos = 0;
           }
-          if (have || ctl->done || *abort_flag) break;
-          if (clock64() - t0 > kWaitCycles) {
-            ctl->abort_flag = 1;
+          if (have || ctl->done || abort_flag->abort_flag) break;
+          if (clock64() - t0 >= abort_flag->limit) {
+            abort_flag->abort_flag = 1;
             atomicMax(&a.hdr->status, (int)RODIMUS_ERR_TIMEOUT);
             break;
           }
@@ -433,11 +446,9 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
       // Leave no bulk copy in flight when the CTA exits: the last fills' barriers complete by
       // byte count, whoever consumed them.
-      const long long t1 = clock64();
       for (uint32_t back = 1; back <= (uint32_t)kStages && back <= f; ++back) {
         const uint32_t ff = f - back;
-        while (!mbar_try(bar(BAR_FULL0 + ff % kStages), (ff / kStages) & 1) &&
-               clock64() - t1 < kWaitCycles) {}
+        mbar_drain(bar(BAR_FULL0 + ff % kStages), (ff / kStages) & 1);
       }
     }
   } else if (warp == 1) {
@@ -794,7 +805,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
     }
     bulk_wait<0>();   // this thread's output copies are complete before the CTA may exit
-  } else if (warp >= kGateWarp0) {
+  } else if (warp >= kGateWarp0 || warp == kCtlWarp) {
     // ============================== gate group and its control warp ==============================
     // The gate warps are workers: for every order of the control warp (a stage and a row count)
     // they run phase 1 on their rows, hand in the column sums, wait for their prefix, run phase
@@ -802,7 +813,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // attempt, the scan over the 16 row groups, decays, verdict exchange, the copies to the
     // partner, refusals and redirects, publishing the pass.
     const int gw = warp - kGateWarp0;                     // rows kGR*gw .. kGR*gw+kGR-1 of the tile
-    const bool is_ctl = gw == kGateWarps;
+    const bool is_ctl = warp == kCtlWarp;
     bool ok = true;
     if (!is_ctl) {
       uint32_t off[kGR]; // swizzled byte offsets of the thread's element pairs inside a slab
@@ -838,6 +849,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       uint32_t fs = 0, fph = 0;                           // stage and phase of the next fill
       uint32_t g = 0, m = 0, oc = 0;                      // passes, exchanged attempts, orders given
       bool armed = false;                                 // attempt m's receive barriers expect bytes
+      uint32_t sent_blk = 0, sent_slab = 0;               // leader: copies issued to the partner
       auto redirect = [&](int jj, int tt) {               // one thread; before the stage is released
         ctl->redir_j = jj;
         ctl->redir_tpos = tt;
@@ -951,6 +963,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           dsmem_bulk_copy(map_to_cta(base + kOffRx + rxi * kBlkBytes, peer),
                           base + kOffTx + rxi * kBlkBytes, kBlkBytes,
                           map_to_cta(bar(BAR_VERD0 + rxi), peer));
+          ++sent_blk;
           // the descriptor of the pass this attempt becomes if both CTAs accept it (slot g & 3
           // is not read before its barrier completes; a refused attempt's entry is overwritten)
           volatile PassDesc* pd = &ctl->pd[g & 3];
@@ -970,6 +983,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const uint32_t pb = map_to_cta(bar(BAR_PEER0 + rxi), peer);
           if (!STATE_ONLY) dsmem_bulk_copy(map_to_cta(dst + kRxQ, peer), st + kStQ, kSlabBytes, pb);
           dsmem_bulk_copy(map_to_cta(dst + kRxK, peer), st + kStK, kSlabBytes, pb);
+          ++sent_slab;
         }
         // both verdicts: the own one and the partner's (came with its decay block)
         if (!(ok = mbar_wait_cluster(bar(BAR_VERD0 + rxi), rxph, abort_flag, a.hdr))) break;
@@ -988,10 +1002,10 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (leader) mbar_arrive_cnt(bar(BAR_EMPTY0 + ahead_s), 2);
             ahead = false;
           }
+          // whatever the partner sent for this attempt must have landed before its buffer
+          // and its stage are declared reusable
+          if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
           if (leader) {
-            // whatever the partner sent for this attempt must have landed before its buffer
-            // and its stage are declared reusable
-            if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), rxph, abort_flag, a.hdr))) break;
             const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]);
             mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
             mbar_arrive_remote(map_to_cta(bar(BAR_RXFREE0 + rxi), peer));
@@ -1025,29 +1039,62 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       give_order(-1, 0);                                  // the workers leave (also after a failed wait)
       if (leader) {
         ctl->done = 1;
-        // nothing the partner sent may still be in flight towards this CTA when it exits
-        const long long t1 = clock64();
-        for (uint32_t back = armed ? 0 : 1; back <= 2 && back <= m; ++back) {
-          const uint32_t mm = m - back;
-          while (!(mbar_try_cluster(bar(BAR_PEER0 + (mm & 1)), (mm >> 1) & 1) &&
-                   mbar_try_cluster(bar(BAR_VERD0 + (mm & 1)), (mm >> 1) & 1)) &&
-                 clock64() - t1 < kWaitCycles) {}
-        }
+        ctl->sent_blk = (int)sent_blk;                    // for the closing handshake
+        ctl->sent_slab = (int)sent_slab;
+        ctl->armed_cnt = (int)(m + (armed ? 1u : 0u));
       }
     }
   }
 
   // ------------------------------------------ teardown ------------------------------------------
+  // Normal end: every copy the pair exchanged has been consumed, nothing is in flight.  After a
+  // wait that ran out the two CTAs may have stopped anywhere, so they tell each other how far
+  // they got and each waits (bounded) for exactly what the other has sent before either leaves;
+  // the issuer first lets the contractions it has issued finish, since they read shared memory
+  // and write tensor memory that is about to be released.
   tc_fence_before();
   __syncthreads();
+  const bool my_abort = ctl->wait.abort_flag != 0;
+  if (tid == 0) {
+    const uint32_t pc = map_to_cta(smem_u32(const_cast<int*>(&ctl->peer_abort)), peer);
+    st_cluster_u32(pc, my_abort ? 1u : 0u);
+    st_cluster_u32(pc + 4, (uint32_t)ctl->sent_blk);
+    st_cluster_u32(pc + 8, (uint32_t)ctl->sent_slab);
+  }
+  if (my_abort && warp == 1) {
+    if (lane == 0) {
+      umma_commit(bar(BAR_DRAIN));
+      mbar_drain(bar(BAR_DRAIN), 0);
+    }
+    __syncwarp();
+  }
+  cluster_arrive();     // release: the stores above; acquire: the partner's
+  cluster_wait();
+  if (my_abort || ctl->peer_abort) {
+    if (tid == 0) {
+      const uint32_t nb = (uint32_t)ctl->peer_sent_blk, ns = (uint32_t)ctl->peer_sent_slab;
+      const uint32_t top = nb > ns ? nb : ns;
+      // receive barriers this CTA never armed, for attempts the partner did send
+      for (uint32_t at = (uint32_t)ctl->armed_cnt; at < top; ++at) {
+        mbar_expect_tx(bar(BAR_VERD0 + (at & 1)), kBlkBytes);
+        mbar_expect_tx(bar(BAR_PEER0 + (at & 1)), STATE_ONLY ? kRxBytes - kSlabBytes : kRxBytes);
+      }
+      // the last attempt of each parity that was sent: its bytes have landed
+      for (uint32_t back = 1; back <= 2; ++back) {
+        if (nb >= back) mbar_drain(bar(BAR_VERD0 + ((nb - back) & 1)), ((nb - back) >> 1) & 1);
+        if (ns >= back) mbar_drain(bar(BAR_PEER0 + ((ns - back) & 1)), ((ns - back) >> 1) & 1);
+      }
+    }
+    __syncthreads();
+    // neither CTA leaves while a copy of the other may still be reading its shared memory
+    cluster_arrive();
+    cluster_wait();
+  }
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
                  : "memory");
   }
-  // neither CTA leaves while the other may still signal one of its barriers
-  cluster_arrive();
-  cluster_wait();
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -1298,6 +1345,7 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   a.pairs = p.dv / (2 * kDVS);
   a.n_items = n_seq0 * p.H * a.pairs;
   a.scale = p.scale;
+  a.wait_cycles = main_loop_wait_cycles();
   a.dtot = nullptr;
   a.sT_only = -1;
   a.state_only = 0;

@@ -59,7 +59,8 @@ constexpr uint32_t kColS = 0, kColO = 128, kColP = 256, kTmemCols = 512;
 
 // mbarrier indices
 enum { BAR_FULL0 = 0, BAR_FULL1, BAR_EMPTY0, BAR_EMPTY1, BAR_GATED0, BAR_GATED1, BAR_PFULL,
-       BAR_PREADY, BAR_SREADY, BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN };
+       BAR_PREADY, BAR_SREADY, BAR_SFULL, BAR_OFULL, BAR_OFREE, BAR_GSCAN,
+       BAR_DRAIN };   // teardown after a timeout: issued contractions are done
 
 
 struct TcArgs {
@@ -72,6 +73,7 @@ struct TcArgs {
   int H, T, dv, n_seq, slices;
   long long n_items;
   float scale;
+  long long wait_cycles;   // limit of one main-loop wait (clock cycles)
 };
 
 struct Item {
@@ -125,8 +127,8 @@ constexpr int kPassFirst = 1, kPassLast = 2;
 
 struct Control {            // lives in shared memory
   uint32_t tmem_base;
-  int abort_flag;
   int done;                 // gate group has finished every item of this CTA
+  WaitCtl wait;             // abort flag and limit shared by every bounded wait of the CTA
   int redir_seq;            // bumped by the gate group after writing redir_j / redir_tpos
   int redir_j, redir_tpos;  // where the producer must continue (CTA-local item index, token)
   int pad[2];
@@ -147,7 +149,7 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   const uint32_t bars = base + kOffBar;
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   volatile Control* ctl = reinterpret_cast<volatile Control*>(gbase + kOffMisc);
-  volatile int* abort_flag = &ctl->abort_flag;
+  volatile WaitCtl* abort_flag = &ctl->wait;
   float* sD = reinterpret_cast<float*>(gbase + kOffD);
   float* sTot = reinterpret_cast<float*>(gbase + kOffTot);
 
@@ -157,7 +159,8 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   if (!a.cu && blockIdx.x == 0 && tid == 0) a.hdr->status = RODIMUS_OK;
 
   if (tid == 0) {
-    ctl->abort_flag = 0;
+    ctl->wait.abort_flag = 0;
+    ctl->wait.limit = a.wait_cycles;
     ctl->done = 0;
     ctl->redir_seq = 0;
     mbar_init(bar(BAR_FULL0), 1);
@@ -173,6 +176,7 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     mbar_init(bar(BAR_OFULL), 1);
     mbar_init(bar(BAR_OFREE), 128);
     mbar_init(bar(BAR_GSCAN), kGateWarps);
+    mbar_init(bar(BAR_DRAIN), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -213,9 +217,9 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             ++j;
             tpos = 0;
           }
-          if (have || ctl->done || *abort_flag) break;
-          if (clock64() - t0 > kWaitCycles) {
-            ctl->abort_flag = 1;
+          if (have || ctl->done || abort_flag->abort_flag) break;
+          if (clock64() - t0 >= abort_flag->limit) {
+            abort_flag->abort_flag = 1;
             atomicMax(&a.hdr->status, (int)RODIMUS_ERR_TIMEOUT);
             break;
           }
@@ -244,10 +248,9 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       }
       // Leave no bulk copy in flight when the CTA exits: the last two fills' barriers complete
       // by byte count, whoever consumed them.
-      const long long t1 = clock64();
       for (uint32_t back = 1; back <= 2 && back <= f; ++back) {
         const uint32_t ff = f - back;
-        while (!mbar_try(bar(BAR_FULL0 + (ff & 1)), (ff >> 1) & 1) && clock64() - t1 < kWaitCycles) {}
+        mbar_drain(bar(BAR_FULL0 + (ff & 1)), (ff >> 1) & 1);
       }
     }
   } else if (warp == 1) {
@@ -613,8 +616,18 @@ ddts_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   }
 
   // ------------------------------------------ teardown ------------------------------------------
+  // After a wait that ran out the roles may have stopped anywhere: the contractions already
+  // issued must finish before the tensor memory they write and the shared memory they read are
+  // released.
   tc_fence_before();
   __syncthreads();
+  if (ctl->wait.abort_flag && warp == 1) {
+    if (lane == 0) {
+      umma_commit(bar(BAR_DRAIN));
+      mbar_drain(bar(BAR_DRAIN), 0);
+    }
+    __syncwarp();
+  }
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
@@ -670,6 +683,7 @@ cudaError_t launch_fwd_tc(const rodimus_ddts_fwd_params& p, int* n_launches) {
   a.slices = p.dv / kDVS;
   a.n_items = (long long)a.n_seq * p.H * a.slices;
   a.scale = p.scale;
+  a.wait_cycles = main_loop_wait_cycles();
   if (a.n_items == 0) return cudaSuccess;
   const uint64_t rows = (uint64_t)p.B * p.H * p.T;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);

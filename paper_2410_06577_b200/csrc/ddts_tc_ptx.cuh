@@ -9,7 +9,18 @@
 namespace ddts {
 namespace {
 
-constexpr long long kWaitCycles = 4000000000LL;  // about two seconds: then give up, never hang
+constexpr long long kWaitCycles = 4000000000LL;   // default limit of a main-loop wait: about two
+                                                  // seconds, then give up, never hang
+constexpr long long kDrainCycles = 4000000000LL;  // limit of the teardown waits (copies in flight)
+
+// What every bounded wait of a CTA shares, in shared memory: the flag a role raises when it gives
+// up (the others then stop waiting too) and the limit of one wait in cycles (a launch argument;
+// 0 makes the first unsuccessful poll a timeout, which is how the tests reach this path).
+struct WaitCtl {
+  int abort_flag;
+  int pad;
+  long long limit;
+};
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -55,28 +66,31 @@ __device__ __forceinline__ bool mbar_try_park(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false (and raises the CTA's abort flag and the device status) if the
 // phase does not complete in time or another role has already given up.  The polling loop is
 // kept out of line: it is cold, and dozens of inlined copies would crowd the instruction cache.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile WaitCtl* wc,
                                             WorkspaceHeader* hdr) {
+  const long long limit = wc->limit;
   const long long t0 = clock64();
   while (true) {
+    if (limit > 0) {
 #pragma unroll 1
-    for (int i = 0; i < 16; ++i)
-      if (mbar_try_park(bar, parity)) return true;
+      for (int i = 0; i < 16; ++i)
+        if (mbar_try_park(bar, parity)) return true;
+    }
     // a completed phase stays visible to every waiter of a group, so re-test before giving up:
     // either all members of a group pass a given wait or none does
-    if (*abort_flag) return mbar_try(bar, parity);
-    if (clock64() - t0 > kWaitCycles) {
+    if (wc->abort_flag) return mbar_try(bar, parity);
+    if (clock64() - t0 >= limit) {
       if (mbar_try(bar, parity)) return true;
-      *abort_flag = 1;
+      wc->abort_flag = 1;
       atomicMax(&hdr->status, (int)RODIMUS_ERR_TIMEOUT);
       return false;
     }
   }
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile WaitCtl* wc,
                                           WorkspaceHeader* hdr) {
   if (mbar_try(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, hdr);
+  return mbar_wait_slow(bar, parity, wc, hdr);
 }
 __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -375,25 +389,40 @@ __device__ __forceinline__ bool mbar_try_park_cluster(uint32_t bar, uint32_t par
   return ok != 0;
 }
 __device__ __noinline__ bool mbar_wait_cluster_slow(uint32_t bar, uint32_t parity,
-                                                    volatile int* abort_flag, WorkspaceHeader* hdr) {
+                                                    volatile WaitCtl* wc, WorkspaceHeader* hdr) {
+  const long long limit = wc->limit;
   const long long t0 = clock64();
   while (true) {
+    if (limit > 0) {
 #pragma unroll 1
-    for (int i = 0; i < 16; ++i)
-      if (mbar_try_park_cluster(bar, parity)) return true;
-    if (*abort_flag) return mbar_try_cluster(bar, parity);
-    if (clock64() - t0 > kWaitCycles) {
+      for (int i = 0; i < 16; ++i)
+        if (mbar_try_park_cluster(bar, parity)) return true;
+    }
+    if (wc->abort_flag) return mbar_try_cluster(bar, parity);
+    if (clock64() - t0 >= limit) {
       if (mbar_try_cluster(bar, parity)) return true;
-      *abort_flag = 1;
+      wc->abort_flag = 1;
       atomicMax(&hdr->status, (int)RODIMUS_ERR_TIMEOUT);
       return false;
     }
   }
 }
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
-                                                  volatile int* abort_flag, WorkspaceHeader* hdr) {
+                                                  volatile WaitCtl* wc, WorkspaceHeader* hdr) {
   if (mbar_try_cluster(bar, parity)) return true;
-  return mbar_wait_cluster_slow(bar, parity, abort_flag, hdr);
+  return mbar_wait_cluster_slow(bar, parity, wc, hdr);
+}
+// Teardown wait (own bound, independent of the launch's limit): true if the phase completed.
+__device__ __noinline__ bool mbar_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try(bar, parity)) {
+    if (clock64() - t0 > kDrainCycles) return false;
+  }
+  return true;
+}
+// Plain 32-bit store into the shared memory of another CTA of the cluster (address from map_to_cta).
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
 // Bulk copy from this CTA's shared memory into another CTA's; completes (by byte count) on an
 // mbarrier of the destination CTA.  Addresses and size are multiples of 16 bytes.

@@ -35,7 +35,14 @@ int check_fwd_sizes(const rodimus_ddts_fwd_params* p, bool varlen) {
 
 }  // namespace
 
+namespace {
+constexpr long long kDefaultWaitCycles = 4000000000LL;   // about two seconds
+std::atomic<long long> g_wait_cycles{kDefaultWaitCycles};
+}  // namespace
+
 namespace ddts {
+
+long long main_loop_wait_cycles() { return g_wait_cycles.load(std::memory_order_relaxed); }
 
 cudaError_t current_device(int* dev, int* sms) {
   static std::atomic<int> cached[64];   // SM count per device ordinal, 0 = not asked yet
@@ -159,6 +166,11 @@ int rodimus_ddts_device_status(const void* workspace, void* stream) {
 }
 
 int rodimus_ddts_last_launch_count(void) { return t_last_launches; }
+
+int rodimus_ddts_test_set_wait_limit(long long cycles) {
+  g_wait_cycles.store(cycles < 0 ? kDefaultWaitCycles : cycles, std::memory_order_relaxed);
+  return RODIMUS_OK;
+}
 
 const char* rodimus_status_str(int status) {
   switch (status) {

@@ -561,3 +561,35 @@ def test_config4_full_size_every_sequence():
         ro, rs = orc.ref_fwd(sl(p.q), sl(p.k), sl(p.x), sl(p.y), sl(p.v), cu_seqlens=cu)
         eo, es = _worst_err(host(o[:, hs]), host(sT[:, hs]), ro, rs, cu)
         assert eo <= TOL_BF16 and es <= TOL_BF16, (h0, eo, es)
+
+
+# ------------------------------------------------------------------------------------------
+# bounded waits: a wait that runs out is reported, nothing hangs, the device stays usable
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dv", [256, 128])      # cluster-pair kernel / single-CTA kernel
+def test_wait_that_runs_out_is_reported_and_the_next_call_is_clean(dv):
+    """The main-loop waits of the tensor-core kernels take their bound from the launch.  With a
+    bound of zero the first wait that is not satisfied at once gives up (at kernel start the
+    issuer always finds no pass published yet): the call itself returns OK, the kernel ends by
+    its teardown path, the status word says TIMEOUT; a normal call on the same workspace then
+    reports OK and matches the oracle."""
+    import torch
+    p = wl.make_prefill(40 + dv, 1, 1, 64, 128, dv, "bf16", s0_std=0.1)
+    d = prefill_to_device(p)
+    o, sT = _nan_outputs(d)
+    prm = rd.fwd_params(d["q"], d["k"], d["x"], d["y"], d["v"], o, d["s0"], sT)
+    ws = rd.new_workspace(prm, "cuda")
+    prm.workspace, prm.workspace_bytes = ws.data_ptr(), ws.numel()
+    try:
+        rd.test_set_wait_limit(0)
+        assert rd.fwd_raw(prm) == rd.OK
+        assert rd.device_status(ws) == rd.ERR_TIMEOUT
+    finally:
+        rd.test_set_wait_limit(-1)
+    o, sT = _nan_outputs(d)
+    prm.o, prm.sT = o.data_ptr(), sT.data_ptr()
+    assert rd.fwd_raw(prm) == rd.OK
+    assert rd.device_status(ws) == rd.OK
+    ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0)
+    assert rel_err(host(o), ro) <= TOL_BF16 and rel_err(host(sT), rs) <= TOL_BF16
