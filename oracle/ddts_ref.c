@@ -8,8 +8,10 @@
  *
  * What it computes (Rodimus paper, Eq. "alpha_def" of Sec. 3.1.2 and
  * Eq. "rodimus_recurrent_form" of Sec. 3.1.3, with the value-side decay
- * beta_t = 1 as Sec. 3.1.1 chooses, and without the value gate and the
- * feed-through term, which the caller applies outside this path):
+ * beta_t = 1 as Sec. 3.1.1 chooses; the value gate beta_hat of Eq. "beta_def" and
+ * the feed-through term d . x' of Eq. "rodimus_recurrent_form" are optional inputs
+ * of the ..._block entry points: v_t is replaced by beta_hat_t . v_t and d . x'_t is
+ * added to o_t; their projections stay with the caller):
  *
  *   g_t     = softplus(x_t)                    selection gate,   per key channel
  *   tau_t   = sigmoid(y_t)                     temperature gate, per key channel
@@ -77,9 +79,14 @@ int ddts_ref_gates(int ingate, int64_t n, const float *x, const float *y, double
 }
 
 /* One sequence, one head: rows [0,len) of q,k,x,y (row stride dk) and v,o (row stride dv). */
+/* Optional terms of the full block (Eq. "beta_def", Eq. "rodimus_recurrent_form"): bh, rows of
+ * the value gate beta_hat (multiplies v_t element by element), and the feed-through d . x'_t
+ * added to o_t after the scaling (d: one weight per value column, fx: rows of x').  NULL = absent,
+ * and then the arithmetic is exactly that of the plain recurrence. */
 static void ref_one_sequence(int ingate, int64_t len, int dk, int dv, double scale, const float *q,
                              const float *k, const float *x, const float *y, const float *v,
-                             const double *s0, double *o, double *sT, double *S) {
+                             const double *s0, double *o, double *sT, double *S, const float *bh,
+                             const float *d_feed, const float *fx) {
   if (s0)
     memcpy(S, s0, sizeof(double) * (size_t)dk * dv);
   else
@@ -95,14 +102,24 @@ static void ref_one_sequence(int ingate, int64_t len, int dk, int dv, double sca
       ref_gate(ingate, (double)xt[d], (double)yt[d], &alpha, &ahat);
       double w = ahat * (double)kt[d];
       double *Sd = S + (size_t)d * dv;
-      for (int j = 0; j < dv; ++j) Sd[j] = alpha * Sd[j] + w * (double)vt[j];
+      if (bh) {
+        const float *bt = bh + t * dv;
+        for (int j = 0; j < dv; ++j) Sd[j] = alpha * Sd[j] + w * ((double)bt[j] * (double)vt[j]);
+      } else {
+        for (int j = 0; j < dv; ++j) Sd[j] = alpha * Sd[j] + w * (double)vt[j];
+      }
       if (ot) {
         double qd = (double)qt[d];
         for (int j = 0; j < dv; ++j) ot[j] += qd * Sd[j];
       }
     }
-    if (ot)
+    if (ot) {
       for (int j = 0; j < dv; ++j) ot[j] *= scale;
+      if (d_feed && fx) {
+        const float *ft = fx + t * dv;
+        for (int j = 0; j < dv; ++j) ot[j] += (double)d_feed[j] * (double)ft[j];
+      }
+    }
   }
   if (sT) memcpy(sT, S, sizeof(double) * (size_t)dk * dv);
 }
@@ -115,9 +132,11 @@ static void ref_one_sequence(int ingate, int64_t len, int dk, int dv, double sca
  * s0/sT are [N,H,dk,dv].  o may be NULL (state only).  Returns 0, or a nonzero
  * code for arguments that make no sense.
  */
-int ddts_ref_fwd(int ingate, int B, int H, int64_t T, int dk, int dv, double scale, const float *q,
-                 const float *k, const float *x, const float *y, const float *v, const double *s0,
-                 double *o, double *sT, const int32_t *cu_seqlens, int N) {
+int ddts_ref_fwd_block(int ingate, int B, int H, int64_t T, int dk, int dv, double scale,
+                       const float *q, const float *k, const float *x, const float *y,
+                       const float *v, const double *s0, double *o, double *sT,
+                       const int32_t *cu_seqlens, int N, const float *beta_hat,
+                       const float *feed_d, const float *feed_x) {
   if (ingate != DDTS_REF_POW_G && ingate != DDTS_REF_POW_SIGMOID) return 3;
   if (B < 0 || H < 0 || T < 0 || dk <= 0 || dv <= 0) return 2;
   int nseq = B;
@@ -152,11 +171,20 @@ int ddts_ref_fwd(int ingate, int B, int H, int64_t T, int dk, int dv, double sca
       size_t so = (size_t)it * dk * dv;
       ref_one_sequence(ingate, len, dk, dv, scale, q + row0 * dk, k + row0 * dk, x + row0 * dk,
                        y + row0 * dk, v + row0 * dv, s0 ? s0 + so : NULL, o ? o + row0 * dv : NULL,
-                       sT ? sT + so : NULL, S);
+                       sT ? sT + so : NULL, S, beta_hat ? beta_hat + row0 * dv : NULL,
+                       feed_d ? feed_d + (size_t)h * dv : NULL, feed_x ? feed_x + row0 * dv : NULL);
     }
     free(S);
   }
   return failed ? 8 : 0;
+}
+
+/* The recurrence alone (no value gate, no feed-through). */
+int ddts_ref_fwd(int ingate, int B, int H, int64_t T, int dk, int dv, double scale, const float *q,
+                 const float *k, const float *x, const float *y, const float *v, const double *s0,
+                 double *o, double *sT, const int32_t *cu_seqlens, int N) {
+  return ddts_ref_fwd_block(ingate, B, H, T, dk, dv, scale, q, k, x, y, v, s0, o, sT, cu_seqlens,
+                            N, NULL, NULL, NULL);
 }
 
 /*
@@ -164,9 +192,10 @@ int ddts_ref_fwd(int ingate, int B, int H, int64_t T, int dk, int dv, double sca
  * [Nseq,H,dv], state is [Nseq,H,dk,dv] and is updated in place; o reads the state
  * after the update (Eq. "rodimus_recurrent_form": o_t = q_t S_t).
  */
-int ddts_ref_step(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
-                  const float *k, const float *x, const float *y, const float *v, double *o,
-                  double *state) {
+int ddts_ref_step_block(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
+                        const float *k, const float *x, const float *y, const float *v, double *o,
+                        double *state, const float *beta_hat, const float *feed_d,
+                        const float *feed_x) {
   if (ingate != DDTS_REF_POW_G && ingate != DDTS_REF_POW_SIGMOID) return 3;
   if (Nseq < 0 || H < 0 || dk <= 0 || dv <= 0) return 2;
   int64_t items = (int64_t)Nseq * H;
@@ -183,14 +212,33 @@ int ddts_ref_step(int ingate, int Nseq, int H, int dk, int dv, double scale, con
       double w = ahat * (double)kt[d];
       double qd = (double)qt[d];
       double *Sd = S + (size_t)d * dv;
-      for (int j = 0; j < dv; ++j) {
-        Sd[j] = alpha * Sd[j] + w * (double)vt[j];
-        ot[j] += qd * Sd[j];
+      if (beta_hat) {
+        const float *bt = beta_hat + it * dv;
+        for (int j = 0; j < dv; ++j) {
+          Sd[j] = alpha * Sd[j] + w * ((double)bt[j] * (double)vt[j]);
+          ot[j] += qd * Sd[j];
+        }
+      } else {
+        for (int j = 0; j < dv; ++j) {
+          Sd[j] = alpha * Sd[j] + w * (double)vt[j];
+          ot[j] += qd * Sd[j];
+        }
       }
     }
     for (int j = 0; j < dv; ++j) ot[j] *= scale;
+    if (feed_d && feed_x) {
+      const float *dh = feed_d + (size_t)(it % H) * dv, *ft = feed_x + it * dv;
+      for (int j = 0; j < dv; ++j) ot[j] += (double)dh[j] * (double)ft[j];
+    }
   }
   return 0;
+}
+
+int ddts_ref_step(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
+                  const float *k, const float *x, const float *y, const float *v, double *o,
+                  double *state) {
+  return ddts_ref_step_block(ingate, Nseq, H, dk, dv, scale, q, k, x, y, v, o, state, NULL, NULL,
+                             NULL);
 }
 
 /* Threads the parallel regions above will use (1 without OpenMP). */

@@ -39,7 +39,7 @@ def _golden_rows():
     path = os.path.join(os.path.dirname(__file__), "golden", "ddts_hand_example.txt")
     rows = []
     for line in open(path):
-        if line.startswith("#") or not line.strip():
+        if line.startswith("#") or not line.strip() or line.startswith("block"):
             continue
         f = line.split()
         rows.append((int(f[0]),) + tuple(float(t) for t in f[1:]))
@@ -271,3 +271,74 @@ def test_strong_decay_and_long_memory_stay_finite():
         assert np.all(np.isfinite(o)) and np.all(np.isfinite(sT))
         ref = orc.parallel_form(q, k, np.full_like(x, xv), np.full_like(y, yv), v)
         assert _rel(o, ref) < 1e-12
+
+
+# -- optional terms of the full block: value gate and feed-through -----------------------------
+
+def _fwd_block(q, k, x, y, v, beta_hat=None, feed_d=None, feed_x=None, **kw):
+    a4 = lambda a: None if a is None else np.asarray(a, dtype=np.float32)[None, None]
+    d = None if feed_d is None else np.asarray(feed_d, dtype=np.float32)[None]
+    o, sT = orc.ref_fwd(a4(q), a4(k), a4(x), a4(y), a4(v), beta_hat=a4(beta_hat), feed_d=d,
+                        feed_x=a4(feed_x), **kw)
+    return o[0, 0], sT[0, 0]
+
+
+def test_block_terms_hand_example():
+    path = os.path.join(os.path.dirname(__file__), "golden", "ddts_hand_example.txt")
+    o1, o2, s2 = [tuple(float(t) for t in l.split()[1:]) for l in open(path) if l.startswith("block")][0]
+    z = np.zeros((2, 1), dtype=np.float32)
+    one = np.ones((2, 1), dtype=np.float32)
+    o, sT = _fwd_block(one, one, z, z, one, beta_hat=[[0.5], [0.25]], feed_d=[3.0], feed_x=[[0.5], [-1.0]])
+    assert abs(o[0, 0] - o1) < 1e-15 and abs(o[1, 0] - o2) < 2e-15 and abs(sT[0, 0] - s2) < 1e-15
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_block_terms_absent_or_neutral_give_the_plain_recurrence(mode):
+    q, k, x, y, v = _draw(41, 23, 6, 5)
+    o, sT = _fwd1(q, k, x, y, v, ingate=mode, scale=0.3)
+    ones = np.ones_like(v)
+    ob, sb = _fwd_block(q, k, x, y, v, beta_hat=ones, feed_d=np.zeros(5), feed_x=v, ingate=mode, scale=0.3)
+    assert np.array_equal(o, ob) and np.array_equal(sT, sb)          # bit for bit
+
+
+def test_value_gate_equals_gating_v_beforehand():
+    # gate values that are powers of two, so that beta_hat * v is exact in the input precision
+    q, k, x, y, v = _draw(42, 19, 4, 6)
+    rng = np.random.default_rng(1)
+    beta = np.float32(2.0) ** (-rng.integers(0, 4, v.shape)).astype(np.float32)
+    ob, sb = _fwd_block(q, k, x, y, v, beta_hat=beta)
+    o, sT = _fwd1(q, k, x, y, (beta * v).astype(np.float32))
+    assert np.array_equal(o, ob) and np.array_equal(sT, sb)
+    # and a gate of zero on one column removes that column from the state
+    beta[:, 2] = 0.0
+    _, s0col = _fwd_block(q, k, x, y, v, beta_hat=beta)
+    assert np.all(s0col[:, 2] == 0.0) and np.any(s0col[:, 3] != 0.0)
+
+
+def test_feed_through_adds_d_times_xprime_after_the_scaling():
+    q, k, x, y, v = _draw(43, 11, 4, 3)
+    rng = np.random.default_rng(2)
+    d = rng.standard_normal(3).astype(np.float32)
+    fx = rng.standard_normal(v.shape).astype(np.float32)
+    o, sT = _fwd1(q, k, x, y, v, scale=0.25)
+    ob, sb = _fwd_block(q, k, x, y, v, feed_d=d, feed_x=fx, scale=0.25)
+    assert np.array_equal(sT, sb)                                     # the state does not see it
+    assert _rel(ob - o, d[None].astype(np.float64) * fx) < 1e-13
+
+
+def test_block_terms_in_decode_steps_and_packed_prefill():
+    rng = np.random.default_rng(3)
+    H, dk, dv, lens = 2, 4, 3, [3, 0, 5]
+    T = sum(lens)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    f = lambda *sh: rng.standard_normal(sh).astype(np.float32)
+    q, k, x, y = f(1, H, T, dk), f(1, H, T, dk), f(1, H, T, dk) - 1, f(1, H, T, dk)
+    v, bh, fx, d = f(1, H, T, dv), rng.random((1, H, T, dv)).astype(np.float32), f(1, H, T, dv), f(H, dv)
+    o, sT = orc.ref_fwd(q, k, x, y, v, cu_seqlens=cu, beta_hat=bh, feed_d=d, feed_x=fx, scale=0.5)
+    for n in range(3):
+        st = np.zeros((1, H, dk, dv))
+        for t in range(cu[n], cu[n + 1]):
+            ot = orc.ref_step(q[:, :, t], k[:, :, t], x[:, :, t], y[:, :, t], v[:, :, t], st, scale=0.5,
+                              beta_hat=bh[:, :, t], feed_d=d, feed_x=fx[:, :, t])
+            assert _rel(ot[0], o[0, :, t]) < 1e-13
+        assert _rel(st[0], sT[n]) < 1e-13 or lens[n] == 0
