@@ -12,8 +12,10 @@
  *   S_t = diag(alpha_t) S_{t-1} + (ahat_t . k_t)^T v_t          S_t is [dk, dv], fp32
  *   o_t = scale * q_t S_t                                       state AFTER the update
  *
- * The projections that produce q, k, v, x, y, the value gate and the feed-through term of
- * the full block are the caller's; v arrives already gated.
+ * The projections that produce q, k, v, x, y and the value gate are the caller's.  The value
+ * gate beta_hat_t (Eq. "beta_def") and the feed-through d . x'_t of Eq. "rodimus_recurrent_form"
+ * can be handed in as optional tensors and are then applied inside the same pass: v_t is
+ * multiplied by beta_hat_t where it is loaded, d . x'_t is added to o_t where it is stored.
  *
  * Conventions shared by every entry point
  *   - All data pointers are DEVICE pointers unless a name ends in "_host".
@@ -101,6 +103,12 @@ typedef struct {
   void *workspace;           /* device, >= rodimus_ddts_fwd_workspace_bytes(), 256-byte aligned */
   size_t workspace_bytes;
   void *stream;              /* cudaStream_t of the caller (NULL = default stream)              */
+  /* Optional terms of the full block, fused into the same pass (all NULL = the recurrence alone): */
+  const void *beta_hat;      /* device [B,H,T,dv], dtype of v: value gate of Eq. "beta_def", already */
+                             /* passed through its sigmoid; v_t enters the state as beta_hat_t * v_t */
+  const float *feed_d;       /* device fp32 [H,dv]: feed-through weight d of Eq.                     */
+                             /* "rodimus_recurrent_form"; given together with feed_x or not at all   */
+  const void *feed_x;        /* device [B,H,T,dv], dtype of v: x'_t; o_t = scale q_t S_t + d . x'_t  */
 } rodimus_ddts_fwd_params;
 
 /*
@@ -121,6 +129,9 @@ typedef struct {
   void *o;                             /* device [Nseq,H,dv], written */
   float *state;                        /* device fp32 [Nseq,H,dk,dv], updated in place */
   void *stream;
+  const void *beta_hat;                /* optional, device [Nseq,H,dv]: value gate (see the prefill) */
+  const float *feed_d;                 /* optional, device fp32 [H,dv]: feed-through weight          */
+  const void *feed_x;                  /* optional with feed_d, device [Nseq,H,dv]: x'_t             */
 } rodimus_ddts_step_params;
 
 /* Bytes of device workspace rodimus_ddts_fwd needs for these sizes (pointers are not read).

@@ -47,6 +47,7 @@ class FwdParams(ctypes.Structure):
         ("cu_seqlens", ctypes.c_void_p), ("cu_seqlens_host", ctypes.c_void_p),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("stream", ctypes.c_void_p),
+        ("beta_hat", ctypes.c_void_p), ("feed_d", ctypes.c_void_p), ("feed_x", ctypes.c_void_p),
     ]
 
 
@@ -59,6 +60,7 @@ class StepParams(ctypes.Structure):
         ("gate_x", ctypes.c_void_p), ("temp_y", ctypes.c_void_p),
         ("v", ctypes.c_void_p), ("o", ctypes.c_void_p),
         ("state", ctypes.c_void_p), ("stream", ctypes.c_void_p),
+        ("beta_hat", ctypes.c_void_p), ("feed_d", ctypes.c_void_p), ("feed_x", ctypes.c_void_p),
     ]
 
 
@@ -133,7 +135,8 @@ def _check_cuda(*tensors):
 
 def fwd_params(q, k, gate_x, temp_y, v, o, s0=None, sT=None, cu_seqlens=None,
                cu_seqlens_host=None, workspace=None, scale: float = 1.0,
-               ingate: int = INGATE_POW_G, stream: Optional[int] = None) -> FwdParams:
+               ingate: int = INGATE_POW_G, stream: Optional[int] = None, beta_hat=None,
+               feed_d=None, feed_x=None) -> FwdParams:
     """Fills a ``rodimus_ddts_fwd_params`` from torch tensors (no checks beyond layout)."""
     import torch
     B, H, T, dk = q.shape
@@ -151,6 +154,7 @@ def fwd_params(q, k, gate_x, temp_y, v, o, s0=None, sT=None, cu_seqlens=None,
     p.workspace = _ptr(workspace)
     p.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     p.stream = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    p.beta_hat, p.feed_d, p.feed_x = _ptr(beta_hat), _ptr(feed_d), _ptr(feed_x)
     return p
 
 
@@ -223,15 +227,18 @@ def new_workspace(p: FwdParams, device):
 
 def ddts_fwd(q, k, gate_x, temp_y, v, s0=None, cu_seqlens=None, cu_seqlens_host=None,
              scale: float = 1.0, ingate: int = INGATE_POW_G, want_final_state: bool = True,
-             out=None, final_state=None, workspace=None) -> Tuple["torch.Tensor", Optional["torch.Tensor"]]:
+             out=None, final_state=None, workspace=None, beta_hat=None, feed_d=None,
+             feed_x=None) -> Tuple["torch.Tensor", Optional["torch.Tensor"]]:
     """Chunked DDTS prefill (``rodimus_ddts_fwd``).
 
     q,k,gate_x,temp_y: [B,H,T,dk]; v: [B,H,T,dv] (bf16 or fp32, all alike); s0: fp32
     [B|N,H,dk,dv] or None; cu_seqlens: int32 CUDA tensor [N+1] for packed sequences (B = 1).
+    Optional, fused into the same pass: beta_hat [B,H,T,dv] (value gate, multiplies v), and the
+    feed-through feed_d fp32 [H,dv] with feed_x [B,H,T,dv] (o += feed_d * feed_x).
     Returns (o, sT) with sT None unless ``want_final_state``.  Asynchronous on the current stream.
     """
     import torch
-    _check_cuda(q, k, gate_x, temp_y, v, s0, cu_seqlens)
+    _check_cuda(q, k, gate_x, temp_y, v, s0, cu_seqlens, beta_hat, feed_d, feed_x)
     B, H, T, dk = q.shape
     dv = v.shape[-1]
     nseq = B if cu_seqlens is None else cu_seqlens.numel() - 1
@@ -240,7 +247,7 @@ def ddts_fwd(q, k, gate_x, temp_y, v, s0=None, cu_seqlens=None, cu_seqlens_host=
     if sT is None and want_final_state:
         sT = torch.empty((nseq, H, dk, dv), dtype=torch.float32, device=q.device)
     p = fwd_params(q, k, gate_x, temp_y, v, o, s0, sT, cu_seqlens, cu_seqlens_host, None, scale,
-                   ingate)
+                   ingate, beta_hat=beta_hat, feed_d=feed_d, feed_x=feed_x)
     ws = workspace if workspace is not None else new_workspace(p, q.device)
     p.workspace = ws.data_ptr()
     p.workspace_bytes = ws.numel() * ws.element_size()
@@ -251,13 +258,13 @@ def ddts_fwd(q, k, gate_x, temp_y, v, s0=None, cu_seqlens=None, cu_seqlens_host=
 
 
 def ddts_step(q, k, gate_x, temp_y, v, state, scale: float = 1.0, ingate: int = INGATE_POW_G,
-              out=None):
+              out=None, beta_hat=None, feed_d=None, feed_x=None):
     """One decode step (``rodimus_ddts_step``): ``state`` fp32 [Nseq,H,dk,dv] is updated in place.
 
     q,k,gate_x,temp_y: [Nseq,H,dk]; v: [Nseq,H,dv].  Returns o [Nseq,H,dv].
     """
     import torch
-    _check_cuda(q, k, gate_x, temp_y, v, state)
+    _check_cuda(q, k, gate_x, temp_y, v, state, beta_hat, feed_d, feed_x)
     Nseq, H, dk = q.shape
     dv = v.shape[-1]
     o = out if out is not None else torch.empty((Nseq, H, dv), dtype=q.dtype, device=q.device)
@@ -270,6 +277,7 @@ def ddts_step(q, k, gate_x, temp_y, v, state, scale: float = 1.0, ingate: int = 
     p.q, p.k, p.gate_x, p.temp_y, p.v, p.o = (_ptr(t) for t in (q, k, gate_x, temp_y, v, o))
     p.state = _ptr(state)
     p.stream = torch.cuda.current_stream().cuda_stream
+    p.beta_hat, p.feed_d, p.feed_x = _ptr(beta_hat), _ptr(feed_d), _ptr(feed_x)
     rc = step_raw(p)
     if rc != OK:
         raise RodimusError(rc, "rodimus_ddts_step")

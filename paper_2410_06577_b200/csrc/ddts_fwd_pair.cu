@@ -86,9 +86,9 @@ constexpr int kGateWarp0 = 12, kGateWarps = 16;
 constexpr int kGR = kC / kGateWarps;                       // rows per gate thread
 constexpr int kOffTot = kOffRx + kRxBufs * kBlkBytes;     // float [2][8][64]: scan partials
 constexpr int kOffBar = kOffTot + 2 * kGateWarps * kCH * 4;
-constexpr int kNumBars = 32;
+constexpr int kNumBars = 40;
 constexpr int kOffMisc = kOffBar + kNumBars * 8;          // control block
-constexpr int kSmemUsed = kOffMisc + 256;
+constexpr int kSmemUsed = kOffMisc + 320;
 constexpr int kSmemBytes = kSmemUsed + 1024;              // slack for manual 1024-byte alignment
 static_assert(kOffTx % 16 == 0 && kOffRx % 16 == 0 && kBlkBytes % 16 == 0, "bulk copy alignment");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
@@ -116,8 +116,9 @@ enum { BAR_FULL0 = 0,                 // [3] TMA fill landed                    
        BAR_GO0, BAR_GO1,              // an order for the gate warps is in its slot              (1)
        BAR_PRE,                       // the row groups' prefixes are in place                   (1)
        BAR_ROWS,                      // every gate warp has rewritten its rows of the pass
-       BAR_DRAIN };                   // teardown after a timeout: issued contractions are done  (1)
-static_assert(BAR_DRAIN < kNumBars, "barrier count");
+       BAR_DRAIN,                     // teardown after a timeout: issued contractions are done  (1)
+       BAR_XFULL0, BAR_XFULL1 };      // feed-through tile x' landed in the output tile (1 + bytes)
+static_assert(BAR_XFULL1 < kNumBars, "barrier count");
 
 struct PairArgs {
   void* o;
@@ -130,6 +131,10 @@ struct PairArgs {
   long long n_items;     // (sequence, head, 256-column slab)
   float scale;
   long long wait_cycles; // limit of one main-loop wait (clock cycles)
+  // optional terms of the full block (BLOCK instantiations only)
+  const __nv_bfloat16* beta_hat;  // [rows, dv] value gate, or nullptr
+  const float* feed_d;            // [H, dv] feed-through weight, or nullptr (then no x' either)
+  int feed_H;                     // heads per sequence of the caller's layout (indexes feed_d)
   float* dtot;           // optional [n_seq, H, dk]: product of all chunk decays of each sequence
   int sT_only;           // >= 0: only this sequence's final state is stored, as if it were number 0
   int state_only;        // 1: launch the state-only instantiation of the kernel
@@ -198,9 +203,11 @@ struct Control {            // lives in shared memory
   int tag[kStages][2];      // per stage: (item index, token position) of the fill it holds
   int pad[2];
   PassDesc pd[4];
-  struct { int stage, nr; } ord[2];   // orders of the control warp to the gate warps (stage < 0: leave)
+  // orders of the control warp to the gate warps (stage < 0: leave); row and col0 locate the
+  // tile in global memory for the value gate
+  struct { int stage, nr, col0, pad; long long row; } ord[2];
 };
-static_assert(sizeof(Control) <= 256, "control block");
+static_assert(sizeof(Control) <= 320, "control block");
 
 // ---------------------------------------------------------------------------------------------
 // gate math on pairs of adjacent key channels (packed fp32x2 adds / multiplies / fmas)
@@ -278,12 +285,16 @@ __device__ __forceinline__ void gate_phase2(uint32_t qs, uint32_t ks, const uint
 
 // STATE_ONLY: only final states and decay products are wanted (no q, scores, outputs); a
 // compile-time switch so that the full kernel carries none of its branches.
-template <int INGATE, bool STATE_ONLY>
+// BLOCK: the optional terms of the full block are compiled in (value gate applied to the v tile
+// in shared memory by the gate warps, feed-through added in the output path); the plain
+// instantiations carry none of that code.
+template <int INGATE, bool STATE_ONLY, bool BLOCK>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
                      const __grid_constant__ CUtensorMap map_o8, const __grid_constant__ CUtensorMap map_o1,
+                     const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_fx,
                      const PairArgs a) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -342,6 +353,8 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     mbar_init(bar(BAR_GO1), 1);
     mbar_init(bar(BAR_PRE), 1);
     mbar_init(bar(BAR_DRAIN), 1);
+    mbar_init(bar(BAR_XFULL0), 1);
+    mbar_init(bar(BAR_XFULL1), 1);
     mbar_init(bar(BAR_ROWS), kGateWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -372,6 +385,14 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       tma_prefetch_2d(&map_k, xc, yp);
       tma_prefetch_2d(&map_v, it.col0, yp);
       tma_prefetch_2d(&map_v, it.col0 + 64, yp);
+      if (BLOCK && a.beta_hat) {
+        tma_prefetch_2d(&map_b, it.col0, yp);
+        tma_prefetch_2d(&map_b, it.col0 + 64, yp);
+      }
+      if (BLOCK && !STATE_ONLY && a.feed_d) {
+        tma_prefetch_2d(&map_fx, it.col0, yp);
+        tma_prefetch_2d(&map_fx, it.col0 + 64, yp);
+      }
     }
   };
   // The first fill touches only this CTA's own barriers and shared memory, so it goes out
@@ -699,6 +720,20 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // address this thread supplies to stmatrix: row block mat_h, row mat_k within it
         const uint32_t ps_mat = stage_base + s * kStageBytes + kStY + (q4 * 16 + mat_h * 8 + mat_k) * 128;
         tc_fence_after();
+        const bool feed = BLOCK && a.feed_d != nullptr;
+        if (feed && q4 == 0) {
+          // Feed-through: the x' tile of this pass is fetched INTO the output tile (same two-slab
+          // swizzled layout), to be combined with the accumulators in place further down.  The
+          // tile must be free first: the copies that read it two passes ago are done.
+          if (!(ok = mbar_wait(bar(BAR_OTFREE0 + ph1), ((g >> 1) & 1) ^ 1, abort_flag, a.hdr))) break;
+          if (lane == 0) {
+            const uint32_t xb = bar(BAR_XFULL0 + ph1);
+            const uint32_t xt = base + kOffOt + ph1 * kOtBytes;
+            mbar_expect_tx(xb, kOtBytes);
+            tma_load_2d(xt, &map_fx, it.col0, (int)row, xb);
+            tma_load_2d(xt + kSlabBytes, &map_fx, it.col0 + 64, (int)row, xb);
+          }
+        }
         if (warp == kScoreWarp0 && lane == 0) {
           // P exists, so the partner's copies out of ITS stage have all landed here (the issuer
           // waited for them): let the partner reuse that stage
@@ -745,8 +780,13 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // still reading while the next pass is written.
         if (!(ok = mbar_wait(bar(BAR_OFULL), ph1, abort_flag, a.hdr))) break;
         tc_fence_after();
-        // the copies that read this tile two passes ago have finished reading
-        if (!(ok = mbar_wait(bar(BAR_OTFREE0 + ph1), ((g >> 1) & 1) ^ 1, abort_flag, a.hdr))) break;
+        // the copies that read this tile two passes ago have finished reading (with the
+        // feed-through, the x' tile that was fetched into it afterwards has landed)
+        if (feed) {
+          if (!(ok = mbar_wait(bar(BAR_XFULL0 + ph1), (g >> 1) & 1, abort_flag, a.hdr))) break;
+        } else {
+          if (!(ok = mbar_wait(bar(BAR_OTFREE0 + ph1), ((g >> 1) & 1) ^ 1, abort_flag, a.hdr))) break;
+        }
         const uint32_t ot = base + kOffOt + ph1 * kOtBytes;
         // this thread addresses output row 8 * (2 jp + mat_j) + mat_k of column block mat_h
         const uint32_t ot_mat = ot + (q4 >> 1) * kSlabBytes + (mat_j * 8 + mat_k) * 128;
@@ -766,6 +806,26 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // 16-byte chunk (8 value columns) of this thread's matrices within the slab
           const uint32_t chunk = (uint32_t)(4 * (q4 & 1) + 2 * hv + mat_h);
           const uint32_t dst = ot_mat + ((chunk ^ (uint32_t)mat_k) << 4);
+          if (feed) {
+            // o = scale q S + d . x': the x' fragments come out of the tile with the transposing
+            // matrix load, which hands thread t exactly the elements (value column, row pair) its
+            // accumulator registers hold; d belongs to the value column, two per thread
+            const float* dh = a.feed_d + (it.seq_head % a.feed_H) * (long long)a.dv + it.col0 + q4 * 32 + 16 * hv + (lane >> 2);
+            const float d_lo = __ldg(dh), d_hi = __ldg(dh + 8);
+#pragma unroll
+            for (int jp = 0; jp < 4; ++jp) {
+              uint32_t xf[4];
+              ldmatrix_x4_trans(dst + jp * 16 * 128, xf);
+#pragma unroll
+              for (int mi = 0; mi < 4; ++mi) {            // (lo, j0) (hi, j0) (lo, j1) (hi, j1)
+                const int ri = 4 * (2 * jp + (mi >> 1)) + 2 * (mi & 1);
+                const float dd = (mi & 1) ? d_hi : d_lo;
+                const float2 xv = bf16x2_to_f2(xf[mi]);
+                r[ri] = __float_as_uint(fmaf(dd, xv.x, __uint_as_float(r[ri])));
+                r[ri + 1] = __float_as_uint(fmaf(dd, xv.y, __uint_as_float(r[ri + 1])));
+              }
+            }
+          }
 #pragma unroll
           for (int jp = 0; jp < 4; ++jp) {                // output rows 16 jp .. 16 jp + 15
             const int j0 = 2 * jp, j1 = 2 * jp + 1;
@@ -834,6 +894,30 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         *reinterpret_cast<float2*>(tot) = run;
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(BAR_GSCAN));
+        if (BLOCK && a.beta_hat) {
+          // Value gate (Eq. "beta_def"): the v tile becomes beta_hat . v in place, while the
+          // control warp scans.  512 threads, two 16-byte chunks (8 value columns) each; the
+          // gate comes straight from global memory (asked into L2 when the stage was filled).
+          const long long row = ctl->ord[oc & 1].row;
+          const int col0 = ctl->ord[oc & 1].col0;
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int ci = gw * 32 + lane + 512 * u;      // chunk of the [64 rows][16 chunks] tile
+            const int r = ci >> 4, c16 = ci & 15;
+            if (r < nr) {
+              const uint4 g4 = __ldg(reinterpret_cast<const uint4*>(
+                  a.beta_hat + (row + r) * a.dv + col0 + c16 * 8));
+              const uint32_t va = st + kStV + (c16 >> 3) * kSlabBytes + r * 128 +
+                                  ((((uint32_t)c16 & 7u) ^ ((uint32_t)r & 7u)) << 4);
+              uint4 v4 = lds128(va);
+              v4.x = hmul2_bf16(v4.x, g4.x);
+              v4.y = hmul2_bf16(v4.y, g4.y);
+              v4.z = hmul2_bf16(v4.z, g4.z);
+              v4.w = hmul2_bf16(v4.w, g4.w);
+              sts128(va, v4.x, v4.y, v4.z, v4.w);
+            }
+          }
+        }
         // the control warp replaces each row group's sum by the sum of the groups before it
         if (!mbar_wait(bar(BAR_PRE), oc & 1, abort_flag, a.hdr)) break;
         const float2 pre = *reinterpret_cast<const float2*>(tot);
@@ -858,10 +942,14 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       };
       // Order number oc goes into slot oc & 1.  The workers read order oc-2 before they reported
       // on it, and at most two orders are outstanding.
-      auto give_order = [&](int stage, int nr) {
+      auto give_order = [&](int stage, int nr, long long row = 0, int col0 = 0) {
         if (leader) {
           ctl->ord[oc & 1].stage = stage;
           ctl->ord[oc & 1].nr = nr;
+          if (BLOCK) {
+            ctl->ord[oc & 1].row = row;
+            ctl->ord[oc & 1].col0 = col0;
+          }
           mbar_arrive(bar(BAR_GO0 + (oc & 1)));
         }
         ++oc;
@@ -905,7 +993,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             continue;
           }
           nr = min(min(kC, left), lcap);
-          give_order((int)s, nr);
+          give_order((int)s, nr, it.row0 + tpos, it.col0);
         }
         const uint32_t st = stage_base + s * kStageBytes;
         const uint32_t ocur = oc - 1;                     // the order of this attempt
@@ -920,7 +1008,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           ahead_s = fs;
           ahead_nr = min(min(kC, nit.len - ntpos), nlcap);
           if (++fs == kStages) { fs = 0; fph ^= 1; }
-          give_order((int)ahead_s, ahead_nr);
+          give_order((int)ahead_s, ahead_nr, nit.row0 + ntpos, nit.col0);
         };
         // ---- attempt m
         const uint32_t rxi = m & 1, rxph = (m >> 1) & 1;
@@ -1134,6 +1222,7 @@ bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uin
 
 struct PairMaps {
   CUtensorMap q, k, x, y, v, o, o8, o1;
+  CUtensorMap b, fx;   // value gate (only ever prefetched through it) and feed-through input
 };
 
 // A tensor map depends only on (address, rows, columns, box rows): each host thread keeps the
@@ -1170,13 +1259,14 @@ bool cached_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, u
   return true;
 }
 
-template <int INGATE, bool STATE_ONLY>
+template <int INGATE, bool STATE_ONLY, bool BLOCK>
 cudaError_t launch_pair(const PairMaps& m, const PairArgs& a, int max_pairs, int dev, cudaStream_t st) {
   static std::atomic<unsigned long long> opted{0};   // one per instantiation
-  cudaError_t e = opt_in_shared_memory(ddts_fwd_pair_kernel<INGATE, STATE_ONLY>, kSmemBytes, dev, opted);
+  cudaError_t e = opt_in_shared_memory(ddts_fwd_pair_kernel<INGATE, STATE_ONLY, BLOCK>, kSmemBytes, dev, opted);
   if (e != cudaSuccess) return e;
   const long long pairs = a.n_items < max_pairs ? a.n_items : max_pairs;
-  ddts_fwd_pair_kernel<INGATE, STATE_ONLY><<<(unsigned)(2 * pairs), kThreads, kSmemBytes, st>>>(m.q, m.k, m.x, m.y, m.v, m.o, m.o8, m.o1, a);
+  ddts_fwd_pair_kernel<INGATE, STATE_ONLY, BLOCK><<<(unsigned)(2 * pairs), kThreads, kSmemBytes, st>>>(
+      m.q, m.k, m.x, m.y, m.v, m.o, m.o8, m.o1, m.b, m.fx, a);
   return cudaGetLastError();
 }
 
@@ -1322,18 +1412,29 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
         !cached_map(&m.v, p.v, rows, dv) || !cached_map(&m.o, p.o, rows, dv) ||
         !cached_map(&m.o8, p.o, rows, dv, 8) || !cached_map(&m.o1, p.o, rows, dv, 1))
       return cudaErrorUnknown;
+    m.b = m.v;      // placeholders where a term is absent (never used then)
+    m.fx = m.v;
+    if (p.beta_hat && !cached_map(&m.b, p.beta_hat, rows, dv)) return cudaErrorUnknown;
+    if (p.feed_x && !cached_map(&m.fx, p.feed_x, rows, dv)) return cudaErrorUnknown;
   } else {
     memset(&m, 0, sizeof(m));   // never dereferenced: no chunks
   }
   const int max_pairs = sms / 2 > 0 ? sms / 2 : 1;   // one CTA per SM; a pair shares a TPC
+  const bool block = p.beta_hat || p.feed_d;
   auto run = [&](const PairArgs& a, cudaStream_t st) {
+    const bool g = p.ingate == RODIMUS_INGATE_POW_G;
+    if (block) {
+      if (a.state_only)
+        return g ? launch_pair<RODIMUS_INGATE_POW_G, true, true>(m, a, max_pairs, dev, st)
+                 : launch_pair<RODIMUS_INGATE_POW_SIGMOID, true, true>(m, a, max_pairs, dev, st);
+      return g ? launch_pair<RODIMUS_INGATE_POW_G, false, true>(m, a, max_pairs, dev, st)
+               : launch_pair<RODIMUS_INGATE_POW_SIGMOID, false, true>(m, a, max_pairs, dev, st);
+    }
     if (a.state_only)
-      return p.ingate == RODIMUS_INGATE_POW_G
-                 ? launch_pair<RODIMUS_INGATE_POW_G, true>(m, a, max_pairs, dev, st)
-                 : launch_pair<RODIMUS_INGATE_POW_SIGMOID, true>(m, a, max_pairs, dev, st);
-    return p.ingate == RODIMUS_INGATE_POW_G
-               ? launch_pair<RODIMUS_INGATE_POW_G, false>(m, a, max_pairs, dev, st)
-               : launch_pair<RODIMUS_INGATE_POW_SIGMOID, false>(m, a, max_pairs, dev, st);
+      return g ? launch_pair<RODIMUS_INGATE_POW_G, true, false>(m, a, max_pairs, dev, st)
+               : launch_pair<RODIMUS_INGATE_POW_SIGMOID, true, false>(m, a, max_pairs, dev, st);
+    return g ? launch_pair<RODIMUS_INGATE_POW_G, false, false>(m, a, max_pairs, dev, st)
+             : launch_pair<RODIMUS_INGATE_POW_SIGMOID, false, false>(m, a, max_pairs, dev, st);
   };
   char* ws = reinterpret_cast<char*>(p.workspace);
   PairArgs a;
@@ -1346,6 +1447,9 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   a.n_items = n_seq0 * p.H * a.pairs;
   a.scale = p.scale;
   a.wait_cycles = main_loop_wait_cycles();
+  a.beta_hat = reinterpret_cast<const __nv_bfloat16*>(p.beta_hat);
+  a.feed_d = p.feed_d;
+  a.feed_H = p.H;
   a.dtot = nullptr;
   a.sT_only = -1;
   a.state_only = 0;

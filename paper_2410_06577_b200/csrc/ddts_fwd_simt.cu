@@ -23,6 +23,8 @@ constexpr int kThreads = 256;
 
 struct SimtArgs {
   const void *q, *k, *gx, *ty, *v;
+  const void *beta_hat, *feed_x;   // optional: value gate [.., dv], feed-through input [.., dv]
+  const float* feed_d;             // optional: feed-through weight [H, dv]
   void* o;
   const float* s0;
   float* sT;
@@ -74,6 +76,9 @@ __global__ void __launch_bounds__(kThreads, 1) ddts_fwd_simt_kernel(const SimtAr
   const T* ty = (const T*)a.ty + row0 * dk;
   const T* v = (const T*)a.v + row0 * dv;
   T* o = (T*)a.o + row0 * dv;
+  const T* bh = a.beta_hat ? (const T*)a.beta_hat + row0 * dv : nullptr;
+  const T* fx = a.feed_d ? (const T*)a.feed_x + row0 * dv : nullptr;
+  const float* fd = a.feed_d ? a.feed_d + (long long)h * dv : nullptr;
   const long long s_off = sh * (long long)dk * dv;
 
   for (int e = tid; e < dk * kTileV; e += kThreads) {
@@ -100,7 +105,13 @@ __global__ void __launch_bounds__(kThreads, 1) ddts_fwd_simt_kernel(const SimtAr
     }
     for (int e = tid; e < kC * kTileV; e += kThreads) {
       const int r = e / kTileV, c = e % kTileV;
-      sV[e] = (r < nr && col0 + c < dv) ? to_f32(v[(long long)(t0 + r) * dv + col0 + c]) : 0.f;
+      float vv = 0.f;
+      if (r < nr && col0 + c < dv) {
+        const long long i = (long long)(t0 + r) * dv + col0 + c;
+        vv = to_f32(v[i]);
+        if (bh) vv *= to_f32(bh[i]);   // value gate (Eq. "beta_def")
+      }
+      sV[e] = vv;
     }
     __syncthreads();
     // (2) intra-chunk scores, causal mask with the diagonal kept
@@ -128,7 +139,10 @@ __global__ void __launch_bounds__(kThreads, 1) ddts_fwd_simt_kernel(const SimtAr
         for (int i = 0; i <= r; ++i) acc = fmaf(sP[r * kC + i], sV[i * kTileV + c], acc);
         const float* qr = sQ + r * ld;
         for (int d = 0; d < dk; ++d) acc = fmaf(qr[d], sS[d * kTileV + c], acc);
-        o[(long long)(t0 + r) * dv + col0 + c] = from_f32<T>(a.scale * acc);
+        const long long i = (long long)(t0 + r) * dv + col0 + c;
+        acc *= a.scale;
+        if (fd) acc = fmaf(fd[col0 + c], to_f32(fx[i]), acc);   // feed-through d . x'
+        o[i] = from_f32<T>(acc);
       }
     }
     __syncthreads();
@@ -166,6 +180,7 @@ cudaError_t launch_fwd_simt(const rodimus_ddts_fwd_params& p, int* n_launches) {
   *n_launches = 0;
   SimtArgs a;
   a.q = p.q; a.k = p.k; a.gx = p.gate_x; a.ty = p.temp_y; a.v = p.v; a.o = p.o;
+  a.beta_hat = p.beta_hat; a.feed_x = p.feed_x; a.feed_d = p.feed_d;
   a.s0 = p.s0; a.sT = p.sT; a.cu = p.cu_seqlens;
   a.hdr = reinterpret_cast<WorkspaceHeader*>(p.workspace);
   a.H = p.H; a.T = p.T; a.dk = p.dk; a.dv = p.dv;

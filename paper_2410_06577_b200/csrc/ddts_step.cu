@@ -26,7 +26,8 @@ __global__ void __launch_bounds__(kStepThreads, 4)
 ddts_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ gx,
                  const T* __restrict__ ty, const T* __restrict__ v, T* __restrict__ o,
                  float* __restrict__ state, int n_seq_heads, int dk, int dv, float scale,
-                 int ingate) {
+                 int ingate, const T* __restrict__ beta_hat, const float* __restrict__ feed_d,
+                 const T* __restrict__ feed_x, int H) {
   __shared__ float s_alpha[kMaxDk];
   __shared__ float s_w[kMaxDk];   // ahat * k
   __shared__ float s_q[kMaxDk];   // scale * q
@@ -64,6 +65,10 @@ ddts_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __re
     if (col_ok) {
       const T* vp = v + nh * dv + col;
       vv = make_float4(to_f32(vp[0]), to_f32(vp[1]), to_f32(vp[2]), to_f32(vp[3]));
+      if (beta_hat) {   // value gate (Eq. "beta_def"): v enters the state as beta_hat * v
+        const T* bp = beta_hat + nh * dv + col;
+        vv.x *= to_f32(bp[0]); vv.y *= to_f32(bp[1]); vv.z *= to_f32(bp[2]); vv.w *= to_f32(bp[3]);
+      }
     }
     __syncthreads();
 
@@ -107,6 +112,12 @@ ddts_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __re
         const float4 u = s_red[w][lane];
         t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
       }
+      if (feed_d) {     // feed-through: o = scale q S + d . x'
+        const float* dp = feed_d + (nh % H) * dv + col;
+        const T* fp = feed_x + nh * dv + col;
+        t.x = fmaf(dp[0], to_f32(fp[0]), t.x); t.y = fmaf(dp[1], to_f32(fp[1]), t.y);
+        t.z = fmaf(dp[2], to_f32(fp[2]), t.z); t.w = fmaf(dp[3], to_f32(fp[3]), t.w);
+      }
       T* op = o + nh * dv + col;
       op[0] = from_f32<T>(t.x);
       op[1] = from_f32<T>(t.y);
@@ -139,12 +150,14 @@ cudaError_t launch_step(const rodimus_ddts_step_params& p, int* n_launches) {
     using T = __nv_bfloat16;
     ddts_step_kernel<T><<<grid, kStepThreads, 0, st>>>(
         (const T*)p.q, (const T*)p.k, (const T*)p.gate_x, (const T*)p.temp_y, (const T*)p.v,
-        (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate);
+        (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate, (const T*)p.beta_hat, p.feed_d,
+        (const T*)p.feed_x, p.H);
   } else {
     using T = float;
     ddts_step_kernel<T><<<grid, kStepThreads, 0, st>>>(
         (const T*)p.q, (const T*)p.k, (const T*)p.gate_x, (const T*)p.temp_y, (const T*)p.v,
-        (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate);
+        (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate, (const T*)p.beta_hat, p.feed_d,
+        (const T*)p.feed_x, p.H);
   }
   *n_launches = 1;
   return cudaGetLastError();

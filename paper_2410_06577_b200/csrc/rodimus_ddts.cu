@@ -65,6 +65,16 @@ bool fwd_tc_supported(const rodimus_ddts_fwd_params& p) {
 
 bool fwd_pair_selected(const rodimus_ddts_fwd_params& p) { return fwd_pair_supported(p); }
 
+bool has_block_terms(const rodimus_ddts_fwd_params& p) { return p.beta_hat || p.feed_d; }
+
+// 0: cluster-pair tensor-core kernel, 1: single-CTA tensor-core kernel (the recurrence alone),
+// 2: fp32 CUDA-core kernel
+int fwd_kernel_choice(const rodimus_ddts_fwd_params& p) {
+  if (fwd_pair_selected(p)) return 0;
+  if (fwd_tc_supported(p) && !has_block_terms(p)) return 1;
+  return 2;
+}
+
 }  // namespace ddts
 
 extern "C" {
@@ -83,7 +93,7 @@ size_t rodimus_ddts_fwd_workspace_bytes(const rodimus_ddts_fwd_params* p) {
 const char* rodimus_ddts_fwd_kernel_name(const rodimus_ddts_fwd_params* p) {
   if (!p) return "invalid";
   if (check_fwd_sizes(p, p->cu_seqlens != nullptr) != RODIMUS_OK) return "invalid";
-  return ddts::fwd_tc_supported(*p) ? "tcgen05" : "simt";
+  return ddts::fwd_kernel_choice(*p) < 2 ? "tcgen05" : "simt";
 }
 
 int rodimus_ddts_fwd(const rodimus_ddts_fwd_params* p) {
@@ -97,7 +107,9 @@ int rodimus_ddts_fwd(const rodimus_ddts_fwd_params* p) {
   const long long n_seq = varlen ? p->N : p->B;
   if (rows > 0 && (!p->q || !p->k || !p->gate_x || !p->temp_y || !p->v || !p->o))
     return RODIMUS_ERR_NULL;
-  const void* ptrs[] = {p->q, p->k, p->gate_x, p->temp_y, p->v, p->o, p->s0, p->sT, p->cu_seqlens};
+  if ((p->feed_d != nullptr) != (p->feed_x != nullptr)) return RODIMUS_ERR_NULL;  // both or neither
+  const void* ptrs[] = {p->q, p->k, p->gate_x, p->temp_y, p->v, p->o, p->s0, p->sT, p->cu_seqlens,
+                        p->beta_hat, p->feed_d, p->feed_x};
   for (const void* ptr : ptrs)
     if (ptr && !aligned16(ptr)) return RODIMUS_ERR_ALIGN;
   if (!p->workspace || p->workspace_bytes < workspace_bytes_for(varlen ? p->N : 0))
@@ -119,9 +131,10 @@ int rodimus_ddts_fwd(const rodimus_ddts_fwd_params* p) {
     launches += n;
   }  // dense: the prefill kernel's first CTA clears the status word itself
   if (e != cudaSuccess) return RODIMUS_ERR_CUDA;
-  if (ddts::fwd_pair_selected(*p))
+  const int choice = ddts::fwd_kernel_choice(*p);
+  if (choice == 0)
     e = ddts::launch_fwd_pair(*p, &n);
-  else if (ddts::fwd_tc_supported(*p))
+  else if (choice == 1)
     e = ddts::launch_fwd_tc(*p, &n);
   else
     e = ddts::launch_fwd_simt(*p, &n);
@@ -145,9 +158,13 @@ int rodimus_ddts_step(const rodimus_ddts_step_params* p) {
   if ((long long)p->Nseq * p->H == 0) return RODIMUS_OK;
   if (!p->q || !p->k || !p->gate_x || !p->temp_y || !p->v || !p->o || !p->state)
     return RODIMUS_ERR_NULL;
+  if ((p->feed_d != nullptr) != (p->feed_x != nullptr)) return RODIMUS_ERR_NULL;
   const void* ptrs[] = {p->q, p->k, p->gate_x, p->temp_y, p->v, p->o, p->state};
   for (const void* ptr : ptrs)
     if (!aligned16(ptr)) return RODIMUS_ERR_ALIGN;
+  const void* opt[] = {p->beta_hat, p->feed_d, p->feed_x};
+  for (const void* ptr : opt)
+    if (ptr && !aligned16(ptr)) return RODIMUS_ERR_ALIGN;
   int n = 0;
   cudaError_t e = ddts::launch_step(*p, &n);
   if (e != cudaSuccess) return RODIMUS_ERR_CUDA;
@@ -188,6 +205,6 @@ const char* rodimus_status_str(int status) {
   }
 }
 
-int rodimus_version(void) { return 100; }
+int rodimus_version(void) { return 101; }
 
 }  // extern "C"

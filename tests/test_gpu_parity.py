@@ -593,3 +593,96 @@ def test_wait_that_runs_out_is_reported_and_the_next_call_is_clean(dv):
     assert rd.device_status(ws) == rd.OK
     ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0)
     assert rel_err(host(o), ro) <= TOL_BF16 and rel_err(host(sT), rs) <= TOL_BF16
+
+
+# ------------------------------------------------------------------------------------------
+# optional terms of the full block: value gate beta_hat (multiplies v) and feed-through d . x'
+# ------------------------------------------------------------------------------------------
+
+def _block_terms(p, seed, H):
+    """Seeded beta_hat in (0, 1) (a sigmoid's range), d ~ N(0, 1), x' ~ N(0, 1), rounded to the
+    workload's dtype where the GPU reads them in it."""
+    rng = np.random.default_rng(seed)
+    dv = p.v.shape[-1]
+    rnd = wl.round_to_bf16 if p.dtype == "bf16" else (lambda a: a.astype(np.float32))
+    beta = rnd(rng.random(p.v.shape, dtype=np.float32))
+    fx = rnd(rng.standard_normal(p.v.shape, dtype=np.float32))
+    d = rng.standard_normal((H, dv), dtype=np.float32)
+    return beta, d, fx
+
+
+def _check_block(p, which="both", ingate=rd.INGATE_POW_G, scale=0.5, expect_kernel=None, ws_bytes=None):
+    import torch
+    B, H, T, dk, dv = p.shape
+    beta, d, fx = _block_terms(p, 5, H)
+    use_b, use_f = which in ("both", "gate"), which in ("both", "feed")
+    dd = prefill_to_device(p)
+    o, sT = _nan_outputs(dd)
+    kw = dict(beta_hat=dev(beta, p.dtype) if use_b else None,
+              feed_d=torch.from_numpy(d).cuda() if use_f else None,
+              feed_x=dev(fx, p.dtype) if use_f else None)
+    prm = rd.fwd_params(dd["q"], dd["k"], dd["x"], dd["y"], dd["v"], o, dd["s0"], sT, dd["cu"],
+                        dd["cu_host"], None, scale, ingate, **kw)
+    if expect_kernel:
+        assert rd.fwd_kernel_name(prm) == expect_kernel
+    need = rd.fwd_workspace_bytes(prm) if ws_bytes is None else ws_bytes
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+    prm.workspace, prm.workspace_bytes = ws.data_ptr(), ws.numel()
+    assert rd.fwd_raw(prm) == rd.OK and rd.device_status(ws) == rd.OK
+    ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0, cu_seqlens=p.cu_seqlens, scale=scale,
+                         ingate=ingate, beta_hat=beta if use_b else None,
+                         feed_d=d if use_f else None, feed_x=fx if use_f else None)
+    tol = _tol(p.dtype)
+    eo, es = _worst_err(host(o), host(sT), ro, rs, p.cu_seqlens)
+    assert eo <= tol and es <= tol, (which, eo, es)
+    return rd.last_launch_count()
+
+
+@pytest.mark.parametrize("which", ["both", "gate", "feed"])
+@pytest.mark.parametrize("ingate", [rd.INGATE_POW_G, rd.INGATE_POW_SIGMOID])
+def test_block_terms_bf16_tensor_core_kernel(which, ingate):
+    p = wl.make_prefill(501, 2, 2, 200, 128, 256, "bf16", s0_std=0.1)       # ragged last tile
+    _check_block(p, which, ingate, expect_kernel="tcgen05")
+    p = wl.make_prefill(502, 1, 3, 64, 128, 512, "bf16")                    # two slabs per head
+    _check_block(p, which, ingate, expect_kernel="tcgen05")
+
+
+def test_block_terms_bf16_packed_sequences_many_items():
+    lens = _mixed_lengths(503, 100)
+    p = _varlen(504, lens, 4, 128, 256, "bf16", s0_std=0.2)
+    _check_block(p, "both")
+
+
+def test_block_terms_with_the_time_split():
+    p = wl.make_prefill(505, 1, 2, 4500, 128, 256, "bf16", s0_std=0.2)
+    assert _check_block(p, "both") == 5                                     # split: five launches
+    assert _check_block(p, "both", ws_bytes=256) == 1                       # same request, unsplit
+
+
+@pytest.mark.parametrize("dtype,dk,dv", [("f32", 64, 64), ("bf16", 128, 128), ("bf16", 48, 80)])
+def test_block_terms_cuda_core_kernel(dtype, dk, dv):
+    p = wl.make_prefill(506, 1, 2, 90, dk, dv, dtype, s0_std=0.2)
+    _check_block(p, "both", expect_kernel="simt")
+    _check_block(p, "gate", rd.INGATE_POW_SIGMOID)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_block_terms_decode_steps(dtype):
+    import torch
+    Nseq, H, dk, dv = 5, 3, 128, 256
+    w = wl.make_decode(507, Nseq, H, dk, dv, ring=4, dtype=dtype)
+    rng = np.random.default_rng(6)
+    rnd = wl.round_to_bf16 if dtype == "bf16" else (lambda a: a.astype(np.float32))
+    beta = rnd(rng.random((4, Nseq, H, dv), dtype=np.float32))
+    fx = rnd(rng.standard_normal((4, Nseq, H, dv), dtype=np.float32))
+    d = rng.standard_normal((H, dv), dtype=np.float32)
+    state = torch.from_numpy(w.state).cuda()
+    ref_state = w.state.astype(np.float64)
+    for s in range(4):
+        o = rd.ddts_step(*(dev(a[s], dtype) for a in (w.q, w.k, w.x, w.y, w.v)), state, scale=0.5,
+                         beta_hat=dev(beta[s], dtype), feed_d=torch.from_numpy(d).cuda(),
+                         feed_x=dev(fx[s], dtype))
+        ro = orc.ref_step(w.q[s], w.k[s], w.x[s], w.y[s], w.v[s], ref_state, scale=0.5,
+                          beta_hat=beta[s], feed_d=d, feed_x=fx[s])
+        assert rel_err(host(o), ro) <= _tol(dtype)
+    assert rel_err(host(state), ref_state) <= TOL_F32
