@@ -238,10 +238,10 @@ __device__ __forceinline__ float2 gate_phase1(uint32_t xs, uint32_t ys, const ui
     const float2 ser = __fmul2_rn(u, __ffma2_rn(u, splat(-0.72134752f), splat(kLog2e)));
     const float2 sp2 = make_float2(u.x < 9.765625e-4f ? ser.x : lg2f(w.x),
                                    u.y < 9.765625e-4f ? ser.y : lg2f(w.y));
-    // -tau = -sigmoid(y) = 1 / (-1 - e^{-y})
-    const float2 yl = __fmul2_rn(y, splat(-kLog2e));
-    const float2 nw = __ffma2_rn(make_float2(ex2f(yl.x), ex2f(yl.y)), splat(-1.f), splat(-1.f));
-    const float2 ntau = make_float2(rcpf(nw.x), rcpf(nw.y));
+    // -tau = -sigmoid(y) = -1/2 - tanh(y/2)/2: one special-function operation instead of two
+    // (the approximation's error, 2^-11 of tanh, is an absolute 2.5e-4 of tau)
+    const float2 yh = __fmul2_rn(y, splat(0.5f));
+    const float2 ntau = __ffma2_rn(make_float2(tanh_approx(yh.x), tanh_approx(yh.y)), splat(-0.5f), splat(-0.5f));
     float2 l2a = __fmul2_rn(sp2, ntau);                                 // log2 alpha <= 0
     l2a.x = fmaxf(l2a.x, -kRange);                                      // per-step floor exp(-60)
     l2a.y = fmaxf(l2a.y, -kRange);
@@ -896,13 +896,13 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (lane == 0) mbar_arrive(bar(BAR_GSCAN));
         if (BLOCK && a.beta_hat) {
           // Value gate (Eq. "beta_def"): the v tile becomes beta_hat . v in place, while the
-          // control warp scans.  512 threads, two 16-byte chunks (8 value columns) each; the
+          // control warp scans.  Every gate thread takes its share of 16-byte chunks (8 value columns); the
           // gate comes straight from global memory (asked into L2 when the stage was filled).
           const long long row = ctl->ord[oc & 1].row;
           const int col0 = ctl->ord[oc & 1].col0;
 #pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const int ci = gw * 32 + lane + 512 * u;      // chunk of the [64 rows][16 chunks] tile
+          for (int u = 0; u < kC * 16 / (kGateWarps * 32); ++u) {
+            const int ci = gw * 32 + lane + kGateWarps * 32 * u;   // chunk of the [64 rows][16 chunks] tile
             const int r = ci >> 4, c16 = ci & 15;
             if (r < nr) {
               const uint4 g4 = __ldg(reinterpret_cast<const uint4*>(

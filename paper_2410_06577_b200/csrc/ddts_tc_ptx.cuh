@@ -69,6 +69,12 @@ __device__ __forceinline__ bool mbar_try_park(uint32_t bar, uint32_t parity) {
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile WaitCtl* wc,
                                             WorkspaceHeader* hdr) {
   const long long limit = wc->limit;
+  // the clock is read only after a first round of parked polls: nearly every wait ends there
+  if (limit > 0) {
+#pragma unroll 1
+    for (int i = 0; i < 4; ++i)
+      if (mbar_try_park(bar, parity)) return true;
+  }
   const long long t0 = clock64();
   while (true) {
     if (limit > 0) {
@@ -236,6 +242,11 @@ __device__ __forceinline__ float ex2f(float x) {
 __device__ __forceinline__ float lg2f(float x) {
   float y;
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float tanh_approx(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 __device__ __forceinline__ float rcpf(float x) {
@@ -409,6 +420,12 @@ __device__ __forceinline__ bool mbar_try_park_cluster(uint32_t bar, uint32_t par
 __device__ __noinline__ bool mbar_wait_cluster_slow(uint32_t bar, uint32_t parity,
                                                     volatile WaitCtl* wc, WorkspaceHeader* hdr) {
   const long long limit = wc->limit;
+  // the clock is read only after a first round of parked polls: nearly every wait ends there
+  if (limit > 0) {
+#pragma unroll 1
+    for (int i = 0; i < 4; ++i)
+      if (mbar_try_park_cluster(bar, parity)) return true;
+  }
   const long long t0 = clock64();
   while (true) {
     if (limit > 0) {
