@@ -240,13 +240,13 @@ def run_reference(args, workload, p):
 # Work per token-head behind the three bound times printed beside every prefill roofline
 # (dk = 128, dv = 256): tensor flops of the chunkwise form at chunk length 64 (state update and
 # readout 2*dk*dv each, causal intra-chunk (C+1)(dk+dv)) and special-function approximations of
-# the gate math (7 per key channel with the paper's input gate: softplus 2, sigmoid 2, log g 1,
+# the gate math (6 per key channel with the paper's input gate: softplus 2, sigmoid 1, log g 1,
 # the two operand exponentials 2).
 DATASHEET = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 
 
 def work_per_token_head(dk: int, dv: int, chunk: int = 64):
-    return {"tensor_flops": 4 * dk * dv + (chunk + 1) * (dk + dv), "sfu_ops": 7 * dk}
+    return {"tensor_flops": 4 * dk * dv + (chunk + 1) * (dk + dv), "sfu_ops": 6 * dk}
 
 
 def measure_sfu_rate(rd, torch, device):
