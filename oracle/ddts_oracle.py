@@ -62,12 +62,16 @@ def _load():
         lib.ddts_ref_fwd.restype = ctypes.c_int
         lib.ddts_ref_fwd_block.argtypes = lib.ddts_ref_fwd.argtypes + [f32p, f32p, f32p]
         lib.ddts_ref_fwd_block.restype = ctypes.c_int
+        lib.ddts_ref_fwd_shared.argtypes = lib.ddts_ref_fwd_block.argtypes
+        lib.ddts_ref_fwd_shared.restype = ctypes.c_int
         lib.ddts_ref_step.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                       ctypes.c_int, ctypes.c_double,
                                       f32p, f32p, f32p, f32p, f32p, f64p, f64p]
         lib.ddts_ref_step.restype = ctypes.c_int
         lib.ddts_ref_step_block.argtypes = lib.ddts_ref_step.argtypes + [f32p, f32p, f32p]
         lib.ddts_ref_step_block.restype = ctypes.c_int
+        lib.ddts_ref_step_shared.argtypes = lib.ddts_ref_step_block.argtypes
+        lib.ddts_ref_step_shared.restype = ctypes.c_int
         lib.ddts_ref_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -100,12 +104,16 @@ def ref_gates(x, y, ingate: int = POW_G):
 
 
 def ref_fwd(q, k, x, y, v, s0=None, cu_seqlens=None, scale: float = 1.0, ingate: int = POW_G,
-            want_o: bool = True, want_sT: bool = True, beta_hat=None, feed_d=None, feed_x=None):
+            want_o: bool = True, want_sT: bool = True, beta_hat=None, feed_d=None, feed_x=None,
+            shared_gates: bool = False):
     """Sequential prefill.  q,k,x,y: [B,H,T,dk]; v: [B,H,T,dv]; s0: [B|N,H,dk,dv] or None.
 
     Optional terms of the full block: beta_hat [B,H,T,dv] (value gate, Eq. "beta_def": v_t is
     replaced by beta_hat_t * v_t) and the feed-through feed_d [H,dv], feed_x [B,H,T,dv]
     (Eq. "rodimus_recurrent_form": o_t = scale * q_t S_t + d * x'_t).
+
+    shared_gates: the layout the paper writes the block in - q,k,x,y are [B,1,T,dk], one set per
+    token shared by all H groups of dv value columns (v, o, states keep their H).
 
     Returns (o [B,H,T,dv] float64 or None, sT [B|N,H,dk,dv] float64 or None).
     """
@@ -115,9 +123,11 @@ def ref_fwd(q, k, x, y, v, s0=None, cu_seqlens=None, scale: float = 1.0, ingate:
     xa, xp = _f32(x)
     ya, yp = _f32(y)
     va, vp = _f32(v)
-    B, H, T, dk = qa.shape
+    B, Hq, T, dk = qa.shape
+    H = va.shape[1]
     dv = va.shape[-1]
     assert ka.shape == qa.shape == xa.shape == ya.shape and va.shape[:3] == (B, H, T)
+    assert Hq == (1 if shared_gates else H)
     cu = None
     cup = None
     nseq = B
@@ -133,7 +143,7 @@ def ref_fwd(q, k, x, y, v, s0=None, cu_seqlens=None, scale: float = 1.0, ingate:
         assert s0a.shape == (nseq, H, dk, dv)
     o = np.empty((B, H, T, dv), dtype=np.float64) if want_o else None
     sT = np.empty((nseq, H, dk, dv), dtype=np.float64) if want_sT else None
-    if beta_hat is None and feed_d is None and feed_x is None:
+    if beta_hat is None and feed_d is None and feed_x is None and not shared_gates:
         rc = lib.ddts_ref_fwd(ingate, B, H, T, dk, dv, float(scale), qp, kp, xp, yp, vp,
                               _f64p(s0a), _f64p(o), _f64p(sT), cup, N)
     else:
@@ -143,15 +153,16 @@ def ref_fwd(q, k, x, y, v, s0=None, cu_seqlens=None, scale: float = 1.0, ingate:
         fa, fp = (None, None) if feed_x is None else _f32(feed_x)
         assert ba is None or ba.shape == va.shape
         assert da is None or (da.shape == (H, dv) and fa.shape == va.shape)
-        rc = lib.ddts_ref_fwd_block(ingate, B, H, T, dk, dv, float(scale), qp, kp, xp, yp, vp,
-                                    _f64p(s0a), _f64p(o), _f64p(sT), cup, N, bp, dp, fp)
+        fn = lib.ddts_ref_fwd_shared if shared_gates else lib.ddts_ref_fwd_block
+        rc = fn(ingate, B, H, T, dk, dv, float(scale), qp, kp, xp, yp, vp,
+                _f64p(s0a), _f64p(o), _f64p(sT), cup, N, bp, dp, fp)
     if rc:
         raise ValueError(f"ddts_ref_fwd returned {rc}")
     return o, sT
 
 
 def ref_step(q, k, x, y, v, state, scale: float = 1.0, ingate: int = POW_G, beta_hat=None,
-             feed_d=None, feed_x=None):
+             feed_d=None, feed_x=None, shared_gates: bool = False):
     """One decode step; ``state`` ([Nseq,H,dk,dv] float64, C-contiguous) is updated in place.
     beta_hat, feed_x: [Nseq,H,dv]; feed_d: [H,dv] (optional, as in ``ref_fwd``)."""
     lib = _load()
@@ -160,12 +171,14 @@ def ref_step(q, k, x, y, v, state, scale: float = 1.0, ingate: int = POW_G, beta
     xa, xp = _f32(x)
     ya, yp = _f32(y)
     va, vp = _f32(v)
-    Nseq, H, dk = qa.shape
+    Nseq, Hq, dk = qa.shape
+    H = va.shape[1]
     dv = va.shape[-1]
+    assert Hq == (1 if shared_gates else H)     # shared: q,k,x,y are [Nseq,1,dk]
     assert state.dtype == np.float64 and state.flags["C_CONTIGUOUS"]
     assert state.shape == (Nseq, H, dk, dv)
     o = np.empty((Nseq, H, dv), dtype=np.float64)
-    if beta_hat is None and feed_d is None and feed_x is None:
+    if beta_hat is None and feed_d is None and feed_x is None and not shared_gates:
         rc = lib.ddts_ref_step(ingate, Nseq, H, dk, dv, float(scale), qp, kp, xp, yp, vp,
                                _f64p(o), _f64p(state))
     else:
@@ -173,8 +186,9 @@ def ref_step(q, k, x, y, v, state, scale: float = 1.0, ingate: int = POW_G, beta
         ba, bp = (None, None) if beta_hat is None else _f32(beta_hat)
         da, dp = (None, None) if feed_d is None else _f32(feed_d)
         fa, fp = (None, None) if feed_x is None else _f32(feed_x)
-        rc = lib.ddts_ref_step_block(ingate, Nseq, H, dk, dv, float(scale), qp, kp, xp, yp, vp,
-                                     _f64p(o), _f64p(state), bp, dp, fp)
+        fn = lib.ddts_ref_step_shared if shared_gates else lib.ddts_ref_step_block
+        rc = fn(ingate, Nseq, H, dk, dv, float(scale), qp, kp, xp, yp, vp,
+                _f64p(o), _f64p(state), bp, dp, fp)
     if rc:
         raise ValueError(f"ddts_ref_step returned {rc}")
     return o

@@ -132,11 +132,15 @@ static void ref_one_sequence(int ingate, int64_t len, int dk, int dv, double sca
  * s0/sT are [N,H,dk,dv].  o may be NULL (state only).  Returns 0, or a nonzero
  * code for arguments that make no sense.
  */
-int ddts_ref_fwd_block(int ingate, int B, int H, int64_t T, int dk, int dv, double scale,
-                       const float *q, const float *k, const float *x, const float *y,
-                       const float *v, const double *s0, double *o, double *sT,
-                       const int32_t *cu_seqlens, int N, const float *beta_hat,
-                       const float *feed_d, const float *feed_x) {
+/* shared != 0: the layout the paper writes the block in (Eq. "rodimus_recurrent_form": the decay
+ * exp(-g.tau)^T 1_m and the input weight multiply ALL m value columns, Table of A_t/B_t: state
+ * "n x 2d"): one q, k, x, y of width dk per token, [B,1,T,dk], shared by the H groups of dv value
+ * columns; v, o and the states keep their H.  Each group then runs the same recurrence. */
+static int ref_fwd_impl(int ingate, int B, int H, int64_t T, int dk, int dv, double scale,
+                        const float *q, const float *k, const float *x, const float *y,
+                        const float *v, const double *s0, double *o, double *sT,
+                        const int32_t *cu_seqlens, int N, const float *beta_hat,
+                        const float *feed_d, const float *feed_x, int shared) {
   if (ingate != DDTS_REF_POW_G && ingate != DDTS_REF_POW_SIGMOID) return 3;
   if (B < 0 || H < 0 || T < 0 || dk <= 0 || dv <= 0) return 2;
   int nseq = B;
@@ -169,14 +173,36 @@ int ddts_ref_fwd_block(int ingate, int B, int H, int64_t T, int dk, int dv, doub
         len = T;
       }
       size_t so = (size_t)it * dk * dv;
-      ref_one_sequence(ingate, len, dk, dv, scale, q + row0 * dk, k + row0 * dk, x + row0 * dk,
-                       y + row0 * dk, v + row0 * dv, s0 ? s0 + so : NULL, o ? o + row0 * dv : NULL,
+      /* rows of q, k, x, y: the head's own, or the single shared set of the sequence */
+      int64_t rq = row0;
+      if (shared) rq = cu_seqlens ? (int64_t)cu_seqlens[n] : n * T;
+      ref_one_sequence(ingate, len, dk, dv, scale, q + rq * dk, k + rq * dk, x + rq * dk,
+                       y + rq * dk, v + row0 * dv, s0 ? s0 + so : NULL, o ? o + row0 * dv : NULL,
                        sT ? sT + so : NULL, S, beta_hat ? beta_hat + row0 * dv : NULL,
                        feed_d ? feed_d + (size_t)h * dv : NULL, feed_x ? feed_x + row0 * dv : NULL);
     }
     free(S);
   }
   return failed ? 8 : 0;
+}
+
+int ddts_ref_fwd_block(int ingate, int B, int H, int64_t T, int dk, int dv, double scale,
+                       const float *q, const float *k, const float *x, const float *y,
+                       const float *v, const double *s0, double *o, double *sT,
+                       const int32_t *cu_seqlens, int N, const float *beta_hat,
+                       const float *feed_d, const float *feed_x) {
+  return ref_fwd_impl(ingate, B, H, T, dk, dv, scale, q, k, x, y, v, s0, o, sT, cu_seqlens, N,
+                      beta_hat, feed_d, feed_x, 0);
+}
+
+/* Shared-gate layout: q, k, x, y are [B,1,T,dk]; everything else as ddts_ref_fwd_block. */
+int ddts_ref_fwd_shared(int ingate, int B, int H, int64_t T, int dk, int dv, double scale,
+                        const float *q, const float *k, const float *x, const float *y,
+                        const float *v, const double *s0, double *o, double *sT,
+                        const int32_t *cu_seqlens, int N, const float *beta_hat,
+                        const float *feed_d, const float *feed_x) {
+  return ref_fwd_impl(ingate, B, H, T, dk, dv, scale, q, k, x, y, v, s0, o, sT, cu_seqlens, N,
+                      beta_hat, feed_d, feed_x, 1);
 }
 
 /* The recurrence alone (no value gate, no feed-through). */
@@ -192,16 +218,17 @@ int ddts_ref_fwd(int ingate, int B, int H, int64_t T, int dk, int dv, double sca
  * [Nseq,H,dv], state is [Nseq,H,dk,dv] and is updated in place; o reads the state
  * after the update (Eq. "rodimus_recurrent_form": o_t = q_t S_t).
  */
-int ddts_ref_step_block(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
-                        const float *k, const float *x, const float *y, const float *v, double *o,
-                        double *state, const float *beta_hat, const float *feed_d,
-                        const float *feed_x) {
+static int ref_step_impl(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
+                         const float *k, const float *x, const float *y, const float *v, double *o,
+                         double *state, const float *beta_hat, const float *feed_d,
+                         const float *feed_x, int shared) {
   if (ingate != DDTS_REF_POW_G && ingate != DDTS_REF_POW_SIGMOID) return 3;
   if (Nseq < 0 || H < 0 || dk <= 0 || dv <= 0) return 2;
   int64_t items = (int64_t)Nseq * H;
 #pragma omp parallel for schedule(static)
   for (int64_t it = 0; it < items; ++it) {
-    const float *qt = q + it * dk, *kt = k + it * dk, *xt = x + it * dk, *yt = y + it * dk;
+    const int64_t iq = shared ? it / H : it; /* shared: one q, k, x, y per sequence, [Nseq,1,dk] */
+    const float *qt = q + iq * dk, *kt = k + iq * dk, *xt = x + iq * dk, *yt = y + iq * dk;
     const float *vt = v + it * dv;
     double *ot = o + it * dv;
     double *S = state + (size_t)it * dk * dv;
@@ -232,6 +259,23 @@ int ddts_ref_step_block(int ingate, int Nseq, int H, int dk, int dv, double scal
     }
   }
   return 0;
+}
+
+int ddts_ref_step_block(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
+                        const float *k, const float *x, const float *y, const float *v, double *o,
+                        double *state, const float *beta_hat, const float *feed_d,
+                        const float *feed_x) {
+  return ref_step_impl(ingate, Nseq, H, dk, dv, scale, q, k, x, y, v, o, state, beta_hat, feed_d,
+                       feed_x, 0);
+}
+
+/* Shared-gate layout for decode: q, k, x, y are [Nseq,1,dk]. */
+int ddts_ref_step_shared(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
+                         const float *k, const float *x, const float *y, const float *v, double *o,
+                         double *state, const float *beta_hat, const float *feed_d,
+                         const float *feed_x) {
+  return ref_step_impl(ingate, Nseq, H, dk, dv, scale, q, k, x, y, v, o, state, beta_hat, feed_d,
+                       feed_x, 1);
 }
 
 int ddts_ref_step(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,

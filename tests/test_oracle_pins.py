@@ -342,3 +342,46 @@ def test_block_terms_in_decode_steps_and_packed_prefill():
                               beta_hat=bh[:, :, t], feed_d=d, feed_x=fx[:, :, t])
             assert _rel(ot[0], o[0, :, t]) < 1e-13
         assert _rel(st[0], sT[n]) < 1e-13 or lens[n] == 0
+
+
+# -- shared-gate layout: one q, k, x, y per token for all groups of value columns --------------
+
+@pytest.mark.parametrize("mode", MODES)
+def test_shared_gate_layout_equals_per_head_inputs_replicated(mode):
+    """Eq. "rodimus_recurrent_form" writes the decay and the input weight as (.)^T 1_m: the same
+    for every value column.  Handing every head a copy of the one q, k, x, y must therefore give
+    the per-head recurrence, bit for bit; and the heads must differ only through v and the state."""
+    rng = np.random.default_rng(50)
+    B, H, T, dk, dv = 2, 3, 13, 4, 5
+    f = lambda *sh: rng.standard_normal(sh).astype(np.float32)
+    q, k, x, y = f(B, 1, T, dk), f(B, 1, T, dk), f(B, 1, T, dk) - 1, f(B, 1, T, dk)
+    v, s0 = f(B, H, T, dv), rng.standard_normal((B, H, dk, dv))
+    o, sT = orc.ref_fwd(q, k, x, y, v, s0=s0, ingate=mode, scale=0.5, shared_gates=True)
+    rep = lambda a: np.ascontiguousarray(np.repeat(a, H, axis=1))
+    o2, sT2 = orc.ref_fwd(rep(q), rep(k), rep(x), rep(y), v, s0=s0, ingate=mode, scale=0.5)
+    assert np.array_equal(o, o2) and np.array_equal(sT, sT2)
+    # same v and state in two heads => same outputs in those heads
+    v[:, 1] = v[:, 0]
+    s0[:, 1] = s0[:, 0]
+    o3, sT3 = orc.ref_fwd(q, k, x, y, v, s0=s0, ingate=mode, shared_gates=True)
+    assert np.array_equal(o3[:, 0], o3[:, 1]) and np.array_equal(sT3[:, 0], sT3[:, 1])
+
+
+def test_shared_gate_layout_packed_and_decode_steps():
+    rng = np.random.default_rng(51)
+    H, dk, dv, lens = 2, 4, 3, [4, 0, 6]
+    T = sum(lens)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    f = lambda *sh: rng.standard_normal(sh).astype(np.float32)
+    q, k, x, y, v = f(1, 1, T, dk), f(1, 1, T, dk), f(1, 1, T, dk) - 1, f(1, 1, T, dk), f(1, H, T, dv)
+    o, sT = orc.ref_fwd(q, k, x, y, v, cu_seqlens=cu, shared_gates=True)
+    rep = lambda a: np.ascontiguousarray(np.repeat(a, H, axis=1))
+    o2, sT2 = orc.ref_fwd(rep(q), rep(k), rep(x), rep(y), v, cu_seqlens=cu)
+    assert np.array_equal(o, o2) and np.array_equal(sT, sT2)
+    for n in range(3):
+        st = np.zeros((1, H, dk, dv))
+        for t in range(cu[n], cu[n + 1]):
+            ot = orc.ref_step(q[:, :, t], k[:, :, t], x[:, :, t], y[:, :, t], v[:, :, t], st,
+                              shared_gates=True)
+            assert _rel(ot[0], o[0, :, t]) < 1e-13
+        assert lens[n] == 0 or _rel(st[0], sT[n]) < 1e-13
