@@ -109,6 +109,12 @@ typedef struct {
   const float *feed_d;       /* device fp32 [H,dv]: feed-through weight d of Eq.                     */
                              /* "rodimus_recurrent_form"; given together with feed_x or not at all   */
   const void *feed_x;        /* device [B,H,T,dv], dtype of v: x'_t; o_t = scale q_t S_t + d . x'_t  */
+  int32_t shared_gates;      /* 0: q,k,gate_x,temp_y are [B,H,T,dk], a set per head (above).          */
+                             /* 1: the layout Eq. "rodimus_recurrent_form" is written in - decay and   */
+                             /* input weight are the same for all value columns (state "n x 2d"):     */
+                             /* q,k,gate_x,temp_y are [B,1,T,dk], one set per token shared by the H    */
+                             /* groups of dv value columns; v, o, s0, sT keep their H.                 */
+  int32_t reserved;          /* 0                                                                    */
 } rodimus_ddts_fwd_params;
 
 /*
@@ -132,6 +138,8 @@ typedef struct {
   const void *beta_hat;                /* optional, device [Nseq,H,dv]: value gate (see the prefill) */
   const float *feed_d;                 /* optional, device fp32 [H,dv]: feed-through weight          */
   const void *feed_x;                  /* optional with feed_d, device [Nseq,H,dv]: x'_t             */
+  int32_t shared_gates;                /* 1: q,k,gate_x,temp_y are [Nseq,1,dk] (see the prefill)     */
+  int32_t reserved;                    /* 0                                                          */
 } rodimus_ddts_step_params;
 
 /* Bytes of device workspace rodimus_ddts_fwd needs for these sizes (pointers are not read).

@@ -48,6 +48,7 @@ class FwdParams(ctypes.Structure):
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("stream", ctypes.c_void_p),
         ("beta_hat", ctypes.c_void_p), ("feed_d", ctypes.c_void_p), ("feed_x", ctypes.c_void_p),
+        ("shared_gates", ctypes.c_int32), ("reserved", ctypes.c_int32),
     ]
 
 
@@ -61,6 +62,7 @@ class StepParams(ctypes.Structure):
         ("v", ctypes.c_void_p), ("o", ctypes.c_void_p),
         ("state", ctypes.c_void_p), ("stream", ctypes.c_void_p),
         ("beta_hat", ctypes.c_void_p), ("feed_d", ctypes.c_void_p), ("feed_x", ctypes.c_void_p),
+        ("shared_gates", ctypes.c_int32), ("reserved", ctypes.c_int32),
     ]
 
 
@@ -139,8 +141,10 @@ def fwd_params(q, k, gate_x, temp_y, v, o, s0=None, sT=None, cu_seqlens=None,
                feed_d=None, feed_x=None) -> FwdParams:
     """Fills a ``rodimus_ddts_fwd_params`` from torch tensors (no checks beyond layout)."""
     import torch
-    B, H, T, dk = q.shape
+    B, Hq, T, dk = q.shape
+    H = v.shape[1]
     p = FwdParams()
+    p.shared_gates = 1 if (Hq == 1 and H > 1) else 0     # q,k,x,y [B,1,T,dk]: one set for all heads
     p.struct_size = ctypes.sizeof(FwdParams)
     p.dtype = _dtype_code(q)
     p.ingate = ingate
@@ -239,7 +243,8 @@ def ddts_fwd(q, k, gate_x, temp_y, v, s0=None, cu_seqlens=None, cu_seqlens_host=
     """
     import torch
     _check_cuda(q, k, gate_x, temp_y, v, s0, cu_seqlens, beta_hat, feed_d, feed_x)
-    B, H, T, dk = q.shape
+    B, _, T, dk = q.shape
+    H = v.shape[1]            # q,k,gate_x,temp_y may have a single head shared by all H of v
     dv = v.shape[-1]
     nseq = B if cu_seqlens is None else cu_seqlens.numel() - 1
     o = out if out is not None else torch.empty((B, H, T, dv), dtype=q.dtype, device=q.device)
@@ -265,7 +270,8 @@ def ddts_step(q, k, gate_x, temp_y, v, state, scale: float = 1.0, ingate: int = 
     """
     import torch
     _check_cuda(q, k, gate_x, temp_y, v, state, beta_hat, feed_d, feed_x)
-    Nseq, H, dk = q.shape
+    Nseq, Hq, dk = q.shape
+    H = v.shape[1]
     dv = v.shape[-1]
     o = out if out is not None else torch.empty((Nseq, H, dv), dtype=q.dtype, device=q.device)
     p = StepParams()
@@ -278,6 +284,7 @@ def ddts_step(q, k, gate_x, temp_y, v, state, scale: float = 1.0, ingate: int = 
     p.state = _ptr(state)
     p.stream = torch.cuda.current_stream().cuda_stream
     p.beta_hat, p.feed_d, p.feed_x = _ptr(beta_hat), _ptr(feed_d), _ptr(feed_x)
+    p.shared_gates = 1 if (Hq == 1 and H > 1) else 0
     rc = step_raw(p)
     if rc != OK:
         raise RodimusError(rc, "rodimus_ddts_step")

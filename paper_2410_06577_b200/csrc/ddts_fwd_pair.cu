@@ -135,6 +135,8 @@ struct PairArgs {
   const __nv_bfloat16* beta_hat;  // [rows, dv] value gate, or nullptr
   const float* feed_d;            // [H, dv] feed-through weight, or nullptr (then no x' either)
   int feed_H;                     // heads per sequence of the caller's layout (indexes feed_d)
+  int gate_div;                   // 1, or for the shared-gate layout the caller's H: q,k,x,y hold
+                                  // one set of rows per sequence, [B,1,T,dk]
   float* dtot;           // optional [n_seq, H, dk]: product of all chunk decays of each sequence
   int sT_only;           // >= 0: only this sequence's final state is stored, as if it were number 0
   int state_only;        // 1: launch the state-only instantiation of the kernel
@@ -142,6 +144,7 @@ struct PairArgs {
 
 struct Item {
   long long row0;      // first global row (in the [rows, d] view) of this sequence and head
+  long long rowq;      // the same in q,k,x,y (differs from row0 in the shared-gate layout)
   long long state_off; // element offset of this CTA's state slice (row 0, first own column)
   long long seq_head;  // sequence * H + head
   int len;             // tokens
@@ -161,9 +164,11 @@ __device__ __forceinline__ Item decode_item(const PairArgs& a, long long item, i
     lo = lo < 0 ? 0 : (lo > a.T ? a.T : lo);
     hi = hi < lo ? lo : (hi > a.T ? a.T : hi);
     it.row0 = (long long)h * a.T + lo;
+    it.rowq = (long long)(h / a.gate_div) * a.T + lo;
     it.len = hi - lo;
   } else {
     it.row0 = (n * a.H + h) * (long long)a.T;
+    it.rowq = ((n * a.H + h) / a.gate_div) * (long long)a.T;
     it.len = a.T;
   }
   it.col0 = (pair * 2 + rank) * kDVS;
@@ -367,22 +372,23 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     mbar_expect_tx(fb, STATE_ONLY ? kStageBytes - kSlabBytes : kStageBytes);
     // rows beyond the tensor read as zeros; rows of the next sequence are masked later
     const int y = (int)(it.row0 + tpos);
+    const int yq = (int)(it.rowq + tpos);
     const int xc = rank * kCH;
-    tma_load_2d(st + kStX, &map_x, xc, y, fb);
-    tma_load_2d(st + kStY, &map_y, xc, y, fb);
-    if (!STATE_ONLY) tma_load_2d(st + kStQ, &map_q, xc, y, fb);
-    tma_load_2d(st + kStK, &map_k, xc, y, fb);
+    tma_load_2d(st + kStX, &map_x, xc, yq, fb);
+    tma_load_2d(st + kStY, &map_y, xc, yq, fb);
+    if (!STATE_ONLY) tma_load_2d(st + kStQ, &map_q, xc, yq, fb);
+    tma_load_2d(st + kStK, &map_k, xc, yq, fb);
     tma_load_2d(st + kStV, &map_v, it.col0, y, fb);
     tma_load_2d(st + kStV + kSlabBytes, &map_v, it.col0 + 64, y, fb);
     // The tile that will go into this stage NEXT time is asked into L2 now: a stage is refilled
     // only when its pass has been consumed, so the fill's latency is on the critical cycle of
     // the ring, and from L2 it is less than half of what it is from HBM.
-    const int yp = y + kStages * kC;
+    const int yp = y + kStages * kC, yqp = yq + kStages * kC;
     if (tpos + kStages * kC < it.len) {
-      tma_prefetch_2d(&map_x, xc, yp);
-      tma_prefetch_2d(&map_y, xc, yp);
-      if (!STATE_ONLY) tma_prefetch_2d(&map_q, xc, yp);
-      tma_prefetch_2d(&map_k, xc, yp);
+      tma_prefetch_2d(&map_x, xc, yqp);
+      tma_prefetch_2d(&map_y, xc, yqp);
+      if (!STATE_ONLY) tma_prefetch_2d(&map_q, xc, yqp);
+      tma_prefetch_2d(&map_k, xc, yqp);
       tma_prefetch_2d(&map_v, it.col0, yp);
       tma_prefetch_2d(&map_v, it.col0 + 64, yp);
       if (BLOCK && a.beta_hat) {
@@ -1398,6 +1404,7 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   const long long n_seq0 = p.cu_seqlens ? p.N : p.B;
   if (n_seq0 * p.H == 0) return cudaSuccess;
   const uint64_t rows = (uint64_t)p.B * p.H * p.T;
+  const uint64_t rows_q = p.shared_gates ? (uint64_t)p.B * p.T : rows;   // rows of q,k,x,y
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
 
   int dev = 0, sms = 0;
@@ -1407,8 +1414,8 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   PairMaps m;
   if (rows > 0) {
     const uint64_t dv = (uint64_t)p.dv;
-    if (!cached_map(&m.q, p.q, rows, kDK) || !cached_map(&m.k, p.k, rows, kDK) ||
-        !cached_map(&m.x, p.gate_x, rows, kDK) || !cached_map(&m.y, p.temp_y, rows, kDK) ||
+    if (!cached_map(&m.q, p.q, rows_q, kDK) || !cached_map(&m.k, p.k, rows_q, kDK) ||
+        !cached_map(&m.x, p.gate_x, rows_q, kDK) || !cached_map(&m.y, p.temp_y, rows_q, kDK) ||
         !cached_map(&m.v, p.v, rows, dv) || !cached_map(&m.o, p.o, rows, dv) ||
         !cached_map(&m.o8, p.o, rows, dv, 8) || !cached_map(&m.o1, p.o, rows, dv, 1))
       return cudaErrorUnknown;
@@ -1450,6 +1457,7 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches) {
   a.beta_hat = reinterpret_cast<const __nv_bfloat16*>(p.beta_hat);
   a.feed_d = p.feed_d;
   a.feed_H = p.H;
+  a.gate_div = p.shared_gates ? p.H : 1;
   a.dtot = nullptr;
   a.sT_only = -1;
   a.state_only = 0;

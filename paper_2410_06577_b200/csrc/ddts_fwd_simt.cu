@@ -33,6 +33,7 @@ struct SimtArgs {
   int H, T, dk, dv, n_seq, tiles;
   float scale;
   int ingate;
+  int shared;   // 1: q,k,gx,ty are [B,1,T,dk], one set per token for all heads
 };
 
 template <typename T>
@@ -70,10 +71,12 @@ __global__ void __launch_bounds__(kThreads, 1) ddts_fwd_simt_kernel(const SimtAr
     row0 = sh * a.T;
     len = a.T;
   }
-  const T* q = (const T*)a.q + row0 * dk;
-  const T* k = (const T*)a.k + row0 * dk;
-  const T* gx = (const T*)a.gx + row0 * dk;
-  const T* ty = (const T*)a.ty + row0 * dk;
+  // rows of q,k,gx,ty: the head's own, or the sequence's single shared set
+  const long long rq = a.shared ? row0 - ((long long)h + (a.cu ? 0 : n * (a.H - 1))) * a.T : row0;
+  const T* q = (const T*)a.q + rq * dk;
+  const T* k = (const T*)a.k + rq * dk;
+  const T* gx = (const T*)a.gx + rq * dk;
+  const T* ty = (const T*)a.ty + rq * dk;
   const T* v = (const T*)a.v + row0 * dv;
   T* o = (T*)a.o + row0 * dv;
   const T* bh = a.beta_hat ? (const T*)a.beta_hat + row0 * dv : nullptr;
@@ -186,7 +189,7 @@ cudaError_t launch_fwd_simt(const rodimus_ddts_fwd_params& p, int* n_launches) {
   a.H = p.H; a.T = p.T; a.dk = p.dk; a.dv = p.dv;
   a.n_seq = p.cu_seqlens ? p.N : p.B;
   a.tiles = (p.dv + kTileV - 1) / kTileV;
-  a.scale = p.scale; a.ingate = p.ingate;
+  a.scale = p.scale; a.ingate = p.ingate; a.shared = p.shared_gates;
   const long long items = (long long)a.n_seq * p.H * a.tiles;
   if (items == 0) return cudaSuccess;
   if (items > 0x7fffffffLL) return cudaErrorInvalidValue;

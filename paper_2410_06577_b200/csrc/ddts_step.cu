@@ -27,7 +27,7 @@ ddts_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __re
                  const T* __restrict__ ty, const T* __restrict__ v, T* __restrict__ o,
                  float* __restrict__ state, int n_seq_heads, int dk, int dv, float scale,
                  int ingate, const T* __restrict__ beta_hat, const float* __restrict__ feed_d,
-                 const T* __restrict__ feed_x, int H) {
+                 const T* __restrict__ feed_x, int H, int shared) {
   __shared__ float s_alpha[kMaxDk];
   __shared__ float s_w[kMaxDk];   // ahat * k
   __shared__ float s_q[kMaxDk];   // scale * q
@@ -54,7 +54,7 @@ ddts_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __re
 
     // Gates of this token (fp32 throughout).
     for (int d = tid; d < dk; d += kStepThreads) {
-      const long long i = nh * dk + d;
+      const long long i = (shared ? nh / H : nh) * dk + d;   // shared: q,k,gx,ty are [Nseq,1,dk]
       float la, lh;
       gate_logs_f32(to_f32(gx[i]), to_f32(ty[i]), ingate, la, lh);
       s_alpha[d] = expf(la);
@@ -151,13 +151,13 @@ cudaError_t launch_step(const rodimus_ddts_step_params& p, int* n_launches) {
     ddts_step_kernel<T><<<grid, kStepThreads, 0, st>>>(
         (const T*)p.q, (const T*)p.k, (const T*)p.gate_x, (const T*)p.temp_y, (const T*)p.v,
         (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate, (const T*)p.beta_hat, p.feed_d,
-        (const T*)p.feed_x, p.H);
+        (const T*)p.feed_x, p.H, p.shared_gates);
   } else {
     using T = float;
     ddts_step_kernel<T><<<grid, kStepThreads, 0, st>>>(
         (const T*)p.q, (const T*)p.k, (const T*)p.gate_x, (const T*)p.temp_y, (const T*)p.v,
         (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate, (const T*)p.beta_hat, p.feed_d,
-        (const T*)p.feed_x, p.H);
+        (const T*)p.feed_x, p.H, p.shared_gates);
   }
   *n_launches = 1;
   return cudaGetLastError();

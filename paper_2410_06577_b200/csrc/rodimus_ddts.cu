@@ -21,6 +21,7 @@ int check_fwd_sizes(const rodimus_ddts_fwd_params* p, bool varlen) {
   if (p->dtype != RODIMUS_BF16 && p->dtype != RODIMUS_F32) return RODIMUS_ERR_DTYPE;
   if (p->ingate != RODIMUS_INGATE_POW_G && p->ingate != RODIMUS_INGATE_POW_SIGMOID)
     return RODIMUS_ERR_DTYPE;
+  if ((p->shared_gates != 0 && p->shared_gates != 1) || p->reserved != 0) return RODIMUS_ERR_DTYPE;
   if (p->B < 0 || p->H < 0 || p->T < 0) return RODIMUS_ERR_SHAPE;
   if (p->dk <= 0 || p->dv <= 0) return RODIMUS_ERR_SHAPE;
   // well-formed widths that none of the kernels covers
@@ -71,7 +72,7 @@ bool has_block_terms(const rodimus_ddts_fwd_params& p) { return p.beta_hat || p.
 // 2: fp32 CUDA-core kernel
 int fwd_kernel_choice(const rodimus_ddts_fwd_params& p) {
   if (fwd_pair_selected(p)) return 0;
-  if (fwd_tc_supported(p) && !has_block_terms(p)) return 1;
+  if (fwd_tc_supported(p) && !has_block_terms(p) && !p.shared_gates) return 1;
   return 2;
 }
 
@@ -151,6 +152,7 @@ int rodimus_ddts_step(const rodimus_ddts_step_params* p) {
   if (p->dtype != RODIMUS_BF16 && p->dtype != RODIMUS_F32) return RODIMUS_ERR_DTYPE;
   if (p->ingate != RODIMUS_INGATE_POW_G && p->ingate != RODIMUS_INGATE_POW_SIGMOID)
     return RODIMUS_ERR_DTYPE;
+  if ((p->shared_gates != 0 && p->shared_gates != 1) || p->reserved != 0) return RODIMUS_ERR_DTYPE;
   if (p->Nseq < 0 || p->H < 0) return RODIMUS_ERR_SHAPE;
   if (p->dk <= 0 || p->dv <= 0) return RODIMUS_ERR_SHAPE;
   if (p->dk % 16 || p->dv % 16 || p->dk > 256 || p->dv > 1024) return RODIMUS_ERR_UNSUPPORTED;
@@ -205,6 +207,6 @@ const char* rodimus_status_str(int status) {
   }
 }
 
-int rodimus_version(void) { return 101; }
+int rodimus_version(void) { return 102; }
 
 }  // extern "C"

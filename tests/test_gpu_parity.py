@@ -686,3 +686,79 @@ def test_block_terms_decode_steps(dtype):
                           beta_hat=beta[s], feed_d=d, feed_x=fx[s])
         assert rel_err(host(o), ro) <= _tol(dtype)
     assert rel_err(host(state), ref_state) <= TOL_F32
+
+
+# ------------------------------------------------------------------------------------------
+# shared-gate layout: q,k,x,y [B,1,T,dk], one set per token for all H groups of value columns
+# ------------------------------------------------------------------------------------------
+
+def _shared_inputs(seed, B, H, T, dk, dv, dtype, s0_std=0.1, cu=None, gate_mean=-3.0):
+    """A workload whose q,k,x,y have a single head; v and the states keep H heads."""
+    pq = wl.make_prefill(seed, B, 1, T, dk, dv, dtype, gate_mean=gate_mean)
+    pv = wl.make_prefill(seed + 1, B, H, T, dk, dv, dtype, s0_std=s0_std, cu_seqlens=cu)
+    return pq, pv
+
+
+def _check_shared(seed, B, H, T, dk, dv, dtype, cu=None, block=False, expect_kernel=None, ingate=rd.INGATE_POW_G):
+    import torch
+    pq, pv = _shared_inputs(seed, B, H, T, dk, dv, dtype, cu=cu)
+    beta, d, fx = _block_terms(pv, 7, H)
+    up = lambda a: dev(a, dtype)
+    q, k, x, y, v = up(pq.q), up(pq.k), up(pq.x), up(pq.y), up(pv.v)
+    s0 = torch.from_numpy(pv.s0).cuda()
+    cu_d = None if cu is None else torch.from_numpy(cu).cuda()
+    cu_h = None if cu is None else torch.from_numpy(cu)
+    nseq = B if cu is None else len(cu) - 1
+    o = torch.full((B, H, T, dv), float("nan"), dtype=q.dtype, device="cuda")
+    sT = torch.full((nseq, H, dk, dv), float("nan"), dtype=torch.float32, device="cuda")
+    kw = dict(beta_hat=up(beta), feed_d=torch.from_numpy(d).cuda(), feed_x=up(fx)) if block else {}
+    prm = rd.fwd_params(q, k, x, y, v, o, s0, sT, cu_d, cu_h, None, 0.5, ingate, **kw)
+    assert prm.shared_gates == 1 and prm.H == H
+    if expect_kernel:
+        assert rd.fwd_kernel_name(prm) == expect_kernel
+    ws = torch.empty(max(rd.fwd_workspace_bytes(prm), 256), dtype=torch.uint8, device="cuda")
+    prm.workspace, prm.workspace_bytes = ws.data_ptr(), ws.numel()
+    assert rd.fwd_raw(prm) == rd.OK and rd.device_status(ws) == rd.OK
+    okw = dict(beta_hat=beta, feed_d=d, feed_x=fx) if block else {}
+    ro, rs = orc.ref_fwd(pq.q, pq.k, pq.x, pq.y, pv.v, s0=pv.s0, cu_seqlens=cu, scale=0.5,
+                         ingate=ingate, shared_gates=True, **okw)
+    eo, es = _worst_err(host(o), host(sT), ro, rs, cu)
+    tol = _tol(dtype)
+    assert eo <= tol and es <= tol, (eo, es)
+    return rd.last_launch_count()
+
+
+@pytest.mark.parametrize("ingate", [rd.INGATE_POW_G, rd.INGATE_POW_SIGMOID])
+def test_shared_gates_tensor_core_kernel(ingate):
+    _check_shared(601, 2, 4, 200, 128, 256, "bf16", expect_kernel="tcgen05", ingate=ingate)
+    _check_shared(603, 1, 3, 130, 128, 512, "bf16", block=True, ingate=ingate)
+
+
+def test_shared_gates_packed_and_time_split():
+    lens = _mixed_lengths(605, 40)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    _check_shared(606, 1, 4, int(cu[-1]), 128, 256, "bf16", cu=cu)
+    assert _check_shared(608, 2, 2, 4500, 128, 256, "bf16") == 5     # (batch, head) units split along time
+
+
+@pytest.mark.parametrize("dtype,dk,dv,H", [("f32", 64, 64, 4), ("bf16", 64, 256, 16), ("bf16", 128, 128, 3)])
+def test_shared_gates_cuda_core_kernel(dtype, dk, dv, H):
+    """dk = 64 with 16 groups of 256 value columns is the paper's own state shape (64 x 2d)."""
+    _check_shared(610, 1, H, 70, dk, dv, dtype, expect_kernel="simt")
+    lens = [5, 0, 33, 17]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    _check_shared(612, 1, H, int(cu[-1]), dk, dv, dtype, cu=cu, block=True)
+
+
+def test_shared_gates_decode_steps():
+    import torch
+    Nseq, H, dk, dv = 6, 4, 64, 256
+    wq = wl.make_decode(620, Nseq, 1, dk, dv, ring=3)
+    wv = wl.make_decode(621, Nseq, H, dk, dv, ring=3)
+    state = torch.from_numpy(wv.state).cuda()
+    ref_state = wv.state.astype(np.float64)
+    for s in range(3):
+        o = rd.ddts_step(*(dev(a[s], "bf16") for a in (wq.q, wq.k, wq.x, wq.y, wv.v)), state)
+        ro = orc.ref_step(wq.q[s], wq.k[s], wq.x[s], wq.y[s], wv.v[s], ref_state, shared_gates=True)
+        assert o.shape == (Nseq, H, dv) and rel_err(host(o), ro) <= TOL_BF16
+    assert rel_err(host(state), ref_state) <= TOL_F32
