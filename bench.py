@@ -268,7 +268,7 @@ def measure_sfu_rate(rd, torch, device):
 
 
 def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sfu_rate,
-            min_region_ms=60.0, with_e2e=True):
+            min_region_ms=60.0, with_e2e=True, variant=None):
     """Times `steps` calls of the workload (regions of exactly `steps` calls, repeated back to
     back until the clock sampler has had at least `min_region_ms` to look at; the median region
     is reported) and returns the record with value, roofline, clocks, e2e and launch count."""
@@ -321,16 +321,31 @@ def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sf
         nseq = B if cu is None else cu.numel() - 1
         o = torch.empty((B, H, T, dv), dtype=tdt, device=device)
         sT = torch.empty((nseq, H, dk, dv), dtype=torch.float32, device=device)
-        prm = rd.fwd_params(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], o, s0, sT, cu, cu_host)
+        # variants of the same workload (the §8(f) rows that are built): "block" adds the value
+        # gate and the feed-through (seeded, +2 tensors of v's shape read per call); "shared" keeps
+        # one q,k,x,y per token for all heads (head 0's), the layout the paper writes the block in
+        kw = {}
+        alg_bytes = prefill_bytes(p)
+        el = 2 if p.dtype == "bf16" else 4
+        if variant == "block":
+            g = torch.Generator(device="cpu").manual_seed(1234)
+            kw = {"beta_hat": torch.rand(p.v.shape, generator=g).to(tdt).to(device),
+                  "feed_x": torch.randn(p.v.shape, generator=g).to(tdt).to(device),
+                  "feed_d": torch.randn((H, dv), generator=g).to(device)}
+            alg_bytes += 2 * B * H * T * dv * el
+        elif variant == "shared":
+            for n in ("q", "k", "x", "y"):
+                devt[n] = devt[n][:, :1].contiguous()
+            alg_bytes -= (H - 1) * B * T * 4 * dk * el
+        prm = rd.fwd_params(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], o, s0, sT, cu, cu_host, **kw)
         ws = rd.new_workspace(prm, device)
         units_per_step = p.tokens
-        alg_bytes = prefill_bytes(p)
         kernel = "ddts_fwd_" + rd.fwd_kernel_name(prm)
         token_heads = B * H * T
 
         def step(i):
             rd.ddts_fwd(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], s0, cu, cu_host,
-                        out=o, final_state=sT, workspace=ws)
+                        out=o, final_state=sT, workspace=ws, **kw)
 
         o_host = torch.empty(o.shape, dtype=tdt).pin_memory()
         sT_host = torch.empty(sT.shape, dtype=torch.float32).pin_memory()
@@ -409,7 +424,11 @@ def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sf
                        "datasheet_peak": DATASHEET["hbm_gbs"],
                        "algorithmic_bytes_per_launch": int(alg_bytes),
                        "bound_times": bounds,
-                       "traffic": load_traffic(kernel, workload)}
+                       "traffic": None if variant else load_traffic(kernel, workload)}
+    if variant:
+        rec["config"] = dict(rec["config"], variant={
+            "block": "value gate beta_hat and feed-through d*x' fused (Eq. beta_def, Eq. rodimus_recurrent_form)",
+            "shared": "one q,k,x,y per token for all 16 heads ([B,1,T,dk])"}[variant])
     if with_e2e:
         e2e_steps = max(1, min(steps, 200 if decode else 5))
         e2e_regions = timed_regions(step_e2e, e2e_steps, 1, 0.0)
@@ -457,6 +476,15 @@ def run_ours(args, workload, p):
             pw = wl.config(WORKLOADS[name])
             k, w = SUB_DEFAULTS[name]
             r = measure(name, pw, k, w, world, rank, local, peaks, peak_kind, sfu_rate, with_e2e=False)
+            extra[name] = {key: r[key] for key in ("metric", "value", "unit", "steps", "warmup", "ms_per_step",
+                                                   "dtype", "config", "timed_regions", "clocks",
+                                                   "gpu_launches", "roofline")}
+            del pw
+        for name, variant in (("cfg1_block_terms", "block"), ("cfg1_shared_gates", "shared")):
+            torch.cuda.empty_cache()
+            pw = wl.config(1)
+            r = measure("cfg1", pw, 500, 5, world, rank, local, peaks, peak_kind, sfu_rate, with_e2e=False,
+                        variant=variant)
             extra[name] = {key: r[key] for key in ("metric", "value", "unit", "steps", "warmup", "ms_per_step",
                                                    "dtype", "config", "timed_regions", "clocks",
                                                    "gpu_launches", "roofline")}
