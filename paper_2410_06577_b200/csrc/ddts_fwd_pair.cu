@@ -80,8 +80,6 @@ constexpr int kBlkFloats = 68;                            // 64 decays, verdict,
 constexpr int kBlkBytes = kBlkFloats * 4;                 // 272 B, a multiple of 16
 constexpr int kOffTx = kOffDp + 4 * kDK * 4;              // float [2][68]: block to send
 constexpr int kOffRx = kOffTx + kRxBufs * kBlkBytes;      // float [2][68]: block received
-constexpr int kCtlWarp = 2;                             // low warp numbers for the single-warp roles:
-                                                      // among ready warps the scheduler favours the oldest
 constexpr int kGateWarp0 = 12, kGateWarps = 16;
 constexpr int kGR = kC / kGateWarps;                       // rows per gate thread
 constexpr int kOffTot = kOffRx + kRxBufs * kBlkBytes;     // float [2][8][64]: scan partials
@@ -93,8 +91,7 @@ constexpr int kSmemBytes = kSmemUsed + 1024;              // slack for manual 10
 static_assert(kOffTx % 16 == 0 && kOffRx % 16 == 0 && kBlkBytes % 16 == 0, "bulk copy alignment");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
-constexpr int kThreads = 32 * (kGateWarp0 + kGateWarps);   // 896 (warp 3 has no role)
-constexpr int kStateWarp0 = 4, kScoreWarp0 = 8;
+constexpr int kThreads = 32 * (kGateWarp0 + kGateWarps);   // 896: 28 warps (warp 24 has no role)
 
 // TMEM columns (32-bit words): two state buffers S^T [lane = value column][128 channels], output
 // O^T [lane = value column][64 rows], scores P [64 rows in 16-lane groups][64], and two buffers
@@ -315,6 +312,22 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
+  // Warp w runs on scheduler w % 4.  The single-warp roles (long straight-line code once per pass)
+  // all sit on scheduler 0 together with one gate worker; schedulers 1-3 run five gate workers,
+  // a state warp and a score warp each, whose loops fit the scheduler's instruction cache.
+  // role: 0 producer, 1 issuer, 2 control, 3 state, 4 score, 5 gate worker, 6 none
+  int role, gw_of_warp = 0;
+  if (warp == 0) role = 0;
+  else if (warp == 4) role = 1;
+  else if (warp == 8) role = 2;
+  else if (warp == 24) role = 6;
+  else if (warp == 12 || warp < 4) role = 3;
+  else if (warp == 16 || warp < 8) role = 4;
+  else {
+    role = 5;
+    // gate warps in increasing warp number: 9,10,11,13,14,15,17,18,19,20,21,22,23,25,26,27
+    gw_of_warp = warp - 9 - (warp > 12) - (warp > 16) - (warp > 24);
+  }
   const int rank = (int)cluster_ctarank();     // 0 or 1: which key-channel half and dv half
   const int peer = rank ^ 1;
   // The state update takes Kt for all 128 channels as ONE operand whose two 64-channel groups
@@ -414,7 +427,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       }
     }
   }
-  if (warp == 1) {
+  if (role == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(base + kOffMisc), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -430,7 +443,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const long long pair_id = blockIdx.x >> 1;
   auto item_of = [&](int j) { return pair_id + (long long)j * n_pairs_grid; };
 
-  if (warp == 0) {
+  if (role == 0) {
     // ===================================== TMA producer =====================================
     if (lane == 0) {
       uint32_t f = early_fills;            // fills issued
@@ -478,7 +491,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         mbar_drain(bar(BAR_FULL0 + ff % kStages), (ff / kStages) & 1);
       }
     }
-  } else if (warp == 1) {
+  } else if (role == 1) {
     // ====================================== MMA issuer ======================================
     // Every lane runs the loop (waits, descriptor arithmetic stay warp-uniform); lane 0 issues.
     {
@@ -559,7 +572,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
       }
     }
-  } else if (warp >= kStateWarp0 && warp < kStateWarp0 + 4) {
+  } else if (role == 3) {
     // ====================================== state group ======================================
     // Each thread owns one value column of the CTA's slice (= one TMEM lane of S^T); the 128
     // key channels are its TMEM columns.  Pass g accumulates its state update in buffer g & 1.
@@ -572,7 +585,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int q4 = warp & 3;                              // TMEM lane quarter this warp may touch
     const int c = q4 * 32 + lane;                         // value column (TMEM lane) of this thread
     const uint32_t t_lane = tmem + ((uint32_t)(q4 * 32) << 16);
-    const bool signaller = warp == kStateWarp0 && lane == 0;
+    const bool signaller = (warp & 3) == 0 && lane == 0;
     uint32_t g = 0;
     int prev_rx = 0;
     bool ok = true;
@@ -683,7 +696,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         tc_fence_before();
       }
     }
-  } else if (warp >= kScoreWarp0 && warp < kScoreWarp0 + 4) {
+  } else if (role == 4) {
     // ================================== score / output group ==================================
     const int q4 = warp & 3;
     // stmatrix roles of this thread: it addresses row mat_k of matrix lane/8 of each x4 group;
@@ -710,7 +723,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const int rxi = ctl->pd[g & 3].rx;
           last = (ctl->pd[g & 3].flags & kPassLast) != 0;
           if (!(ok = mbar_wait_cluster(bar(BAR_PEER0 + rxi), (uint32_t)ctl->pd[g & 3].rxph, abort_flag, a.hdr))) break;
-          if (warp == kScoreWarp0 && lane == 0) {
+          if (q4 == 0 && lane == 0) {
             const int peer_stage = __float_as_int(sRx[rxi * kBlkFloats + 65]);
             mbar_arrive_remote(map_to_cta(bar(BAR_EMPTY0 + peer_stage), peer));
           }
@@ -740,7 +753,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             tma_load_2d(xt + kSlabBytes, &map_fx, it.col0 + 64, (int)row, xb);
           }
         }
-        if (warp == kScoreWarp0 && lane == 0) {
+        if (q4 == 0 && lane == 0) {
           // P exists, so the partner's copies out of ITS stage have all landed here (the issuer
           // waited for them): let the partner reuse that stage
           const int rxi = ctl->pd[g & 3].rx;
@@ -870,16 +883,17 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         ++g;
       }
     }
-    bulk_wait<0>();   // this thread's output copies are complete before the CTA may exit
-  } else if (warp >= kGateWarp0 || warp == kCtlWarp) {
+    bulk_wait_read<0>();   // this thread's output copies have read their tile before the CTA may exit
+                           // (their writes complete with the kernel)
+  } else if (role == 5 || role == 2) {
     // ============================== gate group and its control warp ==============================
     // The gate warps are workers: for every order of the control warp (a stage and a row count)
     // they run phase 1 on their rows, hand in the column sums, wait for their prefix, run phase
     // 2 and report.  Everything serial or rare lives in the control warp: which fill is an
     // attempt, the scan over the 16 row groups, decays, verdict exchange, the copies to the
     // partner, refusals and redirects, publishing the pass.
-    const int gw = warp - kGateWarp0;                     // rows kGR*gw .. kGR*gw+kGR-1 of the tile
-    const bool is_ctl = warp == kCtlWarp;
+    const int gw = gw_of_warp;                            // rows kGR*gw .. kGR*gw+kGR-1 of the tile
+    const bool is_ctl = role == 2;
     bool ok = true;
     if (!is_ctl) {
       uint32_t off[kGR]; // swizzled byte offsets of the thread's element pairs inside a slab
@@ -1155,7 +1169,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     st_cluster_u32(pc + 4, (uint32_t)ctl->sent_blk);
     st_cluster_u32(pc + 8, (uint32_t)ctl->sent_slab);
   }
-  if (my_abort && warp == 1) {
+  if (my_abort && role == 1) {
     if (lane == 0) {
       umma_commit(bar(BAR_DRAIN));
       mbar_drain(bar(BAR_DRAIN), 0);
@@ -1184,7 +1198,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     cluster_arrive();
     cluster_wait();
   }
-  if (warp == 1) {
+  if (role == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
                  : "memory");
