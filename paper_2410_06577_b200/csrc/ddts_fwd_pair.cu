@@ -32,15 +32,18 @@
 // The pair advances in lockstep: which rows form a pass is decided from the decay totals of all
 // 128 channels, so each CTA sends its verdict along with its chunk decays and both take the OR.
 //
-// Roles in one CTA (19 warps), connected by mbarriers; every wait is bounded:
-//   warp 0        TMA producer (own channel slab of q,k,x,y and both slabs of the v slice)
-//   warp 1        tcgen05.mma issuer, owns the TMEM allocation
-//   warps 2-5     state group: TMEM <-> registers trip of S^T, initial / final state I/O
-//   warps 6-9     score / output group
-//   warps 10-17   gate group: 8 rows x 2 channels per thread, packed fp32x2 arithmetic
-//   warp 18       gate control: chunk totals, verdict exchange with the partner, the two slab
-//                 copies (one thread: sixteen small copies issued by the gate warps took them
-//                 ~1400 cycles per pass), publishing
+// Roles in one CTA (28 warps), connected by mbarriers; every wait is bounded.  Warp w runs on
+// scheduler w % 4, and a scheduler's first-level instruction cache holds about 8 KiB, less than
+// the loops of all roles together: the single-warp roles, long straight-line code run once per
+// pass, share scheduler 0, so that the loops of schedulers 1-3 (gate, state, score) stay cached.
+//   warp 0          TMA producer (own channel slab of q,k,x,y and both slabs of the v slice)
+//   warp 4          tcgen05.mma issuer, owns the TMEM allocation
+//   warp 8          control: which fill is an attempt, scan of the row groups' sums, chunk decays,
+//                   verdict exchange and slab copies to the partner, publishing, orders
+//   warps 1-3, 12   state group (TMEM quarter = warp % 4): TMEM <-> registers trip of S^T, state I/O
+//   warps 5-7, 16   score / output group
+//   the other 16    gate workers (one on scheduler 0, five on each other): 4 rows x 2 channels
+//                   per thread, packed fp32x2 arithmetic, on orders of the control warp
 //
 // The loop-carried chain is  state update of pass g -> rescaling of S -> state update of pass
 // g+1 , so the issuer puts the state update of a pass BEFORE its output contractions, and the
@@ -1022,7 +1025,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         Item nit = it;
         const bool nhave = ntpos < it.len ? true : seek(nj, nit, ntpos);
         auto try_ahead = [&]() {
-          if (ahead || !nhave || !mbar_try(bar(BAR_FULL0 + fs), fph)) return;
+          if (ahead || !nhave || !mbar_test(bar(BAR_FULL0 + fs), fph)) return;
           if (ctl->tag[fs][0] != nj || ctl->tag[fs][1] != ntpos) return;
           ahead = true;
           ahead_s = fs;
@@ -1085,6 +1088,7 @@ ddts_fwd_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // both operand slabs of the attempt go to the partner in one copy each (also when the
         // attempt turns out to be abandoned: the byte count the partner's barrier expects is
         // fixed); the partner's receive buffer m&1 is free, see above
+        try_ahead();                                      // second chance: the fill may have landed by now
         if (!(ok = mbar_wait(bar(BAR_ROWS), ocur & 1, abort_flag, a.hdr))) break;
         if (leader) {
           const uint32_t dst = peer_rx_base + rxi * kRxBytes;
