@@ -6,6 +6,8 @@ leg may import this module; the CUDA library and its Python binding never do.
 
 * ``ref_fwd`` / ``ref_step`` / ``ref_gates`` call the sequential recurrence
   (Eq. "alpha_def", Eq. "rodimus_recurrent_form").
+* ``ref_bwd`` calls the adjoint of that recurrence, statement by statement in reverse order
+  (the gradient of a scalar loss with respect to q, k, x, y, v and the initial state).
 * ``parallel_form`` is the O(T^2) masked form of the appendix on the chunkwise
   representation (Eq. "rodimus_parallel_form"), for one sequence and one head.
 * ``unrolled_sum`` is the double sum obtained by unfolding the general gated
@@ -72,6 +74,11 @@ def _load():
         lib.ddts_ref_step_block.restype = ctypes.c_int
         lib.ddts_ref_step_shared.argtypes = lib.ddts_ref_step_block.argtypes
         lib.ddts_ref_step_shared.restype = ctypes.c_int
+        lib.ddts_ref_bwd.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
+                                     ctypes.c_int, ctypes.c_int, ctypes.c_double,
+                                     f32p, f32p, f32p, f32p, f32p, f64p, f32p, f64p,
+                                     f64p, f64p, f64p, f64p, f64p, f64p, i32p, ctypes.c_int]
+        lib.ddts_ref_bwd.restype = ctypes.c_int
         lib.ddts_ref_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -192,6 +199,46 @@ def ref_step(q, k, x, y, v, state, scale: float = 1.0, ingate: int = POW_G, beta
     if rc:
         raise ValueError(f"ddts_ref_step returned {rc}")
     return o
+
+
+def ref_bwd(q, k, x, y, v, do, s0=None, dsT=None, cu_seqlens=None, scale: float = 1.0,
+            ingate: int = POW_G, want_ds0: bool = True):
+    """Gradients of L for given do = dL/do [B,H,T,dv] and dsT = dL/dS_T [B|N,H,dk,dv] (or None).
+
+    Layouts as ``ref_fwd``.  Returns a dict of float64 arrays: dq, dk, dx, dy [B,H,T,dk],
+    dv [B,H,T,dv], ds0 [B|N,H,dk,dv] (None unless wanted).
+    """
+    lib = _load()
+    qa, qp = _f32(q)
+    ka, kp = _f32(k)
+    xa, xp = _f32(x)
+    ya, yp = _f32(y)
+    va, vp = _f32(v)
+    da, dp = _f32(do)
+    B, H, T, dk = qa.shape
+    dv = va.shape[-1]
+    assert ka.shape == qa.shape == xa.shape == ya.shape and va.shape == da.shape == (B, H, T, dv)
+    cup = None
+    nseq = B
+    N = 0
+    if cu_seqlens is not None:
+        cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+        N = cu.size - 1
+        nseq = N
+        cup = cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+    s0a = None if s0 is None else np.ascontiguousarray(s0, dtype=np.float64)
+    dsa = None if dsT is None else np.ascontiguousarray(dsT, dtype=np.float64)
+    assert s0a is None or s0a.shape == (nseq, H, dk, dv)
+    assert dsa is None or dsa.shape == (nseq, H, dk, dv)
+    out = {n: np.zeros((B, H, T, dk), dtype=np.float64) for n in ("dq", "dk", "dx", "dy")}
+    out["dv"] = np.zeros((B, H, T, dv), dtype=np.float64)
+    out["ds0"] = np.zeros((nseq, H, dk, dv), dtype=np.float64) if want_ds0 else None
+    rc = lib.ddts_ref_bwd(ingate, B, H, T, dk, dv, float(scale), qp, kp, xp, yp, vp, _f64p(s0a),
+                          dp, _f64p(dsa), _f64p(out["dq"]), _f64p(out["dk"]), _f64p(out["dx"]),
+                          _f64p(out["dy"]), _f64p(out["dv"]), _f64p(out["ds0"]), cup, N)
+    if rc:
+        raise ValueError(f"ddts_ref_bwd returned {rc}")
+    return out
 
 
 # ----------------------------------------------------------------------------------------------

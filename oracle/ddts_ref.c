@@ -285,6 +285,172 @@ int ddts_ref_step(int ingate, int Nseq, int H, int dk, int dv, double scale, con
                              NULL);
 }
 
+/*
+ * Backward pass: the gradient of a scalar loss L with respect to every input of the prefill,
+ * given dL/do (rows of do) and dL/dS_T (dsT).  The paper trains the block through the
+ * chunkwise form (App. "Chunkwise Parallel Representation of the Rodimus Block") and prints no
+ * backward formulas: the quantity is defined by the forward equations above, and this is their
+ * adjoint written step by step, in reverse order of t, one statement per forward statement:
+ *
+ *   forward, step t, channel d:   w = ahat * k ;  S_t[d,:] = alpha * S_{t-1}[d,:] + w * v_t[:]
+ *                                 o_t[:] = scale * sum_d q_t[d] * S_t[d,:]
+ *   adjoint (G = dL/dS_t, starts at dsT and ends as dL/dS_0):
+ *     G[d,:]   += scale * q_t[d] * do_t[:]             dq_t[d] = scale * sum_j S_t[d,j] do_t[j]
+ *     dalpha    = sum_j G[d,j] * S_{t-1}[d,j]          dw      = sum_j G[d,j] * v_t[j]
+ *     dv_t[:]  += w * G[d,:]                           G[d,:] *= alpha         (now dL/dS_{t-1})
+ *     dk_t[d]   = dw * ahat ;  dahat = dw * k_t[d]
+ *     alpha = exp(-g tau):   dg  = -tau * alpha * dalpha ;  dtau  = -g * alpha * dalpha
+ *     ahat  = u^tau      :   dg += tau * u^(tau-1) * u'(g) * dahat ;  dtau += ahat * ln(u) * dahat
+ *                            (u = g, u' = 1 in mode 0;  u = 1 - e^-g, u' = e^-g in mode 1)
+ *     dx_t[d] = dg * sigmoid(x) ;  dy_t[d] = dtau * tau * (1 - tau)
+ *
+ * The states S_{t-1}, S_t that the adjoint needs are the forward's own: they are recomputed with
+ * the same statements from stored copies taken every kBwdBlock steps (storage only; no step is
+ * reordered or merged).  Pins (tests, CPU only): central finite differences of ddts_ref_fwd,
+ * reverse-mode differentiation of a separately written forward by an autograd library, linearity
+ * in (do, dsT), the chain of two half-length calls through ds0 -> dsT, T = 1 by hand.
+ */
+enum { kBwdBlock = 32 };
+
+/* One forward step of one sequence, the statements of ref_one_sequence without the outputs. */
+static void ref_state_step(int ingate, int dk, int dv, const float *kt, const float *xt,
+                           const float *yt, const float *vt, const double *Sin, double *Sout) {
+  for (int d = 0; d < dk; ++d) {
+    double alpha, ahat;
+    ref_gate(ingate, (double)xt[d], (double)yt[d], &alpha, &ahat);
+    double w = ahat * (double)kt[d];
+    const double *a = Sin + (size_t)d * dv;
+    double *b = Sout + (size_t)d * dv;
+    for (int j = 0; j < dv; ++j) b[j] = alpha * a[j] + w * (double)vt[j];
+  }
+}
+
+static int ref_bwd_one_sequence(int ingate, int64_t len, int dk, int dv, double scale,
+                                const float *q, const float *k, const float *x, const float *y,
+                                const float *v, const double *s0, const float *dout,
+                                const double *dsT, double *dq, double *dkk, double *dx, double *dy,
+                                double *dvv, double *ds0) {
+  const size_t sz = (size_t)dk * dv;
+  const int64_t nblk = (len + kBwdBlock - 1) / kBwdBlock;
+  double *ck = (double *)malloc(sizeof(double) * sz * (size_t)(nblk + 1));
+  double *Sb = (double *)malloc(sizeof(double) * sz * (kBwdBlock + 1));
+  double *G = (double *)malloc(sizeof(double) * sz);
+  if (!ck || !Sb || !G) {
+    free(ck); free(Sb); free(G);
+    return 8;
+  }
+  /* forward: the state at the start of every block */
+  if (s0) memcpy(ck, s0, sizeof(double) * sz); else memset(ck, 0, sizeof(double) * sz);
+  memcpy(Sb, ck, sizeof(double) * sz);
+  for (int64_t t = 0; t < len; ++t) {
+    double *cur = Sb + (size_t)(t & 1) * sz, *nxt = Sb + (size_t)((t + 1) & 1) * sz;
+    ref_state_step(ingate, dk, dv, k + t * dk, x + t * dk, y + t * dk, v + t * dv, cur, nxt);
+    if ((t + 1) % kBwdBlock == 0) memcpy(ck + sz * (size_t)((t + 1) / kBwdBlock), nxt, sizeof(double) * sz);
+  }
+  if (dsT) memcpy(G, dsT, sizeof(double) * sz); else memset(G, 0, sizeof(double) * sz);
+
+  for (int64_t blk = nblk - 1; blk >= 0; --blk) {
+    const int64_t t0 = blk * kBwdBlock;
+    const int n = (int)((len - t0) < kBwdBlock ? (len - t0) : kBwdBlock);
+    memcpy(Sb, ck + sz * (size_t)blk, sizeof(double) * sz);
+    for (int i = 0; i < n; ++i) {
+      const int64_t t = t0 + i;
+      ref_state_step(ingate, dk, dv, k + t * dk, x + t * dk, y + t * dk, v + t * dv,
+                     Sb + sz * (size_t)i, Sb + sz * (size_t)(i + 1));
+    }
+    for (int i = n - 1; i >= 0; --i) {
+      const int64_t t = t0 + i;
+      const double *Sprev = Sb + sz * (size_t)i, *Scur = Sb + sz * (size_t)(i + 1);
+      const float *qt = q + t * dk, *kt = k + t * dk, *xt = x + t * dk, *yt = y + t * dk;
+      const float *vt = v + t * dv, *dot = dout + t * dv;
+      double *dvt = dvv + t * dv;
+      for (int j = 0; j < dv; ++j) dvt[j] = 0.0;
+      for (int d = 0; d < dk; ++d) {
+        const double g = ref_softplus((double)xt[d]), tau = ref_sigmoid((double)yt[d]);
+        double alpha, ahat;
+        ref_gate(ingate, (double)xt[d], (double)yt[d], &alpha, &ahat);
+        const double w = ahat * (double)kt[d];
+        double *Gd = G + (size_t)d * dv;
+        const double *Sp = Sprev + (size_t)d * dv, *Sc = Scur + (size_t)d * dv;
+        double dqd = 0.0, dalpha = 0.0, dw = 0.0;
+        for (int j = 0; j < dv; ++j) {
+          Gd[j] += scale * (double)qt[d] * (double)dot[j];
+          dqd += Sc[j] * (double)dot[j];
+        }
+        for (int j = 0; j < dv; ++j) {
+          dalpha += Gd[j] * Sp[j];
+          dw += Gd[j] * (double)vt[j];
+          dvt[j] += w * Gd[j];
+          Gd[j] *= alpha;
+        }
+        dq[t * dk + d] = scale * dqd;
+        dkk[t * dk + d] = dw * ahat;
+        const double dahat = dw * (double)kt[d];
+        double dg = -tau * alpha * dalpha, dtau = -g * alpha * dalpha;
+        double u, du;
+        if (ingate == DDTS_REF_POW_G) {
+          u = g; du = 1.0;
+        } else {
+          u = -expm1(-g); du = exp(-g);
+        }
+        dg += tau * pow(u, tau - 1.0) * du * dahat;
+        dtau += ahat * log(u) * dahat;
+        dx[t * dk + d] = dg * ref_sigmoid((double)xt[d]);
+        dy[t * dk + d] = dtau * tau * (1.0 - tau);
+      }
+    }
+  }
+  if (ds0) memcpy(ds0, G, sizeof(double) * sz);
+  free(ck); free(Sb); free(G);
+  return 0;
+}
+
+/*
+ * Layouts as ddts_ref_fwd (dense, or packed with cu_seqlens and B = 1).  dout is [B,H,T,dv]
+ * (float, already rounded to the GPU's input type), dsT [B|N,H,dk,dv] or NULL (zero).  Outputs,
+ * all double: dq, dk, dx, dy [B,H,T,dk], dv [B,H,T,dv], ds0 [B|N,H,dk,dv] or NULL (not wanted).
+ */
+int ddts_ref_bwd(int ingate, int B, int H, int64_t T, int dk, int dv, double scale, const float *q,
+                 const float *k, const float *x, const float *y, const float *v, const double *s0,
+                 const float *dout, const double *dsT, double *dq, double *dkk, double *dx,
+                 double *dy, double *dvv, double *ds0, const int32_t *cu_seqlens, int N) {
+  if (ingate != DDTS_REF_POW_G && ingate != DDTS_REF_POW_SIGMOID) return 3;
+  if (B < 0 || H < 0 || T < 0 || dk <= 0 || dv <= 0) return 2;
+  int nseq = B;
+  if (cu_seqlens) {
+    if (B != 1 || N < 0) return 2;
+    if (cu_seqlens[0] != 0 || cu_seqlens[N] != T) return 5;
+    for (int n = 0; n < N; ++n)
+      if (cu_seqlens[n + 1] < cu_seqlens[n]) return 5;
+    nseq = N;
+  }
+  int64_t items = (int64_t)nseq * H;
+  int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t it = 0; it < items; ++it) {
+    int64_t n = it / H, h = it % H;
+    int64_t row0, len;
+    if (cu_seqlens) {
+      row0 = h * T + cu_seqlens[n];
+      len = cu_seqlens[n + 1] - cu_seqlens[n];
+    } else {
+      row0 = (n * H + h) * T;
+      len = T;
+    }
+    size_t so = (size_t)it * dk * dv;
+    int rc = ref_bwd_one_sequence(ingate, len, dk, dv, scale, q + row0 * dk, k + row0 * dk,
+                                  x + row0 * dk, y + row0 * dk, v + row0 * dv, s0 ? s0 + so : NULL,
+                                  dout + row0 * dv, dsT ? dsT + so : NULL, dq + row0 * dk,
+                                  dkk + row0 * dk, dx + row0 * dk, dy + row0 * dk, dvv + row0 * dv,
+                                  ds0 ? ds0 + so : NULL);
+    if (rc) {
+#pragma omp atomic write
+      failed = 1;
+    }
+  }
+  return failed ? 8 : 0;
+}
+
 /* Threads the parallel regions above will use (1 without OpenMP). */
 int ddts_ref_num_threads(void) {
 #ifdef _OPENMP
