@@ -161,6 +161,57 @@ int rodimus_ddts_fwd(const rodimus_ddts_fwd_params *p);
 int rodimus_ddts_step(const rodimus_ddts_step_params *p);
 
 /*
+ * Backward pass of the prefill: the gradient of a scalar loss L with respect to every input of
+ * rodimus_ddts_fwd, given d_o = dL/do and d_sT = dL/dS_T.  The paper trains the block through
+ * the chunkwise form (appendix "Chunkwise Parallel Representation of the Rodimus Block") and
+ * prints no backward formulas; the result is defined by Eq. "alpha_def" and
+ * Eq. "rodimus_recurrent_form" and computed as the adjoint of the chunkwise form (chunk length
+ * internal): a forward sweep over the chunks carries S and yields dq, a reverse sweep carries
+ * dL/dS and yields dk and dv, and the gradients of the two gates follow from suffix sums of
+ * q . dq - (ahat k) . d(ahat k) over the sequence.
+ *
+ * Layouts as rodimus_ddts_fwd_params (dense, or packed with cu_seqlens and B = 1).  Inputs:
+ * q,k,gate_x,temp_y [B,H,T,dk], v and d_o [B,H,T,dv] in `dtype`; s0 and d_sT fp32 [B|N,H,dk,dv]
+ * or NULL (zero).  Outputs, written: d_q,d_k,d_gate_x,d_temp_y [B,H,T,dk] and d_v [B,H,T,dv] in
+ * `dtype`; d_s0 fp32 [B|N,H,dk,dv] or NULL (not wanted).  No output may overlap an input.
+ * Supported widths: dk = 128 and dv = 256 (others: RODIMUS_ERR_UNSUPPORTED); the value gate,
+ * the feed-through and the shared-gate layout of the forward call have no backward here.
+ * dtype BF16 contracts tf32 operands on the tensor cores with fp32 accumulation; dtype F32
+ * splits each operand in two tf32 parts and keeps fp32 accuracy.  The workspace holds the
+ * status word and 8 * dk bytes per token and head of scratch.
+ */
+typedef struct {
+  int32_t struct_size;       /* sizeof(rodimus_ddts_bwd_params), checked                        */
+  int32_t dtype;             /* rodimus_dtype of q,k,gate_x,temp_y,v,d_o and of the d_ outputs  */
+  int32_t ingate;            /* rodimus_ingate                                                  */
+  int32_t B, H, T, dk, dv;
+  float scale;
+  int32_t N;                 /* number of sequences when cu_seqlens != NULL                     */
+  const void *q, *k, *gate_x, *temp_y; /* device [B,H,T,dk]: the forward call's inputs          */
+  const void *v;             /* device [B,H,T,dv]                                               */
+  const float *s0;           /* device fp32 [B|N,H,dk,dv] or NULL: the forward's initial state  */
+  const void *d_o;           /* device [B,H,T,dv]: dL/do                                        */
+  const float *d_sT;         /* device fp32 [B|N,H,dk,dv] or NULL: dL/dS_T                      */
+  void *d_q, *d_k, *d_gate_x, *d_temp_y; /* device [B,H,T,dk], written                          */
+  void *d_v;                 /* device [B,H,T,dv], written                                      */
+  float *d_s0;               /* device fp32 [B|N,H,dk,dv] or NULL, written                      */
+  const int32_t *cu_seqlens; /* device int32 [N+1] or NULL                                      */
+  const int32_t *cu_seqlens_host; /* optional host copy, checked before launch (see the prefill) */
+  void *workspace;           /* device, >= rodimus_ddts_bwd_workspace_bytes(), 256-byte aligned */
+  size_t workspace_bytes;
+  void *stream;
+} rodimus_ddts_bwd_params;
+
+/* Bytes of device workspace rodimus_ddts_bwd needs (pointers are not read, except that a
+ * non-NULL cu_seqlens or cu_seqlens_host marks the call as packed); 0 if the sizes are not valid
+ * or not supported. */
+size_t rodimus_ddts_bwd_workspace_bytes(const rodimus_ddts_bwd_params *p);
+
+/* Backward pass; see rodimus_ddts_bwd_params.  The device-side status (cu_seqlens check) is read
+ * with rodimus_ddts_device_status as for the prefill. */
+int rodimus_ddts_bwd(const rodimus_ddts_bwd_params *p);
+
+/*
  * rodimus_ddts_fwd for callers that cannot allocate device memory.  (A convenience of this
  * library: the paper has no counterpart.)
  *
@@ -201,7 +252,7 @@ int rodimus_ddts_fwd_noalloc(const rodimus_ddts_fwd_params *p, const void **stat
  */
 int rodimus_ddts_device_status(const void *workspace, void *stream);
 
-/* How many kernels the last successful rodimus_ddts_fwd / rodimus_ddts_step call on this host
+/* How many kernels the last successful rodimus_ddts_fwd / _bwd / _step call on this host
  * thread launched (for benchmarks that report launch counts). */
 int rodimus_ddts_last_launch_count(void);
 

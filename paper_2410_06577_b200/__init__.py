@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = (
     "rodimus_ddts_device_status", "rodimus_ddts_last_launch_count",
     "rodimus_ddts_fwd_kernel_name", "rodimus_status_str", "rodimus_version",
     "rodimus_ddts_fwd_noalloc", "rodimus_ddts_sfu_probe", "rodimus_ddts_test_set_wait_limit",
+    "rodimus_ddts_bwd_workspace_bytes", "rodimus_ddts_bwd",
 )
 NOALLOC_MAX_SEQS = 4096
 
@@ -66,6 +67,25 @@ class StepParams(ctypes.Structure):
     ]
 
 
+class BwdParams(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_int32), ("dtype", ctypes.c_int32), ("ingate", ctypes.c_int32),
+        ("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32),
+        ("dk", ctypes.c_int32), ("dv", ctypes.c_int32),
+        ("scale", ctypes.c_float), ("N", ctypes.c_int32),
+        ("q", ctypes.c_void_p), ("k", ctypes.c_void_p),
+        ("gate_x", ctypes.c_void_p), ("temp_y", ctypes.c_void_p),
+        ("v", ctypes.c_void_p), ("s0", ctypes.c_void_p),
+        ("d_o", ctypes.c_void_p), ("d_sT", ctypes.c_void_p),
+        ("d_q", ctypes.c_void_p), ("d_k", ctypes.c_void_p),
+        ("d_gate_x", ctypes.c_void_p), ("d_temp_y", ctypes.c_void_p),
+        ("d_v", ctypes.c_void_p), ("d_s0", ctypes.c_void_p),
+        ("cu_seqlens", ctypes.c_void_p), ("cu_seqlens_host", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+        ("stream", ctypes.c_void_p),
+    ]
+
+
 _lib = None
 
 
@@ -97,6 +117,10 @@ def load_library() -> ctypes.CDLL:
         lib.rodimus_ddts_sfu_probe.restype = ctypes.c_int
         lib.rodimus_ddts_test_set_wait_limit.argtypes = [ctypes.c_longlong]
         lib.rodimus_ddts_test_set_wait_limit.restype = ctypes.c_int
+        lib.rodimus_ddts_bwd_workspace_bytes.argtypes = [ctypes.POINTER(BwdParams)]
+        lib.rodimus_ddts_bwd_workspace_bytes.restype = ctypes.c_size_t
+        lib.rodimus_ddts_bwd.argtypes = [ctypes.POINTER(BwdParams)]
+        lib.rodimus_ddts_bwd.restype = ctypes.c_int
         lib.rodimus_status_str.argtypes = [ctypes.c_int]
         lib.rodimus_status_str.restype = ctypes.c_char_p
         lib.rodimus_version.restype = ctypes.c_int
@@ -227,6 +251,73 @@ def new_workspace(p: FwdParams, device):
     import torch
     n = max(fwd_workspace_bytes(p), 256)
     return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def bwd_params(q, k, gate_x, temp_y, v, d_o, d_q, d_k, d_gate_x, d_temp_y, d_v, s0=None,
+               d_sT=None, d_s0=None, cu_seqlens=None, cu_seqlens_host=None, workspace=None,
+               scale: float = 1.0, ingate: int = INGATE_POW_G,
+               stream: Optional[int] = None) -> BwdParams:
+    """Fills a ``rodimus_ddts_bwd_params`` from torch tensors (no checks beyond layout)."""
+    import torch
+    B, H, T, dk = q.shape
+    p = BwdParams()
+    p.struct_size = ctypes.sizeof(BwdParams)
+    p.dtype = _dtype_code(q)
+    p.ingate = ingate
+    p.B, p.H, p.T, p.dk, p.dv = B, H, T, dk, v.shape[-1]
+    p.scale = scale
+    p.N = 0 if cu_seqlens is None else cu_seqlens.numel() - 1
+    p.q, p.k, p.gate_x, p.temp_y, p.v = (_ptr(t) for t in (q, k, gate_x, temp_y, v))
+    p.s0, p.d_o, p.d_sT = _ptr(s0), _ptr(d_o), _ptr(d_sT)
+    p.d_q, p.d_k, p.d_gate_x, p.d_temp_y = (_ptr(t) for t in (d_q, d_k, d_gate_x, d_temp_y))
+    p.d_v, p.d_s0 = _ptr(d_v), _ptr(d_s0)
+    p.cu_seqlens = _ptr(cu_seqlens)
+    p.cu_seqlens_host = _ptr(cu_seqlens_host)
+    p.workspace = _ptr(workspace)
+    p.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    p.stream = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    return p
+
+
+def bwd_workspace_bytes(p: BwdParams) -> int:
+    return int(load_library().rodimus_ddts_bwd_workspace_bytes(ctypes.byref(p)))
+
+
+def bwd_raw(p: BwdParams) -> int:
+    """Calls ``rodimus_ddts_bwd`` and returns its status without raising."""
+    return int(load_library().rodimus_ddts_bwd(ctypes.byref(p)))
+
+
+def ddts_bwd(q, k, gate_x, temp_y, v, d_o, s0=None, d_sT=None, cu_seqlens=None,
+             cu_seqlens_host=None, scale: float = 1.0, ingate: int = INGATE_POW_G,
+             want_d_s0: bool = True, workspace=None):
+    """Backward pass of the prefill (``rodimus_ddts_bwd``).
+
+    Inputs as ``ddts_fwd`` plus d_o = dL/do [B,H,T,dv] and d_sT = dL/dS_T (fp32 [B|N,H,dk,dv] or
+    None).  Returns a dict with d_q, d_k, d_gate_x, d_temp_y [B,H,T,dk], d_v [B,H,T,dv] (dtype of
+    the inputs) and d_s0 (fp32, None unless wanted).  Asynchronous on the current stream.
+    """
+    import torch
+    _check_cuda(q, k, gate_x, temp_y, v, d_o, s0, d_sT, cu_seqlens)
+    B, H, T, dk = q.shape
+    dv = v.shape[-1]
+    nseq = B if cu_seqlens is None else cu_seqlens.numel() - 1
+    out = {n: torch.empty_like(q) for n in ("d_q", "d_k", "d_gate_x", "d_temp_y")}
+    out["d_v"] = torch.empty_like(v)
+    out["d_s0"] = (torch.empty((nseq, H, dk, dv), dtype=torch.float32, device=q.device)
+                   if want_d_s0 else None)
+    p = bwd_params(q, k, gate_x, temp_y, v, d_o, out["d_q"], out["d_k"], out["d_gate_x"],
+                   out["d_temp_y"], out["d_v"], s0, d_sT, out["d_s0"], cu_seqlens,
+                   cu_seqlens_host, None, scale, ingate)
+    ws = workspace
+    if ws is None:
+        ws = torch.empty(max(bwd_workspace_bytes(p), 256), dtype=torch.uint8, device=q.device)
+    p.workspace = ws.data_ptr()
+    p.workspace_bytes = ws.numel() * ws.element_size()
+    rc = bwd_raw(p)
+    if rc != OK:
+        raise RodimusError(rc, "rodimus_ddts_bwd")
+    return out
 
 
 def ddts_fwd(q, k, gate_x, temp_y, v, s0=None, cu_seqlens=None, cu_seqlens_host=None,

@@ -1,0 +1,610 @@
+// Backward pass of the chunked prefill: gradients with respect to q, k, x, y, v and the initial
+// state, given dL/do and dL/dS_T.  The paper trains the block through the chunkwise form
+// (appendix "Chunkwise Parallel Representation of the Rodimus Block"); this is the adjoint of
+// that form, chunk length 16, with the same notation:
+//
+//   b_r   = sum_{j<=r in chunk} log alpha_j                 (per key channel, b_C at the chunk end)
+//   kt_i  = ahat_i . k_i        q'_r = scale . q_r
+//   A_ri  = sum_d q'_rd kt_id exp(b_rd - b_id),  i <= r     (scores; difference formed BEFORE exp)
+//   dA_ri = sum_j do_rj v_ij,                    i <= r
+//   Qe_r  = q'_r . exp(b_r)     Ke_i = kt_i . exp(b_C - b_i)     D = exp(b_C)
+//
+//   forward sweep  (state S entering the chunk):
+//     dq'_r = sum_{i<=r} dA_ri kt_i exp(b_r - b_i) + exp(b_r) . (S do_r)      S <- D . S + Ke^T V
+//   reverse sweep  (G = dL/dS at the chunk end):
+//     dkt_i = sum_{r>=i} dA_ri q'_r exp(b_r - b_i) + exp(b_C - b_i) . (G v_i)
+//     dv_i  = sum_{r>=i} A_ri do_r + Ke_i G                                   G <- D . G + Qe^T dO
+//   gates: with u_t = q_t . dq_t and w_t = kt_t . dkt_t (= dL/dlog ahat_t),
+//     dL/dlog alpha_t = sum_{s>=t} (u_s - w_s) + sum_j dS_T[.,j] S_T[.,j]
+//   (every pair (r,i) with i < t <= r appears once in the first sum and never in the second),
+//   and dx, dy follow from Eq. "alpha_def" by the chain rule.
+//
+// One launch of 6 CTAs per (sequence, head): the forward sweep for each half of the key channels,
+// the reverse sweep for each half of the key channels (dk), and the reverse sweep with the state
+// transposed for each half of the value columns (dv).  Each CTA keeps its [64 x 256] (or
+// [128 x 128]) slice of the state in REGISTERS as accumulator fragments of mma.sync.m16n8k8
+// (tf32 inputs, fp32 accumulation); the same registers are the A operand of the contraction
+// with dO or V (the k index of that instruction is a free permutation, applied to both
+// operands).  The fp32 build splits every operand into two tf32 parts (three instructions per
+// product), which keeps fp32 accuracy.  A second, small kernel forms the suffix sums and dx, dy.
+#include "ddts_common.cuh"
+
+namespace ddts {
+namespace {
+
+constexpr int kC = 16;            // chunk length
+constexpr int DK = 128, DV = 256; // the widths this kernel is built for
+constexpr int kThreads = 256;
+constexpr int LDK = DK + 8;       // row strides = 8 mod 32 words: fragment loads hit 32 banks
+constexpr int LDV = DV + 8;
+constexpr int LDR = 17;
+
+struct BwdArgs {
+  const void *q, *k, *gx, *ty, *v, *dout;
+  const float *s0, *dsT;
+  void *dq, *dk, *dx, *dy, *dv;
+  float* ds0;
+  float *u, *w, *c;        // scratch: [rows, DK], [rows, DK], [n_seq * H, DK]
+  const int32_t* cu;
+  WorkspaceHeader* hdr;
+  int H, T, n_seq;
+  float scale;
+  int ingate;
+};
+
+template <typename T>
+__device__ __forceinline__ void load8(const T* p, float (&o)[8]);
+template <>
+__device__ __forceinline__ void load8<float>(const float* p, float (&o)[8]) {
+  const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+  o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+}
+template <>
+__device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16* p, float (&o)[8]) {
+  const uint4 a = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    o[2 * i] = __uint_as_float(w[i] << 16);
+    o[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+template <typename T>
+__device__ __forceinline__ void store8(T* p, const float (&o)[8]);
+template <>
+__device__ __forceinline__ void store8<float>(float* p, const float (&o)[8]) {
+  *reinterpret_cast<float4*>(p) = make_float4(o[0], o[1], o[2], o[3]);
+  *reinterpret_cast<float4*>(p + 4) = make_float4(o[4], o[5], o[6], o[7]);
+}
+template <>
+__device__ __forceinline__ void store8<__nv_bfloat16>(__nv_bfloat16* p, const float (&o)[8]) {
+  uint32_t w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+    w[i] = *reinterpret_cast<const uint32_t*>(&h);
+  }
+  *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__device__ __forceinline__ float tf32_round(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return __uint_as_float(r);
+}
+
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const float (&a)[4], const float (&b)[2]) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(__float_as_uint(a[0])), "r"(__float_as_uint(a[1])), "r"(__float_as_uint(a[2])),
+        "r"(__float_as_uint(a[3])), "r"(__float_as_uint(b[0])), "r"(__float_as_uint(b[1])));
+}
+
+// c += a * b for one 16x8x8 tile.  EXACT: operands split as hi + lo (both tf32), the lo*lo term
+// (2^-22 of the product) dropped.
+template <bool EXACT>
+__device__ __forceinline__ void mma_tile(float (&c)[4], const float (&a)[4], const float (&b)[2]) {
+  float ah[4], bh[2];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) ah[i] = tf32_round(a[i]);
+#pragma unroll
+  for (int i = 0; i < 2; ++i) bh[i] = tf32_round(b[i]);
+  if (EXACT) {
+    float al[4], bl[2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) al[i] = tf32_round(a[i] - ah[i]);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) bl[i] = tf32_round(b[i] - bh[i]);
+    mma_tf32(c, al, bh);
+    mma_tf32(c, ah, bl);
+  }
+  mma_tf32(c, ah, bh);
+}
+
+// MODE 0: forward sweep (dq, u, c); 1: reverse sweep, state [d][j] (dk, w, ds0);
+// 2: reverse sweep, state [j][d] (dv).
+template <typename T, int MODE>
+__device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, const int half,
+                          const long long row0, const int len) {
+  constexpr bool EXACT = sizeof(T) == 4;
+  float* sQ = smem;                    // [kC][LDK] scale * q
+  float* sKt = sQ + kC * LDK;          // ahat * k
+  float* sLa = sKt + kC * LDK;         // log alpha
+  float* sB = sLa + kC * LDK;          // b (inclusive cumulative log alpha)
+  float* sQe = sB + kC * LDK;          // q' exp(b)
+  float* sKe = sQe + kC * LDK;         // kt exp(b_C - b)      (MODE 1: ahat instead)
+  float* sV = sKe + kC * LDK;          // [kC][LDV]
+  float* sDO = sV + kC * LDV;          // [kC][LDV]
+  float* sD = sDO + kC * LDV;          // [DK] exp(b_C)
+  float* sP = sD + DK;                 // [kC][LDR] dA (MODE 0, 1) or A (MODE 2), masked
+  float* sRedA = sP + kC * LDR;        // [8][kC][kC] partial dA of each warp
+  float* sRed = sRedA + 8 * kC * kC;   // [8][16][LDR] partial contraction of each warp / dv tile
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const T* q = (const T*)a.q + row0 * DK;
+  const T* k = (const T*)a.k + row0 * DK;
+  const T* gx = (const T*)a.gx + row0 * DK;
+  const T* ty = (const T*)a.ty + row0 * DK;
+  const T* v = (const T*)a.v + row0 * DV;
+  const T* dout = (const T*)a.dout + row0 * DV;
+  const long long s_off = sh * (long long)DK * DV;
+
+  // rows / columns of the state fragments this thread holds
+  const int m0 = MODE == 2 ? 128 * half + 16 * warp : 64 * half + 16 * (warp >> 1);
+  const int nbase = MODE == 2 ? 0 : 128 * (warp & 1);
+  float st[16][4];
+  {
+    const float* init = MODE == 0 ? a.s0 : a.dsT;
+#pragma unroll
+    for (int n = 0; n < 16; ++n) {
+      const int c0 = nbase + 8 * n + 2 * t;
+      if (!init) {
+        st[n][0] = st[n][1] = st[n][2] = st[n][3] = 0.f;
+      } else if (MODE != 2) {
+        const float2 lo = *reinterpret_cast<const float2*>(init + s_off + (long long)(m0 + g) * DV + c0);
+        const float2 hi = *reinterpret_cast<const float2*>(init + s_off + (long long)(m0 + g + 8) * DV + c0);
+        st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y;
+      } else {   // transposed: fragment row = value column, fragment column = key channel
+        st[n][0] = init[s_off + (long long)c0 * DV + m0 + g];
+        st[n][1] = init[s_off + (long long)(c0 + 1) * DV + m0 + g];
+        st[n][2] = init[s_off + (long long)c0 * DV + m0 + g + 8];
+        st[n][3] = init[s_off + (long long)(c0 + 1) * DV + m0 + g + 8];
+      }
+    }
+  }
+
+  const int nchunks = (len + kC - 1) / kC;
+  for (int ci = 0; ci < nchunks; ++ci) {
+    const int t0 = (MODE == 0 ? ci : nchunks - 1 - ci) * kC;
+    const int nr = min(kC, len - t0);
+    // ---- (1) loads and gates: one thread per (row, 8 channels); rows past the end read as zero
+    {
+      const int r = tid >> 4, d8 = (tid & 15) * 8;
+      float fq[8], fk[8], fa[8], la[8];
+      if (r < nr) {
+        float fx[8], fy[8];
+        const long long i = (long long)(t0 + r) * DK + d8;
+        load8<T>(q + i, fq);
+        load8<T>(k + i, fk);
+        load8<T>(gx + i, fx);
+        load8<T>(ty + i, fy);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          float lh;
+          gate_logs_f32(fx[e], fy[e], a.ingate, la[e], lh);
+          fa[e] = expf(lh);
+          fk[e] *= fa[e];
+          fq[e] *= a.scale;
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) fq[e] = fk[e] = fa[e] = la[e] = 0.f;
+      }
+      store8<float>(sQ + r * LDK + d8, fq);
+      store8<float>(sKt + r * LDK + d8, fk);
+      store8<float>(sLa + r * LDK + d8, la);
+      if (MODE == 1) store8<float>(sKe + r * LDK + d8, fa);
+#pragma unroll
+      for (int p = 0; p < 2; ++p) {
+        const int e = tid + p * kThreads, rr = e >> 5, c8 = (e & 31) * 8;
+        float fv[8], fd[8];
+        if (rr < nr) {
+          const long long i = (long long)(t0 + rr) * DV + c8;
+          load8<T>(v + i, fv);
+          load8<T>(dout + i, fd);
+        } else {
+#pragma unroll
+          for (int x = 0; x < 8; ++x) fv[x] = fd[x] = 0.f;
+        }
+        store8<float>(sV + rr * LDV + c8, fv);
+        store8<float>(sDO + rr * LDV + c8, fd);
+      }
+    }
+    __syncthreads();
+    // ---- (2) cumulative decay, scaled operands; partial dA on the tensor cores
+    {
+      const int d = tid & (DK - 1), role = tid >> 7;
+      float b[kC], acc = 0.f;
+#pragma unroll
+      for (int r = 0; r < kC; ++r) {
+        acc += sLa[r * LDK + d];
+        b[r] = acc;
+      }
+      if (role == 0) {
+#pragma unroll
+        for (int r = 0; r < kC; ++r) {
+          sB[r * LDK + d] = b[r];
+          sQe[r * LDK + d] = sQ[r * LDK + d] * expf(b[r]);
+        }
+      } else {
+        sD[d] = expf(acc);
+        if (MODE != 1) {
+#pragma unroll
+          for (int r = 0; r < kC; ++r) sKe[r * LDK + d] = sKt[r * LDK + d] * expf(acc - b[r]);
+        }
+      }
+    }
+    if (MODE != 2) {   // dA[r][i] = sum_j dO[r][j] V[i][j], this warp's 32 value columns
+      float acc[2][4] = {};
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {
+        const int j0 = 32 * warp + 8 * ks + 2 * t;
+        const float2 x0 = *reinterpret_cast<const float2*>(sDO + g * LDV + j0);
+        const float2 x1 = *reinterpret_cast<const float2*>(sDO + (g + 8) * LDV + j0);
+        const float af[4] = {x0.x, x1.x, x0.y, x1.y};
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+          const float2 y = *reinterpret_cast<const float2*>(sV + (nt * 8 + g) * LDV + j0);
+          const float bf[2] = {y.x, y.y};
+          mma_tile<EXACT>(acc[nt], af, bf);
+        }
+      }
+      float* red = sRedA + warp * kC * kC;
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        red[g * kC + nt * 8 + 2 * t] = acc[nt][0];
+        red[g * kC + nt * 8 + 2 * t + 1] = acc[nt][1];
+        red[(g + 8) * kC + nt * 8 + 2 * t] = acc[nt][2];
+        red[(g + 8) * kC + nt * 8 + 2 * t + 1] = acc[nt][3];
+      }
+    }
+    __syncthreads();
+    // ---- (3) masked dA (or scores A), the contraction with the state, the state update
+    if (MODE != 2) {
+      const int r = tid >> 4, i = tid & 15;
+      float s = 0.f;
+      if (i <= r) {
+#pragma unroll
+        for (int w = 0; w < 8; ++w) s += sRedA[w * kC * kC + tid];
+      }
+      sP[r * LDR + i] = s;
+    } else {   // A[r][i]: lanes over key channels, pairs dealt round the warps
+      for (int p = warp; p < kC * (kC + 1) / 2; p += 8) {
+        int r = 0, rem = p;
+        while (rem > r) { rem -= r + 1; ++r; }
+        const int i = rem;
+        float s = 0.f;
+#pragma unroll
+        for (int m = 0; m < DK / 32; ++m) {
+          const int d = lane + 32 * m;
+          s = fmaf(sQ[r * LDK + d] * sKt[i * LDK + d], expf(sB[r * LDK + d] - sB[i * LDK + d]), s);
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) {
+          sP[r * LDR + i] = s;
+          if (i != r) sP[i * LDR + r] = 0.f;
+        }
+      }
+    }
+    {
+      // contraction of the state with the chunk's dO (MODE 0), V (MODE 1) or Ke (MODE 2)
+      float acc[2][4] = {};
+      const float* opB = MODE == 0 ? sDO : (MODE == 1 ? sV : sKe);
+      constexpr int ldb = MODE == 2 ? LDK : LDV;
+#pragma unroll
+      for (int n = 0; n < 16; ++n) {
+        const int c0 = nbase + 8 * n + 2 * t;
+        const float af[4] = {st[n][0], st[n][2], st[n][1], st[n][3]};
+#pragma unroll
+        for (int rt = 0; rt < 2; ++rt) {
+          const float2 y = *reinterpret_cast<const float2*>(opB + (rt * 8 + g) * ldb + c0);
+          const float bf[2] = {y.x, y.y};
+          mma_tile<EXACT>(acc[rt], af, bf);
+        }
+      }
+      if (MODE != 2) {
+        float* red = sRed + warp * 16 * LDR;
+#pragma unroll
+        for (int rt = 0; rt < 2; ++rt) {
+          red[g * LDR + rt * 8 + 2 * t] = acc[rt][0];
+          red[g * LDR + rt * 8 + 2 * t + 1] = acc[rt][1];
+          red[(g + 8) * LDR + rt * 8 + 2 * t] = acc[rt][2];
+          red[(g + 8) * LDR + rt * 8 + 2 * t + 1] = acc[rt][3];
+        }
+      } else {
+        // dv tile [16 rows][128 columns of this half]: the state part now, the score part below
+        constexpr int ldo = 128 + 4;
+        const int jl = 16 * warp + g;
+#pragma unroll
+        for (int rt = 0; rt < 2; ++rt) {
+          sRed[(rt * 8 + 2 * t) * ldo + jl] = acc[rt][0];
+          sRed[(rt * 8 + 2 * t + 1) * ldo + jl] = acc[rt][1];
+          sRed[(rt * 8 + 2 * t) * ldo + jl + 8] = acc[rt][2];
+          sRed[(rt * 8 + 2 * t + 1) * ldo + jl + 8] = acc[rt][3];
+        }
+      }
+      // state update: scale by D, add the chunk's outer products
+      if (MODE != 2) {
+        const float dl = sD[m0 + g], dh = sD[m0 + g + 8];
+#pragma unroll
+        for (int n = 0; n < 16; ++n) {
+          st[n][0] *= dl; st[n][1] *= dl; st[n][2] *= dh; st[n][3] *= dh;
+        }
+        const float* opA = MODE == 0 ? sKe : sQe;
+        const float* opV = MODE == 0 ? sV : sDO;
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+          const int i0 = 8 * ks + t;
+          const float af[4] = {opA[i0 * LDK + m0 + g], opA[i0 * LDK + m0 + g + 8],
+                               opA[(i0 + 4) * LDK + m0 + g], opA[(i0 + 4) * LDK + m0 + g + 8]};
+#pragma unroll
+          for (int n = 0; n < 16; ++n) {
+            const int j = nbase + 8 * n + g;
+            const float bf[2] = {opV[i0 * LDV + j], opV[(i0 + 4) * LDV + j]};
+            mma_tile<EXACT>(st[n], af, bf);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int n = 0; n < 16; ++n) {
+          const float2 dd = *reinterpret_cast<const float2*>(sD + 8 * n + 2 * t);
+          st[n][0] *= dd.x; st[n][1] *= dd.y; st[n][2] *= dd.x; st[n][3] *= dd.y;
+        }
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+          const int r0 = 8 * ks + t;
+          const float af[4] = {sDO[r0 * LDV + m0 + g], sDO[r0 * LDV + m0 + g + 8],
+                               sDO[(r0 + 4) * LDV + m0 + g], sDO[(r0 + 4) * LDV + m0 + g + 8]};
+#pragma unroll
+          for (int n = 0; n < 16; ++n) {
+            const float bf[2] = {sQe[r0 * LDK + 8 * n + g], sQe[(r0 + 4) * LDK + 8 * n + g]};
+            mma_tile<EXACT>(st[n], af, bf);
+          }
+        }
+      }
+    }
+    __syncthreads();
+    // ---- (4) finish the chunk's gradients
+    if (MODE == 0) {
+      const int dl = tid & 63, d = 64 * half + dl;
+      const float* r0p = sRed + (2 * (dl >> 4)) * 16 * LDR + (dl & 15) * LDR;
+      const float* r1p = r0p + 16 * LDR;
+      for (int r = tid >> 6; r < nr; r += 4) {
+        const float br = sB[r * LDK + d];
+        float s = 0.f;
+        for (int i = 0; i <= r; ++i)
+          s = fmaf(sP[r * LDR + i] * sKt[i * LDK + d], expf(br - sB[i * LDK + d]), s);
+        s = fmaf(expf(br), r0p[r] + r1p[r], s);          // dq' = dL/d(scale q)
+        const long long o = (row0 + t0 + r) * DK + d;
+        ((T*)a.dq)[o] = from_f32<T>(a.scale * s);
+        a.u[o] = sQ[r * LDK + d] * s;                    // q . dq
+      }
+    } else if (MODE == 1) {
+      const int dl = tid & 63, d = 64 * half + dl;
+      const float* r0p = sRed + (2 * (dl >> 4)) * 16 * LDR + (dl & 15) * LDR;
+      const float* r1p = r0p + 16 * LDR;
+      const float bc = sB[(kC - 1) * LDK + d];
+      for (int i = tid >> 6; i < nr; i += 4) {
+        const float bi = sB[i * LDK + d];
+        float s = 0.f;
+        for (int r = i; r < nr; ++r)
+          s = fmaf(sP[r * LDR + i] * sQ[r * LDK + d], expf(sB[r * LDK + d] - bi), s);
+        s = fmaf(expf(bc - bi), r0p[i] + r1p[i], s);     // dL/d(ahat k)
+        const long long o = (row0 + t0 + i) * DK + d;
+        ((T*)a.dk)[o] = from_f32<T>(s * sKe[i * LDK + d]);
+        a.w[o] = sKt[i * LDK + d] * s;
+      }
+    } else {
+      constexpr int ldo = 128 + 4;
+      {   // add sum_{r>=i} A[r][i] dO[r][j] to the elements this thread wrote
+        const int jl = 16 * warp + g;
+#pragma unroll
+        for (int rt = 0; rt < 2; ++rt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int i = rt * 8 + 2 * t + (e & 1), j = jl + (e >> 1) * 8;
+            float s = sRed[i * ldo + j];
+            for (int r = i; r < nr; ++r) s = fmaf(sP[r * LDR + i], sDO[r * LDV + 128 * half + j], s);
+            sRed[i * ldo + j] = s;
+          }
+      }
+      __syncthreads();
+      const int i = tid >> 4, c8 = (tid & 15) * 8;
+      if (i < nr) {
+        float o8[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o8[e] = sRed[i * ldo + c8 + e];
+        store8<T>((T*)a.dv + (row0 + t0 + i) * DV + 128 * half + c8, o8);
+      }
+    }
+    __syncthreads();
+  }
+
+  // ---- after the last chunk
+  if (MODE == 0) {   // c[d] = sum_j dS_T[d][j] S_T[d][j]
+    float p0 = 0.f, p1 = 0.f;
+    if (a.dsT) {
+#pragma unroll
+      for (int n = 0; n < 16; ++n) {
+        const int c0 = nbase + 8 * n + 2 * t;
+        const float2 lo = *reinterpret_cast<const float2*>(a.dsT + s_off + (long long)(m0 + g) * DV + c0);
+        const float2 hi = *reinterpret_cast<const float2*>(a.dsT + s_off + (long long)(m0 + g + 8) * DV + c0);
+        p0 = fmaf(lo.x, st[n][0], fmaf(lo.y, st[n][1], p0));
+        p1 = fmaf(hi.x, st[n][2], fmaf(hi.y, st[n][3], p1));
+      }
+    }
+    p0 += __shfl_xor_sync(0xffffffffu, p0, 1);
+    p0 += __shfl_xor_sync(0xffffffffu, p0, 2);
+    p1 += __shfl_xor_sync(0xffffffffu, p1, 1);
+    p1 += __shfl_xor_sync(0xffffffffu, p1, 2);
+    if (t == 0) {
+      sRed[warp * 16 + g] = p0;
+      sRed[warp * 16 + g + 8] = p1;
+    }
+    __syncthreads();
+    if (tid < 64)
+      a.c[sh * DK + 64 * half + tid] = sRed[(2 * (tid >> 4)) * 16 + (tid & 15)] +
+                                        sRed[(2 * (tid >> 4) + 1) * 16 + (tid & 15)];
+  } else if (MODE == 1 && a.ds0) {
+#pragma unroll
+    for (int n = 0; n < 16; ++n) {
+      const int c0 = nbase + 8 * n + 2 * t;
+      *reinterpret_cast<float2*>(a.ds0 + s_off + (long long)(m0 + g) * DV + c0) = make_float2(st[n][0], st[n][1]);
+      *reinterpret_cast<float2*>(a.ds0 + s_off + (long long)(m0 + g + 8) * DV + c0) = make_float2(st[n][2], st[n][3]);
+    }
+  }
+}
+
+constexpr size_t kSweepSmem =
+    sizeof(float) * (6 * kC * LDK + 2 * kC * LDV + DK + kC * LDR + 8 * kC * kC + 8 * 16 * LDR);
+static_assert(16 * (128 + 4) <= 8 * 16 * LDR, "the dv tile fits the space of the partials");
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 2) ddts_bwd_sweep_kernel(const BwdArgs a) {
+  extern __shared__ __align__(16) float smem[];
+  const long long sh = blockIdx.x / 6;     // sequence * H + head
+  const int part = blockIdx.x % 6, mode = part >> 1, half = part & 1;
+  if (!a.cu && blockIdx.x == 0 && threadIdx.x == 0) a.hdr->status = RODIMUS_OK;
+  const int h = (int)(sh % a.H);
+  const long long n = sh / a.H;
+  long long row0;
+  int len;
+  if (a.cu) {
+    int lo = a.cu[n], hi = a.cu[n + 1];
+    lo = lo < 0 ? 0 : (lo > a.T ? a.T : lo);
+    hi = hi < lo ? lo : (hi > a.T ? a.T : hi);
+    row0 = (long long)h * a.T + lo;
+    len = hi - lo;
+  } else {
+    row0 = sh * a.T;
+    len = a.T;
+  }
+  if (mode == 0) bwd_sweep<T, 0>(a, smem, sh, half, row0, len);
+  else if (mode == 1) bwd_sweep<T, 1>(a, smem, sh, half, row0, len);
+  else bwd_sweep<T, 2>(a, smem, sh, half, row0, len);
+}
+
+// dL/dlog alpha by suffix sums over the sequence, then dx, dy (Eq. "alpha_def", chain rule):
+//   log alpha = -g tau,  log ahat = tau ln u(g)   with u = g (paper) or 1 - e^-g = sigmoid(x)
+//   dg   = -tau dla + w tau u'/u        dtau = -g dla + w ln u
+//   dx   = dg sigmoid(x)                dy   = dtau tau (1 - tau)
+// One CTA per (sequence, head): 128 channels x 4 time segments.
+template <typename T>
+__global__ void __launch_bounds__(512) ddts_bwd_gates_kernel(const BwdArgs a) {
+  __shared__ double seg_sum[4][DK];
+  const long long sh = blockIdx.x;
+  const int h = (int)(sh % a.H);
+  const long long n = sh / a.H;
+  long long row0;
+  int len;
+  if (a.cu) {
+    int lo = a.cu[n], hi = a.cu[n + 1];
+    lo = lo < 0 ? 0 : (lo > a.T ? a.T : lo);
+    hi = hi < lo ? lo : (hi > a.T ? a.T : hi);
+    row0 = (long long)h * a.T + lo;
+    len = hi - lo;
+  } else {
+    row0 = sh * a.T;
+    len = a.T;
+  }
+  const int d = threadIdx.x & (DK - 1), seg = threadIdx.x >> 7;
+  const int per = (len + 3) / 4;
+  const int lo = min(len, seg * per), hi = min(len, lo + per);
+  double s = 0.0;
+  for (int r = lo; r < hi; ++r) {
+    const long long i = (row0 + r) * DK + d;
+    s += (double)a.u[i] - (double)a.w[i];
+  }
+  seg_sum[seg][d] = s;
+  __syncthreads();
+  double acc = (double)a.c[sh * DK + d];
+  for (int s2 = seg + 1; s2 < 4; ++s2) acc += seg_sum[s2][d];
+  const T* gx = (const T*)a.gx;
+  const T* ty = (const T*)a.ty;
+  for (int r = hi - 1; r >= lo; --r) {
+    const long long i = (row0 + r) * DK + d;
+    const float w = a.w[i];
+    acc += (double)a.u[i] - (double)w;
+    const float dla = (float)acc;
+    const float x = to_f32(gx[i]), y = to_f32(ty[i]);
+    const float g = softplus_f32(x);
+    const float tau = y >= 0.f ? 1.f / (1.f + expf(-y)) : expf(y) / (1.f + expf(y));
+    const float sx = x >= 0.f ? 1.f / (1.f + expf(-x)) : expf(x) / (1.f + expf(x));
+    float lnu, dgx;   // dgx = (u'/u) * sigmoid(x)
+    if (a.ingate == RODIMUS_INGATE_POW_G) {
+      lnu = logf(g);
+      dgx = sx / g;
+    } else {
+      lnu = -softplus_f32(-x);
+      dgx = x >= 0.f ? expf(-x) / (1.f + expf(-x)) : 1.f / (1.f + expf(x));   // 1 - sigmoid(x)
+    }
+    const float dxv = -tau * dla * sx + w * tau * dgx;
+    const float dyv = (-g * dla + w * lnu) * tau * (1.f - tau);
+    ((T*)a.dx)[i] = from_f32<T>(dxv);
+    ((T*)a.dy)[i] = from_f32<T>(dyv);
+  }
+}
+
+std::atomic<unsigned long long> g_smem_done_bf16{0}, g_smem_done_f32{0};
+
+}  // namespace
+
+bool bwd_supported(const rodimus_ddts_bwd_params& p) { return p.dk == DK && p.dv == DV; }
+
+size_t bwd_scratch_bytes(const rodimus_ddts_bwd_params& p) {
+  const size_t rows = (size_t)p.B * p.H * p.T;
+  const size_t nseq = p.cu_seqlens ? (size_t)p.N : (size_t)p.B;
+  size_t b = sizeof(float) * (2 * rows * DK + nseq * p.H * DK);
+  return (b + 255) & ~(size_t)255;
+}
+
+cudaError_t launch_bwd(const rodimus_ddts_bwd_params& p, size_t scratch_offset, int* n_launches) {
+  *n_launches = 0;
+  BwdArgs a;
+  a.q = p.q; a.k = p.k; a.gx = p.gate_x; a.ty = p.temp_y; a.v = p.v; a.dout = p.d_o;
+  a.s0 = p.s0; a.dsT = p.d_sT;
+  a.dq = p.d_q; a.dk = p.d_k; a.dx = p.d_gate_x; a.dy = p.d_temp_y; a.dv = p.d_v; a.ds0 = p.d_s0;
+  const size_t rows = (size_t)p.B * p.H * p.T;
+  a.u = reinterpret_cast<float*>(reinterpret_cast<char*>(p.workspace) + scratch_offset);
+  a.w = a.u + rows * DK;
+  a.c = a.w + rows * DK;
+  a.cu = p.cu_seqlens;
+  a.hdr = reinterpret_cast<WorkspaceHeader*>(p.workspace);
+  a.H = p.H; a.T = p.T; a.n_seq = p.cu_seqlens ? p.N : p.B;
+  a.scale = p.scale; a.ingate = p.ingate;
+  const long long items = (long long)a.n_seq * p.H;
+  if (items == 0) return cudaSuccess;
+  if (items * 6 > 0x7fffffffLL) return cudaErrorInvalidValue;
+  int dev = 0, sms = 0;
+  cudaError_t e = current_device(&dev, &sms);
+  if (e != cudaSuccess) return e;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
+  if (p.dtype == RODIMUS_BF16) {
+    e = opt_in_shared_memory(ddts_bwd_sweep_kernel<__nv_bfloat16>, (int)kSweepSmem, dev, g_smem_done_bf16);
+    if (e != cudaSuccess) return e;
+    ddts_bwd_sweep_kernel<__nv_bfloat16><<<(unsigned)(items * 6), kThreads, kSweepSmem, st>>>(a);
+    ddts_bwd_gates_kernel<__nv_bfloat16><<<(unsigned)items, 512, 0, st>>>(a);
+  } else {
+    e = opt_in_shared_memory(ddts_bwd_sweep_kernel<float>, (int)kSweepSmem, dev, g_smem_done_f32);
+    if (e != cudaSuccess) return e;
+    ddts_bwd_sweep_kernel<float><<<(unsigned)(items * 6), kThreads, kSweepSmem, st>>>(a);
+    ddts_bwd_gates_kernel<float><<<(unsigned)items, 512, 0, st>>>(a);
+  }
+  *n_launches = 2;
+  return cudaGetLastError();
+}
+
+}  // namespace ddts

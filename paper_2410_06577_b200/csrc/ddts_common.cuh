@@ -44,6 +44,9 @@ cudaError_t launch_plan(const rodimus_ddts_fwd_params& p, int* n_launches);
 cudaError_t launch_fwd_simt(const rodimus_ddts_fwd_params& p, int* n_launches);
 cudaError_t launch_fwd_tc(const rodimus_ddts_fwd_params& p, int* n_launches);
 cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches);
+cudaError_t launch_bwd(const rodimus_ddts_bwd_params& p, size_t scratch_offset, int* n_launches);
+bool bwd_supported(const rodimus_ddts_bwd_params& p);
+size_t bwd_scratch_bytes(const rodimus_ddts_bwd_params& p);   // beyond the header and the order
 bool fwd_tc_supported(const rodimus_ddts_fwd_params& p);
 bool fwd_pair_supported(const rodimus_ddts_fwd_params& p);
 // Workspace a dense call needs if its sequences are to be split along time (0: no split).

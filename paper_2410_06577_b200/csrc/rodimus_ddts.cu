@@ -145,6 +145,77 @@ int rodimus_ddts_fwd(const rodimus_ddts_fwd_params* p) {
   return RODIMUS_OK;
 }
 
+static int check_bwd_sizes(const rodimus_ddts_bwd_params* p, bool varlen) {
+  if (p->struct_size != (int32_t)sizeof(rodimus_ddts_bwd_params)) return RODIMUS_ERR_DTYPE;
+  if (p->dtype != RODIMUS_BF16 && p->dtype != RODIMUS_F32) return RODIMUS_ERR_DTYPE;
+  if (p->ingate != RODIMUS_INGATE_POW_G && p->ingate != RODIMUS_INGATE_POW_SIGMOID)
+    return RODIMUS_ERR_DTYPE;
+  if (p->B < 0 || p->H < 0 || p->T < 0) return RODIMUS_ERR_SHAPE;
+  if (p->dk <= 0 || p->dv <= 0) return RODIMUS_ERR_SHAPE;
+  if (!ddts::bwd_supported(*p)) return RODIMUS_ERR_UNSUPPORTED;
+  if ((long long)p->B * p->H * p->T >= (1LL << 31)) return RODIMUS_ERR_SHAPE;
+  if (varlen) {
+    if (p->B != 1 || p->N < 0) return RODIMUS_ERR_SHAPE;
+    if ((long long)p->N * p->H >= (1LL << 31) / 8) return RODIMUS_ERR_SHAPE;
+  }
+  return RODIMUS_OK;
+}
+
+size_t rodimus_ddts_bwd_workspace_bytes(const rodimus_ddts_bwd_params* p) {
+  if (!p) return 0;
+  const bool varlen = p->cu_seqlens != nullptr || p->cu_seqlens_host != nullptr;
+  if (check_bwd_sizes(p, varlen) != RODIMUS_OK) return 0;
+  rodimus_ddts_bwd_params c = *p;
+  if (varlen && !c.cu_seqlens) c.cu_seqlens = c.cu_seqlens_host;   // only tested against NULL
+  return workspace_bytes_for(varlen ? p->N : 0) + ddts::bwd_scratch_bytes(c);
+}
+
+int rodimus_ddts_bwd(const rodimus_ddts_bwd_params* p) {
+  t_last_launches = 0;
+  if (!p) return RODIMUS_ERR_NULL;
+  const bool varlen = p->cu_seqlens != nullptr;
+  int rc = check_bwd_sizes(p, varlen);
+  if (rc != RODIMUS_OK) return rc;
+  if (!varlen && p->cu_seqlens_host) return RODIMUS_ERR_NULL;
+  const long long rows = (long long)p->B * p->H * p->T;
+  const long long n_seq = varlen ? p->N : p->B;
+  if (rows > 0 && (!p->q || !p->k || !p->gate_x || !p->temp_y || !p->v || !p->d_o || !p->d_q ||
+                   !p->d_k || !p->d_gate_x || !p->d_temp_y || !p->d_v))
+    return RODIMUS_ERR_NULL;
+  const void* ptrs[] = {p->q, p->k, p->gate_x, p->temp_y, p->v, p->d_o, p->s0, p->d_sT, p->d_q,
+                        p->d_k, p->d_gate_x, p->d_temp_y, p->d_v, p->d_s0, p->cu_seqlens};
+  for (const void* ptr : ptrs)
+    if (ptr && !aligned16(ptr)) return RODIMUS_ERR_ALIGN;
+  const size_t base = workspace_bytes_for(varlen ? p->N : 0);
+  if (!p->workspace || p->workspace_bytes < base + ddts::bwd_scratch_bytes(*p))
+    return RODIMUS_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(p->workspace) & 255u) return RODIMUS_ERR_ALIGN;
+  if (varlen && p->cu_seqlens_host) {
+    const int32_t* cu = p->cu_seqlens_host;
+    if (cu[0] != 0 || cu[p->N] != p->T) return RODIMUS_ERR_SEQLENS;
+    for (int n = 0; n < p->N; ++n)
+      if (cu[n + 1] < cu[n]) return RODIMUS_ERR_SEQLENS;
+  }
+  if (varlen && p->N == 0 && p->T != 0) return RODIMUS_ERR_SEQLENS;
+  if (n_seq * p->H == 0) return RODIMUS_OK;
+  int launches = 0, n = 0;
+  cudaError_t e = cudaSuccess;
+  if (varlen) {   // device-side check of cu_seqlens into the status word
+    rodimus_ddts_fwd_params f;
+    std::memset(&f, 0, sizeof(f));
+    f.cu_seqlens = p->cu_seqlens; f.N = p->N; f.T = p->T;
+    f.workspace = p->workspace; f.stream = p->stream;
+    e = ddts::launch_plan(f, &n);
+    launches += n;
+    if (e != cudaSuccess) return RODIMUS_ERR_CUDA;
+  }
+  e = ddts::launch_bwd(*p, base, &n);
+  launches += n;
+  if (e != cudaSuccess) return RODIMUS_ERR_CUDA;
+  t_last_launches = launches;
+  return RODIMUS_OK;
+}
+
 int rodimus_ddts_step(const rodimus_ddts_step_params* p) {
   t_last_launches = 0;
   if (!p) return RODIMUS_ERR_NULL;
@@ -207,6 +278,6 @@ const char* rodimus_status_str(int status) {
   }
 }
 
-int rodimus_version(void) { return 102; }
+int rodimus_version(void) { return 103; }
 
 }  // extern "C"

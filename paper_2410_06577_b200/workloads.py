@@ -5,7 +5,8 @@ fixed order and rounds them to the dtype the GPU consumes, so that the CPU oracl
 the CUDA library see identical bits.  Both the tests and the benchmark import it.
 
 Draw order for every workload: q, k, v, x (gate pre-activation), y (temperature
-pre-activation), s0 (if any).  Varlen lengths are drawn first from their own generator.
+pre-activation), s0 (if any); the gradients fed to the backward pass come from a generator of
+their own (d_o, then dL/dS_T if any).  Varlen lengths are drawn first from their own generator.
 All arrays are returned as float32 whose values are exactly representable in ``dtype``.
 """
 from __future__ import annotations
@@ -82,6 +83,19 @@ def make_prefill(seed: int, B: int, H: int, T: int, dk: int, dv: int, dtype: str
         s0 = (rng.standard_normal((nseq, H, dk, dv), dtype=np.float32) * np.float32(s0_std))
     cu = None if cu_seqlens is None else np.ascontiguousarray(cu_seqlens, dtype=np.int32)
     return PrefillInputs(dtype, q, k, x, y, v, s0, cu, name)
+
+
+def make_grads(seed: int, p: PrefillInputs, with_state: bool = True, state_std: float = 0.1):
+    """Incoming gradients for the backward pass: dL/do ~ N(0,1) in the workload's dtype and, if
+    asked for, dL/dS_T ~ N(0, state_std) in float32.  Returns (d_o [B,H,T,dv], d_sT or None)."""
+    rng = np.random.default_rng(seed)
+    B, H, T, dk, dv = p.shape
+    d_o = _round(rng.standard_normal((B, H, T, dv), dtype=np.float32), p.dtype)
+    d_sT = None
+    if with_state:
+        nseq = B if p.cu_seqlens is None else len(p.cu_seqlens) - 1
+        d_sT = rng.standard_normal((nseq, H, dk, dv), dtype=np.float32) * np.float32(state_std)
+    return d_o, d_sT
 
 
 def varlen_lengths(seed: int, n_seq: int, lo: int, hi: int) -> np.ndarray:

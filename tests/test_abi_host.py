@@ -44,13 +44,18 @@ def test_struct_layout_matches_header(tmp_path):
         "int main(void){printf(\"%zu %zu %zu %zu %zu %zu\\n\", sizeof(rodimus_ddts_fwd_params),"
         " offsetof(rodimus_ddts_fwd_params,q), offsetof(rodimus_ddts_fwd_params,stream),"
         " sizeof(rodimus_ddts_step_params), offsetof(rodimus_ddts_step_params,q),"
-        " offsetof(rodimus_ddts_step_params,stream));return 0;}\n")
+        " offsetof(rodimus_ddts_step_params,stream));"
+        "printf(\"%zu %zu %zu %zu\\n\", sizeof(rodimus_ddts_bwd_params),"
+        " offsetof(rodimus_ddts_bwd_params,q), offsetof(rodimus_ddts_bwd_params,d_s0),"
+        " offsetof(rodimus_ddts_bwd_params,stream));return 0;}\n")
     exe = tmp_path / "sz"
     subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)], check=True)
     out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
     got = [int(t) for t in out]
     want = [ctypes.sizeof(rd.FwdParams), rd.FwdParams.q.offset, rd.FwdParams.stream.offset,
-            ctypes.sizeof(rd.StepParams), rd.StepParams.q.offset, rd.StepParams.stream.offset]
+            ctypes.sizeof(rd.StepParams), rd.StepParams.q.offset, rd.StepParams.stream.offset,
+            ctypes.sizeof(rd.BwdParams), rd.BwdParams.q.offset, rd.BwdParams.d_s0.offset,
+            rd.BwdParams.stream.offset]
     assert got == want
 
 
@@ -153,6 +158,50 @@ def test_step_argument_errors(lib):
     assert rd.step_raw(_step(state=0)) == rd.ERR_NULL
     assert rd.step_raw(_step(v=FAKE + 4)) == rd.ERR_ALIGN
     assert rd.step_raw(_step(Nseq=0)) == rd.OK and rd.last_launch_count() == 0
+
+
+def _bwd(**kw):
+    p = rd.BwdParams()
+    p.struct_size = ctypes.sizeof(rd.BwdParams)
+    p.dtype, p.ingate = rd.BF16, rd.INGATE_POW_G
+    p.B, p.H, p.T, p.dk, p.dv = 2, 2, 64, 128, 256
+    p.scale = 1.0
+    for name in ("q", "k", "gate_x", "temp_y", "v", "d_o", "d_q", "d_k", "d_gate_x", "d_temp_y",
+                 "d_v"):
+        setattr(p, name, FAKE)
+    p.workspace = 0
+    p.workspace_bytes = 0
+    for key, val in kw.items():
+        setattr(p, key, val)
+    return p
+
+
+def test_bwd_argument_errors_and_workspace_size(lib):
+    assert lib.rodimus_ddts_bwd(None) == rd.ERR_NULL
+    assert rd.bwd_raw(_bwd(struct_size=8)) == rd.ERR_DTYPE
+    assert rd.bwd_raw(_bwd(dtype=5)) == rd.ERR_DTYPE
+    assert rd.bwd_raw(_bwd(ingate=2)) == rd.ERR_DTYPE
+    assert rd.bwd_raw(_bwd(T=-1)) == rd.ERR_SHAPE
+    assert rd.bwd_raw(_bwd(dk=64)) == rd.ERR_UNSUPPORTED      # widths the kernel is not built for
+    assert rd.bwd_raw(_bwd(dv=128)) == rd.ERR_UNSUPPORTED
+    assert rd.bwd_raw(_bwd(d_o=0)) == rd.ERR_NULL
+    assert rd.bwd_raw(_bwd(d_v=0)) == rd.ERR_NULL
+    assert rd.bwd_raw(_bwd(d_k=FAKE + 4)) == rd.ERR_ALIGN
+    assert rd.bwd_raw(_bwd(d_sT=FAKE + 8)) == rd.ERR_ALIGN
+    assert rd.bwd_raw(_bwd()) == rd.ERR_WORKSPACE
+    # header + two fp32 scratch rows of dk per token and head + one per (sequence, head)
+    want = 256 + 4 * (2 * 2 * 2 * 64 * 128 + 2 * 2 * 128)
+    assert rd.bwd_workspace_bytes(_bwd()) == want
+    assert rd.bwd_raw(_bwd(workspace=0x7F0000002000, workspace_bytes=want - 256)) == rd.ERR_WORKSPACE
+    assert rd.bwd_workspace_bytes(_bwd(dk=64)) == 0
+    assert rd.bwd_raw(_bwd(cu_seqlens=FAKE, N=3)) == rd.ERR_SHAPE       # packed needs B = 1
+    cu = np.array([0, 10, 5, 64], dtype=np.int32)
+    pv = _bwd(B=1, cu_seqlens=FAKE, cu_seqlens_host=cu.ctypes.data, N=3)
+    pv.workspace, pv.workspace_bytes = 0x7F0000002000, rd.bwd_workspace_bytes(pv)
+    assert pv.workspace_bytes == 256 + 256 + 4 * (2 * 2 * 64 * 128 + 3 * 2 * 128)
+    assert rd.bwd_raw(pv) == rd.ERR_SEQLENS
+    ok = _bwd(B=0, workspace=0x7F0000002000, workspace_bytes=4096)
+    assert rd.bwd_raw(ok) == rd.OK and rd.last_launch_count() == 0
 
 
 def test_missing_library_fails_loudly(tmp_path, monkeypatch):
