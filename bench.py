@@ -243,6 +243,7 @@ def run_reference(args, workload, p):
 # the gate math (6 per key channel with the paper's input gate: softplus 2, sigmoid 1, log g 1,
 # the two operand exponentials 2).
 DATASHEET = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+DATASHEET_TF32_RATIO = 1100.0 / 2250.0   # nominal dense tf32 : bf16
 
 
 def work_per_token_head(dk: int, dv: int, chunk: int = 64):
@@ -337,15 +338,36 @@ def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sf
             for n in ("q", "k", "x", "y"):
                 devt[n] = devt[n][:, :1].contiguous()
             alg_bytes -= (H - 1) * B * T * 4 * dk * el
-        prm = rd.fwd_params(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], o, s0, sT, cu, cu_host, **kw)
-        ws = rd.new_workspace(prm, device)
         units_per_step = p.tokens
-        kernel = "ddts_fwd_" + rd.fwd_kernel_name(prm)
         token_heads = B * H * T
+        if variant == "backward":
+            # the backward pass of the same workload: seeded dL/do and dL/dS_T in, all six
+            # gradients out; bytes = every input and every output once
+            from paper_2410_06577_b200 import workloads as wl_
+            g_o, g_s = wl_.make_grads(4321, p, True)
+            g_o = torch.from_numpy(g_o).to(tdt).to(device)
+            g_s = torch.from_numpy(g_s).to(device)
+            grads = [torch.empty_like(devt["q"]) for _ in range(4)] + [torch.empty_like(devt["v"])]
+            d_s0 = torch.empty_like(sT)
+            bprm = rd.bwd_params(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], g_o, *grads,
+                                 s0=s0, d_sT=g_s, d_s0=d_s0, cu_seqlens=cu, cu_seqlens_host=cu_host)
+            ws = torch.empty(rd.bwd_workspace_bytes(bprm), dtype=torch.uint8, device=device)
+            bprm.workspace, bprm.workspace_bytes = ws.data_ptr(), ws.numel()
+            kernel = "ddts_bwd_sweep_kernel"
+            alg_bytes = token_heads * (8 * dk + 3 * dv) * el + nseq * H * dk * dv * 4 * (2 + (s0 is not None))
 
-        def step(i):
-            rd.ddts_fwd(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], s0, cu, cu_host,
-                        out=o, final_state=sT, workspace=ws, **kw)
+            def step(i):
+                rc = rd.bwd_raw(bprm)
+                if rc != rd.OK:
+                    raise SystemExit(f"rodimus_ddts_bwd: {rd.status_str(rc)}")
+        else:
+            prm = rd.fwd_params(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], o, s0, sT, cu, cu_host, **kw)
+            ws = rd.new_workspace(prm, device)
+            kernel = "ddts_fwd_" + rd.fwd_kernel_name(prm)
+
+            def step(i):
+                rd.ddts_fwd(devt["q"], devt["k"], devt["x"], devt["y"], devt["v"], s0, cu, cu_host,
+                            out=o, final_state=sT, workspace=ws, **kw)
 
         o_host = torch.empty(o.shape, dtype=tdt).pin_memory()
         sT_host = torch.empty(sT.shape, dtype=torch.float32).pin_memory()
@@ -413,7 +435,13 @@ def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sf
     }
     wk = work_per_token_head(128, 256)
     bounds = {"hbm_us": alg_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6}
-    if not decode:
+    if variant == "backward":
+        # five [chunk x dk x dv] contractions per chunk (two in the forward sweep, three in the two
+        # reverse sweeps) on tf32 operands: measured bf16 peak x the nominal tf32/bf16 ratio
+        tf32_peak = peaks["bf16_tflops"] * DATASHEET_TF32_RATIO
+        bounds["tensor_us"] = token_heads * 10 * 128 * 256 / (tf32_peak * 1e12) * 1e6
+        bounds["tensor_peak_tflops"] = tf32_peak
+    elif not decode:
         bounds["tensor_us"] = token_heads * wk["tensor_flops"] / (peaks["bf16_tflops"] * 1e12) * 1e6
         bounds["sfu_us"] = (token_heads * wk["sfu_ops"] / sfu_rate * 1e6) if sfu_rate else "unmeasured"
         bounds["sfu_rate_gops"] = (sfu_rate / 1e9) if sfu_rate else "unmeasured"
@@ -428,7 +456,10 @@ def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sf
     if variant:
         rec["config"] = dict(rec["config"], variant={
             "block": "value gate beta_hat and feed-through d*x' fused (Eq. beta_def, Eq. rodimus_recurrent_form)",
-            "shared": "one q,k,x,y per token for all 16 heads ([B,1,T,dk])"}[variant])
+            "shared": "one q,k,x,y per token for all 16 heads ([B,1,T,dk])",
+            "backward": "backward pass (dq, dk, dx, dy, dv, ds0 from dL/do and dL/dS_T), two launches"}[variant])
+        if variant == "backward":
+            rec["metric"] = "DDTS prefill backward tokens/s"
     if with_e2e:
         e2e_steps = max(1, min(steps, 200 if decode else 5))
         e2e_regions = timed_regions(step_e2e, e2e_steps, 1, 0.0)
@@ -455,8 +486,9 @@ def run_ours(args, workload, p):
     peaks, peak_kind = load_peaks()
     sfu_rate = measure_sfu_rate(rd, torch, device)
 
-    line = measure(workload, p, args.steps, args.warmup, world, rank, local, peaks, peak_kind, sfu_rate)
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    line = measure(workload, p, args.steps, args.warmup, world, rank, local, peaks, peak_kind, sfu_rate,
+                   with_e2e=args.variant is None, variant=args.variant)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.variant is None:
         from oracle import ddts_oracle as orc
         decode = workload == "cfg3"
         u, s, what = oracle_sample_run(workload, p, budget_s=10.0)
@@ -480,11 +512,12 @@ def run_ours(args, workload, p):
                                                    "dtype", "config", "timed_regions", "clocks",
                                                    "gpu_launches", "roofline")}
             del pw
-        for name, variant in (("cfg1_block_terms", "block"), ("cfg1_shared_gates", "shared")):
+        for name, variant in (("cfg1_block_terms", "block"), ("cfg1_shared_gates", "shared"),
+                              ("cfg1_backward", "backward")):
             torch.cuda.empty_cache()
             pw = wl.config(1)
-            r = measure("cfg1", pw, 500, 5, world, rank, local, peaks, peak_kind, sfu_rate, with_e2e=False,
-                        variant=variant)
+            r = measure("cfg1", pw, 40 if variant == "backward" else 500, 5, world, rank, local, peaks,
+                        peak_kind, sfu_rate, with_e2e=False, variant=variant)
             extra[name] = {key: r[key] for key in ("metric", "value", "unit", "steps", "warmup", "ms_per_step",
                                                    "dtype", "config", "timed_regions", "clocks",
                                                    "gpu_launches", "roofline")}
@@ -503,6 +536,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg1")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--variant", choices=["block", "shared", "backward"], default=None,
+                    help="time a variant of the config-1 workload instead (for profiling; no e2e)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true",
                     help="only the workload named by --workload, no sub-records for the others")

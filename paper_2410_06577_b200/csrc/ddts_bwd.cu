@@ -102,25 +102,69 @@ __device__ __forceinline__ void mma_tf32(float (&c)[4], const float (&a)[4], con
         "r"(__float_as_uint(a[3])), "r"(__float_as_uint(b[0])), "r"(__float_as_uint(b[1])));
 }
 
-// c += a * b for one 16x8x8 tile.  EXACT: operands split as hi + lo (both tf32), the lo*lo term
-// (2^-22 of the product) dropped.
+// c += a * b for one 16x8x8 tile.  EXACT (fp32 build): operands split as hi + lo (both tf32),
+// the lo*lo term (2^-22 of the product) dropped.  Otherwise the operands go in as they are: what
+// comes from shared memory is bf16 data or was rounded to tf32 when it was stored, and of the
+// fp32 state fragments the instruction reads the tf32 part.
 template <bool EXACT>
 __device__ __forceinline__ void mma_tile(float (&c)[4], const float (&a)[4], const float (&b)[2]) {
-  float ah[4], bh[2];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) ah[i] = tf32_round(a[i]);
-#pragma unroll
-  for (int i = 0; i < 2; ++i) bh[i] = tf32_round(b[i]);
   if (EXACT) {
-    float al[4], bl[2];
+    float ah[4], bh[2], al[4], bl[2];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) al[i] = tf32_round(a[i] - ah[i]);
+    for (int i = 0; i < 4; ++i) {
+      ah[i] = tf32_round(a[i]);
+      al[i] = tf32_round(a[i] - ah[i]);
+    }
 #pragma unroll
-    for (int i = 0; i < 2; ++i) bl[i] = tf32_round(b[i] - bh[i]);
+    for (int i = 0; i < 2; ++i) {
+      bh[i] = tf32_round(b[i]);
+      bl[i] = tf32_round(b[i] - bh[i]);
+    }
     mma_tf32(c, al, bh);
     mma_tf32(c, ah, bl);
+    mma_tf32(c, ah, bh);
+  } else {
+    mma_tf32(c, a, b);
   }
-  mma_tf32(c, ah, bh);
+}
+
+template <bool FAST>
+__device__ __forceinline__ float exp_f(float x) { return FAST ? __expf(x) : expf(x); }
+
+// log alpha and log ahat of one channel (Eq. "alpha_def").  FAST (bf16 build): hardware
+// exponential / logarithm approximations (relative error about 2^-21, far inside the bf16 bar),
+// with the two places where they would lose everything written out: log(1 + e) for small e, and
+// log(softplus(x)) for very negative x, where softplus(x) = e^x (1 - e^x / 2 + ...).
+template <bool FAST>
+__device__ __forceinline__ void gate_logs(float x, float y, int ingate, float& la, float& lh) {
+  if (!FAST) {
+    gate_logs_f32(x, y, ingate, la, lh);
+    return;
+  }
+  const float e = __expf(-fabsf(x));
+  const float l1p = e < 0.0009765625f ? e * fmaf(-0.5f, e, 1.f) : __logf(1.f + e);
+  const float g = fmaxf(x, 0.f) + l1p;
+  const float tau = __fdividef(1.f, 1.f + __expf(-y));
+  la = -g * tau;
+  if (ingate == RODIMUS_INGATE_POW_G) {
+    lh = tau * (x < -8.f ? fmaf(-0.5f, e, x) : __logf(g));
+  } else {
+    lh = -tau * (fmaxf(-x, 0.f) + l1p);
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void load4(const T* p, float (&o)[4]);
+template <>
+__device__ __forceinline__ void load4<float>(const float* p, float (&o)[4]) {
+  const float4 a = *reinterpret_cast<const float4*>(p);
+  o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w;
+}
+template <>
+__device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16* p, float (&o)[4]) {
+  const uint2 a = *reinterpret_cast<const uint2*>(p);
+  o[0] = __uint_as_float(a.x << 16); o[1] = __uint_as_float(a.x & 0xffff0000u);
+  o[2] = __uint_as_float(a.y << 16); o[3] = __uint_as_float(a.y & 0xffff0000u);
 }
 
 // MODE 0: forward sweep (dq, u, c); 1: reverse sweep, state [d][j] (dk, w, ds0);
@@ -128,7 +172,9 @@ __device__ __forceinline__ void mma_tile(float (&c)[4], const float (&a)[4], con
 template <typename T, int MODE>
 __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, const int half,
                           const long long row0, const int len) {
-  constexpr bool EXACT = sizeof(T) == 4;
+  constexpr bool EXACT = sizeof(T) == 4, FAST = !EXACT;
+  constexpr int NCH = MODE == 2 ? DK : DK / 2;      // key channels whose gates this CTA needs
+  const int ch0 = MODE == 2 ? 0 : 64 * half;
   float* sQ = smem;                    // [kC][LDK] scale * q
   float* sKt = sQ + kC * LDK;          // ahat * k
   float* sLa = sKt + kC * LDK;         // log alpha
@@ -179,34 +225,39 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
   for (int ci = 0; ci < nchunks; ++ci) {
     const int t0 = (MODE == 0 ? ci : nchunks - 1 - ci) * kC;
     const int nr = min(kC, len - t0);
-    // ---- (1) loads and gates: one thread per (row, 8 channels); rows past the end read as zero
+    // ---- (1) loads and gates: a thread per (row, 4 channels) of the channels this CTA needs
+    // (its own half; all of them where the state is transposed); rows past the end read as zero
     {
-      const int r = tid >> 4, d8 = (tid & 15) * 8;
-      float fq[8], fk[8], fa[8], la[8];
-      if (r < nr) {
-        float fx[8], fy[8];
-        const long long i = (long long)(t0 + r) * DK + d8;
-        load8<T>(q + i, fq);
-        load8<T>(k + i, fk);
-        load8<T>(gx + i, fx);
-        load8<T>(ty + i, fy);
+      constexpr int kGroups = NCH / 4;
+#pragma unroll 1
+      for (int e = tid; e < kC * kGroups; e += kThreads) {
+        const int r = e / kGroups, d4 = ch0 + (e % kGroups) * 4;
+        float fq[4], fk[4], fa[4], la[4];
+        if (r < nr) {
+          float fx[4], fy[4];
+          const long long i = (long long)(t0 + r) * DK + d4;
+          load4<T>(q + i, fq);
+          load4<T>(k + i, fk);
+          load4<T>(gx + i, fx);
+          load4<T>(ty + i, fy);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          float lh;
-          gate_logs_f32(fx[e], fy[e], a.ingate, la[e], lh);
-          fa[e] = expf(lh);
-          fk[e] *= fa[e];
-          fq[e] *= a.scale;
+          for (int x = 0; x < 4; ++x) {
+            float lh;
+            gate_logs<FAST>(fx[x], fy[x], a.ingate, la[x], lh);
+            fa[x] = exp_f<FAST>(lh);
+            fk[x] *= fa[x];
+            fq[x] *= a.scale;
+          }
+        } else {
+#pragma unroll
+          for (int x = 0; x < 4; ++x) fq[x] = fk[x] = fa[x] = la[x] = 0.f;
         }
-      } else {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) fq[e] = fk[e] = fa[e] = la[e] = 0.f;
+        *reinterpret_cast<float4*>(sQ + r * LDK + d4) = make_float4(fq[0], fq[1], fq[2], fq[3]);
+        *reinterpret_cast<float4*>(sKt + r * LDK + d4) = make_float4(fk[0], fk[1], fk[2], fk[3]);
+        *reinterpret_cast<float4*>(sLa + r * LDK + d4) = make_float4(la[0], la[1], la[2], la[3]);
+        if (MODE == 1) *reinterpret_cast<float4*>(sKe + r * LDK + d4) = make_float4(fa[0], fa[1], fa[2], fa[3]);
       }
-      store8<float>(sQ + r * LDK + d8, fq);
-      store8<float>(sKt + r * LDK + d8, fk);
-      store8<float>(sLa + r * LDK + d8, la);
-      if (MODE == 1) store8<float>(sKe + r * LDK + d8, fa);
-#pragma unroll
+#pragma unroll 1
       for (int p = 0; p < 2; ++p) {
         const int e = tid + p * kThreads, rr = e >> 5, c8 = (e & 31) * 8;
         float fv[8], fd[8];
@@ -223,28 +274,34 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
       }
     }
     __syncthreads();
-    // ---- (2) cumulative decay, scaled operands; partial dA on the tensor cores
+    // ---- (2) cumulative decay and scaled operands (rounded to tf32 where they only feed the
+    // tensor cores); partial dA on the tensor cores
     {
-      const int d = tid & (DK - 1), role = tid >> 7;
-      float b[kC], acc = 0.f;
-#pragma unroll
+      // job 0: b and Qe, job 1: D and Ke; with half the channels the jobs are split once more
+      constexpr int kJobs = kThreads / NCH;                 // 4 (own half) or 2 (all channels)
+      const int d = ch0 + (tid % NCH), job = tid / NCH;
+      const bool do_b = job == 0, do_qe = MODE != 0 && job == (kJobs == 4 ? 1 : 0);
+      const bool do_ke = MODE != 1 && job == (kJobs == 4 ? 2 : 1), do_d = job == kJobs - 1;
+      float acc = 0.f;
+#pragma unroll 4
       for (int r = 0; r < kC; ++r) {
         acc += sLa[r * LDK + d];
-        b[r] = acc;
+        if (do_b) sB[r * LDK + d] = acc;
+        if (do_qe) {
+          const float x = sQ[r * LDK + d] * exp_f<FAST>(acc);
+          sQe[r * LDK + d] = FAST ? tf32_round(x) : x;
+        }
       }
-      if (role == 0) {
-#pragma unroll
+      if (do_ke) {
+        float part = 0.f;
+#pragma unroll 4
         for (int r = 0; r < kC; ++r) {
-          sB[r * LDK + d] = b[r];
-          sQe[r * LDK + d] = sQ[r * LDK + d] * expf(b[r]);
-        }
-      } else {
-        sD[d] = expf(acc);
-        if (MODE != 1) {
-#pragma unroll
-          for (int r = 0; r < kC; ++r) sKe[r * LDK + d] = sKt[r * LDK + d] * expf(acc - b[r]);
+          part += sLa[r * LDK + d];      // same additions in the same order as above
+          const float x = sKt[r * LDK + d] * exp_f<FAST>(acc - part);
+          sKe[r * LDK + d] = FAST ? tf32_round(x) : x;
         }
       }
+      if (do_d) sD[d] = exp_f<FAST>(acc);
     }
     if (MODE != 2) {   // dA[r][i] = sum_j dO[r][j] V[i][j], this warp's 32 value columns
       float acc[2][4] = {};
@@ -281,6 +338,7 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
       }
       sP[r * LDR + i] = s;
     } else {   // A[r][i]: lanes over key channels, pairs dealt round the warps
+#pragma unroll 1
       for (int p = warp; p < kC * (kC + 1) / 2; p += 8) {
         int r = 0, rem = p;
         while (rem > r) { rem -= r + 1; ++r; }
@@ -289,7 +347,7 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
 #pragma unroll
         for (int m = 0; m < DK / 32; ++m) {
           const int d = lane + 32 * m;
-          s = fmaf(sQ[r * LDK + d] * sKt[i * LDK + d], expf(sB[r * LDK + d] - sB[i * LDK + d]), s);
+          s = fmaf(sQ[r * LDK + d] * sKt[i * LDK + d], exp_f<FAST>(sB[r * LDK + d] - sB[i * LDK + d]), s);
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
@@ -382,12 +440,14 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
       const int dl = tid & 63, d = 64 * half + dl;
       const float* r0p = sRed + (2 * (dl >> 4)) * 16 * LDR + (dl & 15) * LDR;
       const float* r1p = r0p + 16 * LDR;
+#pragma unroll 1
       for (int r = tid >> 6; r < nr; r += 4) {
         const float br = sB[r * LDK + d];
         float s = 0.f;
+#pragma unroll 2
         for (int i = 0; i <= r; ++i)
-          s = fmaf(sP[r * LDR + i] * sKt[i * LDK + d], expf(br - sB[i * LDK + d]), s);
-        s = fmaf(expf(br), r0p[r] + r1p[r], s);          // dq' = dL/d(scale q)
+          s = fmaf(sP[r * LDR + i] * sKt[i * LDK + d], exp_f<FAST>(br - sB[i * LDK + d]), s);
+        s = fmaf(exp_f<FAST>(br), r0p[r] + r1p[r], s);          // dq' = dL/d(scale q)
         const long long o = (row0 + t0 + r) * DK + d;
         ((T*)a.dq)[o] = from_f32<T>(a.scale * s);
         a.u[o] = sQ[r * LDK + d] * s;                    // q . dq
@@ -397,12 +457,14 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
       const float* r0p = sRed + (2 * (dl >> 4)) * 16 * LDR + (dl & 15) * LDR;
       const float* r1p = r0p + 16 * LDR;
       const float bc = sB[(kC - 1) * LDK + d];
+#pragma unroll 1
       for (int i = tid >> 6; i < nr; i += 4) {
         const float bi = sB[i * LDK + d];
         float s = 0.f;
+#pragma unroll 2
         for (int r = i; r < nr; ++r)
-          s = fmaf(sP[r * LDR + i] * sQ[r * LDK + d], expf(sB[r * LDK + d] - bi), s);
-        s = fmaf(expf(bc - bi), r0p[i] + r1p[i], s);     // dL/d(ahat k)
+          s = fmaf(sP[r * LDR + i] * sQ[r * LDK + d], exp_f<FAST>(sB[r * LDK + d] - bi), s);
+        s = fmaf(exp_f<FAST>(bc - bi), r0p[i] + r1p[i], s);     // dL/d(ahat k)
         const long long o = (row0 + t0 + i) * DK + d;
         ((T*)a.dk)[o] = from_f32<T>(s * sKe[i * LDK + d]);
         a.w[o] = sKt[i * LDK + d] * s;
