@@ -275,33 +275,53 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
     }
     __syncthreads();
     // ---- (2) cumulative decay and scaled operands (rounded to tf32 where they only feed the
-    // tensor cores); partial dA on the tensor cores
+    // tensor cores); partial dA on the tensor cores.
+    // Where no channel decays by more than e^-60 over the chunk, exp(b_r - b_i) is factored as
+    // exp(b_r) exp(-b_i) (Ki = kt . exp(-b) stays below e^60 |kt|) and the sums over pairs become
+    // plain contractions; otherwise the chunk takes the pair-by-pair form with the difference
+    // formed before the exponential, which is exact for any decay.
+    bool strong;
     {
-      // job 0: b and Qe, job 1: D and Ke; with half the channels the jobs are split once more
+      // job 0: b (and Qe), last job: D; Ke, Ki on the jobs between (all channels: two jobs only)
       constexpr int kJobs = kThreads / NCH;                 // 4 (own half) or 2 (all channels)
       const int d = ch0 + (tid % NCH), job = tid / NCH;
-      const bool do_b = job == 0, do_qe = MODE != 0 && job == (kJobs == 4 ? 1 : 0);
-      const bool do_ke = MODE != 1 && job == (kJobs == 4 ? 2 : 1), do_d = job == kJobs - 1;
-      float acc = 0.f;
+      float tot = 0.f;
+#pragma unroll
+      for (int r = 0; r < kC; ++r) tot += sLa[r * LDK + d];
+      strong = __syncthreads_or(tot < -60.f) != 0;
+      const bool do_qe = MODE != 0 && job == (kJobs == 4 ? 1 : 0);
+      const bool do_ke = MODE != 1 && job == (kJobs == 4 ? 2 : 1);
+      const bool do_ki = MODE == 0 && job == 1 && !strong;   // all channels: with Ke, below
+      if (job == 0 || do_qe) {
+        float acc = 0.f;
 #pragma unroll 4
-      for (int r = 0; r < kC; ++r) {
-        acc += sLa[r * LDK + d];
-        if (do_b) sB[r * LDK + d] = acc;
-        if (do_qe) {
-          const float x = sQ[r * LDK + d] * exp_f<FAST>(acc);
-          sQe[r * LDK + d] = FAST ? tf32_round(x) : x;
+        for (int r = 0; r < kC; ++r) {
+          acc += sLa[r * LDK + d];
+          if (job == 0) sB[r * LDK + d] = acc;
+          if (do_qe) {
+            const float x = sQ[r * LDK + d] * exp_f<FAST>(acc);
+            sQe[r * LDK + d] = FAST ? tf32_round(x) : x;
+          }
         }
       }
-      if (do_ke) {
+      if (do_ke || do_ki) {
         float part = 0.f;
 #pragma unroll 4
         for (int r = 0; r < kC; ++r) {
           part += sLa[r * LDK + d];      // same additions in the same order as above
-          const float x = sKt[r * LDK + d] * exp_f<FAST>(acc - part);
-          sKe[r * LDK + d] = FAST ? tf32_round(x) : x;
+          const float kt = sKt[r * LDK + d];
+          if (do_ke) {
+            const float x = kt * exp_f<FAST>(tot - part);
+            sKe[r * LDK + d] = FAST ? tf32_round(x) : x;
+          }
+          if (do_ki) sQe[r * LDK + d] = kt * exp_f<FAST>(-part);
+          if (MODE == 2 && !strong) {    // this thread is the array's only reader in this phase
+            const float x = kt * exp_f<FAST>(-part);
+            sKt[r * LDK + d] = FAST ? tf32_round(x) : x;
+          }
         }
       }
-      if (do_d) sD[d] = exp_f<FAST>(acc);
+      if (job == kJobs - 1) sD[d] = exp_f<FAST>(tot);
     }
     if (MODE != 2) {   // dA[r][i] = sum_j dO[r][j] V[i][j], this warp's 32 value columns
       float acc[2][4] = {};
@@ -337,7 +357,7 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
         for (int w = 0; w < 8; ++w) s += sRedA[w * kC * kC + tid];
       }
       sP[r * LDR + i] = s;
-    } else {   // A[r][i]: lanes over key channels, pairs dealt round the warps
+    } else if (strong) {   // A[r][i] pair by pair: lanes over key channels, pairs dealt round the warps
 #pragma unroll 1
       for (int p = warp; p < kC * (kC + 1) / 2; p += 8) {
         int r = 0, rem = p;
@@ -356,10 +376,33 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
           if (i != r) sP[i * LDR + r] = 0.f;
         }
       }
-    }
-    {
-      // contraction of the state with the chunk's dO (MODE 0), V (MODE 1) or Ke (MODE 2)
+    } else {               // A = Qe Ki^T on the tensor cores, this warp's 16 key channels
       float acc[2][4] = {};
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks) {
+        const int d0 = 16 * warp + 8 * ks + 2 * t;
+        const float2 x0 = *reinterpret_cast<const float2*>(sQe + g * LDK + d0);
+        const float2 x1 = *reinterpret_cast<const float2*>(sQe + (g + 8) * LDK + d0);
+        const float af[4] = {x0.x, x1.x, x0.y, x1.y};
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+          const float2 y = *reinterpret_cast<const float2*>(sKt + (nt * 8 + g) * LDK + d0);
+          const float bf[2] = {y.x, y.y};
+          mma_tile<EXACT>(acc[nt], af, bf);
+        }
+      }
+      float* red = sRedA + warp * kC * kC;
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        red[g * kC + nt * 8 + 2 * t] = acc[nt][0];
+        red[g * kC + nt * 8 + 2 * t + 1] = acc[nt][1];
+        red[(g + 8) * kC + nt * 8 + 2 * t] = acc[nt][2];
+        red[(g + 8) * kC + nt * 8 + 2 * t + 1] = acc[nt][3];
+      }
+    }
+    // contraction of the state with the chunk's dO (MODE 0), V (MODE 1) or Ke (MODE 2)
+    float cacc[2][4] = {};
+    {
       const float* opB = MODE == 0 ? sDO : (MODE == 1 ? sV : sKe);
       constexpr int ldb = MODE == 2 ? LDK : LDV;
 #pragma unroll
@@ -370,28 +413,18 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
         for (int rt = 0; rt < 2; ++rt) {
           const float2 y = *reinterpret_cast<const float2*>(opB + (rt * 8 + g) * ldb + c0);
           const float bf[2] = {y.x, y.y};
-          mma_tile<EXACT>(acc[rt], af, bf);
+          mma_tile<EXACT>(cacc[rt], af, bf);
         }
+        if ((n & 3) == 3) asm volatile("" ::: "memory");   // keep the operand loads near their use
       }
       if (MODE != 2) {
         float* red = sRed + warp * 16 * LDR;
 #pragma unroll
         for (int rt = 0; rt < 2; ++rt) {
-          red[g * LDR + rt * 8 + 2 * t] = acc[rt][0];
-          red[g * LDR + rt * 8 + 2 * t + 1] = acc[rt][1];
-          red[(g + 8) * LDR + rt * 8 + 2 * t] = acc[rt][2];
-          red[(g + 8) * LDR + rt * 8 + 2 * t + 1] = acc[rt][3];
-        }
-      } else {
-        // dv tile [16 rows][128 columns of this half]: the state part now, the score part below
-        constexpr int ldo = 128 + 4;
-        const int jl = 16 * warp + g;
-#pragma unroll
-        for (int rt = 0; rt < 2; ++rt) {
-          sRed[(rt * 8 + 2 * t) * ldo + jl] = acc[rt][0];
-          sRed[(rt * 8 + 2 * t + 1) * ldo + jl] = acc[rt][1];
-          sRed[(rt * 8 + 2 * t) * ldo + jl + 8] = acc[rt][2];
-          sRed[(rt * 8 + 2 * t + 1) * ldo + jl + 8] = acc[rt][3];
+          red[g * LDR + rt * 8 + 2 * t] = cacc[rt][0];
+          red[g * LDR + rt * 8 + 2 * t + 1] = cacc[rt][1];
+          red[(g + 8) * LDR + rt * 8 + 2 * t] = cacc[rt][2];
+          red[(g + 8) * LDR + rt * 8 + 2 * t + 1] = cacc[rt][3];
         }
       }
       // state update: scale by D, add the chunk's outer products
@@ -413,6 +446,7 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
             const int j = nbase + 8 * n + g;
             const float bf[2] = {opV[i0 * LDV + j], opV[(i0 + 4) * LDV + j]};
             mma_tile<EXACT>(st[n], af, bf);
+            if ((n & 3) == 3) asm volatile("" ::: "memory");
           }
         }
       } else {
@@ -430,6 +464,7 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
           for (int n = 0; n < 16; ++n) {
             const float bf[2] = {sQe[r0 * LDK + 8 * n + g], sQe[(r0 + 4) * LDK + 8 * n + g]};
             mma_tile<EXACT>(st[n], af, bf);
+            if ((n & 3) == 3) asm volatile("" ::: "memory");
           }
         }
       }
@@ -444,11 +479,18 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
       for (int r = tid >> 6; r < nr; r += 4) {
         const float br = sB[r * LDK + d];
         float s = 0.f;
+        if (strong) {
 #pragma unroll 2
-        for (int i = 0; i <= r; ++i)
-          s = fmaf(sP[r * LDR + i] * sKt[i * LDK + d], exp_f<FAST>(br - sB[i * LDK + d]), s);
-        s = fmaf(exp_f<FAST>(br), r0p[r] + r1p[r], s);          // dq' = dL/d(scale q)
-        const long long o = (row0 + t0 + r) * DK + d;
+          for (int i = 0; i <= r; ++i)
+            s = fmaf(sP[r * LDR + i] * sKt[i * LDK + d], exp_f<FAST>(br - sB[i * LDK + d]), s);
+          s = fmaf(exp_f<FAST>(br), r0p[r] + r1p[r], s);
+        } else {
+          s = r0p[r] + r1p[r];
+#pragma unroll 4
+          for (int i = 0; i <= r; ++i) s = fmaf(sP[r * LDR + i], sQe[i * LDK + d], s);   // Ki
+          s *= exp_f<FAST>(br);
+        }
+        const long long o = (row0 + t0 + r) * DK + d;   // s = dL/d(scale q)
         ((T*)a.dq)[o] = from_f32<T>(a.scale * s);
         a.u[o] = sQ[r * LDK + d] * s;                    // q . dq
       }
@@ -461,27 +503,54 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
       for (int i = tid >> 6; i < nr; i += 4) {
         const float bi = sB[i * LDK + d];
         float s = 0.f;
+        if (strong) {
 #pragma unroll 2
-        for (int r = i; r < nr; ++r)
-          s = fmaf(sP[r * LDR + i] * sQ[r * LDK + d], exp_f<FAST>(sB[r * LDK + d] - bi), s);
-        s = fmaf(exp_f<FAST>(bc - bi), r0p[i] + r1p[i], s);     // dL/d(ahat k)
-        const long long o = (row0 + t0 + i) * DK + d;
+          for (int r = i; r < nr; ++r)
+            s = fmaf(sP[r * LDR + i] * sQ[r * LDK + d], exp_f<FAST>(sB[r * LDK + d] - bi), s);
+          s = fmaf(exp_f<FAST>(bc - bi), r0p[i] + r1p[i], s);
+        } else {
+          s = sD[d] * (r0p[i] + r1p[i]);
+#pragma unroll 4
+          for (int r = i; r < nr; ++r) s = fmaf(sP[r * LDR + i], sQe[r * LDK + d], s);
+          s *= exp_f<FAST>(-bi);
+        }
+        const long long o = (row0 + t0 + i) * DK + d;   // s = dL/d(ahat k)
         ((T*)a.dk)[o] = from_f32<T>(s * sKe[i * LDK + d]);
         a.w[o] = sKt[i * LDK + d] * s;
       }
     } else {
       constexpr int ldo = 128 + 4;
-      {   // add sum_{r>=i} A[r][i] dO[r][j] to the elements this thread wrote
+      if (!strong) {   // finish the scores: sum the warps' parts, keep i <= r
+        const int r = tid >> 4, i = tid & 15;
+        float s = 0.f;
+        if (i <= r) {
+#pragma unroll
+          for (int w = 0; w < 8; ++w) s += sRedA[w * kC * kC + tid];
+        }
+        sP[r * LDR + i] = s;
+      }
+      __syncthreads();
+      // dv^T[j][i] += sum_r dO[r][j] A[r][i] (A is zero above the diagonal and in rows past the end)
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks) {
+        const int r0 = 8 * ks + t;
+        const float af[4] = {sDO[r0 * LDV + m0 + g], sDO[r0 * LDV + m0 + g + 8],
+                             sDO[(r0 + 4) * LDV + m0 + g], sDO[(r0 + 4) * LDV + m0 + g + 8]};
+#pragma unroll
+        for (int rt = 0; rt < 2; ++rt) {
+          const float bf[2] = {sP[r0 * LDR + rt * 8 + g], sP[(r0 + 4) * LDR + rt * 8 + g]};
+          mma_tile<true>(cacc[rt], af, bf);   // scores are fp32 values: keep both tf32 parts
+        }
+      }
+      {
         const int jl = 16 * warp + g;
 #pragma unroll
-        for (int rt = 0; rt < 2; ++rt)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int i = rt * 8 + 2 * t + (e & 1), j = jl + (e >> 1) * 8;
-            float s = sRed[i * ldo + j];
-            for (int r = i; r < nr; ++r) s = fmaf(sP[r * LDR + i], sDO[r * LDV + 128 * half + j], s);
-            sRed[i * ldo + j] = s;
-          }
+        for (int rt = 0; rt < 2; ++rt) {
+          sRed[(rt * 8 + 2 * t) * ldo + jl] = cacc[rt][0];
+          sRed[(rt * 8 + 2 * t + 1) * ldo + jl] = cacc[rt][1];
+          sRed[(rt * 8 + 2 * t) * ldo + jl + 8] = cacc[rt][2];
+          sRed[(rt * 8 + 2 * t + 1) * ldo + jl + 8] = cacc[rt][3];
+        }
       }
       __syncthreads();
       const int i = tid >> 4, c8 = (tid & 15) * 8;

@@ -81,6 +81,12 @@ def test_bwd_alternate_input_gate_and_strong_decay(dtype):
     p = wl.make_prefill(301, 1, 2, 90, 128, 256, dtype, gate_mean=2.0, s0_std=0.1, name="bwd_strong")
     _check(p, 302, True, ingate=rd.INGATE_POW_SIGMOID)
     _check(p, 303, True, ingate=rd.INGATE_POW_G)
+    # pre-activations around +12: a chunk of 16 steps decays by far more than e^-60, which the
+    # kernel answers with its pair-by-pair form; milder chunks of the same call take the factored one
+    p = wl.make_prefill(304, 1, 2, 70, 128, 256, dtype, gate_mean=12.0, s0_std=0.1, name="bwd_very_strong")
+    p.x[:, :, 32:48] = wl.make_prefill(305, 1, 2, 16, 128, 256, dtype, gate_mean=-3.0).x
+    _check(p, 306, True, ingate=rd.INGATE_POW_G)
+    _check(p, 307, True, ingate=rd.INGATE_POW_SIGMOID)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
