@@ -226,38 +226,23 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
     const int t0 = (MODE == 0 ? ci : nchunks - 1 - ci) * kC;
     const int nr = min(kC, len - t0);
     // ---- (1) loads and gates: a thread per (row, 4 channels) of the channels this CTA needs
-    // (its own half; all of them where the state is transposed); rows past the end read as zero
+    // (its own half; all of them where the state is transposed); rows past the end read as zero.
+    // All global loads of the chunk are issued before the first of them is used.
     {
-      constexpr int kGroups = NCH / 4;
-#pragma unroll 1
-      for (int e = tid; e < kC * kGroups; e += kThreads) {
-        const int r = e / kGroups, d4 = ch0 + (e % kGroups) * 4;
-        float fq[4], fk[4], fa[4], la[4];
+      constexpr int kGroups = NCH / 4, kIter = kC * kGroups / kThreads;   // 1 or 2
+      float fq[kIter][4], fk[kIter][4], fx[kIter][4], fy[kIter][4];
+#pragma unroll
+      for (int it = 0; it < kIter; ++it) {
+        const int e = tid + it * kThreads, r = e / kGroups, d4 = ch0 + (e % kGroups) * 4;
         if (r < nr) {
-          float fx[4], fy[4];
           const long long i = (long long)(t0 + r) * DK + d4;
-          load4<T>(q + i, fq);
-          load4<T>(k + i, fk);
-          load4<T>(gx + i, fx);
-          load4<T>(ty + i, fy);
-#pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            float lh;
-            gate_logs<FAST>(fx[x], fy[x], a.ingate, la[x], lh);
-            fa[x] = exp_f<FAST>(lh);
-            fk[x] *= fa[x];
-            fq[x] *= a.scale;
-          }
-        } else {
-#pragma unroll
-          for (int x = 0; x < 4; ++x) fq[x] = fk[x] = fa[x] = la[x] = 0.f;
+          load4<T>(q + i, fq[it]);
+          load4<T>(k + i, fk[it]);
+          load4<T>(gx + i, fx[it]);
+          load4<T>(ty + i, fy[it]);
         }
-        *reinterpret_cast<float4*>(sQ + r * LDK + d4) = make_float4(fq[0], fq[1], fq[2], fq[3]);
-        *reinterpret_cast<float4*>(sKt + r * LDK + d4) = make_float4(fk[0], fk[1], fk[2], fk[3]);
-        *reinterpret_cast<float4*>(sLa + r * LDK + d4) = make_float4(la[0], la[1], la[2], la[3]);
-        if (MODE == 1) *reinterpret_cast<float4*>(sKe + r * LDK + d4) = make_float4(fa[0], fa[1], fa[2], fa[3]);
       }
-#pragma unroll 1
+#pragma unroll
       for (int p = 0; p < 2; ++p) {
         const int e = tid + p * kThreads, rr = e >> 5, c8 = (e & 31) * 8;
         float fv[8], fd[8];
@@ -271,6 +256,28 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
         }
         store8<float>(sV + rr * LDV + c8, fv);
         store8<float>(sDO + rr * LDV + c8, fd);
+      }
+#pragma unroll
+      for (int it = 0; it < kIter; ++it) {
+        const int e = tid + it * kThreads, r = e / kGroups, d4 = ch0 + (e % kGroups) * 4;
+        float fa[4], la[4];
+        if (r < nr) {
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            float lh;
+            gate_logs<FAST>(fx[it][x], fy[it][x], a.ingate, la[x], lh);
+            fa[x] = exp_f<FAST>(lh);
+            fk[it][x] *= fa[x];
+            fq[it][x] *= a.scale;
+          }
+        } else {
+#pragma unroll
+          for (int x = 0; x < 4; ++x) fq[it][x] = fk[it][x] = fa[x] = la[x] = 0.f;
+        }
+        *reinterpret_cast<float4*>(sQ + r * LDK + d4) = make_float4(fq[it][0], fq[it][1], fq[it][2], fq[it][3]);
+        *reinterpret_cast<float4*>(sKt + r * LDK + d4) = make_float4(fk[it][0], fk[it][1], fk[it][2], fk[it][3]);
+        *reinterpret_cast<float4*>(sLa + r * LDK + d4) = make_float4(la[0], la[1], la[2], la[3]);
+        if (MODE == 1) *reinterpret_cast<float4*>(sKe + r * LDK + d4) = make_float4(fa[0], fa[1], fa[2], fa[3]);
       }
     }
     __syncthreads();
@@ -632,11 +639,13 @@ __global__ void __launch_bounds__(kThreads, 2) ddts_bwd_sweep_kernel(const BwdAr
 //   log alpha = -g tau,  log ahat = tau ln u(g)   with u = g (paper) or 1 - e^-g = sigmoid(x)
 //   dg   = -tau dla + w tau u'/u        dtau = -g dla + w ln u
 //   dx   = dg sigmoid(x)                dy   = dtau tau (1 - tau)
-// One CTA per (sequence, head): 128 channels x 4 time segments.
+// One CTA per (sequence, head, 32 channels): 32 channels x 16 time segments.
+constexpr int kGateCh = 32, kGateSegs = 16;
 template <typename T>
-__global__ void __launch_bounds__(512) ddts_bwd_gates_kernel(const BwdArgs a) {
-  __shared__ double seg_sum[4][DK];
-  const long long sh = blockIdx.x;
+__global__ void __launch_bounds__(kGateCh * kGateSegs) ddts_bwd_gates_kernel(const BwdArgs a) {
+  __shared__ double seg_sum[kGateSegs][kGateCh];
+  const long long sh = blockIdx.x / (DK / kGateCh);
+  const int dch = (blockIdx.x % (DK / kGateCh)) * kGateCh;
   const int h = (int)(sh % a.H);
   const long long n = sh / a.H;
   long long row0;
@@ -651,18 +660,18 @@ __global__ void __launch_bounds__(512) ddts_bwd_gates_kernel(const BwdArgs a) {
     row0 = sh * a.T;
     len = a.T;
   }
-  const int d = threadIdx.x & (DK - 1), seg = threadIdx.x >> 7;
-  const int per = (len + 3) / 4;
+  const int dl = threadIdx.x % kGateCh, d = dch + dl, seg = threadIdx.x / kGateCh;
+  const int per = (len + kGateSegs - 1) / kGateSegs;
   const int lo = min(len, seg * per), hi = min(len, lo + per);
   double s = 0.0;
   for (int r = lo; r < hi; ++r) {
     const long long i = (row0 + r) * DK + d;
     s += (double)a.u[i] - (double)a.w[i];
   }
-  seg_sum[seg][d] = s;
+  seg_sum[seg][dl] = s;
   __syncthreads();
   double acc = (double)a.c[sh * DK + d];
-  for (int s2 = seg + 1; s2 < 4; ++s2) acc += seg_sum[s2][d];
+  for (int s2 = seg + 1; s2 < kGateSegs; ++s2) acc += seg_sum[s2][dl];
   const T* gx = (const T*)a.gx;
   const T* ty = (const T*)a.ty;
   for (int r = hi - 1; r >= lo; --r) {
@@ -727,12 +736,12 @@ cudaError_t launch_bwd(const rodimus_ddts_bwd_params& p, size_t scratch_offset, 
     e = opt_in_shared_memory(ddts_bwd_sweep_kernel<__nv_bfloat16>, (int)kSweepSmem, dev, g_smem_done_bf16);
     if (e != cudaSuccess) return e;
     ddts_bwd_sweep_kernel<__nv_bfloat16><<<(unsigned)(items * 6), kThreads, kSweepSmem, st>>>(a);
-    ddts_bwd_gates_kernel<__nv_bfloat16><<<(unsigned)items, 512, 0, st>>>(a);
+    ddts_bwd_gates_kernel<__nv_bfloat16><<<(unsigned)(items * (DK / kGateCh)), kGateCh * kGateSegs, 0, st>>>(a);
   } else {
     e = opt_in_shared_memory(ddts_bwd_sweep_kernel<float>, (int)kSweepSmem, dev, g_smem_done_f32);
     if (e != cudaSuccess) return e;
     ddts_bwd_sweep_kernel<float><<<(unsigned)(items * 6), kThreads, kSweepSmem, st>>>(a);
-    ddts_bwd_gates_kernel<float><<<(unsigned)items, 512, 0, st>>>(a);
+    ddts_bwd_gates_kernel<float><<<(unsigned)(items * (DK / kGateCh)), kGateCh * kGateSegs, 0, st>>>(a);
   }
   *n_launches = 2;
   return cudaGetLastError();
