@@ -66,6 +66,8 @@ def _load():
         lib.ddts_ref_fwd_block.restype = ctypes.c_int
         lib.ddts_ref_fwd_shared.argtypes = lib.ddts_ref_fwd_block.argtypes
         lib.ddts_ref_fwd_shared.restype = ctypes.c_int
+        lib.ddts_ref_fwd_vdecay.argtypes = lib.ddts_ref_fwd_block.argtypes + [f32p, ctypes.c_int]
+        lib.ddts_ref_fwd_vdecay.restype = ctypes.c_int
         lib.ddts_ref_step.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                       ctypes.c_int, ctypes.c_double,
                                       f32p, f32p, f32p, f32p, f32p, f64p, f64p]
@@ -74,6 +76,8 @@ def _load():
         lib.ddts_ref_step_block.restype = ctypes.c_int
         lib.ddts_ref_step_shared.argtypes = lib.ddts_ref_step_block.argtypes
         lib.ddts_ref_step_shared.restype = ctypes.c_int
+        lib.ddts_ref_step_vdecay.argtypes = lib.ddts_ref_step_block.argtypes + [f32p, ctypes.c_int]
+        lib.ddts_ref_step_vdecay.restype = ctypes.c_int
         lib.ddts_ref_bwd.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
                                      ctypes.c_int, ctypes.c_int, ctypes.c_double,
                                      f32p, f32p, f32p, f32p, f32p, f64p, f32p, f64p,
@@ -112,7 +116,7 @@ def ref_gates(x, y, ingate: int = POW_G):
 
 def ref_fwd(q, k, x, y, v, s0=None, cu_seqlens=None, scale: float = 1.0, ingate: int = POW_G,
             want_o: bool = True, want_sT: bool = True, beta_hat=None, feed_d=None, feed_x=None,
-            shared_gates: bool = False):
+            shared_gates: bool = False, value_decay=None):
     """Sequential prefill.  q,k,x,y: [B,H,T,dk]; v: [B,H,T,dv]; s0: [B|N,H,dk,dv] or None.
 
     Optional terms of the full block: beta_hat [B,H,T,dv] (value gate, Eq. "beta_def": v_t is
@@ -121,6 +125,10 @@ def ref_fwd(q, k, x, y, v, s0=None, cu_seqlens=None, scale: float = 1.0, ingate:
 
     shared_gates: the layout the paper writes the block in - q,k,x,y are [B,1,T,dk], one set per
     token shared by all H groups of dv value columns (v, o, states keep their H).
+
+    value_decay: beta_t in (0,1], [B,H,T,dv]: the value-side decay of the general transition
+    (Eq. "general_state_transition"): state element (d, j) decays by alpha_t[d] * beta_t[j].  The
+    paper's model sets it to 1; this is its ablation arm.
 
     Returns (o [B,H,T,dv] float64 or None, sT [B|N,H,dk,dv] float64 or None).
     """
@@ -150,9 +158,20 @@ def ref_fwd(q, k, x, y, v, s0=None, cu_seqlens=None, scale: float = 1.0, ingate:
         assert s0a.shape == (nseq, H, dk, dv)
     o = np.empty((B, H, T, dv), dtype=np.float64) if want_o else None
     sT = np.empty((nseq, H, dk, dv), dtype=np.float64) if want_sT else None
-    if beta_hat is None and feed_d is None and feed_x is None and not shared_gates:
+    if beta_hat is None and feed_d is None and feed_x is None and not shared_gates \
+            and value_decay is None:
         rc = lib.ddts_ref_fwd(ingate, B, H, T, dk, dv, float(scale), qp, kp, xp, yp, vp,
                               _f64p(s0a), _f64p(o), _f64p(sT), cup, N)
+    elif value_decay is not None:
+        assert (feed_d is None) == (feed_x is None)
+        ba, bp = (None, None) if beta_hat is None else _f32(beta_hat)
+        da, dp = (None, None) if feed_d is None else _f32(feed_d)
+        fa, fp = (None, None) if feed_x is None else _f32(feed_x)
+        ga, gp = _f32(value_decay)
+        assert ga.shape == va.shape and (ba is None or ba.shape == va.shape)
+        rc = lib.ddts_ref_fwd_vdecay(ingate, B, H, T, dk, dv, float(scale), qp, kp, xp, yp, vp,
+                                     _f64p(s0a), _f64p(o), _f64p(sT), cup, N, bp, dp, fp, gp,
+                                     1 if shared_gates else 0)
     else:
         assert (feed_d is None) == (feed_x is None)
         ba, bp = (None, None) if beta_hat is None else _f32(beta_hat)
@@ -169,7 +188,7 @@ def ref_fwd(q, k, x, y, v, s0=None, cu_seqlens=None, scale: float = 1.0, ingate:
 
 
 def ref_step(q, k, x, y, v, state, scale: float = 1.0, ingate: int = POW_G, beta_hat=None,
-             feed_d=None, feed_x=None, shared_gates: bool = False):
+             feed_d=None, feed_x=None, shared_gates: bool = False, value_decay=None):
     """One decode step; ``state`` ([Nseq,H,dk,dv] float64, C-contiguous) is updated in place.
     beta_hat, feed_x: [Nseq,H,dv]; feed_d: [H,dv] (optional, as in ``ref_fwd``)."""
     lib = _load()
@@ -185,9 +204,18 @@ def ref_step(q, k, x, y, v, state, scale: float = 1.0, ingate: int = POW_G, beta
     assert state.dtype == np.float64 and state.flags["C_CONTIGUOUS"]
     assert state.shape == (Nseq, H, dk, dv)
     o = np.empty((Nseq, H, dv), dtype=np.float64)
-    if beta_hat is None and feed_d is None and feed_x is None and not shared_gates:
+    if beta_hat is None and feed_d is None and feed_x is None and not shared_gates \
+            and value_decay is None:
         rc = lib.ddts_ref_step(ingate, Nseq, H, dk, dv, float(scale), qp, kp, xp, yp, vp,
                                _f64p(o), _f64p(state))
+    elif value_decay is not None:
+        ba, bp = (None, None) if beta_hat is None else _f32(beta_hat)
+        da, dp = (None, None) if feed_d is None else _f32(feed_d)
+        fa, fp = (None, None) if feed_x is None else _f32(feed_x)
+        ga, gp = _f32(value_decay)
+        rc = lib.ddts_ref_step_vdecay(ingate, Nseq, H, dk, dv, float(scale), qp, kp, xp, yp, vp,
+                                      _f64p(o), _f64p(state), bp, dp, fp, gp,
+                                      1 if shared_gates else 0)
     else:
         assert (feed_d is None) == (feed_x is None)
         ba, bp = (None, None) if beta_hat is None else _f32(beta_hat)
@@ -280,10 +308,13 @@ def parallel_form(q, k, x, y, v, scale: float = 1.0, ingate: int = POW_G):
     return scale * (scores @ v)
 
 
-def unrolled_sum(q, k, x, y, v, scale: float = 1.0, ingate: int = POW_G):
-    """o_t = sum_{i<=t} [q_t (prod_{j=i+1..t} alpha_j . ahat_i . k_i)^T] v_i, by explicit loops.
+def unrolled_sum(q, k, x, y, v, scale: float = 1.0, ingate: int = POW_G, value_decay=None,
+                 beta_hat=None):
+    """o_t = sum_{i<=t} [q_t (prod_{j=i+1..t} alpha_j . ahat_i . k_i)^T]
+                        (prod_{j=i+1..t} beta_j . beta_hat_i . v_i), by explicit loops.
 
-    Sec. 3.1.1, with beta = 1 and no value gate.  Pure Python loops: tiny inputs only.
+    Sec. 3.1.1, the equation obtained by unfolding the general transition; beta (value_decay,
+    [T,dv]) and beta_hat ([T,dv]) default to 1.  Pure Python loops: tiny inputs only.
     """
     q = np.asarray(q, dtype=np.float64)
     k = np.asarray(k, dtype=np.float64)
@@ -291,11 +322,17 @@ def unrolled_sum(q, k, x, y, v, scale: float = 1.0, ingate: int = POW_G):
     log_alpha, ahat = _gates_np(x, y, ingate)
     alpha = np.exp(log_alpha)
     T, dk = q.shape
+    beta = None if value_decay is None else np.asarray(value_decay, dtype=np.float64)
+    bhat = None if beta_hat is None else np.asarray(beta_hat, dtype=np.float64)
     o = np.zeros((T, v.shape[1]), dtype=np.float64)
     for t in range(T):
         for i in range(t + 1):
             prod = np.ones(dk)
+            vprod = np.ones(v.shape[1])
             for j in range(i + 1, t + 1):
                 prod = prod * alpha[j]
-            o[t] += float(np.dot(q[t], prod * ahat[i] * k[i])) * v[i]
+                if beta is not None:
+                    vprod = vprod * beta[j]
+            vi = v[i] if bhat is None else bhat[i] * v[i]
+            o[t] += float(np.dot(q[t], prod * ahat[i] * k[i])) * (vprod * vi)
     return scale * o

@@ -11,7 +11,8 @@
  * beta_t = 1 as Sec. 3.1.1 chooses; the value gate beta_hat of Eq. "beta_def" and
  * the feed-through term d . x' of Eq. "rodimus_recurrent_form" are optional inputs
  * of the ..._block entry points: v_t is replaced by beta_hat_t . v_t and d . x'_t is
- * added to o_t; their projections stay with the caller):
+ * added to o_t; their projections stay with the caller; the ..._vdecay entry points also take the
+ * value-side decay beta_t of the general transition, Eq. "general_state_transition", as numbers):
  *
  *   g_t     = softplus(x_t)                    selection gate,   per key channel
  *   tau_t   = sigmoid(y_t)                     temperature gate, per key channel
@@ -86,7 +87,7 @@ int ddts_ref_gates(int ingate, int64_t n, const float *x, const float *y, double
 static void ref_one_sequence(int ingate, int64_t len, int dk, int dv, double scale, const float *q,
                              const float *k, const float *x, const float *y, const float *v,
                              const double *s0, double *o, double *sT, double *S, const float *bh,
-                             const float *d_feed, const float *fx) {
+                             const float *d_feed, const float *fx, const float *bd) {
   if (s0)
     memcpy(S, s0, sizeof(double) * (size_t)dk * dv);
   else
@@ -102,7 +103,15 @@ static void ref_one_sequence(int ingate, int64_t len, int dk, int dv, double sca
       ref_gate(ingate, (double)xt[d], (double)yt[d], &alpha, &ahat);
       double w = ahat * (double)kt[d];
       double *Sd = S + (size_t)d * dv;
-      if (bh) {
+      if (bd) {
+        /* value-side decay beta_t of Eq. "general_state_transition": the state element (d, j)
+         * decays by alpha_t[d] * beta_t[j]; the input term is as below */
+        const float *dt = bd + t * dv;
+        for (int j = 0; j < dv; ++j) {
+          double vj = bh ? (double)bh[t * dv + j] * (double)vt[j] : (double)vt[j];
+          Sd[j] = (alpha * (double)dt[j]) * Sd[j] + w * vj;
+        }
+      } else if (bh) {
         const float *bt = bh + t * dv;
         for (int j = 0; j < dv; ++j) Sd[j] = alpha * Sd[j] + w * ((double)bt[j] * (double)vt[j]);
       } else {
@@ -140,7 +149,8 @@ static int ref_fwd_impl(int ingate, int B, int H, int64_t T, int dk, int dv, dou
                         const float *q, const float *k, const float *x, const float *y,
                         const float *v, const double *s0, double *o, double *sT,
                         const int32_t *cu_seqlens, int N, const float *beta_hat,
-                        const float *feed_d, const float *feed_x, int shared) {
+                        const float *feed_d, const float *feed_x, int shared,
+                        const float *value_decay) {
   if (ingate != DDTS_REF_POW_G && ingate != DDTS_REF_POW_SIGMOID) return 3;
   if (B < 0 || H < 0 || T < 0 || dk <= 0 || dv <= 0) return 2;
   int nseq = B;
@@ -179,7 +189,8 @@ static int ref_fwd_impl(int ingate, int B, int H, int64_t T, int dk, int dv, dou
       ref_one_sequence(ingate, len, dk, dv, scale, q + rq * dk, k + rq * dk, x + rq * dk,
                        y + rq * dk, v + row0 * dv, s0 ? s0 + so : NULL, o ? o + row0 * dv : NULL,
                        sT ? sT + so : NULL, S, beta_hat ? beta_hat + row0 * dv : NULL,
-                       feed_d ? feed_d + (size_t)h * dv : NULL, feed_x ? feed_x + row0 * dv : NULL);
+                       feed_d ? feed_d + (size_t)h * dv : NULL, feed_x ? feed_x + row0 * dv : NULL,
+                       value_decay ? value_decay + row0 * dv : NULL);
     }
     free(S);
   }
@@ -192,7 +203,21 @@ int ddts_ref_fwd_block(int ingate, int B, int H, int64_t T, int dk, int dv, doub
                        const int32_t *cu_seqlens, int N, const float *beta_hat,
                        const float *feed_d, const float *feed_x) {
   return ref_fwd_impl(ingate, B, H, T, dk, dv, scale, q, k, x, y, v, s0, o, sT, cu_seqlens, N,
-                      beta_hat, feed_d, feed_x, 0);
+                      beta_hat, feed_d, feed_x, 0, NULL);
+}
+
+/* The general transition of Sec. 3.1.1 (Eq. "general_state_transition") with a value-side decay
+ * beta_t in (0,1]^dv, [B,H,T,dv], handed in as numbers: S_t = (alpha_t^T beta_t) . S_{t-1} +
+ * (ahat_t . k_t)^T (beta_hat_t . v_t).  The paper sets beta_t = 1 after its ablation (table
+ * "beta_type"); this entry point exists for that ablation arm.  shared: as ddts_ref_fwd_shared. */
+int ddts_ref_fwd_vdecay(int ingate, int B, int H, int64_t T, int dk, int dv, double scale,
+                        const float *q, const float *k, const float *x, const float *y,
+                        const float *v, const double *s0, double *o, double *sT,
+                        const int32_t *cu_seqlens, int N, const float *beta_hat,
+                        const float *feed_d, const float *feed_x, const float *value_decay,
+                        int shared) {
+  return ref_fwd_impl(ingate, B, H, T, dk, dv, scale, q, k, x, y, v, s0, o, sT, cu_seqlens, N,
+                      beta_hat, feed_d, feed_x, shared, value_decay);
 }
 
 /* Shared-gate layout: q, k, x, y are [B,1,T,dk]; everything else as ddts_ref_fwd_block. */
@@ -202,7 +227,7 @@ int ddts_ref_fwd_shared(int ingate, int B, int H, int64_t T, int dk, int dv, dou
                         const int32_t *cu_seqlens, int N, const float *beta_hat,
                         const float *feed_d, const float *feed_x) {
   return ref_fwd_impl(ingate, B, H, T, dk, dv, scale, q, k, x, y, v, s0, o, sT, cu_seqlens, N,
-                      beta_hat, feed_d, feed_x, 1);
+                      beta_hat, feed_d, feed_x, 1, NULL);
 }
 
 /* The recurrence alone (no value gate, no feed-through). */
@@ -221,7 +246,7 @@ int ddts_ref_fwd(int ingate, int B, int H, int64_t T, int dk, int dv, double sca
 static int ref_step_impl(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
                          const float *k, const float *x, const float *y, const float *v, double *o,
                          double *state, const float *beta_hat, const float *feed_d,
-                         const float *feed_x, int shared) {
+                         const float *feed_x, int shared, const float *value_decay) {
   if (ingate != DDTS_REF_POW_G && ingate != DDTS_REF_POW_SIGMOID) return 3;
   if (Nseq < 0 || H < 0 || dk <= 0 || dv <= 0) return 2;
   int64_t items = (int64_t)Nseq * H;
@@ -239,7 +264,14 @@ static int ref_step_impl(int ingate, int Nseq, int H, int dk, int dv, double sca
       double w = ahat * (double)kt[d];
       double qd = (double)qt[d];
       double *Sd = S + (size_t)d * dv;
-      if (beta_hat) {
+      if (value_decay) {
+        const float *dt = value_decay + it * dv;
+        for (int j = 0; j < dv; ++j) {
+          double vj = beta_hat ? (double)beta_hat[it * dv + j] * (double)vt[j] : (double)vt[j];
+          Sd[j] = (alpha * (double)dt[j]) * Sd[j] + w * vj;
+          ot[j] += qd * Sd[j];
+        }
+      } else if (beta_hat) {
         const float *bt = beta_hat + it * dv;
         for (int j = 0; j < dv; ++j) {
           Sd[j] = alpha * Sd[j] + w * ((double)bt[j] * (double)vt[j]);
@@ -266,7 +298,16 @@ int ddts_ref_step_block(int ingate, int Nseq, int H, int dk, int dv, double scal
                         double *state, const float *beta_hat, const float *feed_d,
                         const float *feed_x) {
   return ref_step_impl(ingate, Nseq, H, dk, dv, scale, q, k, x, y, v, o, state, beta_hat, feed_d,
-                       feed_x, 0);
+                       feed_x, 0, NULL);
+}
+
+/* Decode step with the value-side decay beta_t [Nseq,H,dv] (see ddts_ref_fwd_vdecay). */
+int ddts_ref_step_vdecay(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
+                         const float *k, const float *x, const float *y, const float *v, double *o,
+                         double *state, const float *beta_hat, const float *feed_d,
+                         const float *feed_x, const float *value_decay, int shared) {
+  return ref_step_impl(ingate, Nseq, H, dk, dv, scale, q, k, x, y, v, o, state, beta_hat, feed_d,
+                       feed_x, shared, value_decay);
 }
 
 /* Shared-gate layout for decode: q, k, x, y are [Nseq,1,dk]. */
@@ -275,7 +316,7 @@ int ddts_ref_step_shared(int ingate, int Nseq, int H, int dk, int dv, double sca
                          double *state, const float *beta_hat, const float *feed_d,
                          const float *feed_x) {
   return ref_step_impl(ingate, Nseq, H, dk, dv, scale, q, k, x, y, v, o, state, beta_hat, feed_d,
-                       feed_x, 1);
+                       feed_x, 1, NULL);
 }
 
 int ddts_ref_step(int ingate, int Nseq, int H, int dk, int dv, double scale, const float *q,
