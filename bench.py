@@ -334,6 +334,10 @@ def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sf
                   "feed_x": torch.randn(p.v.shape, generator=g).to(tdt).to(device),
                   "feed_d": torch.randn((H, dv), generator=g).to(device)}
             alg_bytes += 2 * B * H * T * dv * el
+        elif variant == "vdecay":
+            from paper_2410_06577_b200 import workloads as wl_
+            kw = {"value_decay": torch.from_numpy(wl_.make_value_decay(77, p.v.shape, p.dtype)).to(tdt).to(device)}
+            alg_bytes += B * H * T * dv * el
         elif variant == "shared":
             for n in ("q", "k", "x", "y"):
                 devt[n] = devt[n][:, :1].contiguous()
@@ -457,7 +461,8 @@ def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sf
         rec["config"] = dict(rec["config"], variant={
             "block": "value gate beta_hat and feed-through d*x' fused (Eq. beta_def, Eq. rodimus_recurrent_form)",
             "shared": "one q,k,x,y per token for all 16 heads ([B,1,T,dk])",
-            "backward": "backward pass (dq, dk, dx, dy, dv, ds0 from dL/do and dL/dS_T), two launches"}[variant])
+            "backward": "backward pass (dq, dk, dx, dy, dv, ds0 from dL/do and dL/dS_T), two launches",
+            "vdecay": "value-side decay beta_t of the general transition (the paper's ablation arm), fp32 CUDA-core kernel"}[variant])
         if variant == "backward":
             rec["metric"] = "DDTS prefill backward tokens/s"
     if with_e2e:
@@ -513,10 +518,10 @@ def run_ours(args, workload, p):
                                                    "gpu_launches", "roofline")}
             del pw
         for name, variant in (("cfg1_block_terms", "block"), ("cfg1_shared_gates", "shared"),
-                              ("cfg1_backward", "backward")):
+                              ("cfg1_backward", "backward"), ("cfg1_value_decay", "vdecay")):
             torch.cuda.empty_cache()
             pw = wl.config(1)
-            r = measure("cfg1", pw, 40 if variant == "backward" else 500, 5, world, rank, local, peaks,
+            r = measure("cfg1", pw, {"backward": 40, "vdecay": 10}.get(variant, 500), 5, world, rank, local, peaks,
                         peak_kind, sfu_rate, with_e2e=False, variant=variant)
             extra[name] = {key: r[key] for key in ("metric", "value", "unit", "steps", "warmup", "ms_per_step",
                                                    "dtype", "config", "timed_regions", "clocks",
@@ -536,7 +541,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg1")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--variant", choices=["block", "shared", "backward"], default=None,
+    ap.add_argument("--variant", choices=["block", "shared", "backward", "vdecay"], default=None,
                     help="time a variant of the config-1 workload instead (for profiling; no e2e)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true",

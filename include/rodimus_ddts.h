@@ -115,6 +115,11 @@ typedef struct {
                              /* q,k,gate_x,temp_y are [B,1,T,dk], one set per token shared by the H    */
                              /* groups of dv value columns; v, o, s0, sT keep their H.                 */
   int32_t reserved;          /* 0                                                                    */
+  const void *value_decay;   /* optional, device [B,H,T,dv], dtype of v: the value-side decay beta_t of */
+                             /* the general transition (Sec. 3.1.1, Eq. "general_state_transition"),    */
+                             /* numbers in (0,1]: state element (d,j) decays by alpha_t[d]*beta_t[j].   */
+                             /* The paper's model sets beta_t = 1 (NULL) after the ablation of its      */
+                             /* table "beta_type"; requests that give it run the fp32 CUDA-core kernel. */
 } rodimus_ddts_fwd_params;
 
 /*
@@ -140,6 +145,8 @@ typedef struct {
   const void *feed_x;                  /* optional with feed_d, device [Nseq,H,dv]: x'_t             */
   int32_t shared_gates;                /* 1: q,k,gate_x,temp_y are [Nseq,1,dk] (see the prefill)     */
   int32_t reserved;                    /* 0                                                          */
+  const void *value_decay;             /* optional, device [Nseq,H,dv]: value-side decay beta_t      */
+                                       /* (see the prefill); NULL = 1                                */
 } rodimus_ddts_step_params;
 
 /* Bytes of device workspace rodimus_ddts_fwd needs for these sizes (pointers are not read).

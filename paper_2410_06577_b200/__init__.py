@@ -50,6 +50,7 @@ class FwdParams(ctypes.Structure):
         ("stream", ctypes.c_void_p),
         ("beta_hat", ctypes.c_void_p), ("feed_d", ctypes.c_void_p), ("feed_x", ctypes.c_void_p),
         ("shared_gates", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("value_decay", ctypes.c_void_p),
     ]
 
 
@@ -64,6 +65,7 @@ class StepParams(ctypes.Structure):
         ("state", ctypes.c_void_p), ("stream", ctypes.c_void_p),
         ("beta_hat", ctypes.c_void_p), ("feed_d", ctypes.c_void_p), ("feed_x", ctypes.c_void_p),
         ("shared_gates", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("value_decay", ctypes.c_void_p),
     ]
 
 
@@ -162,7 +164,7 @@ def _check_cuda(*tensors):
 def fwd_params(q, k, gate_x, temp_y, v, o, s0=None, sT=None, cu_seqlens=None,
                cu_seqlens_host=None, workspace=None, scale: float = 1.0,
                ingate: int = INGATE_POW_G, stream: Optional[int] = None, beta_hat=None,
-               feed_d=None, feed_x=None) -> FwdParams:
+               feed_d=None, feed_x=None, value_decay=None) -> FwdParams:
     """Fills a ``rodimus_ddts_fwd_params`` from torch tensors (no checks beyond layout)."""
     import torch
     B, Hq, T, dk = q.shape
@@ -183,6 +185,7 @@ def fwd_params(q, k, gate_x, temp_y, v, o, s0=None, sT=None, cu_seqlens=None,
     p.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     p.stream = torch.cuda.current_stream().cuda_stream if stream is None else stream
     p.beta_hat, p.feed_d, p.feed_x = _ptr(beta_hat), _ptr(feed_d), _ptr(feed_x)
+    p.value_decay = _ptr(value_decay)
     return p
 
 
@@ -323,17 +326,19 @@ def ddts_bwd(q, k, gate_x, temp_y, v, d_o, s0=None, d_sT=None, cu_seqlens=None,
 def ddts_fwd(q, k, gate_x, temp_y, v, s0=None, cu_seqlens=None, cu_seqlens_host=None,
              scale: float = 1.0, ingate: int = INGATE_POW_G, want_final_state: bool = True,
              out=None, final_state=None, workspace=None, beta_hat=None, feed_d=None,
-             feed_x=None) -> Tuple["torch.Tensor", Optional["torch.Tensor"]]:
+             feed_x=None, value_decay=None) -> Tuple["torch.Tensor", Optional["torch.Tensor"]]:
     """Chunked DDTS prefill (``rodimus_ddts_fwd``).
 
     q,k,gate_x,temp_y: [B,H,T,dk]; v: [B,H,T,dv] (bf16 or fp32, all alike); s0: fp32
     [B|N,H,dk,dv] or None; cu_seqlens: int32 CUDA tensor [N+1] for packed sequences (B = 1).
     Optional, fused into the same pass: beta_hat [B,H,T,dv] (value gate, multiplies v), and the
     feed-through feed_d fp32 [H,dv] with feed_x [B,H,T,dv] (o += feed_d * feed_x).
+    value_decay [B,H,T,dv] in (0,1]: the value-side decay of the general transition (the arm the
+    paper ablates and drops; fp32 CUDA-core kernel).
     Returns (o, sT) with sT None unless ``want_final_state``.  Asynchronous on the current stream.
     """
     import torch
-    _check_cuda(q, k, gate_x, temp_y, v, s0, cu_seqlens, beta_hat, feed_d, feed_x)
+    _check_cuda(q, k, gate_x, temp_y, v, s0, cu_seqlens, beta_hat, feed_d, feed_x, value_decay)
     B, _, T, dk = q.shape
     H = v.shape[1]            # q,k,gate_x,temp_y may have a single head shared by all H of v
     dv = v.shape[-1]
@@ -343,7 +348,7 @@ def ddts_fwd(q, k, gate_x, temp_y, v, s0=None, cu_seqlens=None, cu_seqlens_host=
     if sT is None and want_final_state:
         sT = torch.empty((nseq, H, dk, dv), dtype=torch.float32, device=q.device)
     p = fwd_params(q, k, gate_x, temp_y, v, o, s0, sT, cu_seqlens, cu_seqlens_host, None, scale,
-                   ingate, beta_hat=beta_hat, feed_d=feed_d, feed_x=feed_x)
+                   ingate, beta_hat=beta_hat, feed_d=feed_d, feed_x=feed_x, value_decay=value_decay)
     ws = workspace if workspace is not None else new_workspace(p, q.device)
     p.workspace = ws.data_ptr()
     p.workspace_bytes = ws.numel() * ws.element_size()
@@ -354,13 +359,13 @@ def ddts_fwd(q, k, gate_x, temp_y, v, s0=None, cu_seqlens=None, cu_seqlens_host=
 
 
 def ddts_step(q, k, gate_x, temp_y, v, state, scale: float = 1.0, ingate: int = INGATE_POW_G,
-              out=None, beta_hat=None, feed_d=None, feed_x=None):
+              out=None, beta_hat=None, feed_d=None, feed_x=None, value_decay=None):
     """One decode step (``rodimus_ddts_step``): ``state`` fp32 [Nseq,H,dk,dv] is updated in place.
 
     q,k,gate_x,temp_y: [Nseq,H,dk]; v: [Nseq,H,dv].  Returns o [Nseq,H,dv].
     """
     import torch
-    _check_cuda(q, k, gate_x, temp_y, v, state, beta_hat, feed_d, feed_x)
+    _check_cuda(q, k, gate_x, temp_y, v, state, beta_hat, feed_d, feed_x, value_decay)
     Nseq, Hq, dk = q.shape
     H = v.shape[1]
     dv = v.shape[-1]
@@ -376,6 +381,7 @@ def ddts_step(q, k, gate_x, temp_y, v, state, scale: float = 1.0, ingate: int = 
     p.stream = torch.cuda.current_stream().cuda_stream
     p.beta_hat, p.feed_d, p.feed_x = _ptr(beta_hat), _ptr(feed_d), _ptr(feed_x)
     p.shared_gates = 1 if (Hq == 1 and H > 1) else 0
+    p.value_decay = _ptr(value_decay)
     rc = step_raw(p)
     if rc != OK:
         raise RodimusError(rc, "rodimus_ddts_step")

@@ -10,6 +10,11 @@
 // Every exponent is <= 0 apart from log ahat, so no input in the documented domain overflows,
 // whatever the decay.
 //
+// Optional value-side decay beta_t (general transition of Sec. 3.1.1, the arm the paper ablates
+// and drops): with c_r = sum_{j<=r in chunk} log beta_j per value column,
+//   O_r   = sum_{i<=r} P_ri (v_i . exp(c_r - c_i)) + exp(c_r) . ((q_r . exp(b_r)) S_in)
+//   S_out = (exp(b_C)^T exp(c_C)) . S_in + sum_i (k_i . ahat_i . exp(b_C - b_i))^T (v_i . exp(c_C - c_i))
+//
 // Work item = (sequence, head, tile of kTileV state columns); one CTA per item keeps its
 // [dk, kTileV] slice of the state in shared memory for the whole sequence.
 #include "ddts_common.cuh"
@@ -24,6 +29,7 @@ constexpr int kThreads = 256;
 struct SimtArgs {
   const void *q, *k, *gx, *ty, *v;
   const void *beta_hat, *feed_x;   // optional: value gate [.., dv], feed-through input [.., dv]
+  const void *vdecay;              // optional: value-side decay beta_t [.., dv], numbers in (0,1]
   const float* feed_d;             // optional: feed-through weight [H, dv]
   void* o;
   const float* s0;
@@ -48,6 +54,7 @@ __global__ void __launch_bounds__(kThreads, 1) ddts_fwd_simt_kernel(const SimtAr
   float* sV = sB + kC * ld;                    // [kC][kTileV]
   float* sP = sV + kC * kTileV;                // [kC][kC]
   float* sE = sP + kC * kC;                    // [dk]          b at the chunk end
+  float* sC = sE + dk;                         // [kC][kTileV]  c (cumulative log beta), if given
 
   const int tid = threadIdx.x;
   const long long item = blockIdx.x;
@@ -82,6 +89,7 @@ __global__ void __launch_bounds__(kThreads, 1) ddts_fwd_simt_kernel(const SimtAr
   const T* bh = a.beta_hat ? (const T*)a.beta_hat + row0 * dv : nullptr;
   const T* fx = a.feed_d ? (const T*)a.feed_x + row0 * dv : nullptr;
   const float* fd = a.feed_d ? a.feed_d + (long long)h * dv : nullptr;
+  const T* bd = a.vdecay ? (const T*)a.vdecay + row0 * dv : nullptr;
   const long long s_off = sh * (long long)dk * dv;
 
   for (int e = tid; e < dk * kTileV; e += kThreads) {
@@ -116,6 +124,16 @@ __global__ void __launch_bounds__(kThreads, 1) ddts_fwd_simt_kernel(const SimtAr
       }
       sV[e] = vv;
     }
+    if (bd) {   // cumulative log of the value-side decay: one thread per state column
+      for (int c = tid; c < kTileV; c += kThreads) {
+        float cum = 0.f;
+        for (int r = 0; r < kC; ++r) {
+          if (r < nr && col0 + c < dv)
+            cum += logf(fmaxf(to_f32(bd[(long long)(t0 + r) * dv + col0 + c]), 1e-37f));
+          sC[r * kTileV + c] = cum;
+        }
+      }
+    }
     __syncthreads();
     // (2) intra-chunk scores, causal mask with the diagonal kept
     {
@@ -139,9 +157,17 @@ __global__ void __launch_bounds__(kThreads, 1) ddts_fwd_simt_kernel(const SimtAr
       const int r = e / kTileV, c = e % kTileV;
       if (r < nr && col0 + c < dv) {
         float acc = 0.f;
-        for (int i = 0; i <= r; ++i) acc = fmaf(sP[r * kC + i], sV[i * kTileV + c], acc);
         const float* qr = sQ + r * ld;
-        for (int d = 0; d < dk; ++d) acc = fmaf(qr[d], sS[d * kTileV + c], acc);
+        if (bd) {
+          const float cr = sC[r * kTileV + c];
+          for (int d = 0; d < dk; ++d) acc = fmaf(qr[d], sS[d * kTileV + c], acc);
+          acc *= expf(cr);
+          for (int i = 0; i <= r; ++i)
+            acc = fmaf(sP[r * kC + i], sV[i * kTileV + c] * expf(cr - sC[i * kTileV + c]), acc);
+        } else {
+          for (int i = 0; i <= r; ++i) acc = fmaf(sP[r * kC + i], sV[i * kTileV + c], acc);
+          for (int d = 0; d < dk; ++d) acc = fmaf(qr[d], sS[d * kTileV + c], acc);
+        }
         const long long i = (long long)(t0 + r) * dv + col0 + c;
         acc *= a.scale;
         if (fd) acc = fmaf(fd[col0 + c], to_f32(fx[i]), acc);   // feed-through d . x'
@@ -154,10 +180,15 @@ __global__ void __launch_bounds__(kThreads, 1) ddts_fwd_simt_kernel(const SimtAr
       const int i = e / dk, d = e % dk;
       sW[i * ld + d] *= expf(sE[d] - sB[i * ld + d]);
     }
+    if (bd) {   // v_i . exp(c_C - c_i), in place (the outputs are done with v)
+      for (int e = tid; e < nr * kTileV; e += kThreads)
+        sV[e] *= expf(sC[(kC - 1) * kTileV + e % kTileV] - sC[e]);
+    }
     __syncthreads();
     for (int e = tid; e < dk * kTileV; e += kThreads) {
       const int d = e / kTileV, c = e % kTileV;
       float acc = expf(sE[d]) * sS[e];
+      if (bd) acc *= expf(sC[(kC - 1) * kTileV + c]);
       for (int i = 0; i < nr; ++i) acc = fmaf(sW[i * ld + d], sV[i * kTileV + c], acc);
       sS[e] = acc;
     }
@@ -174,7 +205,7 @@ __global__ void __launch_bounds__(kThreads, 1) ddts_fwd_simt_kernel(const SimtAr
 
 size_t simt_smem_bytes(int dk) {
   const int ld = dk + 1;
-  return sizeof(float) * ((size_t)dk * kTileV + 3 * (size_t)kC * ld + kC * kTileV + kC * kC + dk);
+  return sizeof(float) * ((size_t)dk * kTileV + 3 * (size_t)kC * ld + 2 * kC * kTileV + kC * kC + dk);
 }
 
 }  // namespace
@@ -183,7 +214,7 @@ cudaError_t launch_fwd_simt(const rodimus_ddts_fwd_params& p, int* n_launches) {
   *n_launches = 0;
   SimtArgs a;
   a.q = p.q; a.k = p.k; a.gx = p.gate_x; a.ty = p.temp_y; a.v = p.v; a.o = p.o;
-  a.beta_hat = p.beta_hat; a.feed_x = p.feed_x; a.feed_d = p.feed_d;
+  a.beta_hat = p.beta_hat; a.feed_x = p.feed_x; a.feed_d = p.feed_d; a.vdecay = p.value_decay;
   a.s0 = p.s0; a.sT = p.sT; a.cu = p.cu_seqlens;
   a.hdr = reinterpret_cast<WorkspaceHeader*>(p.workspace);
   a.H = p.H; a.T = p.T; a.dk = p.dk; a.dv = p.dv;

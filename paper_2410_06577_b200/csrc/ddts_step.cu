@@ -7,6 +7,8 @@
 // access is one 512-byte row segment.  Rows are processed in batches of kBatch per warp with
 // all loads of a batch in flight at once; the first batch is issued before the gate math so
 // that its latency hides the token loads and the transcendental work.
+#include <type_traits>
+
 #include "ddts_common.cuh"
 
 namespace ddts {
@@ -21,13 +23,15 @@ constexpr int kMaxDk = 256;
 __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(float4* p, const float4& v) { __stcs(p, v); }
 
-template <typename T>
+// VDECAY: the value-side decay beta_t of the general transition is given (the paper's ablation
+// arm); a separate instantiation, so that the plain path carries none of it.
+template <typename T, bool VDECAY>
 __global__ void __launch_bounds__(kStepThreads, 4)
 ddts_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ gx,
                  const T* __restrict__ ty, const T* __restrict__ v, T* __restrict__ o,
                  float* __restrict__ state, int n_seq_heads, int dk, int dv, float scale,
                  int ingate, const T* __restrict__ beta_hat, const float* __restrict__ feed_d,
-                 const T* __restrict__ feed_x, int H, int shared) {
+                 const T* __restrict__ feed_x, int H, int shared, const T* __restrict__ vdecay) {
   __shared__ float s_alpha[kMaxDk];
   __shared__ float s_w[kMaxDk];   // ahat * k
   __shared__ float s_q[kMaxDk];   // scale * q
@@ -70,6 +74,11 @@ ddts_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __re
         vv.x *= to_f32(bp[0]); vv.y *= to_f32(bp[1]); vv.z *= to_f32(bp[2]); vv.w *= to_f32(bp[3]);
       }
     }
+    float4 bd = make_float4(1.f, 1.f, 1.f, 1.f);
+    if (VDECAY && col_ok) {
+      const T* dp = vdecay + nh * dv + col;
+      bd = make_float4(to_f32(dp[0]), to_f32(dp[1]), to_f32(dp[2]), to_f32(dp[3]));
+    }
     __syncthreads();
 
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -80,10 +89,17 @@ ddts_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __re
         if (col_ok && r < dk) {
           const float a = s_alpha[r], w = s_w[r], qq = s_q[r];
           float4 s = buf[j];
-          s.x = fmaf(a, s.x, w * vv.x);
-          s.y = fmaf(a, s.y, w * vv.y);
-          s.z = fmaf(a, s.z, w * vv.z);
-          s.w = fmaf(a, s.w, w * vv.w);
+          if (VDECAY) {
+            s.x = fmaf(a * bd.x, s.x, w * vv.x);
+            s.y = fmaf(a * bd.y, s.y, w * vv.y);
+            s.z = fmaf(a * bd.z, s.z, w * vv.z);
+            s.w = fmaf(a * bd.w, s.w, w * vv.w);
+          } else {
+            s.x = fmaf(a, s.x, w * vv.x);
+            s.y = fmaf(a, s.y, w * vv.y);
+            s.z = fmaf(a, s.z, w * vv.z);
+            s.w = fmaf(a, s.w, w * vv.w);
+          }
           acc.x = fmaf(qq, s.x, acc.x);
           acc.y = fmaf(qq, s.y, acc.y);
           acc.z = fmaf(qq, s.z, acc.z);
@@ -146,18 +162,20 @@ cudaError_t launch_step(const rodimus_ddts_step_params& p, int* n_launches) {
   (void)sms;
   const int grid = (int)(items < max_grid ? items : max_grid);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
+  auto launch = [&](auto tag, auto decay) {
+    using T = decltype(tag);
+    constexpr bool VD = decltype(decay)::value;
+    ddts_step_kernel<T, VD><<<grid, kStepThreads, 0, st>>>(
+        (const T*)p.q, (const T*)p.k, (const T*)p.gate_x, (const T*)p.temp_y, (const T*)p.v,
+        (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate, (const T*)p.beta_hat, p.feed_d,
+        (const T*)p.feed_x, p.H, p.shared_gates, (const T*)p.value_decay);
+  };
   if (p.dtype == RODIMUS_BF16) {
-    using T = __nv_bfloat16;
-    ddts_step_kernel<T><<<grid, kStepThreads, 0, st>>>(
-        (const T*)p.q, (const T*)p.k, (const T*)p.gate_x, (const T*)p.temp_y, (const T*)p.v,
-        (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate, (const T*)p.beta_hat, p.feed_d,
-        (const T*)p.feed_x, p.H, p.shared_gates);
+    if (p.value_decay) launch(__nv_bfloat16{}, std::true_type{});
+    else launch(__nv_bfloat16{}, std::false_type{});
   } else {
-    using T = float;
-    ddts_step_kernel<T><<<grid, kStepThreads, 0, st>>>(
-        (const T*)p.q, (const T*)p.k, (const T*)p.gate_x, (const T*)p.temp_y, (const T*)p.v,
-        (T*)p.o, p.state, (int)nh, p.dk, p.dv, p.scale, p.ingate, (const T*)p.beta_hat, p.feed_d,
-        (const T*)p.feed_x, p.H, p.shared_gates);
+    if (p.value_decay) launch(float{}, std::true_type{});
+    else launch(float{}, std::false_type{});
   }
   *n_launches = 1;
   return cudaGetLastError();

@@ -64,7 +64,8 @@ bool fwd_tc_supported(const rodimus_ddts_fwd_params& p) {
   return p.dtype == RODIMUS_BF16 && p.dk == 128 && p.dv % 128 == 0;
 }
 
-bool fwd_pair_selected(const rodimus_ddts_fwd_params& p) { return fwd_pair_supported(p); }
+// the value-side decay (the paper's ablation arm) exists in the fp32 kernel only
+bool fwd_pair_selected(const rodimus_ddts_fwd_params& p) { return fwd_pair_supported(p) && !p.value_decay; }
 
 bool has_block_terms(const rodimus_ddts_fwd_params& p) { return p.beta_hat || p.feed_d; }
 
@@ -72,7 +73,7 @@ bool has_block_terms(const rodimus_ddts_fwd_params& p) { return p.beta_hat || p.
 // 2: fp32 CUDA-core kernel
 int fwd_kernel_choice(const rodimus_ddts_fwd_params& p) {
   if (fwd_pair_selected(p)) return 0;
-  if (fwd_tc_supported(p) && !has_block_terms(p) && !p.shared_gates) return 1;
+  if (fwd_tc_supported(p) && !has_block_terms(p) && !p.shared_gates && !p.value_decay) return 1;
   return 2;
 }
 
@@ -110,7 +111,7 @@ int rodimus_ddts_fwd(const rodimus_ddts_fwd_params* p) {
     return RODIMUS_ERR_NULL;
   if ((p->feed_d != nullptr) != (p->feed_x != nullptr)) return RODIMUS_ERR_NULL;  // both or neither
   const void* ptrs[] = {p->q, p->k, p->gate_x, p->temp_y, p->v, p->o, p->s0, p->sT, p->cu_seqlens,
-                        p->beta_hat, p->feed_d, p->feed_x};
+                        p->beta_hat, p->feed_d, p->feed_x, p->value_decay};
   for (const void* ptr : ptrs)
     if (ptr && !aligned16(ptr)) return RODIMUS_ERR_ALIGN;
   if (!p->workspace || p->workspace_bytes < workspace_bytes_for(varlen ? p->N : 0))
@@ -235,7 +236,7 @@ int rodimus_ddts_step(const rodimus_ddts_step_params* p) {
   const void* ptrs[] = {p->q, p->k, p->gate_x, p->temp_y, p->v, p->o, p->state};
   for (const void* ptr : ptrs)
     if (!aligned16(ptr)) return RODIMUS_ERR_ALIGN;
-  const void* opt[] = {p->beta_hat, p->feed_d, p->feed_x};
+  const void* opt[] = {p->beta_hat, p->feed_d, p->feed_x, p->value_decay};
   for (const void* ptr : opt)
     if (ptr && !aligned16(ptr)) return RODIMUS_ERR_ALIGN;
   int n = 0;
@@ -278,6 +279,6 @@ const char* rodimus_status_str(int status) {
   }
 }
 
-int rodimus_version(void) { return 103; }
+int rodimus_version(void) { return 104; }
 
 }  // extern "C"

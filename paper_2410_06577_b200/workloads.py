@@ -98,6 +98,13 @@ def make_grads(seed: int, p: PrefillInputs, with_state: bool = True, state_std: 
     return d_o, d_sT
 
 
+def make_value_decay(seed: int, shape, dtype: str, low: float = 0.8) -> np.ndarray:
+    """Value-side decay factors beta_t for the ablation arm: uniform in (low, 1], rounded to the
+    workload's dtype."""
+    rng = np.random.default_rng(seed)
+    return _round(np.float32(1.0) - np.float32(1.0 - low) * rng.random(shape, dtype=np.float32), dtype)
+
+
 def varlen_lengths(seed: int, n_seq: int, lo: int, hi: int) -> np.ndarray:
     """Lengths uniform in [lo, hi] and their exclusive prefix sum (int32 [n_seq+1])."""
     rng = np.random.default_rng(seed)

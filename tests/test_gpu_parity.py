@@ -689,6 +689,61 @@ def test_block_terms_decode_steps(dtype):
 
 
 # ------------------------------------------------------------------------------------------
+# value-side decay beta_t of the general transition (the arm the paper ablates and drops)
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype,dk,dv", [("f32", 64, 64), ("bf16", 128, 256), ("f32", 48, 80)])
+@pytest.mark.parametrize("with_gate", [False, True])
+def test_value_decay_prefill(dtype, dk, dv, with_gate):
+    import torch
+    p = wl.make_prefill(801, 2, 2, 90, dk, dv, dtype, s0_std=0.2)            # chunks and a ragged tail
+    beta = wl.make_value_decay(802, p.v.shape, dtype)
+    bhat, d, fx = _block_terms(p, 803, 2)
+    dd = prefill_to_device(p)
+    o, sT = _nan_outputs(dd)
+    kw = dict(value_decay=dev(beta, dtype))
+    ref_kw = dict(value_decay=beta)
+    if with_gate:
+        kw.update(beta_hat=dev(bhat, dtype), feed_d=torch.from_numpy(d).cuda(), feed_x=dev(fx, dtype))
+        ref_kw.update(beta_hat=bhat, feed_d=d, feed_x=fx)
+    prm = rd.fwd_params(dd["q"], dd["k"], dd["x"], dd["y"], dd["v"], o, dd["s0"], sT, scale=0.5, **kw)
+    assert rd.fwd_kernel_name(prm) == "simt"                  # also for the tensor-core shape
+    ws = rd.new_workspace(prm, "cuda")
+    prm.workspace, prm.workspace_bytes = ws.data_ptr(), ws.numel()
+    assert rd.fwd_raw(prm) == rd.OK and rd.device_status(ws) == rd.OK
+    ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0, scale=0.5, **ref_kw)
+    # the fp32 kernel computes in fp32 whatever the token dtype; bf16 only rounds o
+    assert rel_err(host(o), ro) <= _tol(dtype) and rel_err(host(sT), rs) <= TOL_F32
+
+
+def test_value_decay_packed_sequences_and_decode_steps():
+    import torch
+    lens = [33, 0, 1, 70]
+    p = _varlen(811, lens, 2, 128, 256, "bf16", s0_std=0.2)
+    beta = wl.make_value_decay(812, p.v.shape, "bf16")
+    dd = prefill_to_device(p)
+    o, sT = rd.ddts_fwd(dd["q"], dd["k"], dd["x"], dd["y"], dd["v"], dd["s0"], dd["cu"], dd["cu_host"],
+                        value_decay=dev(beta, "bf16"))
+    ro, rs = orc.ref_fwd(p.q, p.k, p.x, p.y, p.v, s0=p.s0, cu_seqlens=p.cu_seqlens, value_decay=beta)
+    eo, es = _worst_err(host(o), host(sT), ro, rs, p.cu_seqlens)
+    assert eo <= TOL_BF16 and es <= TOL_F32
+    # decode: four steps with a decay per step, bf16 and fp32 tokens
+    for dtype in ("bf16", "f32"):
+        Nseq, H, dk, dv = 5, 3, 128, 256
+        w = wl.make_decode(813, Nseq, H, dk, dv, ring=4, dtype=dtype)
+        bd = wl.make_value_decay(814, (4, Nseq, H, dv), dtype)
+        state = torch.from_numpy(w.state).cuda()
+        ref_state = w.state.astype(np.float64)
+        for s in range(4):
+            og = rd.ddts_step(*(dev(a[s], dtype) for a in (w.q, w.k, w.x, w.y, w.v)), state, scale=0.5,
+                              value_decay=dev(bd[s], dtype))
+            rg = orc.ref_step(w.q[s], w.k[s], w.x[s], w.y[s], w.v[s], ref_state, scale=0.5,
+                              value_decay=bd[s])
+            assert rel_err(host(og), rg) <= _tol(dtype)
+        assert rel_err(host(state), ref_state) <= TOL_F32
+
+
+# ------------------------------------------------------------------------------------------
 # shared-gate layout: q,k,x,y [B,1,T,dk], one set per token for all H groups of value columns
 # ------------------------------------------------------------------------------------------
 
