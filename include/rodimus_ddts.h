@@ -219,6 +219,36 @@ size_t rodimus_ddts_bwd_workspace_bytes(const rodimus_ddts_bwd_params *p);
 int rodimus_ddts_bwd(const rodimus_ddts_bwd_params *p);
 
 /*
+ * Sliding-window shared-key attention (SW-SKA), the attention half of the Rodimus+ block
+ * (Sec. "Shared-Key Attention for Lossless Head Compression": softmax attention,
+ * Eq. "attention_parallel", with one key per token shared by all heads, queries and values per
+ * head; combined with a sliding window):
+ *
+ *   s_ti = scale * <q^h_t, k_i>,  t - window < i <= t      p_ti = softmax over those i
+ *   o^h_t = sum_i p_ti v^h_i
+ *
+ * q, v, o are [B,H,T,d]; k is [B,T,d] (no head index).  d = 128 (the paper's head size; other
+ * sizes: RODIMUS_ERR_UNSUPPORTED); window >= 1 (the paper uses half the training context); dense
+ * batches only.  dtype BF16 runs on the tensor cores with a running softmax (cost O(T * window),
+ * nothing of size T x window is stored); dtype F32 is a plain fp32 validation kernel.  Needs no
+ * workspace.  o must not overlap an input.
+ */
+typedef struct {
+  int32_t struct_size; /* sizeof(rodimus_swska_fwd_params), checked */
+  int32_t dtype;       /* rodimus_dtype of q, k, v, o */
+  int32_t B, H, T, d;
+  int32_t window;      /* tokens a query sees, itself included */
+  float scale;         /* multiplies the scores; 1/sqrt(d) for the usual attention */
+  const void *q;       /* device [B,H,T,d] */
+  const void *k;       /* device [B,T,d] */
+  const void *v;       /* device [B,H,T,d] */
+  void *o;             /* device [B,H,T,d], written */
+  void *stream;
+} rodimus_swska_fwd_params;
+
+int rodimus_swska_fwd(const rodimus_swska_fwd_params *p);
+
+/*
  * rodimus_ddts_fwd for callers that cannot allocate device memory.  (A convenience of this
  * library: the paper has no counterpart.)
  *

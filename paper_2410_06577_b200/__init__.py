@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "rodimus_ddts_device_status", "rodimus_ddts_last_launch_count",
     "rodimus_ddts_fwd_kernel_name", "rodimus_status_str", "rodimus_version",
     "rodimus_ddts_fwd_noalloc", "rodimus_ddts_sfu_probe", "rodimus_ddts_test_set_wait_limit",
-    "rodimus_ddts_bwd_workspace_bytes", "rodimus_ddts_bwd",
+    "rodimus_ddts_bwd_workspace_bytes", "rodimus_ddts_bwd", "rodimus_swska_fwd",
 )
 NOALLOC_MAX_SEQS = 4096
 
@@ -88,6 +88,16 @@ class BwdParams(ctypes.Structure):
     ]
 
 
+class SwskaParams(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32), ("d", ctypes.c_int32),
+        ("window", ctypes.c_int32), ("scale", ctypes.c_float),
+        ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
+        ("o", ctypes.c_void_p), ("stream", ctypes.c_void_p),
+    ]
+
+
 _lib = None
 
 
@@ -123,6 +133,8 @@ def load_library() -> ctypes.CDLL:
         lib.rodimus_ddts_bwd_workspace_bytes.restype = ctypes.c_size_t
         lib.rodimus_ddts_bwd.argtypes = [ctypes.POINTER(BwdParams)]
         lib.rodimus_ddts_bwd.restype = ctypes.c_int
+        lib.rodimus_swska_fwd.argtypes = [ctypes.POINTER(SwskaParams)]
+        lib.rodimus_swska_fwd.restype = ctypes.c_int
         lib.rodimus_status_str.argtypes = [ctypes.c_int]
         lib.rodimus_status_str.restype = ctypes.c_char_p
         lib.rodimus_version.restype = ctypes.c_int
@@ -321,6 +333,41 @@ def ddts_bwd(q, k, gate_x, temp_y, v, d_o, s0=None, d_sT=None, cu_seqlens=None,
     if rc != OK:
         raise RodimusError(rc, "rodimus_ddts_bwd")
     return out
+
+
+def swska_params(q, k, v, o, window: int, scale: float, stream: Optional[int] = None) -> SwskaParams:
+    """Fills a ``rodimus_swska_fwd_params`` from torch tensors (no checks beyond layout)."""
+    import torch
+    B, H, T, d = q.shape
+    p = SwskaParams()
+    p.struct_size = ctypes.sizeof(SwskaParams)
+    p.dtype = _dtype_code(q)
+    p.B, p.H, p.T, p.d = B, H, T, d
+    p.window, p.scale = int(window), float(scale)
+    p.q, p.k, p.v, p.o = (_ptr(t) for t in (q, k, v, o))
+    p.stream = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    return p
+
+
+def swska_raw(p: SwskaParams) -> int:
+    """Calls ``rodimus_swska_fwd`` and returns its status without raising."""
+    return int(load_library().rodimus_swska_fwd(ctypes.byref(p)))
+
+
+def swska_fwd(q, k, v, window: int, scale: Optional[float] = None, out=None):
+    """Sliding-window shared-key attention (``rodimus_swska_fwd``): q, v [B,H,T,d], k [B,T,d]
+    (one key per token for all heads); token t attends to tokens t-window+1 .. t.  ``scale``
+    defaults to 1/sqrt(d).  Returns o [B,H,T,d].  Asynchronous on the current stream."""
+    import torch
+    _check_cuda(q, k, v)
+    if k.shape != (q.shape[0], q.shape[2], q.shape[3]) or v.shape != q.shape:
+        raise ValueError("q, v must be [B,H,T,d] and k [B,T,d]")
+    o = out if out is not None else torch.empty_like(q)
+    p = swska_params(q, k, v, o, window, q.shape[-1] ** -0.5 if scale is None else scale)
+    rc = swska_raw(p)
+    if rc != OK:
+        raise RodimusError(rc, "rodimus_swska_fwd")
+    return o
 
 
 def ddts_fwd(q, k, gate_x, temp_y, v, s0=None, cu_seqlens=None, cu_seqlens_host=None,

@@ -47,6 +47,8 @@ cudaError_t launch_fwd_pair(const rodimus_ddts_fwd_params& p, int* n_launches);
 cudaError_t launch_bwd(const rodimus_ddts_bwd_params& p, size_t scratch_offset, int* n_launches);
 bool bwd_supported(const rodimus_ddts_bwd_params& p);
 size_t bwd_scratch_bytes(const rodimus_ddts_bwd_params& p);   // beyond the header and the order
+cudaError_t launch_swska(const rodimus_swska_fwd_params& p, int* n_launches);
+bool swska_supported(const rodimus_swska_fwd_params& p);
 bool fwd_tc_supported(const rodimus_ddts_fwd_params& p);
 bool fwd_pair_supported(const rodimus_ddts_fwd_params& p);
 // Workspace a dense call needs if its sequences are to be split along time (0: no split).

@@ -217,6 +217,26 @@ int rodimus_ddts_bwd(const rodimus_ddts_bwd_params* p) {
   return RODIMUS_OK;
 }
 
+int rodimus_swska_fwd(const rodimus_swska_fwd_params* p) {
+  t_last_launches = 0;
+  if (!p) return RODIMUS_ERR_NULL;
+  if (p->struct_size != (int32_t)sizeof(rodimus_swska_fwd_params)) return RODIMUS_ERR_DTYPE;
+  if (p->dtype != RODIMUS_BF16 && p->dtype != RODIMUS_F32) return RODIMUS_ERR_DTYPE;
+  if (p->B < 0 || p->H < 0 || p->T < 0 || p->d <= 0 || p->window < 1) return RODIMUS_ERR_SHAPE;
+  if (!ddts::swska_supported(*p)) return RODIMUS_ERR_UNSUPPORTED;
+  if ((long long)p->B * p->H * p->T >= (1LL << 31) || p->B > 65535 || p->H > 65535)
+    return RODIMUS_ERR_SHAPE;
+  if ((long long)p->B * p->H * p->T == 0) return RODIMUS_OK;
+  if (!p->q || !p->k || !p->v || !p->o) return RODIMUS_ERR_NULL;
+  const void* ptrs[] = {p->q, p->k, p->v, p->o};
+  for (const void* ptr : ptrs)
+    if (!aligned16(ptr)) return RODIMUS_ERR_ALIGN;
+  int n = 0;
+  if (ddts::launch_swska(*p, &n) != cudaSuccess) return RODIMUS_ERR_CUDA;
+  t_last_launches = n;
+  return RODIMUS_OK;
+}
+
 int rodimus_ddts_step(const rodimus_ddts_step_params* p) {
   t_last_launches = 0;
   if (!p) return RODIMUS_ERR_NULL;
@@ -279,6 +299,6 @@ const char* rodimus_status_str(int status) {
   }
 }
 
-int rodimus_version(void) { return 104; }
+int rodimus_version(void) { return 105; }
 
 }  // extern "C"

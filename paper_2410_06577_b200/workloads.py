@@ -105,6 +105,16 @@ def make_value_decay(seed: int, shape, dtype: str, low: float = 0.8) -> np.ndarr
     return _round(np.float32(1.0) - np.float32(1.0 - low) * rng.random(shape, dtype=np.float32), dtype)
 
 
+def make_swska(seed: int, B: int, H: int, T: int, d: int = 128, dtype: str = "bf16"):
+    """Inputs of the sliding-window shared-key attention: q [B,H,T,d], the shared k [B,T,d] and
+    v [B,H,T,d], all ~ N(0,1), rounded to ``dtype`` (draw order q, k, v)."""
+    rng = np.random.default_rng(seed)
+    q = _round(rng.standard_normal((B, H, T, d), dtype=np.float32), dtype)
+    k = _round(rng.standard_normal((B, T, d), dtype=np.float32), dtype)
+    v = _round(rng.standard_normal((B, H, T, d), dtype=np.float32), dtype)
+    return q, k, v
+
+
 def varlen_lengths(seed: int, n_seq: int, lo: int, hi: int) -> np.ndarray:
     """Lengths uniform in [lo, hi] and their exclusive prefix sum (int32 [n_seq+1])."""
     rng = np.random.default_rng(seed)

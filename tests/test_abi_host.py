@@ -47,7 +47,9 @@ def test_struct_layout_matches_header(tmp_path):
         " offsetof(rodimus_ddts_step_params,stream));"
         "printf(\"%zu %zu %zu %zu\\n\", sizeof(rodimus_ddts_bwd_params),"
         " offsetof(rodimus_ddts_bwd_params,q), offsetof(rodimus_ddts_bwd_params,d_s0),"
-        " offsetof(rodimus_ddts_bwd_params,stream));return 0;}\n")
+        " offsetof(rodimus_ddts_bwd_params,stream));"
+        "printf(\"%zu %zu %zu\\n\", sizeof(rodimus_swska_fwd_params),"
+        " offsetof(rodimus_swska_fwd_params,q), offsetof(rodimus_swska_fwd_params,stream));return 0;}\n")
     exe = tmp_path / "sz"
     subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)], check=True)
     out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
@@ -55,7 +57,8 @@ def test_struct_layout_matches_header(tmp_path):
     want = [ctypes.sizeof(rd.FwdParams), rd.FwdParams.q.offset, rd.FwdParams.stream.offset,
             ctypes.sizeof(rd.StepParams), rd.StepParams.q.offset, rd.StepParams.stream.offset,
             ctypes.sizeof(rd.BwdParams), rd.BwdParams.q.offset, rd.BwdParams.d_s0.offset,
-            rd.BwdParams.stream.offset]
+            rd.BwdParams.stream.offset,
+            ctypes.sizeof(rd.SwskaParams), rd.SwskaParams.q.offset, rd.SwskaParams.stream.offset]
     assert got == want
 
 
@@ -202,6 +205,26 @@ def test_bwd_argument_errors_and_workspace_size(lib):
     assert rd.bwd_raw(pv) == rd.ERR_SEQLENS
     ok = _bwd(B=0, workspace=0x7F0000002000, workspace_bytes=4096)
     assert rd.bwd_raw(ok) == rd.OK and rd.last_launch_count() == 0
+
+
+def test_swska_argument_errors(lib):
+    def mk(**kw):
+        p = rd.SwskaParams()
+        p.struct_size = ctypes.sizeof(rd.SwskaParams)
+        p.dtype, p.B, p.H, p.T, p.d, p.window, p.scale = rd.BF16, 2, 2, 64, 128, 16, 0.1
+        p.q = p.k = p.v = p.o = FAKE
+        for key, val in kw.items():
+            setattr(p, key, val)
+        return p
+    assert lib.rodimus_swska_fwd(None) == rd.ERR_NULL
+    assert rd.swska_raw(mk(struct_size=4)) == rd.ERR_DTYPE
+    assert rd.swska_raw(mk(dtype=3)) == rd.ERR_DTYPE
+    assert rd.swska_raw(mk(window=0)) == rd.ERR_SHAPE
+    assert rd.swska_raw(mk(T=-2)) == rd.ERR_SHAPE
+    assert rd.swska_raw(mk(d=64)) == rd.ERR_UNSUPPORTED
+    assert rd.swska_raw(mk(k=0)) == rd.ERR_NULL
+    assert rd.swska_raw(mk(o=FAKE + 8)) == rd.ERR_ALIGN
+    assert rd.swska_raw(mk(T=0)) == rd.OK and rd.last_launch_count() == 0
 
 
 def test_missing_library_fails_loudly(tmp_path, monkeypatch):
