@@ -474,6 +474,56 @@ def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sf
     return rec
 
 
+def measure_swska(steps, warmup, local, peaks, peak_kind, B=4, H=16, T=2048, d=128, window=1024):
+    """Sub-record for the sliding-window shared-key attention on the layer shape (window = half the
+    context, as the paper sets it): CUDA events around `steps` calls, tensor roofline against the
+    measured bf16 rate.  Flops counted from the definition: 4 d per (query, visible key)."""
+    import torch
+    import paper_2410_06577_b200 as rd
+    from paper_2410_06577_b200 import workloads as wl
+    device = torch.device("cuda", local)
+    q, k, v = (torch.from_numpy(a).to(torch.bfloat16).to(device) for a in wl.make_swska(31, B, H, T, d))
+    o = torch.empty_like(q)
+    prm = rd.swska_params(q, k, v, o, window, d ** -0.5)
+    stream = torch.cuda.current_stream()
+
+    def region(n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            rc = rd.swska_raw(prm)
+            if rc != rd.OK:
+                raise SystemExit(f"rodimus_swska_fwd: {rd.status_str(rc)}")
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    region(warmup)
+    with ClockSampler(local) as clk:
+        times = [region(steps) for _ in range(5)]
+    ms = float(np.median(times)) / steps
+    pairs = sum(min(t + 1, window) for t in range(T))          # visible (query, key) pairs per head
+    flops = 4.0 * d * pairs * B * H
+    alg_bytes = (3 * B * H * T * d + B * T * d) * 2
+    achieved = flops / (ms / 1e3) / 1e12
+    return {
+        "metric": "SW-SKA tokens/s", "value": B * T / (ms / 1e3), "unit": "tokens/s", "steps": steps,
+        "warmup": warmup, "ms_per_step": ms, "dtype": "bf16",
+        "config": {"workload": f"SW-SKA B={B} H={H} T={T} d={d} window={window} bf16, one key per token for all heads",
+                   "l2": "inputs of 105 MB, no flush (the path is bound by the tensor pipe)"},
+        "timed_regions": {"count": len(times), "steps_each": steps, "reported": "median",
+                          "ms_min": float(min(times)), "ms_median": float(np.median(times)),
+                          "ms_max": float(max(times))},
+        "clocks": clk.summary(), "gpu_launches": steps,
+        "roofline": {"bound": "tensor", "kernel": "swska_fwd_bf16_kernel", "achieved": achieved,
+                     "peak": peaks["bf16_tflops"], "peak_kind": f"of {peak_kind} (burst)", "unit": "TFLOP/s",
+                     "frac": achieved / peaks["bf16_tflops"], "algorithmic_flops_per_launch": flops,
+                     "bound_times": {"tensor_us": flops / (peaks["bf16_tflops"] * 1e12) * 1e6,
+                                     "hbm_us": alg_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6},
+                     "traffic": None},
+    }
+
+
 SUB_DEFAULTS = {"cfg1": (500, 5), "cfg2": (100, 5), "cfg4": (40, 5), "cfg3": (1000, 10)}
 
 
@@ -527,6 +577,8 @@ def run_ours(args, workload, p):
                                                    "dtype", "config", "timed_regions", "clocks",
                                                    "gpu_launches", "roofline")}
             del pw
+        torch.cuda.empty_cache()
+        extra["swska_layer"] = measure_swska(50, 5, local, peaks, peak_kind)
         line["workloads"] = extra
     if rank == 0:
         print(json.dumps(line), flush=True)
@@ -541,6 +593,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg1")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--swska", action="store_true",
+                    help="time the sliding-window shared-key attention alone (for profiling)")
     ap.add_argument("--variant", choices=["block", "shared", "backward", "vdecay"], default=None,
                     help="time a variant of the config-1 workload instead (for profiling; no e2e)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -558,6 +612,12 @@ def main():
     from paper_2410_06577_b200 import workloads as wl
     rank = int(os.environ.get("RANK", "0"))
     if args.impl == "reference" and rank != 0:
+        return
+    if args.swska and args.impl == "ours":
+        import torch
+        torch.cuda.set_device(0)
+        peaks, peak_kind = load_peaks()
+        print(json.dumps(measure_swska(args.steps, args.warmup, 0, peaks, peak_kind)), flush=True)
         return
     p = wl.config(WORKLOADS[args.workload])
     if args.impl == "reference":

@@ -147,17 +147,30 @@ __global__ void __launch_bounds__(kThreads, 2) swska_fwd_bf16_kernel(const SwArg
           mma_bf16(s[j + 1], qf[kk], bk[2], bk[3]);
         }
       }
-      // scale into the log2 domain, mask what lies outside (row - W, row]
+      // scale into the log2 domain; where the tile is not wholly inside the window of all 16
+      // rows, mask what lies outside (row - W, row]
       float mx[2] = {-INFINITY, -INFINITY};
+      const bool inside = n0 + kBN - 1 <= wrow0 && n0 > wrow0 + 15 - W;
+      if (inside) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < 8; ++j) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int key = n0 + 8 * j + 2 * t + (e & 1), row = row_lo + (e >> 1) * 8;
-          const bool in = key <= row && key > row - W;
-          const float x = in ? s[j][e] * sc : -INFINITY;
-          s[j][e] = x;
-          mx[e >> 1] = fmaxf(mx[e >> 1], x);
+          for (int e = 0; e < 4; ++e) {
+            s[j][e] *= sc;
+            mx[e >> 1] = fmaxf(mx[e >> 1], s[j][e]);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int key = n0 + 8 * j + 2 * t + (e & 1), row = row_lo + (e >> 1) * 8;
+            const bool in = key <= row && key > row - W;
+            const float x = in ? s[j][e] * sc : -INFINITY;
+            s[j][e] = x;
+            mx[e >> 1] = fmaxf(mx[e >> 1], x);
+          }
         }
       }
       float alpha[2], m_use[2];
