@@ -515,7 +515,7 @@ def measure_swska(steps, warmup, local, peaks, peak_kind, B=4, H=16, T=2048, d=1
                           "ms_min": float(min(times)), "ms_median": float(np.median(times)),
                           "ms_max": float(max(times))},
         "clocks": clk.summary(), "gpu_launches": steps,
-        "roofline": {"bound": "tensor", "kernel": "swska_fwd_bf16_kernel", "achieved": achieved,
+        "roofline": {"bound": "tensor", "kernel": "swska_fwd_tc_kernel", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "peak_kind": f"of {peak_kind} (burst)", "unit": "TFLOP/s",
                      "frac": achieved / peaks["bf16_tflops"], "algorithmic_flops_per_launch": flops,
                      "bound_times": {"tensor_us": flops / (peaks["bf16_tflops"] * 1e12) * 1e6,

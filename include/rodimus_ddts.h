@@ -229,9 +229,11 @@ int rodimus_ddts_bwd(const rodimus_ddts_bwd_params *p);
  *
  * q, v, o are [B,H,T,d]; k is [B,T,d] (no head index).  d = 128 (the paper's head size; other
  * sizes: RODIMUS_ERR_UNSUPPORTED); window >= 1 (the paper uses half the training context); dense
- * batches only.  dtype BF16 runs on the tensor cores with a running softmax (cost O(T * window),
- * nothing of size T x window is stored); dtype F32 is a plain fp32 validation kernel.  Needs no
- * workspace.  o must not overlap an input.
+ * batches only.  dtype BF16 runs on the tcgen05 tensor cores with a running softmax (cost
+ * O(T * window), nothing of size T x window is stored); dtype F32 is a plain fp32 validation
+ * kernel.  o must not overlap an input.  `workspace` is optional: given (>= 256 bytes, 256-byte
+ * aligned), its first word is the status rodimus_ddts_device_status reads (RODIMUS_ERR_TIMEOUT
+ * if a bounded wait inside the kernel ran out; outputs are then unspecified).
  */
 typedef struct {
   int32_t struct_size; /* sizeof(rodimus_swska_fwd_params), checked */
@@ -244,6 +246,8 @@ typedef struct {
   const void *v;       /* device [B,H,T,d] */
   void *o;             /* device [B,H,T,d], written */
   void *stream;
+  void *workspace;     /* optional device status area, see above */
+  size_t workspace_bytes;
 } rodimus_swska_fwd_params;
 
 int rodimus_swska_fwd(const rodimus_swska_fwd_params *p);

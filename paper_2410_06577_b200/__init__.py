@@ -95,6 +95,7 @@ class SwskaParams(ctypes.Structure):
         ("window", ctypes.c_int32), ("scale", ctypes.c_float),
         ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
         ("o", ctypes.c_void_p), ("stream", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
     ]
 
 
@@ -335,7 +336,8 @@ def ddts_bwd(q, k, gate_x, temp_y, v, d_o, s0=None, d_sT=None, cu_seqlens=None,
     return out
 
 
-def swska_params(q, k, v, o, window: int, scale: float, stream: Optional[int] = None) -> SwskaParams:
+def swska_params(q, k, v, o, window: int, scale: float, stream: Optional[int] = None,
+                 workspace=None) -> SwskaParams:
     """Fills a ``rodimus_swska_fwd_params`` from torch tensors (no checks beyond layout)."""
     import torch
     B, H, T, d = q.shape
@@ -346,6 +348,8 @@ def swska_params(q, k, v, o, window: int, scale: float, stream: Optional[int] = 
     p.window, p.scale = int(window), float(scale)
     p.q, p.k, p.v, p.o = (_ptr(t) for t in (q, k, v, o))
     p.stream = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    p.workspace = _ptr(workspace)
+    p.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     return p
 
 

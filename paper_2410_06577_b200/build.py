@@ -14,7 +14,7 @@ CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "librodimus_ddts.so")
 
-SOURCES = ["rodimus_ddts.cu", "ddts_step.cu", "ddts_fwd_simt.cu", "ddts_plan.cu", "ddts_fwd_tc.cu", "ddts_fwd_pair.cu", "ddts_noalloc.cu", "ddts_probe.cu", "ddts_bwd.cu", "swska_fwd.cu"]
+SOURCES = ["rodimus_ddts.cu", "ddts_step.cu", "ddts_fwd_simt.cu", "ddts_plan.cu", "ddts_fwd_tc.cu", "ddts_fwd_pair.cu", "ddts_noalloc.cu", "ddts_probe.cu", "ddts_bwd.cu", "swska_fwd.cu", "swska_fwd_tc.cu"]
 
 
 def _nvcc() -> str:

@@ -48,6 +48,7 @@ cudaError_t launch_bwd(const rodimus_ddts_bwd_params& p, size_t scratch_offset, 
 bool bwd_supported(const rodimus_ddts_bwd_params& p);
 size_t bwd_scratch_bytes(const rodimus_ddts_bwd_params& p);   // beyond the header and the order
 cudaError_t launch_swska(const rodimus_swska_fwd_params& p, int* n_launches);
+cudaError_t launch_swska_tc(const rodimus_swska_fwd_params& p, int* n_launches);   // bf16, tcgen05
 bool swska_supported(const rodimus_swska_fwd_params& p);
 bool fwd_tc_supported(const rodimus_ddts_fwd_params& p);
 bool fwd_pair_supported(const rodimus_ddts_fwd_params& p);

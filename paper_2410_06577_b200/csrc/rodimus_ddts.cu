@@ -231,6 +231,10 @@ int rodimus_swska_fwd(const rodimus_swska_fwd_params* p) {
   const void* ptrs[] = {p->q, p->k, p->v, p->o};
   for (const void* ptr : ptrs)
     if (!aligned16(ptr)) return RODIMUS_ERR_ALIGN;
+  if (p->workspace) {
+    if (p->workspace_bytes < sizeof(ddts::WorkspaceHeader)) return RODIMUS_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(p->workspace) & 255u) return RODIMUS_ERR_ALIGN;
+  }
   int n = 0;
   if (ddts::launch_swska(*p, &n) != cudaSuccess) return RODIMUS_ERR_CUDA;
   t_last_launches = n;

@@ -290,6 +290,7 @@ cudaError_t launch_swska(const rodimus_swska_fwd_params& p, int* n_launches) {
   a.q = p.q; a.k = p.k; a.v = p.v; a.o = p.o;
   a.B = p.B; a.H = p.H; a.T = p.T; a.window = p.window; a.scale = p.scale;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
+  if (p.dtype == RODIMUS_BF16) return launch_swska_tc(p, n_launches);
   if (p.dtype == RODIMUS_BF16) {
     int dev = 0, sms = 0;
     cudaError_t e = current_device(&dev, &sms);

@@ -1,0 +1,360 @@
+// Sliding-window shared-key attention on tcgen05 (bf16 tokens, head size 128):
+//   s_ti = scale <q^h_t, k_i>,  t - W < i <= t      p_ti = softmax_i(s_ti)      o^h_t = sum_i p_ti v^h_i
+// (Sec. "Shared-Key Attention for Lossless Head Compression": one key per token for all heads.)
+//
+// One CTA of 128 threads per (batch, head, 128 queries); thread = query row = tensor-memory lane,
+// so the softmax of a row never leaves its thread.  Per key tile of 128 tokens:
+//   S = Q K^T        tcgen05.mma, Q and K tiles K-major in shared memory (TMA, 128-byte swizzle),
+//                    accumulator [128 x 128] fp32 in tensor memory
+//   softmax          each thread reads its row of S (tcgen05.ld), keeps a running maximum and sum
+//                    in the log2 domain, rescales its row of O in tensor memory when the maximum
+//                    moved, and writes the probabilities back over S as packed bf16 (tcgen05.st)
+//   O += P V         tcgen05.mma with P as the A operand IN TENSOR MEMORY and the V tile
+//                    (token-major, i.e. N-major B operand) from shared memory
+// Tensor memory: 256 columns (S, overwritten by P, and O), shared memory 96 KiB (Q, one K tile,
+// one V tile): two CTAs per SM, one CTA's softmax overlapping the other's contractions.  The K
+// tile of the next step is requested as soon as S is complete, the V tile as soon as the previous
+// O += P V is complete.  Only key tiles that touch the 128 queries' windows are visited.
+// Every wait is bounded; a wait that runs out ends the kernel cleanly (copies and contractions in
+// flight are waited for, tensor memory is freed) and raises RODIMUS_ERR_TIMEOUT in the status word.
+#include "ddts_tc_ptx.cuh"
+
+namespace ddts {
+namespace {
+
+constexpr int kD = 128, kBM = 128, kBN = 128, kThreads = 128;
+constexpr uint32_t kSlabBytes = 128 * 128;            // [128 rows][64 columns] bf16
+constexpr uint32_t kTileBytes = 2 * kSlabBytes;       // 128 x 128 bf16
+constexpr uint32_t kOffQ = 0, kOffK = kTileBytes, kOffV = 2 * kTileBytes, kOffCtl = 3 * kTileBytes;
+constexpr uint32_t kSmemBytes = kOffCtl + 256 + 1024; // + control block + slack for 1024-byte alignment
+constexpr uint32_t kTmemCols = 256, kColS = 0, kColO = 128;
+constexpr float kLog2e = 1.4426950408889634f;
+
+enum { BAR_Q = 0, BAR_K, BAR_V, BAR_S, BAR_O, BAR_DRAIN, kNumBars };
+
+struct SwCtl {
+  uint64_t bar[kNumBars];
+  uint32_t tmem_base;
+  int abort;
+  long long limit;
+};
+
+struct SwTcArgs {
+  void* o;
+  int32_t* status;   // may be nullptr
+  int H, T, window;
+  float scale;
+  long long limit;
+};
+
+__device__ __noinline__ bool sw_wait_slow(uint32_t bar, uint32_t parity, volatile SwCtl* c, int32_t* status) {
+  const long long limit = c->limit, t0 = clock64();
+  while (true) {
+    if (limit > 0) {
+#pragma unroll 1
+      for (int i = 0; i < 16; ++i)
+        if (mbar_try_park(bar, parity)) return true;
+    }
+    if (c->abort) return mbar_try(bar, parity);
+    if (clock64() - t0 >= limit) {
+      if (mbar_try(bar, parity)) return true;
+      c->abort = 1;
+      if (status) atomicMax(status, (int)RODIMUS_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool sw_wait(uint32_t bar, uint32_t parity, volatile SwCtl* c, int32_t* status) {
+  if (mbar_try(bar, parity)) return true;
+  return sw_wait_slow(bar, parity, c, status);
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                    const __grid_constant__ CUtensorMap map_v, const SwTcArgs a) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
+  volatile SwCtl* ctl = reinterpret_cast<volatile SwCtl*>(gen + kOffCtl);
+  auto bar = [&](int i) { return base + kOffCtl + 8u * (uint32_t)i; };
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int m0 = blockIdx.x * kBM, h = blockIdx.y, b = blockIdx.z;
+  const int T = a.T, W = a.window;
+  const long long bh = (long long)b * a.H + h;
+  const int qrow0 = (int)(bh * T) + m0;          // row of the [B*H*T, 128] views of q, v, o
+  const int krow0 = b * T;                       // row of the [B*T, 128] view of k
+  const int vrow0 = (int)(bh * T);
+  const int first_key = max(0, m0 - W + 1);
+  const int nt_lo = first_key / kBN, nt_hi = min(m0 + kBM - 1, T - 1) / kBN;
+
+  if (tid == 0) {
+    ctl->abort = 0;
+    ctl->limit = a.limit;
+    for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(base + kOffCtl + (uint32_t)offsetof(SwCtl, tmem_base)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctl->tmem_base;
+  const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes
+
+  // what thread 0 has asked for and not yet seen complete (for the clean exit)
+  int k_sent = 0, v_sent = 0, q_sent = 0, k_seen = 0, v_seen = 0, q_seen = 0;
+  auto load_tile = [&](const CUtensorMap* map, uint32_t dst, int row, int which) {
+    mbar_expect_tx(bar(which), kTileBytes);
+    tma_load_2d(base + dst, map, 0, row, bar(which));
+    tma_load_2d(base + dst + kSlabBytes, map, 64, row, bar(which));
+  };
+  if (tid == 0) {
+    load_tile(&map_q, kOffQ, qrow0, BAR_Q); q_sent = 1;
+    load_tile(&map_k, kOffK, krow0 + nt_lo * kBN, BAR_K); k_sent = 1;
+    load_tile(&map_v, kOffV, vrow0 + nt_lo * kBN, BAR_V); v_sent = 1;
+  }
+
+  constexpr uint32_t kIdescS = make_idesc(kBM, kBN, 0, 0);   // S = Q K^T, both K-major
+  constexpr uint32_t kIdescO = make_idesc(kBM, kD, 0, 1);    // O += P V, A in tensor memory, B N-major
+  const uint32_t dq0 = desc_lo_kmajor(base + kOffQ), dq1 = desc_lo_kmajor(base + kOffQ + kSlabBytes);
+  const uint32_t dk0 = desc_lo_kmajor(base + kOffK), dk1 = desc_lo_kmajor(base + kOffK + kSlabBytes);
+  const uint32_t dv = desc_lo_mnmajor(base + kOffV, kSlabBytes);
+
+  const int row = m0 + tid;                 // this thread's query
+  const float sc = a.scale * kLog2e;
+  float m_run = -INFINITY, l_run = 0.f;
+  bool ok = true;
+  int it = 0;
+  for (int nt = nt_lo; nt <= nt_hi; ++nt, ++it) {
+    const uint32_t ph = it & 1;
+    const int n0 = nt * kBN;
+    if (tid == 0) {
+      if (it == 0) { ok = sw_wait(bar(BAR_Q), 0, ctl, a.status); q_seen = ok; }
+      if (ok) { ok = sw_wait(bar(BAR_K), ph, ctl, a.status); k_seen += ok; }
+      if (ok) {
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          if (kk == 0) umma_bf16_lo<false>(tmem + kColS, dq0, dk0, kIdescS);
+          else umma_bf16_lo<true>(tmem + kColS, dq0 + 2 * kk, dk0 + 2 * kk, kIdescS);
+        }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColS, dq1 + 2 * kk, dk1 + 2 * kk, kIdescS);
+        umma_commit(bar(BAR_S));
+        // the previous O += P V sits before this S in the pipe: once it is done, the V tile is free
+        if (it > 0) {
+          ok = sw_wait(bar(BAR_O), ph ^ 1, ctl, a.status);
+          if (ok) { load_tile(&map_v, kOffV, vrow0 + n0, BAR_V); ++v_sent; }
+        }
+      }
+    }
+    if (ok) ok = sw_wait(bar(BAR_S), ph, ctl, a.status);
+    ok = __all_sync(0xffffffffu, ok);     // the tensor-memory accesses below need the whole warp
+    tc_fence_after();
+    if (tid == 0 && ok && nt < nt_hi) {       // S is complete: the K tile is free
+      load_tile(&map_k, kOffK, krow0 + n0 + kBN, BAR_K);
+      ++k_sent;
+    }
+    float alpha = 1.f;
+    if (ok) {
+      // ---- this row of S: scale to the log2 domain, mask, maximum
+      float s[kBN];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_row + kColS + 32 * c, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) s[32 * c + e] = __uint_as_float(r[e]) * sc;
+      }
+      const bool inside = n0 + kBN - 1 <= row && n0 > row - W;
+      float mx = -INFINITY;
+      if (inside) {
+#pragma unroll
+        for (int e = 0; e < kBN; ++e) mx = fmaxf(mx, s[e]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < kBN; ++e) {
+          const int key = n0 + e;
+          s[e] = (key <= row && key > row - W) ? s[e] : -INFINITY;
+          mx = fmaxf(mx, s[e]);
+        }
+      }
+      const float m_new = fmaxf(m_run, mx);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;    // a row that has seen no key yet
+      alpha = ex2f(m_run - m_use);
+      m_run = m_new;
+      float psum = 0.f;
+      uint32_t pk[kBN / 2];
+#pragma unroll
+      for (int e = 0; e < kBN; e += 2) {
+        const float p0 = ex2f(s[e] - m_use), p1 = ex2f(s[e + 1] - m_use);
+        psum += p0 + p1;
+        pk[e >> 1] = pack_bf16(p0, p1);
+      }
+      l_run = l_run * alpha + psum;
+      // ---- the previous O += P V must be complete before O is rescaled and P overwritten
+      if (it > 0) ok = sw_wait(bar(BAR_O), ph ^ 1, ctl, a.status);
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after();
+      if (ok) {
+        if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tmem_ld32(t_row + kColO + 32 * c, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+            tmem_st32(t_row + kColO + 32 * c, r);
+          }
+        }
+        {
+          uint32_t r[32];
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) r[e] = pk[32 * c + e];
+            tmem_st32(t_row + kColS + 32 * c, r);
+          }
+        }
+        tmem_st_wait();
+      }
+    }
+    tc_fence_before();
+    ok = __syncthreads_and(ok) != 0;      // every row's P is in place (or everyone gives up)
+    if (!ok) break;
+    if (tid == 0) {
+      tc_fence_after();
+      ok = sw_wait(bar(BAR_V), ph, ctl, a.status);
+      v_seen += ok;
+      if (ok) {
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          if (kk == 0 && it == 0) umma_bf16_atmem<false>(tmem + kColO, tmem + kColS, dv, kIdescO);
+          else umma_bf16_atmem<true>(tmem + kColO, tmem + kColS + 8 * kk, dv + 128 * kk, kIdescO);
+        }
+        umma_commit(bar(BAR_O));
+      }
+    }
+  }
+
+  // ---- the last O += P V, then normalise and store this thread's row
+  if (ok && it > 0) ok = sw_wait(bar(BAR_O), (it - 1) & 1, ctl, a.status);
+  ok = __all_sync(0xffffffffu, ok);
+  tc_fence_after();
+  if (ok && it > 0) {
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    __nv_bfloat16* orow = (__nv_bfloat16*)a.o + ((long long)qrow0 + tid) * kD;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      uint32_t r[32];
+      tmem_ld32(t_row + kColO + 32 * c, r);
+      tmem_ld_wait();
+      if (row < T) {
+#pragma unroll
+      for (int e = 0; e < 32; e += 8) {
+        uint4 w;
+        w.x = pack_bf16(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
+        w.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+        w.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+        w.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+        *reinterpret_cast<uint4*>(orow + 32 * c + e) = w;
+      }
+      }
+    }
+  }
+
+  // ---- clean exit: nothing may still be writing this CTA's shared or tensor memory
+  if (tid == 0 && ctl->abort) {
+    if (q_sent && !q_seen) mbar_drain(bar(BAR_Q), 0);
+    while (k_seen < k_sent) { mbar_drain(bar(BAR_K), k_seen & 1); ++k_seen; }
+    while (v_seen < v_sent) { mbar_drain(bar(BAR_V), v_seen & 1); ++v_seen; }
+    umma_commit(bar(BAR_DRAIN));          // completes when every contraction issued so far has
+    mbar_drain(bar(BAR_DRAIN), 0);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn sw_encode_fn() {
+  static const EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// [rows, 128] bf16 row-major; box = 128 rows x 64 columns (128 bytes), 128-byte swizzle; rows past
+// the end of the tensor read as zeros
+bool sw_make_map(CUtensorMap* m, const void* ptr, uint64_t rows) {
+  EncodeTiledFn fn = sw_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)kD, rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+  const cuuint32_t box[2] = {64u, 128u};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct SwMapCache {     // the three maps of the last call on this host thread
+  const void *q = nullptr, *k = nullptr, *v = nullptr;
+  uint64_t rows_q = 0, rows_k = 0;
+  CUtensorMap mq, mk, mv;
+};
+thread_local SwMapCache t_sw_maps;
+std::atomic<unsigned long long> g_sw_tc_smem_done{0};
+
+}  // namespace
+
+cudaError_t launch_swska_tc(const rodimus_swska_fwd_params& p, int* n_launches) {
+  *n_launches = 0;
+  const uint64_t rows_q = (uint64_t)p.B * p.H * p.T, rows_k = (uint64_t)p.B * p.T;
+  SwMapCache& c = t_sw_maps;
+  if (c.q != p.q || c.k != p.k || c.v != p.v || c.rows_q != rows_q || c.rows_k != rows_k) {
+    if (!sw_make_map(&c.mq, p.q, rows_q) || !sw_make_map(&c.mk, p.k, rows_k) || !sw_make_map(&c.mv, p.v, rows_q)) {
+      c.q = nullptr;
+      return cudaErrorInvalidValue;
+    }
+    c.q = p.q; c.k = p.k; c.v = p.v; c.rows_q = rows_q; c.rows_k = rows_k;
+  }
+  int dev = 0, sms = 0;
+  cudaError_t e = current_device(&dev, &sms);
+  if (e != cudaSuccess) return e;
+  e = opt_in_shared_memory(swska_fwd_tc_kernel, (int)kSmemBytes, dev, g_sw_tc_smem_done);
+  if (e != cudaSuccess) return e;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
+  SwTcArgs a;
+  a.o = p.o;
+  a.status = reinterpret_cast<int32_t*>(p.workspace);
+  a.H = p.H; a.T = p.T; a.window = p.window; a.scale = p.scale;
+  a.limit = main_loop_wait_cycles();
+  if (a.status) {
+    e = cudaMemsetAsync(a.status, 0, sizeof(int32_t), st);
+    if (e != cudaSuccess) return e;
+  }
+  const dim3 grid((p.T + kBM - 1) / kBM, p.H, p.B);
+  swska_fwd_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(c.mq, c.mk, c.mv, a);
+  *n_launches = 1;
+  return cudaGetLastError();
+}
+
+}  // namespace ddts

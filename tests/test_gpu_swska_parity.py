@@ -55,3 +55,26 @@ def test_swska_layer_shape_sampled_heads():
     for b, h in ((0, 0), (3, 11)):
         ref = sw.swska_ref(q[b:b + 1, h:h + 1], k[b:b + 1], v[b:b + 1, h:h + 1], 1024, 128 ** -0.5)
         assert rel_err(got[b:b + 1, h:h + 1], ref) <= TOL_BF16
+
+
+def test_swska_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
+    """With the wait limit set to zero the tensor-core kernel's first unsatisfied wait runs out: the
+    kernel must end by itself, report RODIMUS_ERR_TIMEOUT in the status word and leave the device
+    usable; the next call, with the default limit, is correct."""
+    import torch
+    q, k, v = wl.make_swska(970, 1, 2, 300, 128, "bf16")
+    dq, dk, dv_ = dev(q, "bf16"), dev(k, "bf16"), dev(v, "bf16")
+    o = torch.zeros_like(dq)
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    prm = rd.swska_params(dq, dk, dv_, o, 100, 128 ** -0.5, workspace=ws)
+    rd.test_set_wait_limit(0)
+    try:
+        assert rd.swska_raw(prm) == rd.OK
+        assert rd.device_status(ws) == rd.ERR_TIMEOUT
+    finally:
+        rd.test_set_wait_limit(-1)
+    o = torch.full_like(dq, float("nan"))
+    prm = rd.swska_params(dq, dk, dv_, o, 100, 128 ** -0.5, workspace=ws)
+    assert rd.swska_raw(prm) == rd.OK
+    assert rd.device_status(ws) == rd.OK
+    assert rel_err(host(o), sw.swska_ref(q, k, v, 100, 128 ** -0.5)) <= TOL_BF16
