@@ -240,7 +240,7 @@ typedef struct {
   int32_t dtype;       /* rodimus_dtype of q, k, v, o */
   int32_t B, H, T, d;
   int32_t window;      /* tokens a query sees, itself included */
-  float scale;         /* multiplies the scores; 1/sqrt(d) for the usual attention */
+  float scale;         /* multiplies the scores, > 0; 1/sqrt(d) for the usual attention */
   const void *q;       /* device [B,H,T,d] */
   const void *k;       /* device [B,T,d] */
   const void *v;       /* device [B,H,T,d] */

@@ -223,6 +223,7 @@ int rodimus_swska_fwd(const rodimus_swska_fwd_params* p) {
   if (p->struct_size != (int32_t)sizeof(rodimus_swska_fwd_params)) return RODIMUS_ERR_DTYPE;
   if (p->dtype != RODIMUS_BF16 && p->dtype != RODIMUS_F32) return RODIMUS_ERR_DTYPE;
   if (p->B < 0 || p->H < 0 || p->T < 0 || p->d <= 0 || p->window < 1) return RODIMUS_ERR_SHAPE;
+  if (!(p->scale > 0.f) || !(p->scale < 1e30f)) return RODIMUS_ERR_SHAPE;   // positive and finite
   if (!ddts::swska_supported(*p)) return RODIMUS_ERR_UNSUPPORTED;
   if ((long long)p->B * p->H * p->T >= (1LL << 31) || p->B > 65535 || p->H > 65535)
     return RODIMUS_ERR_SHAPE;

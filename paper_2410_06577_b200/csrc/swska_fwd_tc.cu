@@ -2,13 +2,16 @@
 //   s_ti = scale <q^h_t, k_i>,  t - W < i <= t      p_ti = softmax_i(s_ti)      o^h_t = sum_i p_ti v^h_i
 // (Sec. "Shared-Key Attention for Lossless Head Compression": one key per token for all heads.)
 //
-// One CTA of 128 threads per (batch, head, 128 queries); thread = query row = tensor-memory lane,
-// so the softmax of a row never leaves its thread.  Per key tile of 128 tokens:
+// One CTA of 256 threads per (batch, head, 128 queries): query row = tensor-memory lane, two
+// threads per row (64 of the 128 key columns each; they exchange one maximum per tile and one sum
+// at the end through shared memory).  Per key tile of 128 tokens:
 //   S = Q K^T        tcgen05.mma, Q and K tiles K-major in shared memory (TMA, 128-byte swizzle),
 //                    accumulator [128 x 128] fp32 in tensor memory
-//   softmax          each thread reads its row of S (tcgen05.ld), keeps a running maximum and sum
-//                    in the log2 domain, rescales its row of O in tensor memory when the maximum
-//                    moved, and writes the probabilities back over S as packed bf16 (tcgen05.st)
+//   softmax          each thread reads its part of a row of S (tcgen05.ld), keeps a reference
+//                    exponent and a sum in the log2 domain, rescales its part of the row of O in
+//                    tensor memory when the reference moved (lazily: only when a tile's maximum
+//                    exceeds it by more than 2^8), and writes the probabilities back over S as
+//                    packed bf16 (tcgen05.st)
 //   O += P V         tcgen05.mma with P as the A operand IN TENSOR MEMORY and the V tile
 //                    (token-major, i.e. N-major B operand) from shared memory
 // Tensor memory: 256 columns (S, overwritten by P, and O), shared memory 96 KiB (Q, one K tile,
@@ -22,11 +25,12 @@
 namespace ddts {
 namespace {
 
-constexpr int kD = 128, kBM = 128, kBN = 128, kThreads = 128;
+constexpr int kD = 128, kBM = 128, kBN = 128, kThreads = 256, kHalf = 64;
 constexpr uint32_t kSlabBytes = 128 * 128;            // [128 rows][64 columns] bf16
 constexpr uint32_t kTileBytes = 2 * kSlabBytes;       // 128 x 128 bf16
 constexpr uint32_t kOffQ = 0, kOffK = kTileBytes, kOffV = 2 * kTileBytes, kOffCtl = 3 * kTileBytes;
-constexpr uint32_t kSmemBytes = kOffCtl + 256 + 1024; // + control block + slack for 1024-byte alignment
+constexpr uint32_t kOffMax = kOffCtl + 256;            // [2][128] floats: the halves' row maxima / sums
+constexpr uint32_t kSmemBytes = kOffMax + 1024 + 1024; // + slack for 1024-byte alignment
 constexpr uint32_t kTmemCols = 256, kColS = 0, kColO = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -79,6 +83,10 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   auto bar = [&](int i) { return base + kOffCtl + 8u * (uint32_t)i; };
 
   const int tid = threadIdx.x, warp = tid >> 5;
+  // thread = (query row, half of the 128 columns): warps 0-3 columns 0-63, warps 4-7 columns 64-127;
+  // a warp reaches the 32 tensor-memory lanes of its number mod 4
+  const int rowl = tid & (kBM - 1), half = tid >> 7, col0 = half * kHalf;
+  float* sMax = reinterpret_cast<float*>(gen + kOffMax);
   const int m0 = blockIdx.x * kBM, h = blockIdx.y, b = blockIdx.z;
   const int T = a.T, W = a.window;
   const long long bh = (long long)b * a.H + h;
@@ -103,7 +111,7 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = ctl->tmem_base;
-  const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes
+  const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's 32 lanes
 
   // what thread 0 has asked for and not yet seen complete (for the clean exit)
   int k_sent = 0, v_sent = 0, q_sent = 0, k_seen = 0, v_seen = 0, q_seen = 0;
@@ -124,9 +132,12 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const uint32_t dk0 = desc_lo_kmajor(base + kOffK), dk1 = desc_lo_kmajor(base + kOffK + kSlabBytes);
   const uint32_t dv = desc_lo_mnmajor(base + kOffV, kSlabBytes);
 
-  const int row = m0 + tid;                 // this thread's query
-  const float sc = a.scale * kLog2e;
-  float m_run = -INFINITY, l_run = 0.f;
+  const int row = m0 + rowl;                // this thread's query
+  const float sc = a.scale * kLog2e;        // > 0 (checked by the host)
+  // Reference exponent of the row (log2 domain).  It follows the running maximum lazily: it moves
+  // only when a tile's maximum exceeds it by more than 8, so probabilities stay below 2^8 and O, l
+  // are rescaled rarely; the final division by l makes the result independent of the reference.
+  float m_ref = -INFINITY, l_run = 0.f;
   bool ok = true;
   int it = 0;
   for (int nt = nt_lo; nt <= nt_hi; ++nt, ++it) {
@@ -159,69 +170,68 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       load_tile(&map_k, kOffK, krow0 + n0 + kBN, BAR_K);
       ++k_sent;
     }
-    float alpha = 1.f;
+    // ---- this thread's 64 columns of its row of S: mask, maximum
+    float sv[kHalf];
+    float mx = -INFINITY;
     if (ok) {
-      // ---- this row of S: scale to the log2 domain, mask, maximum
-      float s[kBN];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t r[32];
-        tmem_ld32(t_row + kColS + 32 * c, r);
+        tmem_ld32(t_row + kColS + col0 + 32 * c, r);
         tmem_ld_wait();
 #pragma unroll
-        for (int e = 0; e < 32; ++e) s[32 * c + e] = __uint_as_float(r[e]) * sc;
+        for (int e = 0; e < 32; ++e) sv[32 * c + e] = __uint_as_float(r[e]);
       }
-      const bool inside = n0 + kBN - 1 <= row && n0 > row - W;
-      float mx = -INFINITY;
-      if (inside) {
+      const int k0 = n0 + col0;
+      if (!(k0 + kHalf - 1 <= row && k0 > row - W)) {
 #pragma unroll
-        for (int e = 0; e < kBN; ++e) mx = fmaxf(mx, s[e]);
-      } else {
-#pragma unroll
-        for (int e = 0; e < kBN; ++e) {
-          const int key = n0 + e;
-          s[e] = (key <= row && key > row - W) ? s[e] : -INFINITY;
-          mx = fmaxf(mx, s[e]);
+        for (int e = 0; e < kHalf; ++e) {
+          const int key = k0 + e;
+          sv[e] = (key <= row && key > row - W) ? sv[e] : -INFINITY;
         }
       }
-      const float m_new = fmaxf(m_run, mx);
-      const float m_use = m_new == -INFINITY ? 0.f : m_new;    // a row that has seen no key yet
-      alpha = ex2f(m_run - m_use);
-      m_run = m_new;
-      float psum = 0.f;
-      uint32_t pk[kBN / 2];
 #pragma unroll
-      for (int e = 0; e < kBN; e += 2) {
-        const float p0 = ex2f(s[e] - m_use), p1 = ex2f(s[e + 1] - m_use);
+      for (int e = 0; e < kHalf; ++e) mx = fmaxf(mx, sv[e]);
+    }
+    sMax[half * kBM + rowl] = mx * sc;          // (-inf stays -inf: sc > 0)
+    tc_fence_before();
+    ok = __syncthreads_and(ok) != 0;            // both halves of every row have read S
+    if (!ok) break;
+    tc_fence_after();
+    {
+      const float m_tile = fmaxf(sMax[rowl], sMax[kBM + rowl]);
+      float alpha = 1.f;
+      if (m_tile > m_ref + 8.f) {               // also the first tile with a visible key
+        alpha = ex2f(m_ref - m_tile);           // 0 when nothing had been seen
+        m_ref = m_tile;
+      }
+      const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
+      float psum = 0.f;
+      uint32_t pk[kHalf / 2];
+#pragma unroll
+      for (int e = 0; e < kHalf; e += 2) {
+        const float p0 = ex2f(fmaf(sv[e], sc, -m_use)), p1 = ex2f(fmaf(sv[e + 1], sc, -m_use));
         psum += p0 + p1;
         pk[e >> 1] = pack_bf16(p0, p1);
       }
       l_run = l_run * alpha + psum;
-      // ---- the previous O += P V must be complete before O is rescaled and P overwritten
+      // the previous O += P V must be complete before O is rescaled and P overwritten
       if (it > 0) ok = sw_wait(bar(BAR_O), ph ^ 1, ctl, a.status);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
       if (ok) {
         if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 2; ++c) {
             uint32_t r[32];
-            tmem_ld32(t_row + kColO + 32 * c, r);
+            tmem_ld32(t_row + kColO + col0 + 32 * c, r);
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-            tmem_st32(t_row + kColO + 32 * c, r);
+            tmem_st32(t_row + kColO + col0 + 32 * c, r);
           }
         }
-        {
-          uint32_t r[32];
-#pragma unroll
-          for (int c = 0; c < 2; ++c) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) r[e] = pk[32 * c + e];
-            tmem_st32(t_row + kColS + 32 * c, r);
-          }
-        }
+        tmem_st32(t_row + kColS + 32 * half, pk);     // keys col0 .. col0+63, two per column
         tmem_st_wait();
       }
     }
@@ -243,28 +253,31 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
   }
 
-  // ---- the last O += P V, then normalise and store this thread's row
+  // ---- the last O += P V, then normalise and store this thread's 64 columns of its row
   if (ok && it > 0) ok = sw_wait(bar(BAR_O), (it - 1) & 1, ctl, a.status);
   ok = __all_sync(0xffffffffu, ok);
+  sMax[half * kBM + rowl] = l_run;
+  __syncthreads();
   tc_fence_after();
   if (ok && it > 0) {
-    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-    __nv_bfloat16* orow = (__nv_bfloat16*)a.o + ((long long)qrow0 + tid) * kD;
+    const float l = sMax[rowl] + sMax[kBM + rowl];
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    __nv_bfloat16* orow = (__nv_bfloat16*)a.o + ((long long)qrow0 + rowl) * kD + col0;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 2; ++c) {
       uint32_t r[32];
-      tmem_ld32(t_row + kColO + 32 * c, r);
+      tmem_ld32(t_row + kColO + col0 + 32 * c, r);
       tmem_ld_wait();
       if (row < T) {
 #pragma unroll
-      for (int e = 0; e < 32; e += 8) {
-        uint4 w;
-        w.x = pack_bf16(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
-        w.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-        w.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-        w.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-        *reinterpret_cast<uint4*>(orow + 32 * c + e) = w;
-      }
+        for (int e = 0; e < 32; e += 8) {
+          uint4 w;
+          w.x = pack_bf16(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
+          w.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+          w.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+          w.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+          *reinterpret_cast<uint4*>(orow + 32 * c + e) = w;
+        }
       }
     }
   }
