@@ -2,45 +2,55 @@
 //   s_ti = scale <q^h_t, k_i>,  t - W < i <= t      p_ti = softmax_i(s_ti)      o^h_t = sum_i p_ti v^h_i
 // (Sec. "Shared-Key Attention for Lossless Head Compression": one key per token for all heads.)
 //
-// One CTA of 256 threads per (batch, head, 128 queries): query row = tensor-memory lane, two
-// threads per row (64 of the 128 key columns each; they exchange one maximum per tile and one sum
-// at the end through shared memory).  Per key tile of 128 tokens:
-//   S = Q K^T        tcgen05.mma, Q and K tiles K-major in shared memory (TMA, 128-byte swizzle),
-//                    accumulator [128 x 128] fp32 in tensor memory
+// One CTA per (batch, head, 128 queries): 8 softmax warps, one warp that issues the contractions
+// and one that issues the TMA loads.  Query row =
+// tensor-memory lane; two softmax threads per row (32 of a tile's 64 key columns each; they
+// exchange one maximum per tile and one sum at the end through shared memory).  Per key tile of
+// 64 tokens:
+//   S = Q K^T        tcgen05.mma, Q tile and K tile K-major in shared memory (TMA, 128-byte
+//                    swizzle), accumulator [128 x 64] fp32 in tensor memory, TWO buffers: the
+//                    scores of tile i+1 are computed while the softmax of tile i runs
 //   softmax          each thread reads its part of a row of S (tcgen05.ld), keeps a reference
 //                    exponent and a sum in the log2 domain, rescales its part of the row of O in
 //                    tensor memory when the reference moved (lazily: only when a tile's maximum
 //                    exceeds it by more than 2^8), and writes the probabilities back over S as
 //                    packed bf16 (tcgen05.st)
-//   O += P V         tcgen05.mma with P as the A operand IN TENSOR MEMORY and the V tile
-//                    (token-major, i.e. N-major B operand) from shared memory
-// Tensor memory: 256 columns (S, overwritten by P, and O), shared memory 96 KiB (Q, one K tile,
-// one V tile): two CTAs per SM, one CTA's softmax overlapping the other's contractions.  The K
-// tile of the next step is requested as soon as S is complete, the V tile as soon as the previous
-// O += P V is complete.  Only key tiles that touch the 128 queries' windows are visited.
-// Every wait is bounded; a wait that runs out ends the kernel cleanly (copies and contractions in
-// flight are waited for, tensor memory is freed) and raises RODIMUS_ERR_TIMEOUT in the status word.
+//   O += P V         tcgen05.mma, A = P from tensor memory, B = the V tile (token-major, i.e.
+//                    N-major) from shared memory
+// Issuing a tcgen05.mma or a TMA load costs its thread about a hundred cycles here, which is why
+// two threads of two warps share that work and the softmax warps do none of it.  Tensor memory: 256 columns
+// (S twice 64, O 128); shared memory 96 KiB (Q 32, two K tiles, two V tiles; a tile is requested
+// two tiles ahead, as soon as the contraction that read its slot is complete): two CTAs per SM.  Only key tiles that
+// touch the 128 queries' windows are visited.  Every wait is bounded; a wait that runs out ends
+// the kernel cleanly (copies and contractions in flight are waited for, tensor memory is freed)
+// and raises RODIMUS_ERR_TIMEOUT in the status word.  No hardware barrier is used inside the
+// loop (a role that gave up would leave the others at it).
 #include "ddts_tc_ptx.cuh"
 
 namespace ddts {
 namespace {
 
-constexpr int kD = 128, kBM = 128, kBN = 128, kThreads = 256, kHalf = 64;
-constexpr uint32_t kSlabBytes = 128 * 128;            // [128 rows][64 columns] bf16
-constexpr uint32_t kTileBytes = 2 * kSlabBytes;       // 128 x 128 bf16
-constexpr uint32_t kOffQ = 0, kOffK = kTileBytes, kOffV = 2 * kTileBytes, kOffCtl = 3 * kTileBytes;
-constexpr uint32_t kOffMax = kOffCtl + 256;            // [2][128] floats: the halves' row maxima / sums
-constexpr uint32_t kSmemBytes = kOffMax + 1024 + 1024; // + slack for 1024-byte alignment
+constexpr int kD = 128, kBM = 128, kBN = 64, kHalf = kBN / 2;
+constexpr int kSoftmaxWarps = 8, kIssuerWarp = 8, kProducerWarp = 9, kThreads = 32 * (kSoftmaxWarps + 2);
+constexpr uint32_t kQSlabBytes = kBM * 128;           // [128 rows][64 columns] bf16
+constexpr uint32_t kSlabBytes = kBN * 128;            // [64 rows][64 columns] bf16
+constexpr uint32_t kTileBytes = 2 * kSlabBytes;       // 64 x 128 bf16
+constexpr uint32_t kOffQ = 0, kOffK = 2 * kQSlabBytes, kOffV = kOffK + 2 * kTileBytes;
+constexpr uint32_t kOffCtl = kOffV + 2 * kTileBytes;
+constexpr uint32_t kOffMax = kOffCtl + 256;            // [2][2][128] floats: the halves' row maxima (by buffer) / sums
+constexpr uint32_t kSmemBytes = kOffMax + 2048 + 1024; // + slack for 1024-byte alignment
 constexpr uint32_t kTmemCols = 256, kColS = 0, kColO = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 
-enum { BAR_Q = 0, BAR_K, BAR_V, BAR_S, BAR_O, BAR_DRAIN, kNumBars };
+enum { BAR_Q = 0, BAR_K0, BAR_K1, BAR_V0, BAR_V1, BAR_S0, BAR_S1, BAR_P0, BAR_P1, BAR_O0, BAR_O1, BAR_PAIR0,
+       BAR_DRAIN = BAR_PAIR0 + 4, kNumBars };
 
 struct SwCtl {
   uint64_t bar[kNumBars];
   uint32_t tmem_base;
   int abort;
   long long limit;
+  int k_sent, v_sent, k_seen, v_seen;   // loads asked for / seen complete (for the clean exit)
 };
 
 struct SwTcArgs {
@@ -81,28 +91,31 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   unsigned char* gen = smem_raw + (base - smem_u32(smem_raw));
   volatile SwCtl* ctl = reinterpret_cast<volatile SwCtl*>(gen + kOffCtl);
   auto bar = [&](int i) { return base + kOffCtl + 8u * (uint32_t)i; };
-
-  const int tid = threadIdx.x, warp = tid >> 5;
-  // thread = (query row, half of the 128 columns): warps 0-3 columns 0-63, warps 4-7 columns 64-127;
-  // a warp reaches the 32 tensor-memory lanes of its number mod 4
-  const int rowl = tid & (kBM - 1), half = tid >> 7, col0 = half * kHalf;
   float* sMax = reinterpret_cast<float*>(gen + kOffMax);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int m0 = blockIdx.x * kBM, h = blockIdx.y, b = blockIdx.z;
   const int T = a.T, W = a.window;
   const long long bh = (long long)b * a.H + h;
-  const int qrow0 = (int)(bh * T) + m0;          // row of the [B*H*T, 128] views of q, v, o
+  const long long qrow0 = bh * T + m0;           // row of the [B*H*T, 128] views of q, o
   const int krow0 = b * T;                       // row of the [B*T, 128] view of k
-  const int vrow0 = (int)(bh * T);
+  const int vrow0 = (int)(bh * T);               // row of the [B*H*T, 128] view of v
   const int first_key = max(0, m0 - W + 1);
   const int nt_lo = first_key / kBN, nt_hi = min(m0 + kBM - 1, T - 1) / kBN;
+  const int n_tiles = nt_hi - nt_lo + 1;
 
   if (tid == 0) {
     ctl->abort = 0;
     ctl->limit = a.limit;
-    for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), 1);
+    ctl->k_sent = ctl->v_sent = ctl->k_seen = ctl->v_seen = 0;
+    for (int i = 0; i < kNumBars; ++i) {
+      const bool per_warp = i == BAR_P0 || i == BAR_P1;
+      const bool pair = i >= BAR_PAIR0 && i < BAR_PAIR0 + 4;
+      mbar_init(bar(i), per_warp ? kSoftmaxWarps : (pair ? 2 : 1));
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 0) {
+  if (warp == kIssuerWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(base + kOffCtl + (uint32_t)offsetof(SwCtl, tmem_base)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -111,95 +124,144 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = ctl->tmem_base;
-  const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's 32 lanes
 
-  // what thread 0 has asked for and not yet seen complete (for the clean exit)
-  int k_sent = 0, v_sent = 0, q_sent = 0, k_seen = 0, v_seen = 0, q_seen = 0;
-  auto load_tile = [&](const CUtensorMap* map, uint32_t dst, int row, int which) {
-    mbar_expect_tx(bar(which), kTileBytes);
-    tma_load_2d(base + dst, map, 0, row, bar(which));
-    tma_load_2d(base + dst + kSlabBytes, map, 64, row, bar(which));
-  };
-  if (tid == 0) {
-    load_tile(&map_q, kOffQ, qrow0, BAR_Q); q_sent = 1;
-    load_tile(&map_k, kOffK, krow0 + nt_lo * kBN, BAR_K); k_sent = 1;
-    load_tile(&map_v, kOffV, vrow0 + nt_lo * kBN, BAR_V); v_sent = 1;
-  }
-
-  constexpr uint32_t kIdescS = make_idesc(kBM, kBN, 0, 0);   // S = Q K^T, both K-major
-  constexpr uint32_t kIdescO = make_idesc(kBM, kD, 0, 1);    // O += P V, A in tensor memory, B N-major
-  const uint32_t dq0 = desc_lo_kmajor(base + kOffQ), dq1 = desc_lo_kmajor(base + kOffQ + kSlabBytes);
-  const uint32_t dk0 = desc_lo_kmajor(base + kOffK), dk1 = desc_lo_kmajor(base + kOffK + kSlabBytes);
-  const uint32_t dv = desc_lo_mnmajor(base + kOffV, kSlabBytes);
-
-  const int row = m0 + rowl;                // this thread's query
-  const float sc = a.scale * kLog2e;        // > 0 (checked by the host)
-  // Reference exponent of the row (log2 domain).  It follows the running maximum lazily: it moves
-  // only when a tile's maximum exceeds it by more than 8, so probabilities stay below 2^8 and O, l
-  // are rescaled rarely; the final division by l makes the result independent of the reference.
-  float m_ref = -INFINITY, l_run = 0.f;
-  bool ok = true;
-  int it = 0;
-  for (int nt = nt_lo; nt <= nt_hi; ++nt, ++it) {
-    const uint32_t ph = it & 1;
-    const int n0 = nt * kBN;
-    if (tid == 0) {
-      if (it == 0) { ok = sw_wait(bar(BAR_Q), 0, ctl, a.status); q_seen = ok; }
-      if (ok) { ok = sw_wait(bar(BAR_K), ph, ctl, a.status); k_seen += ok; }
-      if (ok) {
+  if (warp == kProducerWarp) {
+    // =========================== producer warp: every TMA load ================================
+    if (lane == 0) {
+      int k_sent = 0, v_sent = 0;
+      auto load = [&](const CUtensorMap* map, uint32_t dst, uint32_t slab, int row, int which, uint32_t bytes) {
+        mbar_expect_tx(bar(which), bytes);
+        tma_load_2d(base + dst, map, 0, row, bar(which));
+        tma_load_2d(base + dst + slab, map, 64, row, bar(which));
+      };
+      auto fill_k = [&](int j) {
+        load(&map_k, kOffK + (j & 1) * kTileBytes, kSlabBytes, krow0 + (nt_lo + j) * kBN, BAR_K0 + (j & 1), kTileBytes);
+        ++k_sent;
+      };
+      auto fill_v = [&](int j) {
+        load(&map_v, kOffV + (j & 1) * kTileBytes, kSlabBytes, vrow0 + (nt_lo + j) * kBN, BAR_V0 + (j & 1), kTileBytes);
+        ++v_sent;
+      };
+      load(&map_q, kOffQ, kQSlabBytes, (int)qrow0, BAR_Q, 2 * kQSlabBytes);
+      fill_k(0);
+      fill_v(0);
+      if (n_tiles > 1) { fill_k(1); fill_v(1); }
+      bool ok = true;
+      // a slot is refilled as soon as the contraction that read it is complete: K two tiles ahead
+      // of the scores that will read it, V two tiles ahead of its O += P V
+      for (int it = 0; ok && it + 2 < n_tiles; ++it) {
+        if (!(ok = sw_wait(bar(BAR_S0 + (it & 1)), (it >> 1) & 1, ctl, a.status))) break;
+        fill_k(it + 2);
+        if (!(ok = sw_wait(bar(BAR_O0 + (it & 1)), (it >> 1) & 1, ctl, a.status))) break;
+        fill_v(it + 2);
+      }
+      ctl->k_sent = k_sent;
+      ctl->v_sent = v_sent;
+    }
+    __syncwarp();
+  } else if (warp == kIssuerWarp) {
+    // =========================== issuing warp: every contraction ==============================
+    if (lane == 0) {
+      constexpr uint32_t kIdescS = make_idesc(kBM, kBN, 0, 0);   // S = Q K^T, both K-major
+      constexpr uint32_t kIdescO = make_idesc(kBM, kD, 0, 1);    // O += P V: A in tensor memory, B N-major
+      int k_seen = 0, v_seen = 0;
+      auto issue_s = [&](int j) {   // scores of tile j into buffer j & 1
+        const uint32_t dq0 = desc_lo_kmajor(base + kOffQ), dq1 = desc_lo_kmajor(base + kOffQ + kQSlabBytes);
+        const uint32_t ks = base + kOffK + (j & 1) * kTileBytes;
+        const uint32_t dk0 = desc_lo_kmajor(ks), dk1 = desc_lo_kmajor(ks + kSlabBytes);
+        const uint32_t d = tmem + kColS + (j & 1) * kBN;
+        umma_bf16_lo<false>(d, dq0, dk0, kIdescS);
+#pragma unroll
+        for (int kk = 1; kk < 4; ++kk) umma_bf16_lo<true>(d, dq0 + 2 * kk, dk0 + 2 * kk, kIdescS);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) umma_bf16_lo<true>(d, dq1 + 2 * kk, dk1 + 2 * kk, kIdescS);
+        umma_commit(bar(BAR_S0 + (j & 1)));
+      };
+      bool ok = sw_wait(bar(BAR_Q), 0, ctl, a.status);
+      if (ok) { ok = sw_wait(bar(BAR_K0), 0, ctl, a.status); k_seen += ok; }
+      if (ok) { tc_fence_after(); issue_s(0); }
+      for (int it = 0; ok && it < n_tiles; ++it) {
+        const int sb = it & 1;
+        const uint32_t ph = (it >> 1) & 1;
+        if (it + 1 < n_tiles) {            // the next tile's scores, while this tile's softmax runs
+          ok = sw_wait(bar(BAR_K0 + (sb ^ 1)), ((it + 1) >> 1) & 1, ctl, a.status);
+          k_seen += ok;
+          if (!ok) break;
+          tc_fence_after();
+          issue_s(it + 1);
+        }
+        if (!(ok = sw_wait(bar(BAR_P0 + sb), ph, ctl, a.status))) break;   // probabilities in place
+        ok = sw_wait(bar(BAR_V0 + sb), ph, ctl, a.status);
+        v_seen += ok;
+        if (!ok) break;
         tc_fence_after();
+        const uint32_t dv = desc_lo_mnmajor(base + kOffV + sb * kTileBytes, kSlabBytes);
+        const uint32_t pa = tmem + kColS + sb * kBN;
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
-          if (kk == 0) umma_bf16_lo<false>(tmem + kColS, dq0, dk0, kIdescS);
-          else umma_bf16_lo<true>(tmem + kColS, dq0 + 2 * kk, dk0 + 2 * kk, kIdescS);
+          if (kk == 0 && it == 0) umma_bf16_atmem<false>(tmem + kColO, pa, dv, kIdescO);
+          else umma_bf16_atmem<true>(tmem + kColO, pa + 8 * kk, dv + 128 * kk, kIdescO);
         }
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) umma_bf16_lo<true>(tmem + kColS, dq1 + 2 * kk, dk1 + 2 * kk, kIdescS);
-        umma_commit(bar(BAR_S));
-        // the previous O += P V sits before this S in the pipe: once it is done, the V tile is free
-        if (it > 0) {
-          ok = sw_wait(bar(BAR_O), ph ^ 1, ctl, a.status);
-          if (ok) { load_tile(&map_v, kOffV, vrow0 + n0, BAR_V); ++v_sent; }
-        }
+        umma_commit(bar(BAR_O0 + sb));   // (two barriers, by tile parity: a waiter is never two phases behind)
       }
+      ctl->k_seen = k_seen;
+      ctl->v_seen = v_seen;
     }
-    if (ok) ok = sw_wait(bar(BAR_S), ph, ctl, a.status);
-    ok = __all_sync(0xffffffffu, ok);     // the tensor-memory accesses below need the whole warp
-    tc_fence_after();
-    if (tid == 0 && ok && nt < nt_hi) {       // S is complete: the K tile is free
-      load_tile(&map_k, kOffK, krow0 + n0 + kBN, BAR_K);
-      ++k_sent;
-    }
-    // ---- this thread's 64 columns of its row of S: mask, maximum
-    float sv[kHalf];
-    float mx = -INFINITY;
-    if (ok) {
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
+    __syncwarp();
+  } else {
+    // =========================== softmax warps =================================================
+    // thread = (query row, half of a tile's 64 key columns): warps 0-3 the first half, warps 4-7
+    // the second; a warp reaches the 32 tensor-memory lanes of its number mod 4
+    const int rowl = tid & (kBM - 1), half = tid >> 7, col0 = half * kHalf;
+    const int row = m0 + rowl;
+    const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t pair_bar = bar(BAR_PAIR0 + (warp & 3));   // this warp and the one with the other half
+    const float sc = a.scale * kLog2e;        // > 0 (checked by the host)
+    // Reference exponent of the row (log2 domain).  It follows the running maximum lazily: it
+    // moves only when a tile's maximum exceeds it by more than 8, so probabilities stay below 2^8
+    // and O, l are rescaled rarely; the final division by l makes the result independent of it.
+    float m_ref = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    int it = 0;
+    for (; it < n_tiles; ++it) {
+      const int sb = it & 1;
+      const uint32_t ph = (it >> 1) & 1;
+      const int n0 = (nt_lo + it) * kBN;
+      ok = sw_wait(bar(BAR_S0 + sb), ph, ctl, a.status);
+      ok = __all_sync(0xffffffffu, ok);     // the tensor-memory accesses below need the whole warp
+      if (!ok) break;
+      tc_fence_after();
+      // ---- this thread's 32 columns of its row of S: mask, maximum
+      float sv[kHalf];
+      float mx = -INFINITY;
+      {
         uint32_t r[32];
-        tmem_ld32(t_row + kColS + col0 + 32 * c, r);
+        tmem_ld32(t_row + kColS + sb * kBN + col0, r);
         tmem_ld_wait();
+        const int k0 = n0 + col0;
+        if (k0 + kHalf - 1 <= row && k0 > row - W) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) sv[32 * c + e] = __uint_as_float(r[e]);
-      }
-      const int k0 = n0 + col0;
-      if (!(k0 + kHalf - 1 <= row && k0 > row - W)) {
+          for (int e = 0; e < kHalf; ++e) sv[e] = __uint_as_float(r[e]);
+        } else {
 #pragma unroll
-        for (int e = 0; e < kHalf; ++e) {
-          const int key = k0 + e;
-          sv[e] = (key <= row && key > row - W) ? sv[e] : -INFINITY;
+          for (int e = 0; e < kHalf; ++e) {
+            const int key = k0 + e;
+            sv[e] = (key <= row && key > row - W) ? __uint_as_float(r[e]) : -INFINITY;
+          }
         }
-      }
 #pragma unroll
-      for (int e = 0; e < kHalf; ++e) mx = fmaxf(mx, sv[e]);
-    }
-    sMax[half * kBM + rowl] = mx * sc;          // (-inf stays -inf: sc > 0)
-    tc_fence_before();
-    ok = __syncthreads_and(ok) != 0;            // both halves of every row have read S
-    if (!ok) break;
-    tc_fence_after();
-    {
-      const float m_tile = fmaxf(sMax[rowl], sMax[kBM + rowl]);
+        for (int e = 0; e < kHalf; ++e) mx = fmaxf(mx, sv[e]);
+      }
+      sMax[(sb * 2 + half) * kBM + rowl] = mx * sc;   // (-inf stays -inf: sc > 0)
+      // both threads of a row have read S (the probabilities overwrite it) and left their maximum
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pair_bar);
+      ok = sw_wait(pair_bar, it & 1, ctl, a.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const float m_tile = fmaxf(sMax[(sb * 2) * kBM + rowl], sMax[(sb * 2 + 1) * kBM + rowl]);
       float alpha = 1.f;
       if (m_tile > m_ref + 8.f) {               // also the first tile with a visible key
         alpha = ex2f(m_ref - m_tile);           // 0 when nothing had been seen
@@ -215,84 +277,75 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         pk[e >> 1] = pack_bf16(p0, p1);
       }
       l_run = l_run * alpha + psum;
-      // the previous O += P V must be complete before O is rescaled and P overwritten
-      if (it > 0) ok = sw_wait(bar(BAR_O), ph ^ 1, ctl, a.status);
-      ok = __all_sync(0xffffffffu, ok);
-      tc_fence_after();
-      if (ok) {
-        if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+      // the previous O += P V must be complete before O is rescaled
+      if (it > 0) {
+        ok = sw_wait(bar(BAR_O0 + ((it - 1) & 1)), ((it - 1) >> 1) & 1, ctl, a.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
             uint32_t r[32];
-            tmem_ld32(t_row + kColO + col0 + 32 * c, r);
+            tmem_ld32(t_row + kColO + 64 * half + 32 * c, r);
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-            tmem_st32(t_row + kColO + col0 + 32 * c, r);
+            tmem_st32(t_row + kColO + 64 * half + 32 * c, r);
           }
         }
-        tmem_st32(t_row + kColS + 32 * half, pk);     // keys col0 .. col0+63, two per column
-        tmem_st_wait();
       }
+      tmem_st16(t_row + kColS + sb * kBN + 16 * half, pk);     // keys col0 .. col0+31, two per column
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_P0 + sb));
     }
-    tc_fence_before();
-    ok = __syncthreads_and(ok) != 0;      // every row's P is in place (or everyone gives up)
-    if (!ok) break;
-    if (tid == 0) {
+    // ---- the last O += P V, then normalise and store this thread's 64 columns of its row
+    if (ok) ok = sw_wait(bar(BAR_O0 + ((n_tiles - 1) & 1)), ((n_tiles - 1) >> 1) & 1, ctl, a.status);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
       tc_fence_after();
-      ok = sw_wait(bar(BAR_V), ph, ctl, a.status);
-      v_seen += ok;
-      if (ok) {
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          if (kk == 0 && it == 0) umma_bf16_atmem<false>(tmem + kColO, tmem + kColS, dv, kIdescO);
-          else umma_bf16_atmem<true>(tmem + kColO, tmem + kColS + 8 * kk, dv + 128 * kk, kIdescO);
-        }
-        umma_commit(bar(BAR_O));
-      }
+      sMax[half * kBM + rowl] = l_run;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pair_bar);
+      ok = sw_wait(pair_bar, n_tiles & 1, ctl, a.status);
+      ok = __all_sync(0xffffffffu, ok);
     }
-  }
-
-  // ---- the last O += P V, then normalise and store this thread's 64 columns of its row
-  if (ok && it > 0) ok = sw_wait(bar(BAR_O), (it - 1) & 1, ctl, a.status);
-  ok = __all_sync(0xffffffffu, ok);
-  sMax[half * kBM + rowl] = l_run;
-  __syncthreads();
-  tc_fence_after();
-  if (ok && it > 0) {
-    const float l = sMax[rowl] + sMax[kBM + rowl];
-    const float inv = l > 0.f ? 1.f / l : 0.f;
-    __nv_bfloat16* orow = (__nv_bfloat16*)a.o + ((long long)qrow0 + rowl) * kD + col0;
+    if (ok) {
+      const float l = sMax[rowl] + sMax[kBM + rowl];
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      __nv_bfloat16* orow = (__nv_bfloat16*)a.o + (qrow0 + rowl) * kD + 64 * half;
 #pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      uint32_t r[32];
-      tmem_ld32(t_row + kColO + col0 + 32 * c, r);
-      tmem_ld_wait();
-      if (row < T) {
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_row + kColO + 64 * half + 32 * c, r);
+        tmem_ld_wait();
+        if (row < T) {
 #pragma unroll
-        for (int e = 0; e < 32; e += 8) {
-          uint4 w;
-          w.x = pack_bf16(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
-          w.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-          w.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-          w.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-          *reinterpret_cast<uint4*>(orow + 32 * c + e) = w;
+          for (int e = 0; e < 32; e += 8) {
+            uint4 w;
+            w.x = pack_bf16(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + 32 * c + e) = w;
+          }
         }
       }
     }
-  }
-
-  // ---- clean exit: nothing may still be writing this CTA's shared or tensor memory
-  if (tid == 0 && ctl->abort) {
-    if (q_sent && !q_seen) mbar_drain(bar(BAR_Q), 0);
-    while (k_seen < k_sent) { mbar_drain(bar(BAR_K), k_seen & 1); ++k_seen; }
-    while (v_seen < v_sent) { mbar_drain(bar(BAR_V), v_seen & 1); ++v_seen; }
-    umma_commit(bar(BAR_DRAIN));          // completes when every contraction issued so far has
-    mbar_drain(bar(BAR_DRAIN), 0);
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0)
+  if (tid == 0 && ctl->abort) {   // clean exit: nothing may still be writing this CTA's shared or tensor memory
+    mbar_drain(bar(BAR_Q), 0);
+    for (int j = ctl->k_seen; j < ctl->k_sent; ++j) mbar_drain(bar(BAR_K0 + (j & 1)), (j >> 1) & 1);
+    for (int j = ctl->v_seen; j < ctl->v_sent; ++j) mbar_drain(bar(BAR_V0 + (j & 1)), (j >> 1) & 1);
+    umma_commit(bar(BAR_DRAIN));      // completes when every contraction issued so far has
+    mbar_drain(bar(BAR_DRAIN), 0);
+  }
+  __syncthreads();
+  if (warp == kIssuerWarp)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
@@ -314,14 +367,14 @@ EncodeTiledFn sw_encode_fn() {
   return fn;
 }
 
-// [rows, 128] bf16 row-major; box = 128 rows x 64 columns (128 bytes), 128-byte swizzle; rows past
-// the end of the tensor read as zeros
-bool sw_make_map(CUtensorMap* m, const void* ptr, uint64_t rows) {
+// [rows, 128] bf16 row-major; box = box_rows rows x 64 columns (128 bytes), 128-byte swizzle; rows
+// past the end of the tensor read as zeros
+bool sw_make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint32_t box_rows) {
   EncodeTiledFn fn = sw_encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)kD, rows};
   const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
-  const cuuint32_t box[2] = {64u, 128u};
+  const cuuint32_t box[2] = {64u, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -343,7 +396,8 @@ cudaError_t launch_swska_tc(const rodimus_swska_fwd_params& p, int* n_launches) 
   const uint64_t rows_q = (uint64_t)p.B * p.H * p.T, rows_k = (uint64_t)p.B * p.T;
   SwMapCache& c = t_sw_maps;
   if (c.q != p.q || c.k != p.k || c.v != p.v || c.rows_q != rows_q || c.rows_k != rows_k) {
-    if (!sw_make_map(&c.mq, p.q, rows_q) || !sw_make_map(&c.mk, p.k, rows_k) || !sw_make_map(&c.mv, p.v, rows_q)) {
+    if (!sw_make_map(&c.mq, p.q, rows_q, kBM) || !sw_make_map(&c.mk, p.k, rows_k, kBN) ||
+        !sw_make_map(&c.mv, p.v, rows_q, kBN)) {
       c.q = nullptr;
       return cudaErrorInvalidValue;
     }
