@@ -277,13 +277,13 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         pk[e >> 1] = pack_bf16(p0, p1);
       }
       l_run = l_run * alpha + psum;
-      // the previous O += P V must be complete before O is rescaled
-      if (it > 0) {
+      // rescaling O (rare) needs the previous O += P V complete; writing P does not
+      if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
         ok = sw_wait(bar(BAR_O0 + ((it - 1) & 1)), ((it - 1) >> 1) & 1, ctl, a.status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+        {
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
             uint32_t r[32];
