@@ -322,7 +322,7 @@ def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sf
         nseq = B if cu is None else cu.numel() - 1
         o = torch.empty((B, H, T, dv), dtype=tdt, device=device)
         sT = torch.empty((nseq, H, dk, dv), dtype=torch.float32, device=device)
-        # variants of the same workload (the §8(f) rows that are built): "block" adds the value
+        # variants of the same workload: "block" adds the value
         # gate and the feed-through (seeded, +2 tensors of v's shape read per call); "shared" keeps
         # one q,k,x,y per token for all heads (head 0's), the layout the paper writes the block in
         kw = {}
