@@ -94,7 +94,8 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   float* sMax = reinterpret_cast<float*>(gen + kOffMax);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int m0 = blockIdx.x * kBM, h = blockIdx.y, b = blockIdx.z;
+  // query tiles late in the sequence see the most keys: they are started first, the short ones fill the tail
+  const int m0 = (int)(gridDim.x - 1 - blockIdx.x) * kBM, h = blockIdx.y, b = blockIdx.z;
   const int T = a.T, W = a.window;
   const long long bh = (long long)b * a.H + h;
   const long long qrow0 = bh * T + m0;           // row of the [B*H*T, 128] views of q, o
