@@ -250,8 +250,14 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             sv[e] = (key <= row && key > row - W) ? __uint_as_float(r[e]) : -INFINITY;
           }
         }
+        // maximum as a tree: four independent chains instead of one of 32 dependent steps
+        float m4[4] = {sv[0], sv[1], sv[2], sv[3]};
 #pragma unroll
-        for (int e = 0; e < kHalf; ++e) mx = fmaxf(mx, sv[e]);
+        for (int e = 4; e < kHalf; e += 4) {
+          m4[0] = fmaxf(m4[0], sv[e]); m4[1] = fmaxf(m4[1], sv[e + 1]);
+          m4[2] = fmaxf(m4[2], sv[e + 2]); m4[3] = fmaxf(m4[3], sv[e + 3]);
+        }
+        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       }
       sMax[(sb * 2 + half) * kBM + rowl] = mx * sc;   // (-inf stays -inf: sc > 0)
       // both threads of a row have read S (the probabilities overwrite it) and left their maximum
@@ -269,15 +275,15 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         m_ref = m_tile;
       }
       const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
-      float psum = 0.f;
+      float ps[4] = {0.f, 0.f, 0.f, 0.f};     // four partial sums: no chain of 16 dependent additions
       uint32_t pk[kHalf / 2];
 #pragma unroll
       for (int e = 0; e < kHalf; e += 2) {
         const float p0 = ex2f(fmaf(sv[e], sc, -m_use)), p1 = ex2f(fmaf(sv[e + 1], sc, -m_use));
-        psum += p0 + p1;
+        ps[(e >> 1) & 3] += p0 + p1;
         pk[e >> 1] = pack_bf16(p0, p1);
       }
-      l_run = l_run * alpha + psum;
+      l_run = l_run * alpha + ((ps[0] + ps[1]) + (ps[2] + ps[3]));
       // rescaling O (rare) needs the previous O += P V complete; writing P does not
       if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
         ok = sw_wait(bar(BAR_O0 + ((it - 1) & 1)), ((it - 1) >> 1) & 1, ctl, a.status);
