@@ -130,3 +130,14 @@ def test_bwd_config1_shape_sampled_heads():
         for a, r in PAIRS:
             assert rel_err(got[a][sl], ref[r]) <= TOL_BF16, (a, b, h)
         assert rel_err(got["d_s0"][sl], ref["ds0"]) <= TOL_BF16
+
+
+def test_bwd_long_sequence_and_many_packed_sequences():
+    # 1000 steps (63 chunks): the suffix sums run over the whole sequence in 16 time segments
+    p = wl.make_prefill(701, 1, 2, 1000, 128, 256, "bf16", s0_std=0.1, name="bwd_long")
+    _check(p, 702, True)
+    # 40 packed sequences of mixed lengths, several of them shorter than a chunk
+    lens = list(np.random.default_rng(703).integers(0, 90, 40))
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    p = wl.make_prefill(704, 1, 2, int(cu[-1]), 128, 256, "bf16", s0_std=0.1, cu_seqlens=cu, name="bwd_many")
+    _check(p, 705, True)

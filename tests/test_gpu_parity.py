@@ -716,6 +716,18 @@ def test_value_decay_prefill(dtype, dk, dv, with_gate):
     assert rel_err(host(o), ro) <= _tol(dtype) and rel_err(host(sT), rs) <= TOL_F32
 
 
+def test_value_decay_with_shared_gates():
+    """The value-side decay together with the one-set-per-token layout (both go to the fp32 kernel)."""
+    pq, pv = _shared_inputs(821, 2, 3, 75, 64, 64, "f32")
+    beta = wl.make_value_decay(822, pv.v.shape, "f32")
+    dq_ = {n: dev(getattr(pq, n), "f32") for n in ("q", "k", "x", "y")}
+    import torch
+    o, sT = rd.ddts_fwd(dq_["q"], dq_["k"], dq_["x"], dq_["y"], dev(pv.v, "f32"),
+                        torch.from_numpy(pv.s0).cuda(), value_decay=dev(beta, "f32"))
+    ro, rs = orc.ref_fwd(pq.q, pq.k, pq.x, pq.y, pv.v, s0=pv.s0, shared_gates=True, value_decay=beta)
+    assert rel_err(host(o), ro) <= TOL_F32 and rel_err(host(sT), rs) <= TOL_F32
+
+
 def test_value_decay_packed_sequences_and_decode_steps():
     import torch
     lens = [33, 0, 1, 70]

@@ -30,6 +30,8 @@ def _run(q, k, v, window, scale, dtype):
     (1, 2, 200, 1),        # every token sees only itself
     (1, 2, 260, 1000),     # window longer than the sequence: plain causal attention
     (1, 1, 300, 65),       # window one past a tile: three tiles touch a query tile
+    (3, 5, 129, 129),      # one row past a query tile, odd batch and head counts
+    (1, 2, 513, 200),      # five query tiles, window of three key tiles and a bit
 ])
 def test_swska_matches_oracle(dtype, B, H, T, window):
     q, k, v = wl.make_swska(900 + T, B, H, T, 128, dtype)
