@@ -456,7 +456,7 @@ def measure(workload, p, steps, warmup, world, rank, local, peaks, peak_kind, sf
                        "datasheet_peak": DATASHEET["hbm_gbs"],
                        "algorithmic_bytes_per_launch": int(alg_bytes),
                        "bound_times": bounds,
-                       "traffic": None if variant else load_traffic(kernel, workload)}
+                       "traffic": load_traffic(kernel, f"{workload}_{variant}" if variant else workload)}
     if variant:
         rec["config"] = dict(rec["config"], variant={
             "block": "value gate beta_hat and feed-through d*x' fused (Eq. beta_def, Eq. rodimus_recurrent_form)",
@@ -520,7 +520,7 @@ def measure_swska(steps, warmup, local, peaks, peak_kind, B=4, H=16, T=2048, d=1
                      "frac": achieved / peaks["bf16_tflops"], "algorithmic_flops_per_launch": flops,
                      "bound_times": {"tensor_us": flops / (peaks["bf16_tflops"] * 1e12) * 1e6,
                                      "hbm_us": alg_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6},
-                     "traffic": None},
+                     "traffic": load_traffic("swska_fwd_tc_kernel", "layer")},
     }
 
 
