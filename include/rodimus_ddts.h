@@ -231,7 +231,9 @@ int rodimus_ddts_bwd(const rodimus_ddts_bwd_params *p);
  * sizes: RODIMUS_ERR_UNSUPPORTED); window >= 1 (the paper uses half the training context); dense
  * batches only.  dtype BF16 runs on the tcgen05 tensor cores with a running softmax (cost
  * O(T * window), nothing of size T x window is stored); dtype F32 is a plain fp32 validation
- * kernel.  o must not overlap an input.  `workspace` is optional: given (>= 256 bytes, 256-byte
+ * kernel.  Inputs must be finite (a tile may span the rows of two heads; what lies outside a
+ * query's window is weighted by zero, which a NaN or infinity would not survive).  o must not
+ * overlap an input.  `workspace` is optional: given (>= 256 bytes, 256-byte
  * aligned), its first word is the status rodimus_ddts_device_status reads (RODIMUS_ERR_TIMEOUT
  * if a bounded wait inside the kernel ran out; outputs are then unspecified).
  */
