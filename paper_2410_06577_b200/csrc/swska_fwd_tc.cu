@@ -53,10 +53,37 @@ struct SwCtl {
   int k_sent, v_sent, k_seen, v_seen;   // loads asked for / seen complete (for the clean exit)
 };
 
+// Two fp32 operations in one instruction (packed pairs in 64-bit registers) and the three-input
+// maximum: the softmax loop is bound by instruction issue and by the special-function unit, and
+// these halve the count of everything around the exponentials.
+__device__ __forceinline__ uint64_t pair_f32(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpair_f32(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 struct SwTcArgs {
   void* o;
   int32_t* status;   // may be nullptr
-  int H, T, window;
+  int B, H, T, window, n_qtiles;
   float scale;
   long long limit;
 };
@@ -94,10 +121,15 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   float* sMax = reinterpret_cast<float*>(gen + kOffMax);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // query tiles late in the sequence see the most keys: they are started first, the short ones fill the tail
-  const int m0 = (int)(gridDim.x - 1 - blockIdx.x) * kBM, h = blockIdx.y, b = blockIdx.z;
+  // Query tiles late in the sequence see the most keys.  CTAs are handed out in the order of
+  // their index, so the index runs over the query tiles from the last one down and, within one
+  // tile position, over all (batch, head): every long tile of the call starts before any short
+  // one, and the short ones fill the tail.
   const int T = a.T, W = a.window;
-  const long long bh = (long long)b * a.H + h;
+  const int n_bh = a.B * a.H;
+  const int m0 = (a.n_qtiles - 1 - (int)(blockIdx.x / (unsigned)n_bh)) * kBM;
+  const long long bh = blockIdx.x % (unsigned)n_bh;
+  const int b = (int)(bh / a.H);
   const long long qrow0 = bh * T + m0;           // row of the [B*H*T, 128] views of q, o
   const int krow0 = b * T;                       // row of the [B*T, 128] view of k
   const int vrow0 = (int)(bh * T);               // row of the [B*H*T, 128] view of v
@@ -250,14 +282,14 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             sv[e] = (key <= row && key > row - W) ? __uint_as_float(r[e]) : -INFINITY;
           }
         }
-        // maximum as a tree: four independent chains instead of one of 32 dependent steps
-        float m4[4] = {sv[0], sv[1], sv[2], sv[3]};
+        // maximum as a tree: four independent chains of three-input steps over eight values each
+        float m4[4];
 #pragma unroll
-        for (int e = 4; e < kHalf; e += 4) {
-          m4[0] = fmaxf(m4[0], sv[e]); m4[1] = fmaxf(m4[1], sv[e + 1]);
-          m4[2] = fmaxf(m4[2], sv[e + 2]); m4[3] = fmaxf(m4[3], sv[e + 3]);
+        for (int c = 0; c < 4; ++c) {
+          const float* s8 = sv + 8 * c;
+          m4[c] = fmaxf(max3(max3(max3(s8[0], s8[1], s8[2]), s8[3], s8[4]), s8[5], s8[6]), s8[7]);
         }
-        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        mx = fmaxf(max3(m4[0], m4[1], m4[2]), m4[3]);
       }
       sMax[(sb * 2 + half) * kBM + rowl] = mx * sc;   // (-inf stays -inf: sc > 0)
       // both threads of a row have read S (the probabilities overwrite it) and left their maximum
@@ -275,15 +307,22 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         m_ref = m_tile;
       }
       const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
-      float ps[4] = {0.f, 0.f, 0.f, 0.f};     // four partial sums: no chain of 16 dependent additions
+      uint64_t ps[4] = {0ull, 0ull, 0ull, 0ull};     // four pairs of partial sums: short dependent chains
       uint32_t pk[kHalf / 2];
+      const uint64_t sc2 = pair_f32(sc, sc), nm2 = pair_f32(-m_use, -m_use);
 #pragma unroll
       for (int e = 0; e < kHalf; e += 2) {
-        const float p0 = ex2f(fmaf(sv[e], sc, -m_use)), p1 = ex2f(fmaf(sv[e + 1], sc, -m_use));
-        ps[(e >> 1) & 3] += p0 + p1;
+        float x0, x1;
+        unpair_f32(fma2(pair_f32(sv[e], sv[e + 1]), sc2, nm2), x0, x1);
+        const float p0 = ex2f(x0), p1 = ex2f(x1);
+        ps[(e >> 1) & 3] = add2(ps[(e >> 1) & 3], pair_f32(p0, p1));
         pk[e >> 1] = pack_bf16(p0, p1);
       }
-      l_run = l_run * alpha + ((ps[0] + ps[1]) + (ps[2] + ps[3]));
+      {
+        float s0, s1;
+        unpair_f32(add2(add2(ps[0], ps[1]), add2(ps[2], ps[3])), s0, s1);
+        l_run = l_run * alpha + (s0 + s1);
+      }
       // rescaling O (rare) needs the previous O += P V complete; writing P does not
       if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
         ok = sw_wait(bar(BAR_O0 + ((it - 1) & 1)), ((it - 1) >> 1) & 1, ctl, a.status);
@@ -419,13 +458,16 @@ cudaError_t launch_swska_tc(const rodimus_swska_fwd_params& p, int* n_launches) 
   SwTcArgs a;
   a.o = p.o;
   a.status = reinterpret_cast<int32_t*>(p.workspace);
-  a.H = p.H; a.T = p.T; a.window = p.window; a.scale = p.scale;
+  a.B = p.B; a.H = p.H; a.T = p.T; a.window = p.window; a.scale = p.scale;
+  a.n_qtiles = (p.T + kBM - 1) / kBM;
+  const long long n_ctas = (long long)a.n_qtiles * p.B * p.H;
+  if (n_ctas > 0x7fffffffLL) return cudaErrorInvalidValue;
   a.limit = main_loop_wait_cycles();
   if (a.status) {
     e = cudaMemsetAsync(a.status, 0, sizeof(int32_t), st);
     if (e != cudaSuccess) return e;
   }
-  const dim3 grid((p.T + kBM - 1) / kBM, p.H, p.B);
+  const dim3 grid((unsigned)n_ctas);
   swska_fwd_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(c.mq, c.mk, c.mv, a);
   *n_launches = 1;
   return cudaGetLastError();
