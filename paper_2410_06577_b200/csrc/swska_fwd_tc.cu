@@ -256,6 +256,51 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     float m_ref = -INFINITY, l_run = 0.f;
     bool ok = true;
     int it = 0;
+    // the two threads of a row exchange their maxima of a tile (both have then read S, which the
+    // probabilities overwrite); the reference exponent follows; returns the factor for O and l
+    auto exchange = [&](int sb, int it, float mx, float& alpha) -> bool {
+      sMax[(sb * 2 + half) * kBM + rowl] = mx * sc;   // (-inf stays -inf: sc > 0)
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pair_bar);
+      bool good = sw_wait(pair_bar, it & 1, ctl, a.status);
+      good = __all_sync(0xffffffffu, good);
+      if (!good) return false;
+      tc_fence_after();
+      const float m_tile = fmaxf(sMax[(sb * 2) * kBM + rowl], sMax[(sb * 2 + 1) * kBM + rowl]);
+      alpha = 1.f;
+      if (m_tile > m_ref + 8.f) {               // also the first tile with a visible key
+        alpha = ex2f(m_ref - m_tile);           // 0 when nothing had been seen
+        m_ref = m_tile;
+      }
+      return true;
+    };
+    // rescaling O (rare) needs the previous O += P V complete; writing P does not
+    auto rescale = [&](int it, float alpha) -> bool {
+      if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+        bool good = sw_wait(bar(BAR_O0 + ((it - 1) & 1)), ((it - 1) >> 1) & 1, ctl, a.status);
+        good = __all_sync(0xffffffffu, good);
+        if (!good) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_row + kColO + 64 * half + 32 * c, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+          tmem_st32(t_row + kColO + 64 * half + 32 * c, r);
+        }
+      }
+      return true;
+    };
+    auto publish = [&](int sb, const uint32_t (&pk)[kHalf / 2]) {
+      tmem_st16(t_row + kColS + sb * kBN + 16 * half, pk);     // keys col0 .. col0+31, two per column
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_P0 + sb));
+    };
     for (; it < n_tiles; ++it) {
       const int sb = it & 1;
       const uint32_t ph = (it >> 1) & 1;
@@ -264,23 +309,36 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       ok = __all_sync(0xffffffffu, ok);     // the tensor-memory accesses below need the whole warp
       if (!ok) break;
       tc_fence_after();
+      // the visible keys of this thread's 32 are e_lo .. e_hi (none when e_lo > e_hi)
+      const int k0 = n0 + col0;
+      const int e_lo = max(0, row - W + 1 - k0), e_hi = min(kHalf - 1, row - k0);
+      if (__all_sync(0xffffffffu, e_lo > e_hi)) {
+        // on the diagonal and at the window's far edge whole warps see no key of a tile: they
+        // take part in the hand-offs and write zeros, without the arithmetic
+        float alpha;
+        if (!(ok = exchange(sb, it, -INFINITY, alpha))) break;
+        l_run *= alpha;
+        if (!(ok = rescale(it, alpha))) break;
+        uint32_t pk[kHalf / 2];
+#pragma unroll
+        for (int e = 0; e < kHalf / 2; ++e) pk[e] = 0u;
+        publish(sb, pk);
+        continue;
+      }
       // ---- this thread's 32 columns of its row of S: mask, maximum
       float sv[kHalf];
-      float mx = -INFINITY;
+      float mx;
       {
         uint32_t r[32];
         tmem_ld32(t_row + kColS + sb * kBN + col0, r);
         tmem_ld_wait();
-        const int k0 = n0 + col0;
-        if (k0 + kHalf - 1 <= row && k0 > row - W) {
+        if (e_lo == 0 && e_hi == kHalf - 1) {
 #pragma unroll
           for (int e = 0; e < kHalf; ++e) sv[e] = __uint_as_float(r[e]);
         } else {
+          const uint32_t bits = e_lo > e_hi ? 0u : ((0xffffffffu >> (kHalf - 1 - e_hi)) & (0xffffffffu << e_lo));
 #pragma unroll
-          for (int e = 0; e < kHalf; ++e) {
-            const int key = k0 + e;
-            sv[e] = (key <= row && key > row - W) ? __uint_as_float(r[e]) : -INFINITY;
-          }
+          for (int e = 0; e < kHalf; ++e) sv[e] = ((bits >> e) & 1u) ? __uint_as_float(r[e]) : -INFINITY;
         }
         // maximum as a tree: four independent chains of three-input steps over eight values each
         float m4[4];
@@ -291,21 +349,8 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         mx = fmaxf(max3(m4[0], m4[1], m4[2]), m4[3]);
       }
-      sMax[(sb * 2 + half) * kBM + rowl] = mx * sc;   // (-inf stays -inf: sc > 0)
-      // both threads of a row have read S (the probabilities overwrite it) and left their maximum
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(pair_bar);
-      ok = sw_wait(pair_bar, it & 1, ctl, a.status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
-      const float m_tile = fmaxf(sMax[(sb * 2) * kBM + rowl], sMax[(sb * 2 + 1) * kBM + rowl]);
-      float alpha = 1.f;
-      if (m_tile > m_ref + 8.f) {               // also the first tile with a visible key
-        alpha = ex2f(m_ref - m_tile);           // 0 when nothing had been seen
-        m_ref = m_tile;
-      }
+      float alpha;
+      if (!(ok = exchange(sb, it, mx, alpha))) break;
       const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
       uint64_t ps[4] = {0ull, 0ull, 0ull, 0ull};     // four pairs of partial sums: short dependent chains
       uint32_t pk[kHalf / 2];
@@ -323,29 +368,8 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         unpair_f32(add2(add2(ps[0], ps[1]), add2(ps[2], ps[3])), s0, s1);
         l_run = l_run * alpha + (s0 + s1);
       }
-      // rescaling O (rare) needs the previous O += P V complete; writing P does not
-      if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-        ok = sw_wait(bar(BAR_O0 + ((it - 1) & 1)), ((it - 1) >> 1) & 1, ctl, a.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tc_fence_after();
-        {
-#pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            uint32_t r[32];
-            tmem_ld32(t_row + kColO + 64 * half + 32 * c, r);
-            tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-            tmem_st32(t_row + kColO + 64 * half + 32 * c, r);
-          }
-        }
-      }
-      tmem_st16(t_row + kColS + sb * kBN + 16 * half, pk);     // keys col0 .. col0+31, two per column
-      tmem_st_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_P0 + sb));
+      if (!(ok = rescale(it, alpha))) break;
+      publish(sb, pk);
     }
     // ---- the last O += P V, then normalise and store this thread's 64 columns of its row
     if (ok) ok = sw_wait(bar(BAR_O0 + ((n_tiles - 1) & 1)), ((n_tiles - 1) >> 1) & 1, ctl, a.status);
