@@ -407,12 +407,16 @@ swska_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   }
   tc_fence_before();
   __syncthreads();
-  if (tid == 0 && ctl->abort) {   // clean exit: nothing may still be writing this CTA's shared or tensor memory
-    mbar_drain(bar(BAR_Q), 0);
-    for (int j = ctl->k_seen; j < ctl->k_sent; ++j) mbar_drain(bar(BAR_K0 + (j & 1)), (j >> 1) & 1);
-    for (int j = ctl->v_seen; j < ctl->v_sent; ++j) mbar_drain(bar(BAR_V0 + (j & 1)), (j >> 1) & 1);
-    umma_commit(bar(BAR_DRAIN));      // completes when every contraction issued so far has
-    mbar_drain(bar(BAR_DRAIN), 0);
+  if (ctl->abort) {   // clean exit: nothing may still be writing this CTA's shared or tensor memory
+    if (tid == 0) {
+      mbar_drain(bar(BAR_Q), 0);
+      for (int j = ctl->k_seen; j < ctl->k_sent; ++j) mbar_drain(bar(BAR_K0 + (j & 1)), (j >> 1) & 1);
+      for (int j = ctl->v_seen; j < ctl->v_sent; ++j) mbar_drain(bar(BAR_V0 + (j & 1)), (j >> 1) & 1);
+    }
+    if (warp == kIssuerWarp && lane == 0) {   // (a commit follows the contractions of the thread that makes it)
+      umma_commit(bar(BAR_DRAIN));            // completes when every contraction issued so far has
+      mbar_drain(bar(BAR_DRAIN), 0);
+    }
   }
   __syncthreads();
   if (warp == kIssuerWarp)
