@@ -185,7 +185,11 @@ int rodimus_ddts_step(const rodimus_ddts_step_params *p);
  * the feed-through and the shared-gate layout of the forward call have no backward here.
  * dtype BF16 contracts tf32 operands on the tensor cores with fp32 accumulation; dtype F32
  * splits each operand in two tf32 parts and keeps fp32 accuracy.  The workspace holds the
- * status word and 8 * dk bytes per token and head of scratch.
+ * status word, 8 * dk bytes per token and head of scratch, and 6 * dk/2 * dv * 4 bytes per
+ * (sequence, head): each sweep may be cut into time segments that run as thread blocks of their
+ * own and hand their slice of the state to the next one through that area.  A segment waits
+ * for the one before it under the same limit as every other wait (rodimus_ddts_test_set_wait_limit);
+ * if that ran out the status word holds RODIMUS_ERR_TIMEOUT and the outputs are unspecified.
  */
 typedef struct {
   int32_t struct_size;       /* sizeof(rodimus_ddts_bwd_params), checked                        */

@@ -45,12 +45,25 @@ struct BwdArgs {
   void *dq, *dk, *dx, *dy, *dv;
   float* ds0;
   float *u, *w, *c;        // scratch: [rows, DK], [rows, DK], [n_seq * H, DK]
+  float* seg_state;        // scratch: [n_seq * H * 6][64][256] state fragments handed from one time segment to the next
+  int32_t* seg_flag;       // scratch: [n_seq * H * 6] number of segments of the sweep that have finished
+  int nseg;                // time segments per sweep (1: a sweep is one CTA)
+  long long limit;         // cycles a CTA waits for the segment before it
   const int32_t* cu;
   WorkspaceHeader* hdr;
   int H, T, n_seq;
   float scale;
   int ingate;
 };
+
+__device__ __forceinline__ int32_t ld_acquire_s32(const int32_t* p) {
+  int32_t v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_s32(int32_t* p, int32_t v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 
 template <typename T>
 __device__ __forceinline__ void load8(const T* p, float (&o)[8]);
@@ -169,9 +182,14 @@ __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16* p, flo
 
 // MODE 0: forward sweep (dq, u, c); 1: reverse sweep, state [d][j] (dk, w, ds0);
 // 2: reverse sweep, state [j][d] (dv).
+// CTA index = ((segment * 6 + sweep slot) * items + item): all first segments, then all second ones ..
+__device__ __forceinline__ int segment_of_this_cta(const BwdArgs& a) {
+  return (int)(blockIdx.x / (gridDim.x / a.nseg));
+}
+
 template <typename T, int MODE>
 __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, const int half,
-                          const long long row0, const int len) {
+                          const long long row0, const int len, const int seg) {
   constexpr bool EXACT = sizeof(T) == 4, FAST = !EXACT;
   constexpr int NCH = MODE == 2 ? DK : DK / 2;      // key channels whose gates this CTA needs
   const int ch0 = MODE == 2 ? 0 : 64 * half;
@@ -201,8 +219,11 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
   const int m0 = MODE == 2 ? 128 * half + 16 * warp : 64 * half + 16 * (warp >> 1);
   const int nbase = MODE == 2 ? 0 : 128 * (warp & 1);
   float st[16][4];
+  // A sweep may be cut into time segments that run as CTAs of their own; a segment after the
+  // first starts from the state the one before it left in the workspace, in the layout of s0.
   {
-    const float* init = MODE == 0 ? a.s0 : a.dsT;
+    const float* init = seg > 0 ? a.seg_state : (MODE == 0 ? a.s0 : a.dsT);
+    const long long s_off = (seg > 0 ? sh * 3 + MODE : sh) * (long long)DK * DV;
 #pragma unroll
     for (int n = 0; n < 16; ++n) {
       const int c0 = nbase + 8 * n + 2 * t;
@@ -571,6 +592,26 @@ __device__ void bwd_sweep(const BwdArgs& a, float* smem, const long long sh, con
     __syncthreads();
   }
 
+  if (segment_of_this_cta(a) + 1 < a.nseg) {   // hand the state to the next segment
+    float* hand = a.seg_state + (sh * 3 + MODE) * (long long)DK * DV;
+#pragma unroll
+    for (int n = 0; n < 16; ++n) {
+      const int c0 = nbase + 8 * n + 2 * t;
+      if (MODE != 2) {
+        *reinterpret_cast<float2*>(hand + (long long)(m0 + g) * DV + c0) = make_float2(st[n][0], st[n][1]);
+        *reinterpret_cast<float2*>(hand + (long long)(m0 + g + 8) * DV + c0) = make_float2(st[n][2], st[n][3]);
+      } else {
+        hand[(long long)c0 * DV + m0 + g] = st[n][0];
+        hand[(long long)(c0 + 1) * DV + m0 + g] = st[n][1];
+        hand[(long long)c0 * DV + m0 + g + 8] = st[n][2];
+        hand[(long long)(c0 + 1) * DV + m0 + g + 8] = st[n][3];
+      }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) st_release_s32(a.seg_flag + sh * 6 + (MODE * 2 + half), segment_of_this_cta(a) + 1);
+    return;
+  }
   // ---- after the last chunk
   if (MODE == 0) {   // c[d] = sum_j dS_T[d][j] S_T[d][j]
     float p0 = 0.f, p1 = 0.f;
@@ -613,8 +654,15 @@ static_assert(16 * (128 + 4) <= 8 * 16 * LDR, "the dv tile fits the space of the
 template <typename T>
 __global__ void __launch_bounds__(kThreads, 2) ddts_bwd_sweep_kernel(const BwdArgs a) {
   extern __shared__ __align__(16) float smem[];
-  const long long sh = blockIdx.x / 6;     // sequence * H + head
-  const int part = blockIdx.x % 6, mode = part >> 1, half = part & 1;
+  // The three sweeps differ in length (on the layer shape: the transposed reverse sweep 1.14 ms,
+  // the forward sweep 0.99, the reverse sweep 0.91) and the grid is about 1.3 times the resident
+  // CTAs, so the index runs over the sweeps from the longest to the shortest and, within a sweep,
+  // over all (sequence, head): what starts late is short.
+  const unsigned n_items = gridDim.x / (6 * a.nseg);
+  const long long sh = blockIdx.x % n_items;     // sequence * H + head
+  const int seg = segment_of_this_cta(a);
+  const int slot = (int)(blockIdx.x / n_items) % 6;
+  const int part = slot < 2 ? 4 + slot : slot - 2, mode = part >> 1, half = part & 1;
   if (!a.cu && blockIdx.x == 0 && threadIdx.x == 0) a.hdr->status = RODIMUS_OK;
   const int h = (int)(sh % a.H);
   const long long n = sh / a.H;
@@ -630,9 +678,36 @@ __global__ void __launch_bounds__(kThreads, 2) ddts_bwd_sweep_kernel(const BwdAr
     row0 = sh * a.T;
     len = a.T;
   }
-  if (mode == 0) bwd_sweep<T, 0>(a, smem, sh, half, row0, len);
-  else if (mode == 1) bwd_sweep<T, 1>(a, smem, sh, half, row0, len);
-  else bwd_sweep<T, 2>(a, smem, sh, half, row0, len);
+  if (a.nseg > 1) {
+    // this segment's rows: chunks c_lo .. c_hi-1 of the sweep, counted from the sequence's start
+    // (forward sweep) or from its end (reverse sweeps); row0, len become those of the segment
+    const int nchunks = (len + kC - 1) / kC;
+    const int c_lo = (int)((long long)nchunks * seg / a.nseg), c_hi = (int)((long long)nchunks * (seg + 1) / a.nseg);
+    const int r_lo = (mode == 0 ? c_lo : nchunks - c_hi) * kC;
+    const int r_hi = min((mode == 0 ? c_hi : nchunks - c_lo) * kC, len);
+    row0 += r_lo;
+    len = r_hi > r_lo ? r_hi - r_lo : 0;
+  }
+  if (seg > 0) {
+    // The segment before this one belongs to a CTA with a lower index, and CTAs start in the
+    // order of their index: it is running or done.  The wait is bounded all the same.
+    const int32_t* flag = a.seg_flag + sh * 6 + part;
+    int late = 0;
+    if (threadIdx.x == 0) {
+      const long long t_start = clock64();
+      while (ld_acquire_s32(flag) < seg) {
+        if (clock64() - t_start > a.limit) { late = 1; break; }
+        __nanosleep(256);
+      }
+    }
+    if (__syncthreads_or(late)) {
+      if (threadIdx.x == 0) atomicMax(&a.hdr->status, (int)RODIMUS_ERR_TIMEOUT);
+      return;
+    }
+  }
+  if (mode == 0) bwd_sweep<T, 0>(a, smem, sh, half, row0, len, seg);
+  else if (mode == 1) bwd_sweep<T, 1>(a, smem, sh, half, row0, len, seg);
+  else bwd_sweep<T, 2>(a, smem, sh, half, row0, len, seg);
 }
 
 // dL/dlog alpha by suffix sums over the sequence, then dx, dy (Eq. "alpha_def", chain rule):
@@ -708,7 +783,10 @@ size_t bwd_scratch_bytes(const rodimus_ddts_bwd_params& p) {
   const size_t rows = (size_t)p.B * p.H * p.T;
   const size_t nseq = p.cu_seqlens ? (size_t)p.N : (size_t)p.B;
   size_t b = sizeof(float) * (2 * rows * DK + nseq * p.H * DK);
-  return (b + 255) & ~(size_t)255;
+  b = (b + 255) & ~(size_t)255;
+  b += nseq * p.H * 6 * (sizeof(float) * 64 * kThreads);        // state fragments between time segments
+  b += (nseq * p.H * 6 * sizeof(int32_t) + 255) & ~(size_t)255; // and their flags
+  return b;
 }
 
 cudaError_t launch_bwd(const rodimus_ddts_bwd_params& p, size_t scratch_offset, int* n_launches) {
@@ -721,6 +799,12 @@ cudaError_t launch_bwd(const rodimus_ddts_bwd_params& p, size_t scratch_offset, 
   a.u = reinterpret_cast<float*>(reinterpret_cast<char*>(p.workspace) + scratch_offset);
   a.w = a.u + rows * DK;
   a.c = a.w + rows * DK;
+  {
+    const size_t nseq = p.cu_seqlens ? (size_t)p.N : (size_t)p.B;
+    const size_t first = (sizeof(float) * (2 * rows * DK + nseq * p.H * DK) + 255) & ~(size_t)255;
+    a.seg_state = reinterpret_cast<float*>(reinterpret_cast<char*>(p.workspace) + scratch_offset + first);
+    a.seg_flag = reinterpret_cast<int32_t*>(a.seg_state + nseq * p.H * 6 * (size_t)64 * kThreads);
+  }
   a.cu = p.cu_seqlens;
   a.hdr = reinterpret_cast<WorkspaceHeader*>(p.workspace);
   a.H = p.H; a.T = p.T; a.n_seq = p.cu_seqlens ? p.N : p.B;
@@ -732,15 +816,39 @@ cudaError_t launch_bwd(const rodimus_ddts_bwd_params& p, size_t scratch_offset, 
   cudaError_t e = current_device(&dev, &sms);
   if (e != cudaSuccess) return e;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(p.stream);
+  // Time segments per sweep: a sweep is one serial scan, and 6 CTAs per (sequence, head) seldom
+  // fill the resident CTA slots evenly (the layer shape: 384 CTAs of ~1 ms on 296 slots = two
+  // rounds).  Cutting every sweep into n segments gives n times the CTAs at 1/n the length; n of
+  // 1..8 minimises rounds(n) / n, with at least four chunks per segment.  Equal costs go to the
+  // finer cut while the grid is only a few rounds (the three sweeps differ in length, and finer
+  // pieces pack better: 1.87 ms for n = 3, 1.81 for 6 on the layer shape), else to the coarser.
+  {
+    const long long slots = 2LL * sms, per_seq = p.T / (p.cu_seqlens ? (a.n_seq > 0 ? a.n_seq : 1) : 1);
+    const bool few_rounds = items * 6 < 4 * slots;
+    int best = 1;
+    double best_cost = 1e30;
+    for (int n = 1; n <= 8; ++n) {
+      if (n > 1 && per_seq < (long long)n * 4 * kC) break;
+      const double cost = (double)((items * 6 * n + slots - 1) / slots) / n;
+      if (cost < best_cost * 0.999 || (few_rounds && cost < best_cost * 1.001)) { best_cost = cost; best = n; }
+    }
+    a.nseg = best;
+    a.limit = main_loop_wait_cycles();
+    if (items * 6 * a.nseg > 0x7fffffffLL) return cudaErrorInvalidValue;
+    if (a.nseg > 1) {
+      e = cudaMemsetAsync(a.seg_flag, 0, sizeof(int32_t) * (size_t)items * 6, st);
+      if (e != cudaSuccess) return e;
+    }
+  }
   if (p.dtype == RODIMUS_BF16) {
     e = opt_in_shared_memory(ddts_bwd_sweep_kernel<__nv_bfloat16>, (int)kSweepSmem, dev, g_smem_done_bf16);
     if (e != cudaSuccess) return e;
-    ddts_bwd_sweep_kernel<__nv_bfloat16><<<(unsigned)(items * 6), kThreads, kSweepSmem, st>>>(a);
+    ddts_bwd_sweep_kernel<__nv_bfloat16><<<(unsigned)(items * 6 * a.nseg), kThreads, kSweepSmem, st>>>(a);
     ddts_bwd_gates_kernel<__nv_bfloat16><<<(unsigned)(items * (DK / kGateCh)), kGateCh * kGateSegs, 0, st>>>(a);
   } else {
     e = opt_in_shared_memory(ddts_bwd_sweep_kernel<float>, (int)kSweepSmem, dev, g_smem_done_f32);
     if (e != cudaSuccess) return e;
-    ddts_bwd_sweep_kernel<float><<<(unsigned)(items * 6), kThreads, kSweepSmem, st>>>(a);
+    ddts_bwd_sweep_kernel<float><<<(unsigned)(items * 6 * a.nseg), kThreads, kSweepSmem, st>>>(a);
     ddts_bwd_gates_kernel<float><<<(unsigned)(items * (DK / kGateCh)), kGateCh * kGateSegs, 0, st>>>(a);
   }
   *n_launches = 2;

@@ -193,7 +193,8 @@ def test_bwd_argument_errors_and_workspace_size(lib):
     assert rd.bwd_raw(_bwd(d_sT=FAKE + 8)) == rd.ERR_ALIGN
     assert rd.bwd_raw(_bwd()) == rd.ERR_WORKSPACE
     # header + two fp32 scratch rows of dk per token and head + one per (sequence, head)
-    want = 256 + 4 * (2 * 2 * 2 * 64 * 128 + 2 * 2 * 128)
+    # + six 64 x 256 fp32 state slices per (sequence, head) and their flags (a multiple of 256 bytes)
+    want = 256 + 4 * (2 * 2 * 2 * 64 * 128 + 2 * 2 * 128) + 2 * 2 * 6 * 65536 + 256
     assert rd.bwd_workspace_bytes(_bwd()) == want
     assert rd.bwd_raw(_bwd(workspace=0x7F0000002000, workspace_bytes=want - 256)) == rd.ERR_WORKSPACE
     assert rd.bwd_workspace_bytes(_bwd(dk=64)) == 0
@@ -201,7 +202,7 @@ def test_bwd_argument_errors_and_workspace_size(lib):
     cu = np.array([0, 10, 5, 64], dtype=np.int32)
     pv = _bwd(B=1, cu_seqlens=FAKE, cu_seqlens_host=cu.ctypes.data, N=3)
     pv.workspace, pv.workspace_bytes = 0x7F0000002000, rd.bwd_workspace_bytes(pv)
-    assert pv.workspace_bytes == 256 + 256 + 4 * (2 * 2 * 64 * 128 + 3 * 2 * 128)
+    assert pv.workspace_bytes == 256 + 256 + 4 * (2 * 2 * 64 * 128 + 3 * 2 * 128) + 3 * 2 * 6 * 65536 + 256
     assert rd.bwd_raw(pv) == rd.ERR_SEQLENS
     ok = _bwd(B=0, workspace=0x7F0000002000, workspace_bytes=4096)
     assert rd.bwd_raw(ok) == rd.OK and rd.last_launch_count() == 0

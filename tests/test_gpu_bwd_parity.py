@@ -141,3 +141,27 @@ def test_bwd_long_sequence_and_many_packed_sequences():
     cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
     p = wl.make_prefill(704, 1, 2, int(cu[-1]), 128, 256, "bf16", s0_std=0.1, cu_seqlens=cu, name="bwd_many")
     _check(p, 705, True)
+
+
+def test_bwd_segment_wait_that_runs_out_reports_timeout():
+    """A long sweep is cut into time segments that run as thread blocks of their own; each waits,
+    with a limit, for the one before it.  With the limit at zero the later segments find their
+    predecessors unfinished, give up and return: the call reports TIMEOUT, nothing hangs, and the
+    next call is clean."""
+    import torch
+    p = wl.make_prefill(801, 1, 2, 1000, 128, 256, "bf16", s0_std=0.1, name="bwd_wait")
+    d = prefill_to_device(p)
+    d_o, d_sT = wl.make_grads(802, p, True)
+    outs = [torch.zeros_like(d["q"]) for _ in range(4)] + [torch.zeros_like(d["v"])]
+    prm = rd.bwd_params(d["q"], d["k"], d["x"], d["y"], d["v"], dev(d_o, "bf16"), *outs,
+                        s0=d["s0"], d_sT=torch.from_numpy(d_sT).cuda())
+    ws = torch.empty(rd.bwd_workspace_bytes(prm), dtype=torch.uint8, device="cuda")
+    prm.workspace, prm.workspace_bytes = ws.data_ptr(), ws.numel()
+    rd.test_set_wait_limit(0)
+    try:
+        assert rd.bwd_raw(prm) == rd.OK
+        assert rd.device_status(ws) == rd.ERR_TIMEOUT
+    finally:
+        rd.test_set_wait_limit(-1)
+    torch.cuda.synchronize()
+    _check(p, 802, True)
