@@ -165,3 +165,15 @@ def test_bwd_segment_wait_that_runs_out_reports_timeout():
         rd.test_set_wait_limit(-1)
     torch.cuda.synchronize()
     _check(p, 802, True)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_bwd_packed_sequences_cut_into_time_segments(dtype):
+    # long enough on average for the sweeps to be cut into time segments, with an empty sequence,
+    # one of two chunks (one row in the second) and ragged tails among them
+    lens = [300, 0, 200, 17, 129]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    p = wl.make_prefill(901, 1, 2, int(cu[-1]), 128, 256, dtype, s0_std=0.1, cu_seqlens=cu,
+                        name="bwd_packed_segments")
+    _check(p, 902, True)
+    _check(p, 903, False, host_cu=False, want_d_s0=False)
