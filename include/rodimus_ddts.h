@@ -315,8 +315,8 @@ const char *rodimus_ddts_fwd_kernel_name(const rodimus_ddts_fwd_params *p);
  * `sink` is one device float (written only in a case that does not occur).  iters in 1 .. 2^24. */
 int rodimus_ddts_sfu_probe(int iters, float *sink, void *stream, long long *ops);
 
-/* Test hook (the paper has no counterpart).  Every wait inside the tensor-core prefill kernels is
- * bounded: when one runs out, the kernel stops early, frees what it holds and records
+/* Test hook (the paper has no counterpart).  Every wait inside the tensor-core prefill kernels,
+ * the attention kernel and between the time segments of the backward sweeps is bounded: when one runs out, the kernel stops early, frees what it holds and records
  * RODIMUS_ERR_TIMEOUT in the workspace status word (outputs are then unspecified, the device
  * stays usable).  The bound is a launch argument of about two seconds' worth of clock cycles;
  * this call replaces it, process-wide, for the launches that follow: 0 makes the first wait that
